@@ -1,0 +1,166 @@
+/*
+ * mwu.h -- C ABI of the micro-structured weight unification / pruning library
+ *          (method of arXiv 2106.08301), CUDA, sm_100a only.
+ *
+ * Conventions that hold for every entry point
+ *   - All tensor pointers are DEVICE pointers owned by the caller, 16-byte aligned unless
+ *     stated otherwise; the library allocates nothing and keeps no state between calls.
+ *   - Descriptors (mwu_proj_desc) and scalar arguments are HOST values.
+ *   - Work is enqueued on `cuda_stream` (a cudaStream_t passed as void*, NULL = default
+ *     stream).  No call synchronises with the host.
+ *   - Argument errors are returned before anything is launched.  Conditions that only the
+ *     device can see set bits in *dev_status (a device uint32_t the caller zeroes and reads
+ *     after synchronising); outputs are then unspecified but every access stays in bounds.
+ *   - There is no CPU fallback: on a device that is not compute capability 10.x the calls
+ *     return MWU_ERR_UNSUPPORTED_DEVICE.
+ *
+ * Notation (paper, Section 3.1): a layer's weight tensor is viewed as W[rows][cols]
+ * (rows = output features / filters, cols = the reduction axis; for a convolution
+ * cols = cin*kh*kw in [cout, cin, kh, kw] order).  It is divided into Mb = rows*cols/block
+ * micro-blocks of `block` consecutive entries of one row; block j = n*(cols/block) + kb
+ * covers W[n][kb*block .. kb*block+block-1].
+ */
+#ifndef MWU_H_
+#define MWU_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    MWU_OK = 0,
+    MWU_ERR_INVALID_ARG = 1,        /* null pointer, negative size, unknown enum value        */
+    MWU_ERR_SHAPE = 2,              /* cols % block != 0, block not in {2,4,8,16}, bad counts */
+    MWU_ERR_ALIGNMENT = 3,          /* a pointer or leading dimension is not aligned          */
+    MWU_ERR_WORKSPACE = 4,          /* workspace / packed buffer too small                    */
+    MWU_ERR_UNSUPPORTED_DEVICE = 5, /* current device is not sm_100                           */
+    MWU_ERR_CUDA = 6                /* a CUDA runtime or driver call failed                   */
+} mwu_status;
+
+/* bits of the device status word */
+enum {
+    MWU_DEV_NONFINITE = 1,  /* an input weight was NaN or Inf                                 */
+    MWU_DEV_TIMEOUT = 2,    /* a bounded wait inside a kernel ran out                         */
+    MWU_DEV_BOUNDS = 4,     /* packed data inconsistent with the descriptor (nothing written
+                               out of bounds)                                                 */
+    MWU_DEV_SELECT = 8      /* internal selection invariant violated                          */
+};
+
+typedef enum {
+    MWU_PRUNE_KEY_L2SQ = 0, /* sum v^2: squared distance to the zero block (Eq. 7, q = 0)     */
+    MWU_PRUNE_KEY_L1 = 1    /* sum |v|: the norm Section 3.1's pruning example names          */
+} mwu_prune_key;
+
+typedef struct {
+    int64_t rows, cols;     /* W[rows][cols], row-major, cols % block == 0                    */
+    int32_t block;          /* micro-block width along cols: 2, 4, 8 or 16                    */
+    int32_t prune_key;      /* mwu_prune_key                                                  */
+    int64_t k_unify;        /* number of blocks unified OR pruned (0 <= k_prune <= k_unify)   */
+    int64_t k_prune;        /* number of blocks pruned to zero                                */
+} mwu_proj_desc;
+
+const char *mwu_status_string(int status);
+
+/* Ratio -> integer count, (permille * n_blocks + 500) / 1000 in integers.  The paper gives
+ * ratios (Section 1, "unification ratio"); counts cross this ABI as integers so that no
+ * floating-point rounding can make caller and library disagree. */
+int64_t mwu_count_from_permille(int64_t n_blocks, int32_t permille);
+
+/*
+ * mwu_project -- the Q-step of ADMM: Q = Unify(W + U)   (Algorithm 1; Eq. 7: a Euclidean
+ * projection onto the set of tensors with k_prune zero blocks and k_unify - k_prune further
+ * blocks whose entries share one absolute value).
+ *
+ * Per block (Section 3.1, Eq. 2 and the text after it) with v = W, or fp32(W + U_dual):
+ *   q   = mean |v_l|                    unified value
+ *   L_u = sum (|v_l| - q)^2             unification loss  (distance^2 to the unified block)
+ *   L_p = sum v_l^2  (or sum |v_l|)     prune key         (distance^2 to the zero block)
+ * evaluated in fp64, each operation rounded on its own, block sums as a balanced pairwise
+ * tree.  Selection: the k_prune blocks with the smallest prune key are pruned; among the
+ * others the k_unify - k_prune blocks with the smallest L_u are unified; equal keys are
+ * ordered by block index.  Output of a pruned block is +0; of a unified block +q where
+ * v_l >= 0 (this includes -0.0) and -q otherwise, q rounded to fp32; other blocks are
+ * copied bit for bit.
+ *
+ *   W, U_dual      in   fp32 [rows*cols]; U_dual may be NULL
+ *   Q              out  fp32 [rows*cols]; may be NULL (only the compressed form is wanted)
+ *   u              out  fp32 [Mb]: fp32(q) for unified blocks, +0 otherwise
+ *   pruned_bitmap, unified_bitmap
+ *                  out  uint32 [ceil(Mb/32)], bit (j%32) of word (j/32); unused bits 0
+ *   sign_bits      out  uint32 [ceil(rows*cols/32)], bit = (v_l < 0) for every weight
+ *   loss_u, loss_p out  fp64 [Mb] each, may be NULL: L_u and the prune key of every block
+ *   dev_status     i/o  device uint32, bits OR-ed in
+ *   workspace      device scratch of at least mwu_project_workspace_bytes(desc) bytes,
+ *                  256-byte aligned; contents undefined on entry and exit
+ * Errors: MWU_ERR_* as listed above; nothing is launched on error.
+ */
+size_t mwu_project_workspace_bytes(const mwu_proj_desc *desc);
+int mwu_project(const mwu_proj_desc *desc, const float *W, const float *U_dual, float *Q,
+                float *u, uint32_t *pruned_bitmap, uint32_t *unified_bitmap,
+                uint32_t *sign_bits, double *loss_u, double *loss_p, uint32_t *dev_status,
+                void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
+ * mwu_pack -- the storage form of Section 3.1 / Table 1: a unified block keeps one
+ * magnitude, a pruned block nothing, every weight one sign bit, the remaining blocks their
+ * values (here rounded to bf16, the type the GEMM multiplies in).
+ *
+ * Needs cols % 64 == 0.  Inputs are mwu_project's inputs and outputs for the same desc.
+ * `packed` receives exactly mwu_packed_bytes(desc) bytes (256-byte aligned buffer):
+ *   header   256 B : u64 magic "MWUPACK1", version, rows, cols, block, rows_padded, n_tiles,
+ *                    n_stages, n_pruned, n_unified, n_dense, byte offsets of the five sections,
+ *                    total bytes
+ *   rec      16 B per record (row tile of 128 rows x 64 columns), tile-major:
+ *                    u32 ubase, dbase (index of the record's first entry in ustream/dstream),
+ *                    u32 live (bit s set if some row has a non-pruned block overlapping columns
+ *                    [16s,16s+16) of the record), u32 0
+ *   meta     16 B per (record, row): u64 sign bits of the 64 columns, u32 pruned bits and
+ *                    u32 unified bits of the 64/block blocks (bit i = block i of the row)
+ *   rel      4 B per (record, row): u16 unified and u16 dense blocks in earlier rows of the
+ *                    record
+ *   ustream  fp32 unified value per unified block, ordered by record, row, position
+ *   dstream  bf16 (round to nearest even) values of the other non-pruned blocks, same order
+ * Rows beyond `rows` up to the next multiple of 128 are padding and count as pruned.
+ * Sections start on 256-byte boundaries, gaps are zero.  A mismatch between the bitmaps and
+ * desc's counts sets MWU_DEV_BOUNDS.
+ */
+size_t mwu_packed_bytes(const mwu_proj_desc *desc);
+int mwu_pack(const mwu_proj_desc *desc, const float *W, const float *U_dual, const float *u,
+             const uint32_t *pruned_bitmap, const uint32_t *unified_bitmap,
+             const uint32_t *sign_bits, void *packed, size_t packed_bytes,
+             uint32_t *dev_status, void *cuda_stream);
+
+/*
+ * mwu_gemm -- layer forward on the compressed weights (Section 3.2): Y = X . W_hat^T with
+ * W_hat decoded from `packed` (0 for pruned blocks, +-bf16(u) by sign bit for unified blocks,
+ * the stored bf16 values otherwise).  Column slices that are pruned in every row of a weight
+ * tile are skipped; products are bf16 x bf16 accumulated in fp32.
+ *
+ *   X        in   bf16 [M][ldx], ldx >= cols, ldx % 8 == 0
+ *   Y        out  [M][ldy], ldy >= rows; y_dtype 0: bf16 (round to nearest even, ldy % 8 == 0),
+ *                 1: fp32 (ldy % 4 == 0)
+ * M may be any positive value (ragged last tile is handled); M == 0 is a no-op.
+ */
+int mwu_gemm(const mwu_proj_desc *desc, const void *packed, const void *X, int64_t M,
+             int64_t ldx, void *Y, int64_t ldy, int32_t y_dtype, uint32_t *dev_status,
+             void *cuda_stream);
+
+/*
+ * mwu_conv_implicit -- the same contraction for a convolution lowered to GEMM without
+ * materialising the lowered matrix (Section 3.2: "convolution ... implemented by GEMM"):
+ *   A[(n,oh,ow)][(c,i,j)] = x[n][c][oh*stride+i-pad][ow*stride+j-pad]  (0 outside),
+ *   y[n][o][oh][ow] = sum_k A[(n,oh,ow)][k] * W_hat[o][k],  desc->cols == c*kh*kw.
+ *   X  in  bf16 NCHW [n][c][h][w];   Y  out NCHW [n][rows][oh][ow], y_dtype as above.
+ */
+int mwu_conv_implicit(const mwu_proj_desc *desc, const void *packed, const void *X_nchw,
+                      int32_t n, int32_t c, int32_t h, int32_t w, int32_t kh, int32_t kw,
+                      int32_t stride, int32_t pad, void *Y_nchw, int32_t y_dtype,
+                      uint32_t *dev_status, void *cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MWU_H_ */

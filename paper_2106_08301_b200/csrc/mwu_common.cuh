@@ -1,0 +1,66 @@
+// Shared host/device helpers of the CUDA library: argument validation, the packed-format
+// layout arithmetic, and small device utilities.  Nothing here is used by the CPU checker.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <stddef.h>
+
+#include "mwu.h"
+
+namespace mwu {
+
+constexpr int kTileRows = 128;     // rows of W per packed record
+constexpr int kStageK = 64;        // reduction-axis extent per packed record
+constexpr int kHeaderBytes = 256;
+constexpr size_t kAlign = 256;
+constexpr unsigned long long kMagic = 0x314B43415055574Dull;   // "MWUPACK1" little-endian
+
+inline size_t align_up(size_t x, size_t a = kAlign) { return (x + a - 1) / a * a; }
+
+struct PackedLayout {
+    int64_t n_pad, n_tiles, n_stages, n_unified, n_dense, n_pruned;
+    size_t off_rec, off_meta, off_rel, off_ustream, off_dstream, total;
+};
+
+inline PackedLayout packed_layout(const mwu_proj_desc *d) {
+    PackedLayout L;
+    const int64_t mb = d->rows * d->cols / d->block;
+    L.n_pad = (d->rows + kTileRows - 1) / kTileRows * kTileRows;
+    L.n_tiles = L.n_pad / kTileRows;
+    L.n_stages = d->cols / kStageK;
+    L.n_pruned = d->k_prune;
+    L.n_unified = d->k_unify - d->k_prune;
+    L.n_dense = mb - d->k_unify;
+    const size_t n_rs = (size_t)L.n_tiles * L.n_stages * kTileRows;
+    L.off_rec = kHeaderBytes;
+    L.off_meta = align_up(L.off_rec + 16 * (size_t)L.n_tiles * L.n_stages);
+    L.off_rel = align_up(L.off_meta + 16 * n_rs);
+    L.off_ustream = align_up(L.off_rel + 4 * n_rs);
+    L.off_dstream = align_up(L.off_ustream + 4 * (size_t)L.n_unified);
+    L.total = align_up(L.off_dstream + 2 * (size_t)d->block * L.n_dense);
+    return L;
+}
+
+// MWU_OK or the error that describes what is wrong with the descriptor.
+inline int validate_desc(const mwu_proj_desc *d, bool need_stage_multiple) {
+    if (!d) return MWU_ERR_INVALID_ARG;
+    if (d->rows <= 0 || d->cols <= 0) return MWU_ERR_SHAPE;
+    if (d->block != 2 && d->block != 4 && d->block != 8 && d->block != 16) return MWU_ERR_SHAPE;
+    if (d->cols % d->block != 0) return MWU_ERR_SHAPE;
+    if (need_stage_multiple && d->cols % kStageK != 0) return MWU_ERR_SHAPE;
+    if (d->prune_key != MWU_PRUNE_KEY_L2SQ && d->prune_key != MWU_PRUNE_KEY_L1)
+        return MWU_ERR_INVALID_ARG;
+    const int64_t mb = d->rows * d->cols / d->block;
+    if (mb >= (int64_t(1) << 31)) return MWU_ERR_SHAPE;
+    if (d->k_prune < 0 || d->k_prune > d->k_unify || d->k_unify > mb) return MWU_ERR_SHAPE;
+    return MWU_OK;
+}
+
+inline bool aligned_to(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+// MWU_OK when the current device is compute capability 10.x; also reports its SM count.
+int check_device(int *sm_count);
+
+}  // namespace mwu

@@ -1,0 +1,157 @@
+"""GPU parity: mwu_project / mwu_pack through the C ABI against the CPU checker."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import mwu_oracle as O
+from paper_2106_08301_b200 import binding as B
+from paper_2106_08301_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+
+
+def run_project(W, b, ku, kp, U=None, prune_key=0, want_loss=True):
+    rows, cols = W.shape
+    desc = B.make_desc(rows, cols, b, ku, kp, prune_key)
+    bufs = B.ProjectionBuffers(desc, want_q=True, want_loss=want_loss)
+    Wd = W.cuda().contiguous()
+    Ud = U.cuda().contiguous() if U is not None else None
+    bufs.project(Wd, Ud)
+    torch.cuda.synchronize()
+    return desc, bufs, Wd, Ud
+
+
+def check_against_oracle(W, b, ku, kp, U=None, prune_key=0):
+    desc, bufs, Wd, Ud = run_project(W, b, ku, kp, U, prune_key)
+    assert int(bufs.dev_status.item()) == 0
+    p = O.project(W.numpy(), b, ku, kp, U=None if U is None else U.numpy(),
+                  prune_key="l1" if prune_key else "l2sq")
+    # keys: bit-exact fp64
+    lu = bufs.loss_u.cpu().numpy()
+    lp = bufs.loss_p.cpu().numpy()
+    assert np.array_equal(lu.view(np.uint64), p.stats.L_u.view(np.uint64))
+    kp_ref = p.stats.S if prune_key else p.stats.L_p
+    assert np.array_equal(lp.view(np.uint64), kp_ref.view(np.uint64))
+    # selection, sign plane: bit-exact
+    pb = bufs.pruned_bitmap.cpu().numpy().view(np.uint32)
+    ub = bufs.unified_bitmap.cpu().numpy().view(np.uint32)
+    assert np.array_equal(pb, O.bitmap_words(p.pruned))
+    assert np.array_equal(ub, O.bitmap_words(p.unified))
+    sb = bufs.sign_bits.cpu().numpy().view(np.uint32)
+    assert np.array_equal(sb, O.bitmap_words(p.sign.reshape(-1)))
+    # unified values within 1e-6 relative (they are in fact the same fp32 numbers)
+    u = bufs.u.cpu().numpy()
+    assert np.allclose(u, p.u, rtol=1e-6, atol=0)
+    assert np.array_equal(u, p.u)
+    Q = bufs.Q.cpu().numpy().reshape(W.shape)
+    assert np.array_equal(Q.view(np.uint32), p.Q.view(np.uint32))
+    return desc, bufs, Wd, Ud, p
+
+
+@pytest.mark.parametrize("b", [2, 4, 8, 16])
+@pytest.mark.parametrize("rows,cols", [(64, 64), (96, 160), (7, 48), (300, 1008)])
+def test_projection_parity_small(b, rows, cols):
+    W = inputs.normal_weights(rows, cols, 0.02, 1234 + b)
+    Mb = rows * cols // b
+    check_against_oracle(W, b, O.count_from_permille(Mb, 600), O.count_from_permille(Mb, 300))
+
+
+@pytest.mark.parametrize("ku,kp", [(0, 0), (1, 0), (1, 1), (2048, 0), (2048, 2048), (4096, 1),
+                                   (4096, 4096), (4096, 4095), (3000, 2999)])
+def test_projection_edge_counts(ku, kp):
+    W = inputs.normal_weights(64, 256, 0.02, 77)
+    check_against_oracle(W, 4, ku, kp)
+
+
+def test_projection_l1_key_and_dual():
+    W = inputs.normal_weights(128, 256, 0.02, 5)
+    U = inputs.normal_weights(128, 256, 0.004, 6)
+    Mb = 128 * 256 // 8
+    check_against_oracle(W, 8, Mb // 2, Mb // 4, U=U)
+    check_against_oracle(W, 8, Mb // 2, Mb // 4, prune_key=1)
+
+
+def test_projection_ties_zeros_and_negative_zero():
+    g = torch.Generator().manual_seed(3)
+    W = inputs.normal_weights(64, 128, 0.02, 9)
+    W[:, 0:32] = 0.0                 # whole zero blocks: exact ties at key 0
+    W[5, 0:4] = -0.0
+    W[:, 64:96] = W[0:1, 64:96]      # identical blocks in every row
+    W[:, 96:128] = 0.5 * torch.sign(torch.randn(64, 32, generator=g))   # equal magnitudes: L_u == 0
+    for b in (4, 16):
+        Mb = W.numel() // b
+        check_against_oracle(W, b, Mb * 3 // 4, Mb // 8)
+        check_against_oracle(W, b, Mb // 8, Mb // 16)
+
+
+def test_projection_idempotent_on_device():
+    W = inputs.normal_weights(256, 256, 0.02, 11)
+    b = 8
+    Mb = W.numel() // b
+    ku, kp = Mb * 6 // 10, Mb * 3 // 10
+    desc, bufs, Wd, _, p = check_against_oracle(W, b, ku, kp)
+    Q1 = bufs.Q.clone().reshape(256, 256)
+    # projecting the projection: massive exact ties (all pruned blocks 0, all unified L_u = 0)
+    desc2, bufs2, _, _, p2 = check_against_oracle(Q1.cpu(), b, ku, kp)
+    assert torch.equal(bufs2.Q.view(torch.int32), Q1.reshape(-1).view(torch.int32))
+
+
+def test_projection_large_tie_group_refinement():
+    """All blocks identical: the threshold is decided by block index alone."""
+    blk = torch.tensor([0.5, -0.25, 0.125, 1.0])
+    W = blk.repeat(256 * 64).reshape(256, 256).contiguous()
+    check_against_oracle(W, 4, 9000, 5000)
+
+
+def test_nonfinite_sets_status():
+    W = inputs.normal_weights(64, 64, 0.02, 1)
+    W[3, 7] = float("inf")
+    desc, bufs, _, _ = run_project(W, 4, 100, 50, want_loss=False)
+    assert int(bufs.dev_status.item()) & B.MWU_DEV_NONFINITE
+
+
+@pytest.mark.parametrize("name", ["c1_linear", "c2_conv3x3", "c3_conv1x1"])
+def test_projection_and_pack_parity_configs(name):
+    wl = inputs.WORKLOADS[name]
+    W = wl.weights()
+    Mb = wl.n_blocks
+    ku = B.mwu_count_from_permille(Mb, wl.unified_permille)
+    kp = B.mwu_count_from_permille(Mb, wl.pruned_permille)
+    assert ku == O.count_from_permille(Mb, wl.unified_permille)
+    assert kp == O.count_from_permille(Mb, wl.pruned_permille)
+    desc, bufs, Wd, _, p = check_against_oracle(W, wl.block, ku, kp)
+    packed = bufs.pack(Wd)
+    torch.cuda.synchronize()
+    assert int(bufs.dev_status.item()) == 0
+    ref = O.pack(p, wl.block)
+    got = packed.cpu().numpy()
+    assert got.shape == ref.shape
+    assert np.array_equal(got, ref)
+
+
+@pytest.mark.parametrize("b,rows,cols", [(2, 100, 128), (4, 130, 64), (8, 257, 192), (16, 128, 256)])
+def test_pack_parity_ragged_rows(b, rows, cols):
+    W = inputs.normal_weights(rows, cols, 0.02, 99 + b)
+    Mb = rows * cols // b
+    desc, bufs, Wd, _, p = check_against_oracle(W, b, Mb * 7 // 10, Mb * 4 // 10)
+    packed = bufs.pack(Wd)
+    torch.cuda.synchronize()
+    assert int(bufs.dev_status.item()) == 0
+    assert np.array_equal(packed.cpu().numpy(), O.pack(p, b))
+
+
+def test_pack_with_dual_and_structured_pruning():
+    rows, cols, b = 256, 256, 16
+    W = inputs.normal_weights(rows, cols, 0.02, 21)
+    U = inputs.normal_weights(rows, cols, 0.002, 22)
+    W[:, 64:128] = 0.0
+    U[:, 64:128] = 0.0               # a whole 64-column stage is zero in every row
+    Mb = rows * cols // b
+    desc, bufs, Wd, Ud, p = check_against_oracle(W, b, Mb // 2, Mb // 4, U=U)
+    packed = bufs.pack(Wd, Ud)
+    torch.cuda.synchronize()
+    ref = O.pack(p, b)
+    assert np.array_equal(packed.cpu().numpy(), ref)
+    h = O.parse_header(ref)
+    rec = ref[h["off_rec"]:h["off_rec"] + 16 * 8].view(np.uint32).reshape(-1, 4)
+    assert rec[1, 2] == 0 and rec[5, 2] == 0          # stage 1 of both row tiles is dead
