@@ -109,23 +109,24 @@ int mwu_project(const mwu_proj_desc *desc, const float *W, const float *U_dual, 
  * values (here rounded to bf16, the type the GEMM multiplies in).
  *
  * Needs cols % 64 == 0.  Inputs are mwu_project's inputs and outputs for the same desc.
- * `packed` receives exactly mwu_packed_bytes(desc) bytes (256-byte aligned buffer):
- *   header   256 B : u64 magic "MWUPACK1", version, rows, cols, block, rows_padded, n_tiles,
- *                    n_stages, n_pruned, n_unified, n_dense, byte offsets of the five sections,
- *                    total bytes
- *   rec      16 B per record (row tile of 128 rows x 64 columns), tile-major:
- *                    u32 ubase, dbase (index of the record's first entry in ustream/dstream),
- *                    u32 live (bit s set if some row has a non-pruned block overlapping columns
- *                    [16s,16s+16) of the record), u32 0
- *   meta     16 B per (record, row): u64 sign bits of the 64 columns, u32 pruned bits and
- *                    u32 unified bits of the 64/block blocks (bit i = block i of the row)
- *   rel      4 B per (record, row): u16 unified and u16 dense blocks in earlier rows of the
- *                    record
- *   ustream  fp32 unified value per unified block, ordered by record, row, position
- *   dstream  bf16 (round to nearest even) values of the other non-pruned blocks, same order
- * Rows beyond `rows` up to the next multiple of 128 are padding and count as pruned.
- * Sections start on 256-byte boundaries, gaps are zero.  A mismatch between the bitmaps and
- * desc's counts sets MWU_DEV_BOUNDS.
+ * `packed` receives exactly mwu_packed_bytes(desc) bytes (256-byte aligned buffer).  A record is
+ * a row tile of 128 rows x 64 columns; it has 128 * 64/block block slots with slot code
+ * pos = row_in_tile * (64/block) + block_in_record.  Per record the blocks are listed by class,
+ * each list in ascending pos order, records in tile-major order:
+ *   header  256 B : u64 magic "MWUPACK1", version 2, rows, cols, block, rows_padded, n_tiles,
+ *                   n_stages, n_pruned, n_unified, n_dense, n_plist, byte offsets of rec, ulist,
+ *                   dpos, dpay, ppos, total bytes
+ *   rec     16 B per record plus one closing entry: u32 ubase, dbase, pbase (index of the
+ *                   record's first entry in ulist, dpos/dpay, ppos; the closing entry holds the
+ *                   totals), u32 live (bit s set if some row has a non-pruned block overlapping
+ *                   columns [16s,16s+16) of the record)
+ *   ulist   8 B per unified block: u32 (pos | sign bits << 16; bit l = (v_l < 0)), fp32 value
+ *   dpos    u16 pos per remaining non-pruned ("dense") block
+ *   dpay    the dense block's `block` values as bf16 (round to nearest even), same order
+ *   ppos    u16 pos per pruned block
+ * Rows beyond `rows` up to the next multiple of 128 are padding and are listed as pruned
+ * (n_plist = n_pruned + padding blocks).  Sections start on 256-byte boundaries, gaps are
+ * zero.  A mismatch between the bitmaps and desc's counts sets MWU_DEV_BOUNDS.
  */
 size_t mwu_packed_bytes(const mwu_proj_desc *desc);
 int mwu_pack(const mwu_proj_desc *desc, const float *W, const float *U_dual, const float *u,

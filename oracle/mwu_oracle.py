@@ -48,7 +48,7 @@ STAGE_K = 64             # reduction-axis extent per record
 HEADER_BYTES = 256
 SECTION_ALIGN = 256
 MAGIC = b"MWUPACK1"
-VERSION = 1
+VERSION = 2
 
 
 def count_from_permille(n_blocks: int, permille: int) -> int:
@@ -188,42 +188,53 @@ def _align(x: int, a: int = SECTION_ALIGN) -> int:
     return (x + a - 1) // a * a
 
 
-def packed_layout(N: int, K: int, b: int, n_unified: int, n_dense: int) -> dict:
+def packed_layout(N: int, K: int, b: int, n_unified: int, n_dense: int, n_pruned: int) -> dict:
     assert K % STAGE_K == 0 and STAGE_K % b == 0
     n_pad = _align(N, TILE_ROWS)
     n_tiles = n_pad // TILE_ROWS
     n_stages = K // STAGE_K
-    n_rs = n_tiles * n_stages * TILE_ROWS
+    n_plist = n_pruned + (n_pad - N) * (K // b)          # padding rows count as pruned
     off_rec = HEADER_BYTES
-    off_meta = _align(off_rec + 16 * n_tiles * n_stages)
-    off_rel = _align(off_meta + 16 * n_rs)
-    off_ustream = _align(off_rel + 4 * n_rs)
-    off_dstream = _align(off_ustream + 4 * n_unified)
-    total = _align(off_dstream + 2 * b * n_dense)
-    return dict(n_pad=n_pad, n_tiles=n_tiles, n_stages=n_stages, off_rec=off_rec,
-                off_meta=off_meta, off_rel=off_rel, off_ustream=off_ustream,
-                off_dstream=off_dstream, total=total)
+    off_ulist = _align(off_rec + 16 * (n_tiles * n_stages + 1))
+    off_dpos = _align(off_ulist + 8 * n_unified)
+    off_dpay = _align(off_dpos + 2 * n_dense)
+    off_ppos = _align(off_dpay + 2 * b * n_dense)
+    total = _align(off_ppos + 2 * n_plist)
+    return dict(n_pad=n_pad, n_tiles=n_tiles, n_stages=n_stages, n_plist=n_plist, off_rec=off_rec,
+                off_ulist=off_ulist, off_dpos=off_dpos, off_dpay=off_dpay, off_ppos=off_ppos,
+                total=total)
+
+
+HEADER_FIELDS = ["magic", "version", "N", "K", "b", "n_pad", "n_tiles", "n_stages", "n_pruned",
+                 "n_unified", "n_dense", "n_plist", "off_rec", "off_ulist", "off_dpos", "off_dpay",
+                 "off_ppos", "total"]
 
 
 def pack(p: Projection, b: int) -> np.ndarray:
     """Serialise a projection into the packed byte format (uint8 array).
 
-    Records are (row tile of 128 rows) x (64 reduction-axis entries); inside a
-    record blocks are ordered by row, then by position.  Rows beyond N are
-    padding and count as pruned.
+    A record is (row tile of 128 rows) x (64 reduction-axis entries) and holds 128 * 64/b
+    block slots; slot code pos = row_in_tile * (64/b) + block_in_stage.  Per record the blocks
+    are listed by class, each list in ascending pos order:
+      ulist  8 B per unified block: u32 (pos | sign bits << 16), fp32 unified value
+      dpos   u16 pos per dense block;  dpay  its b values as bf16 (round to nearest even)
+      ppos   u16 pos per pruned block (rows beyond N are padding and count as pruned)
+    rec[i] = (u32 ubase, dbase, pbase, live) gives where record i starts in each list; rec has
+    one extra entry holding the totals.  live bit s = some row of the record has a non-pruned
+    block overlapping columns [16s, 16s+16).
     """
     N, K = p.V.shape
     nb = STAGE_K // b
     n_unified = int(p.unified.sum())
     n_pruned = int(p.pruned.sum())
     n_dense = p.unified.shape[0] - n_unified - n_pruned
-    L = packed_layout(N, K, b, n_unified, n_dense)
+    L = packed_layout(N, K, b, n_unified, n_dense, n_pruned)
     n_pad, n_tiles, n_stages = L["n_pad"], L["n_tiles"], L["n_stages"]
     buf = np.zeros(L["total"], dtype=np.uint8)
 
     hdr = [int.from_bytes(MAGIC, "little"), VERSION, N, K, b, n_pad, n_tiles, n_stages,
-           n_pruned, n_unified, n_dense, L["off_rec"], L["off_meta"], L["off_rel"],
-           L["off_ustream"], L["off_dstream"], L["total"]]
+           n_pruned, n_unified, n_dense, L["n_plist"], L["off_rec"], L["off_ulist"],
+           L["off_dpos"], L["off_dpay"], L["off_ppos"], L["total"]]
     buf[:8 * len(hdr)] = np.frombuffer(struct.pack("<%dQ" % len(hdr), *hdr), dtype=np.uint8)
 
     pruned = np.ones((n_pad, K // b), dtype=bool)
@@ -237,15 +248,11 @@ def pack(p: Projection, b: int) -> np.ndarray:
     vbf = np.zeros((n_pad, K), dtype=np.uint16)
     vbf[:N] = bf16_bits_rne(p.V)
 
-    rec = np.zeros((n_tiles * n_stages, 4), dtype=np.uint32)
-    meta_sgn = np.zeros(n_tiles * n_stages * TILE_ROWS, dtype=np.uint64)
-    meta_pu = np.zeros((n_tiles * n_stages * TILE_ROWS, 2), dtype=np.uint32)
-    rel = np.zeros((n_tiles * n_stages * TILE_ROWS, 2), dtype=np.uint16)
-    ustream = []
-    dstream = []
-    n_u = 0
-    n_d = 0
-    bitw = (np.uint64(1) << np.arange(64, dtype=np.uint64))
+    n_rec = n_tiles * n_stages
+    rec = np.zeros((n_rec + 1, 4), dtype=np.uint32)
+    ulist_w0, ulist_u, dpos, dpay, ppos = [], [], [], [], []
+    n_u = n_d = n_p = 0
+    bitw = (np.uint32(1) << np.arange(b, dtype=np.uint32))
     for t in range(n_tiles):
         r0 = t * TILE_ROWS
         for s in range(n_stages):
@@ -259,47 +266,45 @@ def pack(p: Projection, b: int) -> np.ndarray:
                 hi = max(lo + 1, ((sl + 1) * 16) // b)
                 if (~P[:, lo:hi]).any():
                     live |= 1 << sl
-            rec[ri] = (n_u, n_d, live, 0)
-            sg = sign[r0:r0 + TILE_ROWS, s * STAGE_K:(s + 1) * STAGE_K]
-            base = ri * TILE_ROWS
-            meta_sgn[base:base + TILE_ROWS] = (sg.astype(np.uint64) * bitw).sum(axis=1)
-            w32 = (np.uint64(1) << np.arange(nb, dtype=np.uint64))
-            meta_pu[base:base + TILE_ROWS, 0] = (P.astype(np.uint64) * w32).sum(axis=1).astype(np.uint32)
-            meta_pu[base:base + TILE_ROWS, 1] = (Uf.astype(np.uint64) * w32).sum(axis=1).astype(np.uint32)
-            cu = Uf.sum(axis=1)
-            cd = D.sum(axis=1)
-            rel[base:base + TILE_ROWS, 0] = (np.cumsum(cu) - cu).astype(np.uint16)
-            rel[base:base + TILE_ROWS, 1] = (np.cumsum(cd) - cd).astype(np.uint16)
-            ustream.append(u[r0:r0 + TILE_ROWS, s * nb:(s + 1) * nb][Uf])        # row-major order
-            vb = vbf[r0:r0 + TILE_ROWS, s * STAGE_K:(s + 1) * STAGE_K].reshape(TILE_ROWS, nb, b)
-            dstream.append(vb[D].reshape(-1))
-            n_u += int(cu.sum())
-            n_d += int(cd.sum())
-    assert n_u == n_unified and n_d == n_dense
+            rec[ri] = (n_u, n_d, n_p, live)
+            pos_u = np.flatnonzero(Uf.reshape(-1)).astype(np.uint32)      # ascending pos
+            pos_d = np.flatnonzero(D.reshape(-1)).astype(np.uint16)
+            pos_p = np.flatnonzero(P.reshape(-1)).astype(np.uint16)
+            sg = sign[r0:r0 + TILE_ROWS, s * STAGE_K:(s + 1) * STAGE_K].reshape(TILE_ROWS * nb, b)
+            sbits = (sg.astype(np.uint32) * bitw).sum(axis=1).astype(np.uint32)
+            ulist_w0.append(pos_u | (sbits[pos_u] << np.uint32(16)))
+            ulist_u.append(u[r0:r0 + TILE_ROWS, s * nb:(s + 1) * nb].reshape(-1)[pos_u])
+            dpos.append(pos_d)
+            vb = vbf[r0:r0 + TILE_ROWS, s * STAGE_K:(s + 1) * STAGE_K].reshape(TILE_ROWS * nb, b)
+            dpay.append(vb[pos_d].reshape(-1))
+            ppos.append(pos_p)
+            n_u += pos_u.shape[0]
+            n_d += pos_d.shape[0]
+            n_p += pos_p.shape[0]
+    assert n_u == n_unified and n_d == n_dense and n_p == L["n_plist"]
+    rec[n_rec] = (n_u, n_d, n_p, 0)
 
     def put(off, arr):
         raw = np.ascontiguousarray(arr).view(np.uint8).reshape(-1)
         buf[off:off + raw.shape[0]] = raw
 
     put(L["off_rec"], rec)
-    meta = np.zeros((meta_sgn.shape[0], 2), dtype=np.uint64)
-    meta[:, 0] = meta_sgn
-    meta[:, 1] = meta_pu[:, 0].astype(np.uint64) | (meta_pu[:, 1].astype(np.uint64) << np.uint64(32))
-    put(L["off_meta"], meta)
-    put(L["off_rel"], rel)
     if n_unified:
-        put(L["off_ustream"], np.concatenate(ustream).astype(np.float32))
+        ul = np.zeros((n_unified, 2), dtype=np.uint32)
+        ul[:, 0] = np.concatenate(ulist_w0)
+        ul[:, 1] = np.concatenate(ulist_u).astype(np.float32).view(np.uint32)
+        put(L["off_ulist"], ul)
     if n_dense:
-        put(L["off_dstream"], np.concatenate(dstream).astype(np.uint16))
+        put(L["off_dpos"], np.concatenate(dpos).astype(np.uint16))
+        put(L["off_dpay"], np.concatenate(dpay).astype(np.uint16))
+    if L["n_plist"]:
+        put(L["off_ppos"], np.concatenate(ppos).astype(np.uint16))
     return buf
 
 
 def parse_header(buf: np.ndarray) -> dict:
-    names = ["magic", "version", "N", "K", "b", "n_pad", "n_tiles", "n_stages", "n_pruned",
-             "n_unified", "n_dense", "off_rec", "off_meta", "off_rel", "off_ustream",
-             "off_dstream", "total"]
-    vals = struct.unpack("<%dQ" % len(names), bytes(buf[:8 * len(names)]))
-    h = dict(zip(names, vals))
+    vals = struct.unpack("<%dQ" % len(HEADER_FIELDS), bytes(buf[:8 * len(HEADER_FIELDS)]))
+    h = dict(zip(HEADER_FIELDS, vals))
     assert h["magic"] == int.from_bytes(MAGIC, "little") and h["version"] == VERSION
     return h
 
@@ -314,38 +319,32 @@ def decode(buf: np.ndarray) -> np.ndarray:
     N, K, b = h["N"], h["K"], h["b"]
     nb = STAGE_K // b
     n_tiles, n_stages = h["n_tiles"], h["n_stages"]
-    n_rs = n_tiles * n_stages * TILE_ROWS
-    rec = buf[h["off_rec"]:h["off_rec"] + 16 * n_tiles * n_stages].view(np.uint32).reshape(-1, 4)
-    meta = buf[h["off_meta"]:h["off_meta"] + 16 * n_rs].view(np.uint64).reshape(-1, 2)
-    rel = buf[h["off_rel"]:h["off_rel"] + 4 * n_rs].view(np.uint16).reshape(-1, 2)
-    ustream = buf[h["off_ustream"]:h["off_ustream"] + 4 * h["n_unified"]].view(np.float32)
-    dstream = buf[h["off_dstream"]:h["off_dstream"] + 2 * b * h["n_dense"]].view(np.uint16)
-    u_bf = bf16_bits_to_f64(bf16_bits_rne(ustream)) if h["n_unified"] else np.zeros(0)
-    d_f = bf16_bits_to_f64(dstream) if h["n_dense"] else np.zeros(0)
-    What = np.zeros((h["n_pad"], K), dtype=np.float64)
+    n_rec = n_tiles * n_stages
+    rec = buf[h["off_rec"]:h["off_rec"] + 16 * (n_rec + 1)].view(np.uint32).reshape(-1, 4)
+    ulist = buf[h["off_ulist"]:h["off_ulist"] + 8 * h["n_unified"]].view(np.uint32).reshape(-1, 2)
+    dpos = buf[h["off_dpos"]:h["off_dpos"] + 2 * h["n_dense"]].view(np.uint16)
+    dpay = buf[h["off_dpay"]:h["off_dpay"] + 2 * b * h["n_dense"]].view(np.uint16)
+    ppos = buf[h["off_ppos"]:h["off_ppos"] + 2 * h["n_plist"]].view(np.uint16)
+    What = np.full((h["n_pad"], K), np.nan, dtype=np.float64)     # every slot must be listed once
     for t in range(n_tiles):
         for s in range(n_stages):
             ri = t * n_stages + s
-            ub, db = int(rec[ri, 0]), int(rec[ri, 1])
-            for r in range(TILE_ROWS):
-                rs = ri * TILE_ROWS + r
-                sgn = int(meta[rs, 0])
-                P = int(meta[rs, 1]) & 0xFFFFFFFF
-                Uf = int(meta[rs, 1]) >> 32
-                ui = ub + int(rel[rs, 0])
-                di = db + int(rel[rs, 1])
-                for i in range(nb):
-                    k0 = s * STAGE_K + i * b
-                    if (P >> i) & 1:
-                        continue
-                    if (Uf >> i) & 1:
-                        for l in range(b):
-                            neg = (sgn >> (i * b + l)) & 1
-                            What[t * TILE_ROWS + r, k0 + l] = -u_bf[ui] if neg else u_bf[ui]
-                        ui += 1
-                    else:
-                        What[t * TILE_ROWS + r, k0:k0 + b] = d_f[di * b:(di + 1) * b]
-                        di += 1
+            for e in range(int(rec[ri, 0]), int(rec[ri + 1, 0])):
+                w0 = int(ulist[e, 0])
+                pos, sbits = w0 & 0xFFFF, w0 >> 16
+                uval = float(bf16_bits_to_f64(bf16_bits_rne(ulist[e:e + 1, 1].view(np.float32)))[0])
+                r, i = divmod(pos, nb)
+                for l in range(b):
+                    What[t * TILE_ROWS + r, s * STAGE_K + i * b + l] = -uval if (sbits >> l) & 1 else uval
+            for e in range(int(rec[ri, 1]), int(rec[ri + 1, 1])):
+                r, i = divmod(int(dpos[e]), nb)
+                k0 = s * STAGE_K + i * b
+                What[t * TILE_ROWS + r, k0:k0 + b] = bf16_bits_to_f64(dpay[e * b:(e + 1) * b])
+            for e in range(int(rec[ri, 2]), int(rec[ri + 1, 2])):
+                r, i = divmod(int(ppos[e]), nb)
+                k0 = s * STAGE_K + i * b
+                What[t * TILE_ROWS + r, k0:k0 + b] = 0.0
+    assert not np.isnan(What).any()
     return What[:N]
 
 

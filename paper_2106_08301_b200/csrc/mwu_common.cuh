@@ -20,9 +20,12 @@ constexpr unsigned long long kMagic = 0x314B43415055574Dull;   // "MWUPACK1" lit
 inline size_t align_up(size_t x, size_t a = kAlign) { return (x + a - 1) / a * a; }
 
 struct PackedLayout {
-    int64_t n_pad, n_tiles, n_stages, n_unified, n_dense, n_pruned;
-    size_t off_rec, off_meta, off_rel, off_ustream, off_dstream, total;
+    int64_t n_pad, n_tiles, n_stages, n_unified, n_dense, n_pruned, n_plist;
+    size_t off_rec, off_ulist, off_dpos, off_dpay, off_ppos, total;
 };
+
+// one entry of the record table: where the record starts in each class list
+struct PackedRec { unsigned ubase, dbase, pbase, live; };
 
 inline PackedLayout packed_layout(const mwu_proj_desc *d) {
     PackedLayout L;
@@ -33,13 +36,13 @@ inline PackedLayout packed_layout(const mwu_proj_desc *d) {
     L.n_pruned = d->k_prune;
     L.n_unified = d->k_unify - d->k_prune;
     L.n_dense = mb - d->k_unify;
-    const size_t n_rs = (size_t)L.n_tiles * L.n_stages * kTileRows;
+    L.n_plist = L.n_pruned + (L.n_pad - d->rows) * (d->cols / d->block);
     L.off_rec = kHeaderBytes;
-    L.off_meta = align_up(L.off_rec + 16 * (size_t)L.n_tiles * L.n_stages);
-    L.off_rel = align_up(L.off_meta + 16 * n_rs);
-    L.off_ustream = align_up(L.off_rel + 4 * n_rs);
-    L.off_dstream = align_up(L.off_ustream + 4 * (size_t)L.n_unified);
-    L.total = align_up(L.off_dstream + 2 * (size_t)d->block * L.n_dense);
+    L.off_ulist = align_up(L.off_rec + 16 * ((size_t)L.n_tiles * L.n_stages + 1));
+    L.off_dpos = align_up(L.off_ulist + 8 * (size_t)L.n_unified);
+    L.off_dpay = align_up(L.off_dpos + 2 * (size_t)L.n_dense);
+    L.off_ppos = align_up(L.off_dpay + 2 * (size_t)d->block * L.n_dense);
+    L.total = align_up(L.off_ppos + 2 * (size_t)L.n_plist);
     return L;
 }
 

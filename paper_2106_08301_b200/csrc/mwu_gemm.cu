@@ -1,7 +1,683 @@
-// placeholder until the tensor-core kernel lands
+// mwu_gemm / mwu_conv_implicit: Y = X . W_hat^T on the packed weights (Section 3.2).
+//
+// One persistent CTA per SM, warp-specialised:
+//   warp 0        producer of the activation tile (A operand, 128 rows x 64 k, bf16): one thread
+//                 issues a TMA load per stage (GEMM); for the convolution four extra warps gather
+//                 the im2col rows with plain loads instead.
+//   warp 1        allocates tensor memory and issues tcgen05.mma (one thread); fp32 accumulators
+//                 live in TMEM, two buffers so that the epilogue of tile i overlaps tile i+1.
+//   warps 2-5     epilogue: tcgen05.ld -> bf16/fp32 -> global.
+//   warps 6-13    decode the weight tile (B operand) from the packed class lists into the
+//                 128-byte-swizzled K-major layout the MMA reads: pruned blocks -> zeros,
+//                 unified blocks -> sign . bf16(u), dense blocks -> stored bf16 values.
+// A 64-wide k stage whose blocks are pruned in every row of the weight tile is skipped by all
+// roles (no load, no decode, no MMA); inside a live stage the MMA skips dead 16-wide slices.
+// Every wait on an mbarrier is bounded; when one runs out the kernel raises MWU_DEV_TIMEOUT,
+// drains what it issued, frees its tensor memory and returns.
+#include <cuda.h>
+
 #include "mwu_common.cuh"
-extern "C" int mwu_gemm(const mwu_proj_desc *, const void *, const void *, int64_t, int64_t, void *,
-                        int64_t, int32_t, uint32_t *, void *) { return MWU_ERR_CUDA; }
-extern "C" int mwu_conv_implicit(const mwu_proj_desc *, const void *, const void *, int32_t, int32_t,
-                                 int32_t, int32_t, int32_t, int32_t, int32_t, int32_t, void *, int32_t,
-                                 uint32_t *, void *) { return MWU_ERR_CUDA; }
+
+namespace mwu {
+namespace gemm {
+
+constexpr int BM = 128;                 // rows of X per tile
+constexpr int BK = kStageK;             // 64
+constexpr int STAGES = 4;
+constexpr int A_BYTES = BM * BK * 2;    // 16 KiB
+constexpr int REC_BYTES = kTileRows * BK * 2;
+constexpr int NDEC_WARPS = 8;
+constexpr int NGATHER_WARPS = 4;
+constexpr int THREADS_GEMM = 32 * (6 + NDEC_WARPS);
+constexpr int THREADS_CONV = THREADS_GEMM + 32 * NGATHER_WARPS;
+constexpr long long WAIT_LIMIT_CYCLES = 4000000000ll;   // about two seconds
+
+struct Params {
+    const unsigned char *packed;
+    size_t off_rec, off_ulist, off_dpos, off_dpay, off_ppos;
+    long long n_rec_tiles;              // 128-row tiles of W
+    long long n_stages;                 // K / 64
+    long long M, N, K;
+    void *Y;
+    long long ldy;
+    int y_fp32;
+    unsigned *dev_status;
+    // convolution only
+    const __nv_bfloat16 *X;
+    int C, H, W, KH, KW, stride, pad, OH, OW;
+};
+
+// ------------------------------------------------------------------------------------------
+// PTX wrappers
+// ------------------------------------------------------------------------------------------
+__device__ __forceinline__ unsigned smem_u32(const void *p) {
+    return (unsigned)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ void mbar_init(unsigned bar, unsigned count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(unsigned bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(unsigned bar, unsigned bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(unsigned bar, unsigned parity) {
+    unsigned ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// bounded wait: false when aborted or out of time (then *abort is set)
+__device__ __forceinline__ bool mbar_wait(unsigned bar, unsigned parity, volatile int *abort) {
+#pragma unroll 1
+    for (int i = 0; i < 128; ++i)
+        if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+#pragma unroll 1
+    while (true) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (*abort) return false;
+        if (clock64() - t0 > WAIT_LIMIT_CYCLES) { *abort = 1; return false; }
+    }
+}
+__device__ __forceinline__ void fence_proxy_async() {
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tma_load_2d(unsigned dst, const CUtensorMap *map, unsigned bar, int x, int y) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void tmem_alloc(unsigned dst_smem, unsigned ncols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(unsigned taddr, unsigned ncols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void umma_bf16(unsigned d_tmem, unsigned long long adesc, unsigned long long bdesc,
+                                          unsigned idesc, unsigned accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit(unsigned bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(unsigned taddr, unsigned (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr) : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// K-major operand, 128-byte swizzle: rows of 128 bytes, 8-row groups 1024 bytes apart
+__device__ __forceinline__ unsigned long long make_desc(unsigned smem_addr) {
+    unsigned long long d = 0;
+    d |= (unsigned long long)((smem_addr & 0x3FFFFu) >> 4);
+    d |= (unsigned long long)1 << 16;                    // leading byte offset (unused for this layout)
+    d |= (unsigned long long)(1024 >> 4) << 32;          // stride between 8-row groups
+    d |= (unsigned long long)1 << 46;                    // descriptor version of this architecture
+    d |= (unsigned long long)2 << 61;                    // 128-byte swizzle
+    return d;
+}
+// bf16 x bf16 -> fp32, both operands K-major, M = 128
+__device__ __forceinline__ unsigned make_idesc(int n) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((unsigned)(n >> 3) << 17) | ((unsigned)(BM >> 4) << 24);
+}
+
+// byte offset of 16-byte chunk c of row r inside a swizzled K-major tile
+__device__ __forceinline__ unsigned swz(unsigned r, unsigned c) {
+    return (r >> 3) * 1024u + (r & 7u) * 128u + ((c ^ (r & 7u)) << 4);
+}
+
+// ------------------------------------------------------------------------------------------
+// decode of one record's class lists into its 128 x 64 tile
+// ------------------------------------------------------------------------------------------
+__device__ __forceinline__ unsigned sign_word(unsigned u2, unsigned sbits, int w) {
+    const unsigned t = (sbits >> (2 * w)) & 3u;          // signs of weights 2w, 2w+1
+    return ((t * 0x40008000u) & 0x80008000u) ^ u2;        // bit0 -> bit 15, bit1 -> bit 31
+}
+
+template <int BW>
+__device__ __forceinline__ void decode_record(unsigned char *tile, const PackedRec r0, const PackedRec r1,
+                                              const Params &p, int tid, int nthr) {
+    constexpr int NBK = BK / BW;                          // blocks per row
+    const uint2 *ulist = reinterpret_cast<const uint2 *>(p.packed + p.off_ulist);
+    const unsigned short *dpos = reinterpret_cast<const unsigned short *>(p.packed + p.off_dpos);
+    const unsigned char *dpay = p.packed + p.off_dpay;
+    const unsigned short *ppos = reinterpret_cast<const unsigned short *>(p.packed + p.off_ppos);
+    // pruned blocks: zeros
+    for (unsigned e = r0.pbase + tid; e < r1.pbase; e += nthr) {
+        const unsigned pos = __ldg(ppos + e) & (kTileRows * NBK - 1);
+        const unsigned r = pos / NBK, i = pos % NBK;
+        if (BW == 16) {
+            const unsigned a = swz(r, 2 * i);
+            *reinterpret_cast<uint4 *>(tile + a) = make_uint4(0, 0, 0, 0);
+            *reinterpret_cast<uint4 *>(tile + (a ^ 16u)) = make_uint4(0, 0, 0, 0);
+        } else if (BW == 8) {
+            *reinterpret_cast<uint4 *>(tile + swz(r, i)) = make_uint4(0, 0, 0, 0);
+        } else if (BW == 4) {
+            *reinterpret_cast<uint2 *>(tile + swz(r, i >> 1) + (i & 1) * 8) = make_uint2(0, 0);
+        } else {
+            *reinterpret_cast<unsigned *>(tile + swz(r, i >> 2) + (i & 3) * 4) = 0u;
+        }
+    }
+    // dense blocks: copy the stored bf16 values
+    for (unsigned e = r0.dbase + tid; e < r1.dbase; e += nthr) {
+        const unsigned pos = __ldg(dpos + e) & (kTileRows * NBK - 1);
+        const unsigned r = pos / NBK, i = pos % NBK;
+        const unsigned char *src = dpay + (size_t)e * (2 * BW);
+        if (BW == 16) {
+            const uint4 v0 = __ldg(reinterpret_cast<const uint4 *>(src));
+            const uint4 v1 = __ldg(reinterpret_cast<const uint4 *>(src + 16));
+            const unsigned a = swz(r, 2 * i);
+            *reinterpret_cast<uint4 *>(tile + a) = v0;
+            *reinterpret_cast<uint4 *>(tile + (a ^ 16u)) = v1;
+        } else if (BW == 8) {
+            *reinterpret_cast<uint4 *>(tile + swz(r, i)) = __ldg(reinterpret_cast<const uint4 *>(src));
+        } else if (BW == 4) {
+            *reinterpret_cast<uint2 *>(tile + swz(r, i >> 1) + (i & 1) * 8) =
+                __ldg(reinterpret_cast<const uint2 *>(src));
+        } else {
+            *reinterpret_cast<unsigned *>(tile + swz(r, i >> 2) + (i & 3) * 4) =
+                __ldg(reinterpret_cast<const unsigned *>(src));
+        }
+    }
+    // unified blocks: sign . bf16(u)
+    for (unsigned e = r0.ubase + tid; e < r1.ubase; e += nthr) {
+        const uint2 ent = __ldg(ulist + e);
+        const unsigned pos = ent.x & (kTileRows * NBK - 1);
+        const unsigned sbits = ent.x >> 16;
+        const unsigned r = pos / NBK, i = pos % NBK;
+        const __nv_bfloat16 ub = __float2bfloat16_rn(__uint_as_float(ent.y));
+        const unsigned u1 = (unsigned)__bfloat16_as_ushort(ub);
+        const unsigned u2 = u1 | (u1 << 16);
+        if (BW == 16) {
+            const unsigned a = swz(r, 2 * i);
+            *reinterpret_cast<uint4 *>(tile + a) = make_uint4(sign_word(u2, sbits, 0), sign_word(u2, sbits, 1),
+                                                              sign_word(u2, sbits, 2), sign_word(u2, sbits, 3));
+            *reinterpret_cast<uint4 *>(tile + (a ^ 16u)) = make_uint4(sign_word(u2, sbits, 4), sign_word(u2, sbits, 5),
+                                                                      sign_word(u2, sbits, 6), sign_word(u2, sbits, 7));
+        } else if (BW == 8) {
+            *reinterpret_cast<uint4 *>(tile + swz(r, i)) = make_uint4(sign_word(u2, sbits, 0), sign_word(u2, sbits, 1),
+                                                                      sign_word(u2, sbits, 2), sign_word(u2, sbits, 3));
+        } else if (BW == 4) {
+            *reinterpret_cast<uint2 *>(tile + swz(r, i >> 1) + (i & 1) * 8) =
+                make_uint2(sign_word(u2, sbits, 0), sign_word(u2, sbits, 1));
+        } else {
+            *reinterpret_cast<unsigned *>(tile + swz(r, i >> 2) + (i & 3) * 4) = sign_word(u2, sbits, 0);
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// the kernel
+// ------------------------------------------------------------------------------------------
+struct Smem {
+    unsigned long long full_a[STAGES], full_b[STAGES], empty[STAGES], tfull[2], tempty[2], drain;
+    unsigned tmem_base;
+    int abort;
+};
+
+template <int MODE, int NREC, int BW>
+__global__ void __launch_bounds__(MODE ? THREADS_CONV : THREADS_GEMM, 1)
+mwu_gemm_kernel(const __grid_constant__ CUtensorMap tmap, const Params p) {
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char *base = reinterpret_cast<unsigned char *>(
+        (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    unsigned char *sA = base;
+    unsigned char *sB = base + STAGES * A_BYTES;
+    constexpr int B_BYTES = NREC * REC_BYTES;
+    Smem *sm = reinterpret_cast<Smem *>(sB + STAGES * B_BYTES);
+    int2 *ktab = reinterpret_cast<int2 *>(reinterpret_cast<unsigned char *>(sm) + 256);   // conv only
+    volatile int *abort = &sm->abort;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const PackedRec *recs = reinterpret_cast<const PackedRec *>(p.packed + p.off_rec);
+    const long long m_tiles = (p.M + BM - 1) / BM;
+    const long long n_tiles = (p.n_rec_tiles + NREC - 1) / NREC;
+    const long long total_tiles = m_tiles * n_tiles;
+    const int n_stages = (int)p.n_stages;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(smem_u32(&sm->full_a[s]), MODE ? NGATHER_WARPS : 1);
+            mbar_init(smem_u32(&sm->full_b[s]), NDEC_WARPS);
+            mbar_init(smem_u32(&sm->empty[s]), 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(smem_u32(&sm->tfull[b]), 1);
+            mbar_init(smem_u32(&sm->tempty[b]), 4);
+        }
+        mbar_init(smem_u32(&sm->drain), 1);
+        sm->abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (MODE) {
+        for (int k = threadIdx.x; k < (int)p.K; k += blockDim.x) {
+            const int c = k / (p.KH * p.KW), rem = k % (p.KH * p.KW);
+            const int di = rem / p.KW - p.pad, dj = rem % p.KW - p.pad;
+            ktab[k] = make_int2(c * p.H * p.W + di * p.W + dj, (di & 0xffff) | (dj << 16));
+        }
+    }
+    if (warp == 1) tmem_alloc(smem_u32(&sm->tmem_base), 512);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const unsigned tmem_base = *reinterpret_cast<volatile unsigned *>(&sm->tmem_base);
+
+    // live mask of stage ks for weight tile nt (OR over its records)
+    auto live_of = [&](long long nt, int ks) -> unsigned {
+        unsigned live = 0;
+#pragma unroll
+        for (int q = 0; q < NREC; ++q) {
+            const long long rt = nt * NREC + q;
+            if (rt < p.n_rec_tiles) live |= __ldg(&recs[rt * n_stages + ks].live);
+        }
+        return live;
+    };
+
+    if (warp == 0 && MODE == 0) {
+        // ---------------- TMA producer ----------------
+        if (lane == 0) {
+            int stage = 0;
+            unsigned phase = 0;
+            bool ok = true;
+            for (long long t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+                const long long mt = t % m_tiles, nt = t / m_tiles;
+                for (int ks = 0; ks < n_stages; ++ks) {
+                    if (!live_of(nt, ks)) continue;
+                    if (!mbar_wait(smem_u32(&sm->empty[stage]), phase ^ 1u, abort)) { ok = false; break; }
+                    const unsigned bar = smem_u32(&sm->full_a[stage]);
+                    mbar_expect_tx(bar, A_BYTES);
+                    tma_load_2d(smem_u32(sA + stage * A_BYTES), &tmap, bar, ks * BK, (int)(mt * BM));
+                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer ----------------
+        if (lane == 0) {
+            int stage = 0;
+            unsigned phase = 0;
+            unsigned acc_phase[2] = {0, 0};
+            long long it = 0;
+            bool ok = true;
+            bool issued_any = false;
+            for (long long t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++it) {
+                const long long nt = t / m_tiles;
+                const int buf = (int)(it & 1);
+                const int nrec_here = (int)((p.n_rec_tiles - nt * NREC) < NREC ? (p.n_rec_tiles - nt * NREC) : NREC);
+                const unsigned idesc = make_idesc(nrec_here * kTileRows);
+                if (!mbar_wait(smem_u32(&sm->tempty[buf]), acc_phase[buf] ^ 1u, abort)) { ok = false; break; }
+                acc_phase[buf] ^= 1u;
+                tc_fence_after();
+                const unsigned d_tmem = tmem_base + (unsigned)(buf * 256);
+                bool first = true;
+                for (int ks = 0; ks < n_stages; ++ks) {
+                    const unsigned live = live_of(nt, ks);
+                    if (!live) continue;
+                    if (!mbar_wait(smem_u32(&sm->full_a[stage]), phase, abort)) { ok = false; break; }
+                    if (!mbar_wait(smem_u32(&sm->full_b[stage]), phase, abort)) { ok = false; break; }
+                    tc_fence_after();
+                    const unsigned long long adesc = make_desc(smem_u32(sA + stage * A_BYTES));
+                    const unsigned long long bdesc = make_desc(smem_u32(sB + stage * B_BYTES));
+#pragma unroll
+                    for (int k4 = 0; k4 < 4; ++k4) {
+                        if ((live >> k4) & 1u) {
+                            umma_bf16(d_tmem, adesc + (unsigned long long)(k4 * 2), bdesc + (unsigned long long)(k4 * 2),
+                                      idesc, first ? 0u : 1u);
+                            first = false;
+                            issued_any = true;
+                        }
+                    }
+                    umma_commit(smem_u32(&sm->empty[stage]));
+                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                }
+                if (!ok) break;
+                if (!first) umma_commit(smem_u32(&sm->tfull[buf]));
+                else mbar_arrive(smem_u32(&sm->tfull[buf]));
+            }
+            // everything this thread issued must have retired before tensor memory is freed
+            if (issued_any) {
+                umma_commit(smem_u32(&sm->drain));
+                mbar_wait(smem_u32(&sm->drain), 0, abort);
+            }
+        }
+    } else if (warp >= 2 && warp < 6) {
+        // ---------------- epilogue ----------------
+        const int quarter = warp & 3;                       // TMEM lanes this warp may read
+        unsigned acc_phase[2] = {0, 0};
+        long long it = 0;
+        bool ok = true;
+        for (long long t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++it) {
+            const long long mt = t % m_tiles, nt = t / m_tiles;
+            const int buf = (int)(it & 1);
+            unsigned any = 0;
+            for (int ks = lane; ks < n_stages; ks += 32) any |= live_of(nt, ks);
+            any = __reduce_or_sync(0xffffffffu, any);
+            if (!mbar_wait(smem_u32(&sm->tfull[buf]), acc_phase[buf], abort)) { ok = false; }
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            acc_phase[buf] ^= 1u;
+            tc_fence_after();
+            const long long m = mt * BM + quarter * 32 + lane;
+            const int ncols_tile = (int)(((p.n_rec_tiles - nt * NREC) < NREC ? (p.n_rec_tiles - nt * NREC) : NREC) * kTileRows);
+            for (int c0 = 0; c0 < ncols_tile; c0 += 32) {
+                unsigned v[32];
+                if (any) {
+                    tmem_ld32(tmem_base + ((unsigned)(quarter * 32) << 16) + (unsigned)(buf * 256 + c0), v);
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) v[j] = 0u;
+                }
+                const long long n0 = nt * (NREC * kTileRows) + c0;
+                if (MODE == 0) {
+                    if (m < p.M) {
+                        if (p.y_fp32) {
+                            float *dst = reinterpret_cast<float *>(p.Y) + m * p.ldy + n0;
+                            if (n0 + 32 <= p.N) {
+#pragma unroll
+                                for (int j = 0; j < 32; j += 4)
+                                    *reinterpret_cast<uint4 *>(dst + j) = make_uint4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+                            } else {
+                                for (int j = 0; j < 32; ++j)
+                                    if (n0 + j < p.N) dst[j] = __uint_as_float(v[j]);
+                            }
+                        } else {
+                            __nv_bfloat16 *dst = reinterpret_cast<__nv_bfloat16 *>(p.Y) + m * p.ldy + n0;
+                            if (n0 + 32 <= p.N) {
+#pragma unroll
+                                for (int j = 0; j < 32; j += 8) {
+                                    uint4 o;
+                                    __nv_bfloat162 h;
+                                    h = __floats2bfloat162_rn(__uint_as_float(v[j]), __uint_as_float(v[j + 1]));
+                                    o.x = *reinterpret_cast<unsigned *>(&h);
+                                    h = __floats2bfloat162_rn(__uint_as_float(v[j + 2]), __uint_as_float(v[j + 3]));
+                                    o.y = *reinterpret_cast<unsigned *>(&h);
+                                    h = __floats2bfloat162_rn(__uint_as_float(v[j + 4]), __uint_as_float(v[j + 5]));
+                                    o.z = *reinterpret_cast<unsigned *>(&h);
+                                    h = __floats2bfloat162_rn(__uint_as_float(v[j + 6]), __uint_as_float(v[j + 7]));
+                                    o.w = *reinterpret_cast<unsigned *>(&h);
+                                    *reinterpret_cast<uint4 *>(dst + j) = o;
+                                }
+                            } else {
+                                for (int j = 0; j < 32; ++j)
+                                    if (n0 + j < p.N) dst[j] = __float2bfloat16_rn(__uint_as_float(v[j]));
+                            }
+                        }
+                    }
+                } else {
+                    // NCHW output: row m = (img, oh, ow); consecutive lanes write consecutive pixels
+                    if (m < p.M) {
+                        const long long hw = (long long)p.OH * p.OW;
+                        const long long img = m / hw, pix = m % hw;
+                        for (int j = 0; j < 32; ++j) {
+                            const long long o = n0 + j;
+                            if (o < p.N) {
+                                const long long idx = (img * p.N + o) * hw + pix;
+                                if (p.y_fp32) reinterpret_cast<float *>(p.Y)[idx] = __uint_as_float(v[j]);
+                                else reinterpret_cast<__nv_bfloat16 *>(p.Y)[idx] = __float2bfloat16_rn(__uint_as_float(v[j]));
+                            }
+                        }
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&sm->tempty[buf]));
+        }
+    } else if (warp >= 6 && warp < 6 + NDEC_WARPS) {
+        // ---------------- weight decode ----------------
+        const int tid = threadIdx.x - 6 * 32;
+        constexpr int NTHR = NDEC_WARPS * 32;
+        int stage = 0;
+        unsigned phase = 0;
+        bool ok = true;
+        for (long long t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+            const long long nt = t / m_tiles;
+            for (int ks = 0; ks < n_stages; ++ks) {
+                if (!live_of(nt, ks)) continue;
+                if (!mbar_wait(smem_u32(&sm->empty[stage]), phase ^ 1u, abort)) ok = false;
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+#pragma unroll
+                for (int q = 0; q < NREC; ++q) {
+                    const long long rt = nt * NREC + q;
+                    if (rt < p.n_rec_tiles) {
+                        const uint4 a = __ldg(reinterpret_cast<const uint4 *>(&recs[rt * n_stages + ks]));
+                        const uint4 b = __ldg(reinterpret_cast<const uint4 *>(&recs[rt * n_stages + ks + 1]));
+                        PackedRec r0, r1;
+                        r0.ubase = a.x; r0.dbase = a.y; r0.pbase = a.z; r0.live = a.w;
+                        r1.ubase = b.x; r1.dbase = b.y; r1.pbase = b.z; r1.live = b.w;
+                        decode_record<BW>(sB + stage * B_BYTES + q * REC_BYTES, r0, r1, p, tid, NTHR);
+                    }
+                }
+                fence_proxy_async();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&sm->full_b[stage]));
+                if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+            }
+        }
+    } else if (MODE == 1 && warp >= 6 + NDEC_WARPS) {
+        // ---------------- im2col gather of the A tile (convolution) ----------------
+        const int r = threadIdx.x - (6 + NDEC_WARPS) * 32;      // row of the tile, 0..127
+        const unsigned short *X = reinterpret_cast<const unsigned short *>(p.X);
+        int stage = 0;
+        unsigned phase = 0;
+        bool ok = true;
+        const long long hw = (long long)p.OH * p.OW;
+        for (long long t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+            const long long mt = t % m_tiles, nt = t / m_tiles;
+            const long long m = mt * BM + r;
+            const bool row_ok = m < p.M;
+            const long long img = row_ok ? m / hw : 0, pix = row_ok ? m % hw : 0;
+            const int ih0 = (int)(pix / p.OW) * p.stride, iw0 = (int)(pix % p.OW) * p.stride;
+            const long long xbase = img * (long long)p.C * p.H * p.W + (long long)ih0 * p.W + iw0;
+            for (int ks = 0; ks < n_stages; ++ks) {
+                if (!live_of(nt, ks)) continue;
+                if (!mbar_wait(smem_u32(&sm->empty[stage]), phase ^ 1u, abort)) ok = false;
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                unsigned char *tile = sA + stage * A_BYTES;
+#pragma unroll 1
+                for (int c = 0; c < 8; ++c) {
+                    unsigned w[4];
+#pragma unroll
+                    for (int h = 0; h < 4; ++h) {
+                        unsigned pair = 0;
+#pragma unroll
+                        for (int e = 0; e < 2; ++e) {
+                            const int2 tb = ktab[ks * BK + c * 8 + h * 2 + e];
+                            const int ih = ih0 + (int)(short)(tb.y & 0xffff), iw = iw0 + (tb.y >> 16);
+                            unsigned val = 0;
+                            if (row_ok && (unsigned)ih < (unsigned)p.H && (unsigned)iw < (unsigned)p.W)
+                                val = __ldg(X + xbase + tb.x);
+                            pair |= val << (16 * e);
+                        }
+                        w[h] = pair;
+                    }
+                    *reinterpret_cast<uint4 *>(tile + swz((unsigned)r, (unsigned)c)) = make_uint4(w[0], w[1], w[2], w[3]);
+                }
+                fence_proxy_async();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&sm->full_a[stage]));
+                if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+            }
+        }
+    }
+
+    // teardown
+    if (*abort && threadIdx.x == 0) atomicOr(p.dev_status, (unsigned)MWU_DEV_TIMEOUT);
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, 512);
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// host
+// ------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn get_encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void *ptr = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) != cudaSuccess ||
+            qres != cudaDriverEntryPointSuccess)
+            return nullptr;
+        fn = reinterpret_cast<EncodeTiledFn>(ptr);
+    }
+    return fn;
+}
+
+static size_t smem_bytes(int nrec, long long conv_k) {
+    return 1024 + (size_t)STAGES * (A_BYTES + nrec * REC_BYTES) + 256 + (size_t)conv_k * sizeof(int2);
+}
+
+template <int MODE, int NREC, int BW>
+static cudaError_t launch(const CUtensorMap &tmap, const Params &p, int grid, size_t smem, cudaStream_t st) {
+    auto kern = mwu_gemm_kernel<MODE, NREC, BW>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    kern<<<grid, MODE ? THREADS_CONV : THREADS_GEMM, smem, st>>>(tmap, p);
+    return cudaGetLastError();
+}
+
+template <int MODE, int NREC>
+static cudaError_t launch_bw(int bw, const CUtensorMap &tmap, const Params &p, int grid, size_t smem, cudaStream_t st) {
+    switch (bw) {
+        case 2: return launch<MODE, NREC, 2>(tmap, p, grid, smem, st);
+        case 4: return launch<MODE, NREC, 4>(tmap, p, grid, smem, st);
+        case 8: return launch<MODE, NREC, 8>(tmap, p, grid, smem, st);
+        default: return launch<MODE, NREC, 16>(tmap, p, grid, smem, st);
+    }
+}
+
+static void fill_common(Params &p, const mwu_proj_desc *desc, const void *packed, void *Y, int y_dtype,
+                        uint32_t *dev_status) {
+    const PackedLayout L = packed_layout(desc);
+    p.packed = (const unsigned char *)packed;
+    p.off_rec = L.off_rec; p.off_ulist = L.off_ulist; p.off_dpos = L.off_dpos;
+    p.off_dpay = L.off_dpay; p.off_ppos = L.off_ppos;
+    p.n_rec_tiles = L.n_tiles;
+    p.n_stages = L.n_stages;
+    p.N = desc->rows;
+    p.K = desc->cols;
+    p.Y = Y;
+    p.y_fp32 = y_dtype;
+    p.dev_status = dev_status;
+}
+
+}  // namespace gemm
+}  // namespace mwu
+
+extern "C" int mwu_gemm(const mwu_proj_desc *desc, const void *packed, const void *X, int64_t M,
+                        int64_t ldx, void *Y, int64_t ldy, int32_t y_dtype, uint32_t *dev_status,
+                        void *cuda_stream) {
+    using namespace mwu;
+    using namespace mwu::gemm;
+    int rc = validate_desc(desc, true);
+    if (rc != MWU_OK) return rc;
+    if (!packed || !X || !Y || !dev_status || M < 0) return MWU_ERR_INVALID_ARG;
+    if (y_dtype != 0 && y_dtype != 1) return MWU_ERR_INVALID_ARG;
+    if (ldx < desc->cols || ldy < desc->rows) return MWU_ERR_SHAPE;
+    if (M >= (int64_t(1) << 31) || ldx >= (int64_t(1) << 31)) return MWU_ERR_SHAPE;
+    if (!aligned_to(packed, 256) || !aligned_to(X, 16) || !aligned_to(Y, 16) || ldx % 8 != 0 ||
+        ldy % (y_dtype ? 4 : 8) != 0 || !aligned_to(dev_status, 4))
+        return MWU_ERR_ALIGNMENT;
+    if (M == 0) return MWU_OK;
+    int sm_count = 0;
+    rc = check_device(&sm_count);
+    if (rc != MWU_OK) return rc;
+    EncodeTiledFn encode = get_encode_fn();
+    if (!encode) return MWU_ERR_CUDA;
+
+    CUtensorMap tmap;
+    const cuuint64_t gdim[2] = {(cuuint64_t)desc->cols, (cuuint64_t)M};
+    const cuuint64_t gstride[1] = {(cuuint64_t)ldx * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)BM};
+    const cuuint32_t estr[2] = {1, 1};
+    if (encode(&tmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(X), gdim, gstride, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return MWU_ERR_CUDA;
+
+    Params p = {};
+    fill_common(p, desc, packed, Y, y_dtype, dev_status);
+    p.M = M;
+    p.ldy = ldy;
+    const int nrec = p.n_rec_tiles >= 2 ? 2 : 1;
+    const long long tiles = ((M + BM - 1) / BM) * ((p.n_rec_tiles + nrec - 1) / nrec);
+    const int grid = (int)(tiles < sm_count ? tiles : sm_count);
+    const size_t smem = smem_bytes(nrec, 0);
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    cudaError_t e = (nrec == 2) ? launch_bw<0, 2>(desc->block, tmap, p, grid, smem, st)
+                                : launch_bw<0, 1>(desc->block, tmap, p, grid, smem, st);
+    return e == cudaSuccess ? MWU_OK : MWU_ERR_CUDA;
+}
+
+extern "C" int mwu_conv_implicit(const mwu_proj_desc *desc, const void *packed, const void *X_nchw,
+                                 int32_t n, int32_t c, int32_t h, int32_t w, int32_t kh, int32_t kw,
+                                 int32_t stride, int32_t pad, void *Y_nchw, int32_t y_dtype,
+                                 uint32_t *dev_status, void *cuda_stream) {
+    using namespace mwu;
+    using namespace mwu::gemm;
+    int rc = validate_desc(desc, true);
+    if (rc != MWU_OK) return rc;
+    if (!packed || !X_nchw || !Y_nchw || !dev_status) return MWU_ERR_INVALID_ARG;
+    if (y_dtype != 0 && y_dtype != 1) return MWU_ERR_INVALID_ARG;
+    if (n <= 0 || c <= 0 || h <= 0 || w <= 0 || kh <= 0 || kw <= 0 || stride <= 0 || pad < 0)
+        return MWU_ERR_INVALID_ARG;
+    if ((int64_t)c * kh * kw != desc->cols) return MWU_ERR_SHAPE;
+    if (h + 2 * pad < kh || w + 2 * pad < kw || pad > 32767 || kh > 32767 || kw > 32767) return MWU_ERR_SHAPE;
+    if ((int64_t)c * h * w >= (int64_t(1) << 31)) return MWU_ERR_SHAPE;
+    if (!aligned_to(packed, 256) || !aligned_to(X_nchw, 16) || !aligned_to(Y_nchw, 16) ||
+        !aligned_to(dev_status, 4))
+        return MWU_ERR_ALIGNMENT;
+    int sm_count = 0;
+    rc = check_device(&sm_count);
+    if (rc != MWU_OK) return rc;
+
+    Params p = {};
+    fill_common(p, desc, packed, Y_nchw, y_dtype, dev_status);
+    p.X = (const __nv_bfloat16 *)X_nchw;
+    p.C = c; p.H = h; p.W = w; p.KH = kh; p.KW = kw; p.stride = stride; p.pad = pad;
+    p.OH = (h + 2 * pad - kh) / stride + 1;
+    p.OW = (w + 2 * pad - kw) / stride + 1;
+    p.M = (long long)n * p.OH * p.OW;
+    p.ldy = 0;
+    const int nrec = p.n_rec_tiles >= 2 ? 2 : 1;
+    const size_t smem = smem_bytes(nrec, desc->cols);
+    if (smem > 227 * 1024) return MWU_ERR_SHAPE;
+    const long long tiles = ((p.M + BM - 1) / BM) * ((p.n_rec_tiles + nrec - 1) / nrec);
+    const int grid = (int)(tiles < sm_count ? tiles : sm_count);
+    CUtensorMap tmap;
+    memset(&tmap, 0, sizeof(tmap));
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    cudaError_t e = (nrec == 2) ? launch_bw<1, 2>(desc->block, tmap, p, grid, smem, st)
+                                : launch_bw<1, 1>(desc->block, tmap, p, grid, smem, st);
+    return e == cudaSuccess ? MWU_OK : MWU_ERR_CUDA;
+}

@@ -1,11 +1,13 @@
 // mwu_pack: serialise a projection into the packed storage form (Section 3.1 / Table 1: one
-// magnitude per unified block, nothing for a pruned block, one sign bit per weight).
+// magnitude per unified block, nothing but its position for a pruned block, one sign bit per
+// weight of a unified block, bf16 values for the rest), arranged per GEMM tile.
 //
-//   count_kernel  one CTA per record (128 rows x 64 columns): per-row class bits, sign word,
-//                 counts of unified / dense blocks and their exclusive scan over the rows.
+//   count_kernel  one CTA per record (128 rows x 64 columns): number of unified / dense / pruned
+//                 blocks and the record's live-slice mask.
 //   scan_kernel   one CTA: exclusive scan of the per-record counts over all records, header.
-//   fill_kernel   one CTA per record: writes the unified values and the bf16 payload of the
-//                 dense blocks; each warp reads one row segment (256 contiguous bytes) at a time.
+//   fill_kernel   one CTA per record: per-row class masks, scan over the rows, then the three
+//                 class lists; the dense payload is written warp-per-row so that every row
+//                 segment (256 contiguous bytes of W) is read with one coalesced request.
 #include "mwu_common.cuh"
 
 namespace mwu {
@@ -25,161 +27,210 @@ struct Params {
     PackedLayout L;
 };
 
-struct Rec { unsigned ubase, dbase, live, zero; };
-struct Meta { unsigned long long sgn; unsigned P, U; };
+// class masks of row r of a record; padding rows are all-pruned
+__device__ __forceinline__ void row_masks(const Params &p, long long tile, long long stage, int r,
+                                          unsigned *P, unsigned *U, unsigned long long *sgn) {
+    const int nb = kStageK / p.b;
+    const unsigned mask = (nb >= 32) ? 0xffffffffu : ((1u << nb) - 1u);
+    const long long n = tile * kTileRows + r;
+    *P = mask;
+    *U = 0;
+    *sgn = 0;
+    if (n < p.rows) {
+        const long long j0 = n * (p.cols / p.b) + stage * nb;
+        *P = (p.pruned_bitmap[j0 >> 5] >> (j0 & 31)) & mask;
+        *U = (p.unified_bitmap[j0 >> 5] >> (j0 & 31)) & mask & ~*P;
+        const long long f = n * p.cols + stage * kStageK;
+        *sgn = (unsigned long long)p.sign_bits[f >> 5] |
+               ((unsigned long long)p.sign_bits[(f >> 5) + 1] << 32);
+    }
+}
+
+__device__ __forceinline__ unsigned live_of(unsigned P, int b) {
+    const int nb = kStageK / b;
+    const unsigned mask = (nb >= 32) ? 0xffffffffu : ((1u << nb) - 1u);
+    const unsigned notP = ~P & mask;
+    const int bps = (16 / b) > 0 ? (16 / b) : 1;            // blocks per 16-column slice
+    unsigned live = 0;
+    for (int s = 0; s < 4; ++s) {
+        const unsigned m = (b >= 16) ? (1u << s) : (((1u << bps) - 1u) << (s * bps));
+        if (notP & m) live |= 1u << s;
+    }
+    return live;
+}
 
 __global__ void __launch_bounds__(128) count_kernel(Params p) {
     const int r = threadIdx.x;
     const long long rec = blockIdx.x;
     const long long tile = rec / p.L.n_stages, stage = rec % p.L.n_stages;
-    const long long n = tile * kTileRows + r;
     const int nb = kStageK / p.b;
-    const unsigned mask = (nb >= 32) ? 0xffffffffu : ((1u << nb) - 1u);
-    unsigned P = mask, U = 0;
-    unsigned long long sgn = 0;
-    if (n < p.rows) {
-        const long long j0 = n * (p.cols / p.b) + stage * nb;
-        P = (p.pruned_bitmap[j0 >> 5] >> (j0 & 31)) & mask;
-        U = (p.unified_bitmap[j0 >> 5] >> (j0 & 31)) & mask;
-        const long long f = n * p.cols + stage * kStageK;
-        sgn = (unsigned long long)p.sign_bits[f >> 5] | ((unsigned long long)p.sign_bits[(f >> 5) + 1] << 32);
+    unsigned P, U;
+    unsigned long long sgn;
+    row_masks(p, tile, stage, r, &P, &U, &sgn);
+    unsigned cu = __popc(U), cp = __popc(P);
+    unsigned live = live_of(P, p.b);
+    for (int m = 16; m > 0; m >>= 1) {
+        cu += __shfl_xor_sync(0xffffffffu, cu, m);
+        cp += __shfl_xor_sync(0xffffffffu, cp, m);
+        live |= __shfl_xor_sync(0xffffffffu, live, m);
     }
-    if (P & U) { atomicOr(p.dev_status, (unsigned)MWU_DEV_BOUNDS); U &= ~P; }
-    const unsigned cu = __popc(U), cd = nb - __popc(P) - cu;
-    // live 16-column slices of this row
-    unsigned live = 0;
-    const unsigned notP = ~P & mask;
-    const int bps = (16 / p.b) > 0 ? (16 / p.b) : 1;            // blocks per 16-column slice
-    for (int s = 0; s < 4; ++s) {
-        const unsigned m = (p.b >= 16) ? (1u << s) : (((1u << bps) - 1u) << (s * bps));
-        if (notP & m) live |= 1u << s;
-    }
-    // exclusive scan of (cu, cd) over the 128 rows: packed in one 32-bit word (each <= 4096)
-    unsigned both = cu | (cd << 16);
-    unsigned incl = both;
-    const int lane = r & 31, warp = r >> 5;
-    for (int off = 1; off < 32; off <<= 1) {
-        const unsigned t = __shfl_up_sync(0xffffffffu, incl, off);
-        if (lane >= off) incl += t;
-    }
-    __shared__ unsigned s_wsum[4];
-    __shared__ unsigned s_live;
-    if (r == 0) s_live = 0;
-    if (lane == 31) s_wsum[warp] = incl;
+    __shared__ unsigned s_cu[4], s_cp[4], s_live[4];
+    if ((r & 31) == 0) { s_cu[r >> 5] = cu; s_cp[r >> 5] = cp; s_live[r >> 5] = live; }
     __syncthreads();
-    unsigned base = 0;
-    for (int w = 0; w < warp; ++w) base += s_wsum[w];
-    const unsigned excl = base + incl - both;
-    if (live) atomicOr(&s_live, live);
-    __syncthreads();
-    const long long rs = rec * kTileRows + r;
-    Meta *meta = reinterpret_cast<Meta *>(p.packed + p.L.off_meta);
-    meta[rs].sgn = sgn;
-    meta[rs].P = P;
-    meta[rs].U = U;
-    reinterpret_cast<unsigned *>(p.packed + p.L.off_rel)[rs] = excl;     // u16 urel | u16 drel << 16
-    if (r == 127) {
-        const unsigned tot = excl + both;
-        Rec *recs = reinterpret_cast<Rec *>(p.packed + p.L.off_rec);
-        recs[rec].ubase = tot & 0xffffu;        // counts for now; scan_kernel turns them into bases
-        recs[rec].dbase = tot >> 16;
-        recs[rec].live = s_live;
-        recs[rec].zero = 0;
+    if (r == 0) {
+        const unsigned tu = s_cu[0] + s_cu[1] + s_cu[2] + s_cu[3];
+        const unsigned tp = s_cp[0] + s_cp[1] + s_cp[2] + s_cp[3];
+        PackedRec *recs = reinterpret_cast<PackedRec *>(p.packed + p.L.off_rec);
+        recs[rec].ubase = tu;                         // counts for now; scan_kernel makes bases
+        recs[rec].dbase = kTileRows * nb - tu - tp;
+        recs[rec].pbase = tp;
+        recs[rec].live = s_live[0] | s_live[1] | s_live[2] | s_live[3];
     }
 }
 
 __global__ void __launch_bounds__(1024) scan_kernel(Params p) {
     const long long n_rec = p.L.n_tiles * p.L.n_stages;
-    Rec *recs = reinterpret_cast<Rec *>(p.packed + p.L.off_rec);
-    __shared__ unsigned long long s_u[1024], s_d[1024];
+    PackedRec *recs = reinterpret_cast<PackedRec *>(p.packed + p.L.off_rec);
+    __shared__ unsigned long long s_u[1024], s_d[1024], s_p[1024];
     const long long per = (n_rec + 1023) / 1024;
     const long long lo = threadIdx.x * per;
     const long long hi = (lo + per < n_rec) ? lo + per : n_rec;
-    unsigned long long su = 0, sd = 0;
-    for (long long i = lo; i < hi; ++i) { su += recs[i].ubase; sd += recs[i].dbase; }
-    s_u[threadIdx.x] = su;
-    s_d[threadIdx.x] = sd;
+    unsigned long long su = 0, sd = 0, sp = 0;
+    for (long long i = lo; i < hi; ++i) { su += recs[i].ubase; sd += recs[i].dbase; sp += recs[i].pbase; }
+    s_u[threadIdx.x] = su; s_d[threadIdx.x] = sd; s_p[threadIdx.x] = sp;
     __syncthreads();
     for (int off = 1; off < 1024; off <<= 1) {
-        unsigned long long au = 0, ad = 0;
-        if ((int)threadIdx.x >= off) { au = s_u[threadIdx.x - off]; ad = s_d[threadIdx.x - off]; }
+        unsigned long long au = 0, ad = 0, ap = 0;
+        if ((int)threadIdx.x >= off) {
+            au = s_u[threadIdx.x - off]; ad = s_d[threadIdx.x - off]; ap = s_p[threadIdx.x - off];
+        }
         __syncthreads();
-        s_u[threadIdx.x] += au;
-        s_d[threadIdx.x] += ad;
+        s_u[threadIdx.x] += au; s_d[threadIdx.x] += ad; s_p[threadIdx.x] += ap;
         __syncthreads();
     }
-    unsigned long long ru = s_u[threadIdx.x] - su, rd = s_d[threadIdx.x] - sd;
+    unsigned long long ru = s_u[threadIdx.x] - su, rd = s_d[threadIdx.x] - sd, rp = s_p[threadIdx.x] - sp;
     for (long long i = lo; i < hi; ++i) {
-        const unsigned cu = recs[i].ubase, cd = recs[i].dbase;
-        recs[i].ubase = (unsigned)ru;
-        recs[i].dbase = (unsigned)rd;
-        ru += cu;
-        rd += cd;
+        const unsigned cu = recs[i].ubase, cd = recs[i].dbase, cp = recs[i].pbase;
+        recs[i].ubase = (unsigned)ru; recs[i].dbase = (unsigned)rd; recs[i].pbase = (unsigned)rp;
+        ru += cu; rd += cd; rp += cp;
     }
     if (threadIdx.x == 1023) {
-        if (s_u[1023] != (unsigned long long)p.L.n_unified || s_d[1023] != (unsigned long long)p.L.n_dense)
+        const unsigned long long tu = s_u[1023], td = s_d[1023], tp = s_p[1023];
+        if (tu != (unsigned long long)p.L.n_unified || td != (unsigned long long)p.L.n_dense ||
+            tp != (unsigned long long)p.L.n_plist)
             atomicOr(p.dev_status, (unsigned)MWU_DEV_BOUNDS);
+        recs[n_rec].ubase = (unsigned)tu; recs[n_rec].dbase = (unsigned)td;
+        recs[n_rec].pbase = (unsigned)tp; recs[n_rec].live = 0;
     }
     if (threadIdx.x < 32) {
         unsigned long long *h = reinterpret_cast<unsigned long long *>(p.packed);
-        const unsigned long long vals[32] = {
-            kMagic, 1ull, (unsigned long long)p.rows, (unsigned long long)p.cols,
-            (unsigned long long)p.b, (unsigned long long)p.L.n_pad, (unsigned long long)p.L.n_tiles,
-            (unsigned long long)p.L.n_stages, (unsigned long long)p.L.n_pruned,
-            (unsigned long long)p.L.n_unified, (unsigned long long)p.L.n_dense,
-            (unsigned long long)p.L.off_rec, (unsigned long long)p.L.off_meta,
-            (unsigned long long)p.L.off_rel, (unsigned long long)p.L.off_ustream,
-            (unsigned long long)p.L.off_dstream, (unsigned long long)p.L.total,
-            0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
-        h[threadIdx.x] = vals[threadIdx.x];
+        unsigned long long v = 0;
+        switch (threadIdx.x) {
+            case 0: v = kMagic; break;
+            case 1: v = 2; break;
+            case 2: v = (unsigned long long)p.rows; break;
+            case 3: v = (unsigned long long)p.cols; break;
+            case 4: v = (unsigned long long)p.b; break;
+            case 5: v = (unsigned long long)p.L.n_pad; break;
+            case 6: v = (unsigned long long)p.L.n_tiles; break;
+            case 7: v = (unsigned long long)p.L.n_stages; break;
+            case 8: v = (unsigned long long)p.L.n_pruned; break;
+            case 9: v = (unsigned long long)p.L.n_unified; break;
+            case 10: v = (unsigned long long)p.L.n_dense; break;
+            case 11: v = (unsigned long long)p.L.n_plist; break;
+            case 12: v = (unsigned long long)p.L.off_rec; break;
+            case 13: v = (unsigned long long)p.L.off_ulist; break;
+            case 14: v = (unsigned long long)p.L.off_dpos; break;
+            case 15: v = (unsigned long long)p.L.off_dpay; break;
+            case 16: v = (unsigned long long)p.L.off_ppos; break;
+            case 17: v = (unsigned long long)p.L.total; break;
+            default: v = 0;
+        }
+        h[threadIdx.x] = v;
     }
 }
 
 __global__ void __launch_bounds__(128) fill_kernel(Params p) {
     const long long rec = blockIdx.x;
     const long long tile = rec / p.L.n_stages, stage = rec % p.L.n_stages;
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const Rec *recs = reinterpret_cast<const Rec *>(p.packed + p.L.off_rec);
-    const Meta *meta = reinterpret_cast<const Meta *>(p.packed + p.L.off_meta);
-    const unsigned *rel = reinterpret_cast<const unsigned *>(p.packed + p.L.off_rel);
-    float *ustream = reinterpret_cast<float *>(p.packed + p.L.off_ustream);
-    __nv_bfloat162 *dstream = reinterpret_cast<__nv_bfloat162 *>(p.packed + p.L.off_dstream);
-    const unsigned ubase = recs[rec].ubase, dbase = recs[rec].dbase;
+    const int r = threadIdx.x, lane = r & 31, warp = r >> 5;
     const int b = p.b;
     const int nb = kStageK / b;
     const unsigned mask = (nb >= 32) ? 0xffffffffu : ((1u << nb) - 1u);
+    const PackedRec *recs = reinterpret_cast<const PackedRec *>(p.packed + p.L.off_rec);
+    uint2 *ulist = reinterpret_cast<uint2 *>(p.packed + p.L.off_ulist);
+    unsigned short *dpos = reinterpret_cast<unsigned short *>(p.packed + p.L.off_dpos);
+    __nv_bfloat162 *dpay = reinterpret_cast<__nv_bfloat162 *>(p.packed + p.L.off_dpay);
+    unsigned short *ppos = reinterpret_cast<unsigned short *>(p.packed + p.L.off_ppos);
+    const unsigned long long ubase = recs[rec].ubase, dbase = recs[rec].dbase, pbase = recs[rec].pbase;
+
+    __shared__ unsigned s_D[kTileRows], s_doff[kTileRows];
+    __shared__ unsigned s_w[3][4];
+    unsigned P, U;
+    unsigned long long sgn;
+    row_masks(p, tile, stage, r, &P, &U, &sgn);
+    const unsigned D = ~P & ~U & mask;
+    const unsigned cu = __popc(U), cd = __popc(D), cp = __popc(P);
+    unsigned iu = cu, id = cd, ip = cp;
+    for (int off = 1; off < 32; off <<= 1) {
+        const unsigned tu = __shfl_up_sync(0xffffffffu, iu, off);
+        const unsigned td = __shfl_up_sync(0xffffffffu, id, off);
+        const unsigned tp = __shfl_up_sync(0xffffffffu, ip, off);
+        if (lane >= off) { iu += tu; id += td; ip += tp; }
+    }
+    if (lane == 31) { s_w[0][warp] = iu; s_w[1][warp] = id; s_w[2][warp] = ip; }
+    __syncthreads();
+    unsigned bu = 0, bd = 0, bp = 0;
+    for (int w = 0; w < warp; ++w) { bu += s_w[0][w]; bd += s_w[1][w]; bp += s_w[2][w]; }
+    const unsigned eu = bu + iu - cu, ed = bd + id - cd, ep = bp + ip - cp;   // exclusive over rows
+    s_D[r] = D;
+    s_doff[r] = ed;
     bool bad = false;
-    for (int rr = 0; rr < 32; ++rr) {
-        const int r = warp * 32 + rr;
-        const long long n = tile * kTileRows + r;
-        if (n >= p.rows) break;                       // padding rows hold nothing
-        const long long rs = rec * kTileRows + r;
-        const unsigned P = meta[rs].P, U = meta[rs].U;
-        const unsigned D = ~P & ~U & mask;
-        const unsigned rl = rel[rs];
-        const unsigned long long ui0 = (unsigned long long)ubase + (rl & 0xffffu);
-        const unsigned long long di0 = (unsigned long long)dbase + (rl >> 16);
-        if (D) {
-            const long long f = n * p.cols + stage * kStageK + 2 * lane;
-            float2 v = __ldg(reinterpret_cast<const float2 *>(p.W + f));
-            if (p.U) {
-                const float2 d = __ldg(reinterpret_cast<const float2 *>(p.U + f));
-                v.x = __fadd_rn(v.x, d.x);
-                v.y = __fadd_rn(v.y, d.y);
-            }
-            const int i = (2 * lane) / b;             // block of this lane's pair
-            if ((D >> i) & 1u) {
-                const unsigned long long di = di0 + __popc(D & ((1u << i) - 1u));
-                if (di < (unsigned long long)p.L.n_dense)
-                    dstream[(di * b + (2 * lane - i * b)) >> 1] = __floats2bfloat162_rn(v.x, v.y);
-                else
-                    bad = true;
+    const long long n = tile * kTileRows + r;
+    // unified, dense-position and pruned lists: one thread per row, ascending pos
+    {
+        unsigned long long ui = ubase + eu, di = dbase + ed, pi = pbase + ep;
+        const unsigned bmask = (b >= 32) ? 0xffffffffu : ((1u << b) - 1u);
+        for (int i = 0; i < nb; ++i) {
+            const unsigned pos = (unsigned)(r * nb + i);
+            if ((U >> i) & 1u) {
+                const unsigned sb = (unsigned)(sgn >> (i * b)) & bmask;
+                const long long j = n * (p.cols / b) + stage * nb + i;
+                if (ui < (unsigned long long)p.L.n_unified)
+                    ulist[ui] = make_uint2(pos | (sb << 16), __float_as_uint(p.u[j]));
+                else bad = true;
+                ++ui;
+            } else if ((D >> i) & 1u) {
+                if (di < (unsigned long long)p.L.n_dense) dpos[di] = (unsigned short)pos;
+                else bad = true;
+                ++di;
+            } else {
+                if (pi < (unsigned long long)p.L.n_plist) ppos[pi] = (unsigned short)pos;
+                else bad = true;
+                ++pi;
             }
         }
-        if (lane < nb && ((U >> lane) & 1u)) {
-            const unsigned long long ui = ui0 + __popc(U & ((1u << lane) - 1u));
-            const long long j = n * (p.cols / b) + stage * nb + lane;
-            if (ui < (unsigned long long)p.L.n_unified) ustream[ui] = p.u[j];
+    }
+    __syncthreads();
+    // dense payload: each warp walks its 32 rows, lanes cover the 64 columns two at a time
+    for (int rr = 0; rr < 32; ++rr) {
+        const int row = warp * 32 + rr;
+        const long long nn = tile * kTileRows + row;
+        if (nn >= p.rows) break;
+        const unsigned Dr = s_D[row];
+        if (!Dr) continue;
+        const long long f = nn * p.cols + stage * kStageK + 2 * lane;
+        float2 v = __ldg(reinterpret_cast<const float2 *>(p.W + f));
+        if (p.U) {
+            const float2 d = __ldg(reinterpret_cast<const float2 *>(p.U + f));
+            v.x = __fadd_rn(v.x, d.x);
+            v.y = __fadd_rn(v.y, d.y);
+        }
+        const int i = (2 * lane) / b;
+        if ((Dr >> i) & 1u) {
+            const unsigned long long di = dbase + s_doff[row] + __popc(Dr & ((1u << i) - 1u));
+            if (di < (unsigned long long)p.L.n_dense)
+                dpay[(di * b + (2 * lane - i * b)) >> 1] = __floats2bfloat162_rn(v.x, v.y);
             else bad = true;
         }
     }
@@ -219,21 +270,21 @@ extern "C" int mwu_pack(const mwu_proj_desc *desc, const float *W, const float *
     p.dev_status = dev_status;
     p.rows = desc->rows; p.cols = desc->cols; p.b = desc->block;
     cudaStream_t st = (cudaStream_t)cuda_stream;
-    // gaps between sections and the tail of the last section must read as zero
+    // header, and the gaps between sections, must read as zero
     if (cudaMemsetAsync(packed, 0, kHeaderBytes, st) != cudaSuccess) return MWU_ERR_CUDA;
+    const size_t n_rec = (size_t)p.L.n_tiles * p.L.n_stages;
     const size_t gaps[5][2] = {
-        {p.L.off_rec + 16 * (size_t)p.L.n_tiles * p.L.n_stages, p.L.off_meta},
-        {p.L.off_meta + 16 * (size_t)p.L.n_tiles * p.L.n_stages * kTileRows, p.L.off_rel},
-        {p.L.off_rel + 4 * (size_t)p.L.n_tiles * p.L.n_stages * kTileRows, p.L.off_ustream},
-        {p.L.off_ustream + 4 * (size_t)p.L.n_unified, p.L.off_dstream},
-        {p.L.off_dstream + 2 * (size_t)desc->block * p.L.n_dense, p.L.total}};
+        {p.L.off_rec + 16 * (n_rec + 1), p.L.off_ulist},
+        {p.L.off_ulist + 8 * (size_t)p.L.n_unified, p.L.off_dpos},
+        {p.L.off_dpos + 2 * (size_t)p.L.n_dense, p.L.off_dpay},
+        {p.L.off_dpay + 2 * (size_t)desc->block * p.L.n_dense, p.L.off_ppos},
+        {p.L.off_ppos + 2 * (size_t)p.L.n_plist, p.L.total}};
     for (int g = 0; g < 5; ++g)
         if (gaps[g][1] > gaps[g][0])
             if (cudaMemsetAsync((char *)packed + gaps[g][0], 0, gaps[g][1] - gaps[g][0], st) != cudaSuccess)
                 return MWU_ERR_CUDA;
-    const int n_rec = (int)(p.L.n_tiles * p.L.n_stages);
-    pack::count_kernel<<<n_rec, 128, 0, st>>>(p);
+    pack::count_kernel<<<(unsigned)n_rec, 128, 0, st>>>(p);
     pack::scan_kernel<<<1, 1024, 0, st>>>(p);
-    pack::fill_kernel<<<n_rec, 128, 0, st>>>(p);
+    pack::fill_kernel<<<(unsigned)n_rec, 128, 0, st>>>(p);
     return cudaGetLastError() == cudaSuccess ? MWU_OK : MWU_ERR_CUDA;
 }

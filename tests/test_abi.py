@@ -73,4 +73,4 @@ def test_packed_bytes_matches_the_format_arithmetic():
                                   (16384, 4096, 16, 3355443, 2516582), (100, 128, 2, 6400, 0)]:
         d = B.make_desc(rows, cols, b, ku, kp)
         mb = rows * cols // b
-        assert B.mwu_packed_bytes(d) == O.packed_layout(rows, cols, b, ku - kp, mb - ku)["total"]
+        assert B.mwu_packed_bytes(d) == O.packed_layout(rows, cols, b, ku - kp, mb - ku, kp)["total"]

@@ -1,0 +1,182 @@
+"""GPU parity: mwu_gemm / mwu_conv_implicit through the C ABI against the CPU checker.
+
+Tolerances: bf16 output -- relative Frobenius error <= 2e-3 and max element error
+<= 1e-2 * max|y| (output rounding alone is about 1.5e-3); fp32 output -- 1e-5 relative
+Frobenius, so that an indexing or decode mistake cannot hide under output rounding.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import mwu_oracle as O
+from paper_2106_08301_b200 import binding as B
+from paper_2106_08301_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+
+
+def project_and_pack(W, b, ku, kp):
+    rows, cols = W.shape
+    desc = B.make_desc(rows, cols, b, ku, kp)
+    bufs = B.ProjectionBuffers(desc, want_q=False)
+    Wd = W.cuda().contiguous()
+    bufs.project(Wd)
+    packed = bufs.pack(Wd)
+    torch.cuda.synchronize()
+    assert int(bufs.dev_status.item()) == 0
+    p = O.project(W.numpy(), b, ku, kp)
+    return desc, bufs, packed, p
+
+
+def errors(Y, ref):
+    Y = Y.astype(np.float64)
+    fro = np.linalg.norm(Y - ref) / max(np.linalg.norm(ref), 1e-300)
+    mx = np.abs(Y - ref).max() / max(np.abs(ref).max(), 1e-300)
+    return fro, mx
+
+
+def run_gemm(desc, bufs, packed, X, y_dtype, ldy=None):
+    M = X.shape[0]
+    N = desc.rows
+    ldy = ldy or N
+    Y = torch.full((M, ldy), float("nan"), dtype=torch.float32 if y_dtype else torch.bfloat16, device="cuda")
+    Xd = X.cuda().contiguous()
+    B.mwu_gemm(desc, packed, Xd, M, X.shape[1], Y, ldy, y_dtype, bufs.dev_status)
+    torch.cuda.synchronize()
+    assert int(bufs.dev_status.item()) == 0
+    return Y.float().cpu().numpy()[:, :N]
+
+
+def check_gemm(W, b, ku, kp, M, seed=0):
+    desc, bufs, packed, p = project_and_pack(W, b, ku, kp)
+    X = inputs.normal_activations_bf16((M, W.shape[1]), 4242 + seed)
+    What = O.decoded_weights(p, b)
+    ref = O.gemm(X.to(torch.float64).numpy(), What)
+    Y32 = run_gemm(desc, bufs, packed, X, 1)
+    fro, mx = errors(Y32, ref)
+    assert fro <= 1e-5, (fro, mx)
+    Y16 = run_gemm(desc, bufs, packed, X, 0)
+    fro, mx = errors(Y16, ref)
+    assert fro <= 2e-3 and mx <= 1e-2, (fro, mx)
+    return desc, bufs, packed, p
+
+
+def test_gemm_config1_linear():
+    wl = inputs.WORKLOADS["c1_linear"]
+    Mb = wl.n_blocks
+    check_gemm(wl.weights(), wl.block, B.mwu_count_from_permille(Mb, wl.unified_permille),
+               B.mwu_count_from_permille(Mb, wl.pruned_permille), wl.m)
+
+
+@pytest.mark.parametrize("b", [2, 4, 8, 16])
+def test_gemm_block_widths_and_ragged_shapes(b):
+    # N = 384 -> three 128-row weight tiles (an odd count: last CTA tile has one record);
+    # M = 300 -> ragged last row tile; K = 192 -> three stages
+    W = inputs.normal_weights(384, 192, 0.02, 50 + b)
+    Mb = W.numel() // b
+    check_gemm(W, b, Mb * 6 // 10, Mb * 3 // 10, 300, seed=b)
+
+
+def test_gemm_ragged_weight_rows():
+    W = inputs.normal_weights(200, 128, 0.02, 61)       # N not a multiple of 128, single CTA tile
+    Mb = W.numel() // 8
+    check_gemm(W, 8, Mb // 2, Mb // 4, 130)
+    W = inputs.normal_weights(72, 64, 0.02, 62)         # one record, N = 72
+    check_gemm(W, 4, 100, 50, 5)
+
+
+def test_gemm_all_classes_degenerate():
+    W = inputs.normal_weights(256, 256, 0.02, 63)
+    Mb = W.numel() // 16
+    check_gemm(W, 16, 0, 0, 64)            # all dense: an ordinary GEMM
+    check_gemm(W, 16, Mb, 0, 64)           # all unified
+    check_gemm(W, 16, Mb, Mb, 64)          # all pruned: exactly zero, every stage skipped
+    desc, bufs, packed, p = project_and_pack(W, 16, Mb, Mb)
+    X = inputs.normal_activations_bf16((64, 256), 1)
+    assert np.all(run_gemm(desc, bufs, packed, X, 0) == 0)
+
+
+def test_gemm_skips_dead_stages_and_slices():
+    """Structured pruning: whole 64-column stages and single 16-column slices are zero in every
+    row, so the kernel's skip paths run; results must not change."""
+    W = inputs.normal_weights(256, 512, 0.02, 64)
+    W[:, 64:192] = 0.0                  # stages 1 and 2 dead in every tile
+    W[:, 272:288] = 0.0                 # slice 1 of stage 4 dead
+    W[:128, 448:512] = 0.0              # stage 7 dead in the first row tile only (not skippable with 2-tile CTAs)
+    b = 16
+    Mb = W.numel() // b
+    n_zero = int((W.reshape(-1, b).abs().sum(dim=1) == 0).sum())
+    desc, bufs, packed, p = check_gemm(W, b, n_zero + 500, n_zero, 200)
+    h = O.parse_header(O.pack(p, b))
+    rec = O.pack(p, b)[h["off_rec"]:h["off_rec"] + 16 * 17].view(np.uint32).reshape(-1, 4)
+    assert rec[1, 3] == 0 and rec[2, 3] == 0 and rec[8 + 1, 3] == 0 and rec[4, 3] == 0b1101
+
+
+def test_gemm_output_leading_dimension():
+    W = inputs.normal_weights(256, 128, 0.02, 65)
+    desc, bufs, packed, p = project_and_pack(W, 8, 2000, 1000)
+    X = inputs.normal_activations_bf16((100, 128), 3)
+    ref = O.gemm(X.to(torch.float64).numpy(), O.decoded_weights(p, 8))
+    Y = run_gemm(desc, bufs, packed, X, 1, ldy=264)
+    assert errors(Y, ref)[0] <= 1e-5
+
+
+def test_gemm_argument_errors():
+    W = inputs.normal_weights(128, 64, 0.02, 66)
+    desc, bufs, packed, p = project_and_pack(W, 4, 100, 50)
+    X = inputs.normal_activations_bf16((16, 64), 3).cuda()
+    Y = torch.empty((16, 128), dtype=torch.bfloat16, device="cuda")
+    assert B.mwu_gemm(desc, packed, X, 16, 60, Y, 128, 0, bufs.dev_status, check=False) == 2   # ldx < cols
+    assert B.mwu_gemm(desc, packed, X, 16, 64, Y, 100, 0, bufs.dev_status, check=False) == 2   # ldy < rows
+    assert B.mwu_gemm(desc, packed, X, 16, 64, Y, 132, 0, bufs.dev_status, check=False) == 3   # ldy % 8
+    assert B.mwu_gemm(desc, packed, X, 16, 64, Y, 128, 7, bufs.dev_status, check=False) == 1
+    assert B.mwu_gemm(desc, packed, X, 0, 64, Y, 128, 0, bufs.dev_status, check=False) == 0    # no-op
+
+
+def test_gemm_config3_shape_sampled_rows():
+    """1x1 conv as GEMM (K = 256, N = 1024) on a reduced M; full M is exercised by the benchmark."""
+    wl = inputs.WORKLOADS["c3_conv1x1"]
+    Mb = wl.n_blocks
+    check_gemm(wl.weights(), wl.block, B.mwu_count_from_permille(Mb, wl.unified_permille),
+               B.mwu_count_from_permille(Mb, wl.pruned_permille), 1000)
+
+
+def conv_case(W, b, ku, kp, x, kh, kw, stride, pad):
+    desc, bufs, packed, p = project_and_pack(W, b, ku, kp)
+    n, c, h, w = x.shape
+    oh = (h + 2 * pad - kh) // stride + 1
+    ow = (w + 2 * pad - kw) // stride + 1
+    ref = O.conv2d_direct(x.to(torch.float64).numpy(), O.decoded_weights(p, b), kh, kw, stride, pad)
+    xd = x.cuda().contiguous()
+    for y_dtype, tol in [(1, 1e-5), (0, 2e-3)]:
+        Y = torch.full((n, W.shape[0], oh, ow), float("nan"),
+                       dtype=torch.float32 if y_dtype else torch.bfloat16, device="cuda")
+        B.mwu_conv_implicit(desc, packed, xd, n, c, h, w, kh, kw, stride, pad, Y, y_dtype, bufs.dev_status)
+        torch.cuda.synchronize()
+        assert int(bufs.dev_status.item()) == 0
+        fro, mx = errors(Y.float().cpu().numpy(), ref)
+        assert fro <= tol and mx <= 1e-2, (y_dtype, fro, mx)
+
+
+def test_conv_small_cases():
+    # 3x3 s1 p1, K = 64*9 = 576; M = 2*9*7 = 126 (ragged)
+    W = inputs.normal_weights(128, 576, 0.05, 70)
+    x = inputs.normal_activations_bf16((2, 64, 9, 7), 71)
+    Mb = W.numel() // 4
+    conv_case(W, 4, Mb * 6 // 10, Mb * 3 // 10, x, 3, 3, 1, 1)
+    # stride 2, no padding, 256 filters (two records per CTA tile), b = 16
+    W = inputs.normal_weights(256, 576, 0.05, 72)
+    Mb = W.numel() // 16
+    conv_case(W, 16, Mb // 2, Mb // 4, x, 3, 3, 2, 0)
+    # 1x1 convolution equals a GEMM over channels
+    W = inputs.normal_weights(128, 64, 0.05, 73)
+    conv_case(W, 8, 300, 100, x, 1, 1, 1, 0)
+
+
+def test_conv_config2():
+    wl = inputs.WORKLOADS["c2_conv3x3"]
+    Mb = wl.n_blocks
+    x = wl.activations()
+    n, c, h, w, kh, kw, stride, pad = wl.conv
+    conv_case(wl.weights(), wl.block, B.mwu_count_from_permille(Mb, wl.unified_permille),
+              B.mwu_count_from_permille(Mb, wl.pruned_permille), x, kh, kw, stride, pad)

@@ -153,5 +153,6 @@ def test_pack_with_dual_and_structured_pruning():
     ref = O.pack(p, b)
     assert np.array_equal(packed.cpu().numpy(), ref)
     h = O.parse_header(ref)
-    rec = ref[h["off_rec"]:h["off_rec"] + 16 * 8].view(np.uint32).reshape(-1, 4)
-    assert rec[1, 2] == 0 and rec[5, 2] == 0          # stage 1 of both row tiles is dead
+    rec = ref[h["off_rec"]:h["off_rec"] + 16 * 9].view(np.uint32).reshape(-1, 4)
+    assert rec[1, 3] == 0 and rec[5, 3] == 0          # stage 1 of both row tiles is dead
+    assert rec[0, 3] == 0xF

@@ -56,10 +56,11 @@ def test_packed_size_accounting():
     ku, kp = Mb * 3 // 4, Mb // 2
     p = O.project(W, b, ku, kp)
     h = O.parse_header(O.pack(p, b))
-    assert h["off_dstream"] - h["off_ustream"] >= 4 * (ku - kp)
-    assert h["total"] - h["off_dstream"] >= 2 * b * (Mb - ku)
-    assert h["total"] - h["off_dstream"] < 2 * b * (Mb - ku) + 256
-    assert h["n_dense"] == Mb - ku
+    assert h["off_dpos"] - h["off_ulist"] >= 8 * (ku - kp)
+    assert h["off_ppos"] - h["off_dpay"] >= 2 * b * (Mb - ku)
+    assert h["off_ppos"] - h["off_dpay"] < 2 * b * (Mb - ku) + 256
+    assert h["total"] - h["off_ppos"] >= 2 * kp
+    assert h["n_dense"] == Mb - ku and h["n_plist"] == kp
 
 
 def test_live_mask_and_padding():
@@ -72,10 +73,15 @@ def test_live_mask_and_padding():
     assert p.pruned.reshape(N, K // b)[:, 1].all()
     buf = O.pack(p, b)
     h = O.parse_header(buf)
-    rec = buf[h["off_rec"]:h["off_rec"] + 16 * 2].view(np.uint32).reshape(2, 4)
-    assert rec[0, 2] == 0b1101 and rec[1, 2] == 0b1111
-    meta = buf[h["off_meta"]:h["off_meta"] + 16 * 256].view(np.uint64).reshape(-1, 2)
-    assert (meta[100:128, 1] & np.uint64(0xFFFFFFFF) == 0xF).all()      # padding rows pruned
+    rec = buf[h["off_rec"]:h["off_rec"] + 16 * 3].view(np.uint32).reshape(3, 4)
+    assert rec[0, 3] == 0b1101 and rec[1, 3] == 0b1111
+    nb = 64 // b
+    assert h["n_plist"] == kp + 28 * (K // b)                           # padding rows pruned
+    ppos = buf[h["off_ppos"]:h["off_ppos"] + 2 * h["n_plist"]].view(np.uint16)
+    first = ppos[rec[0, 2]:rec[1, 2]]
+    assert np.all(np.diff(first.astype(int)) > 0)                       # ascending slot codes
+    assert set(range(100 * nb, 128 * nb)) <= set(first.tolist())
+    assert rec[2].tolist() == [h["n_unified"], h["n_dense"], h["n_plist"], 0]
     assert O.decode(buf).shape == (N, K)
 
 
