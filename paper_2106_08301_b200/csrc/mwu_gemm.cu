@@ -7,9 +7,13 @@
 //   warp 1        allocates tensor memory and issues tcgen05.mma (one thread); fp32 accumulators
 //                 live in TMEM, two buffers so that the epilogue of tile i overlaps tile i+1.
 //   warps 2-5     epilogue: tcgen05.ld -> bf16/fp32 -> global.
-//   warps 6-13    decode the weight tile (B operand) from the packed class lists into the
+//   warps 6-21    decode the weight tile (B operand) from the packed class lists into the
 //                 128-byte-swizzled K-major layout the MMA reads: pruned blocks -> zeros,
-//                 unified blocks -> sign . bf16(u), dense blocks -> stored bf16 values.
+//                 unified blocks -> sign . bf16(u), dense blocks -> stored bf16 values.  Four
+//                 groups of four warps, one per pipeline slot, take every fourth live stage, so
+//                 a group has four stage times to hide the latency of its list reads; each
+//                 thread reads a fixed number of list entries per stage (all loads first, then
+//                 the stores).
 // A 64-wide k stage whose blocks are pruned in every row of the weight tile is skipped by all
 // roles (no load, no decode, no MMA); inside a live stage the MMA skips dead 16-wide slices.
 // Every wait on an mbarrier is bounded; when one runs out the kernel raises MWU_DEV_TIMEOUT,
@@ -26,15 +30,20 @@ constexpr int BK = kStageK;             // 64
 constexpr int STAGES = 4;
 constexpr int A_BYTES = BM * BK * 2;    // 16 KiB
 constexpr int REC_BYTES = kTileRows * BK * 2;
-constexpr int NDEC_WARPS = 8;
+constexpr int NDEC_WARPS = 4;           // warps per decode group
+constexpr int NDEC_GROUPS = 4;          // one group per pipeline slot
+constexpr int NDEC_THREADS = NDEC_WARPS * 32;
 constexpr int NGATHER_WARPS = 4;
-constexpr int THREADS_GEMM = 32 * (6 + NDEC_WARPS);
+constexpr int FIRST_GATHER_WARP = 6 + NDEC_WARPS * NDEC_GROUPS;
+constexpr int THREADS_GEMM = 32 * FIRST_GATHER_WARP;
+constexpr int MAX_STAGES_K = 256;       // cols <= 16384
 constexpr int THREADS_CONV = THREADS_GEMM + 32 * NGATHER_WARPS;
 constexpr long long WAIT_LIMIT_CYCLES = 4000000000ll;   // about two seconds
 
 struct Params {
     const unsigned char *packed;
     size_t off_rec, off_ulist, off_dpos, off_dpay, off_ppos;
+    unsigned n_unified, n_dense, n_plist;   // list lengths, to keep every index in bounds
     long long n_rec_tiles;              // 128-row tiles of W
     long long n_stages;                 // K / 64
     long long M, N, K;
@@ -154,74 +163,94 @@ __device__ __forceinline__ unsigned sign_word(unsigned u2, unsigned sbits, int w
 }
 
 template <int BW>
+__device__ __forceinline__ void store_block(unsigned char *tile, unsigned pos, const unsigned (&w)[8]) {
+    constexpr int NBK = BK / BW;
+    const unsigned r = pos / NBK, i = pos % NBK;
+    if (BW == 16) {
+        const unsigned a = swz(r, 2 * i);
+        *reinterpret_cast<uint4 *>(tile + a) = make_uint4(w[0], w[1], w[2], w[3]);
+        *reinterpret_cast<uint4 *>(tile + (a ^ 16u)) = make_uint4(w[4], w[5], w[6], w[7]);
+    } else if (BW == 8) {
+        *reinterpret_cast<uint4 *>(tile + swz(r, i)) = make_uint4(w[0], w[1], w[2], w[3]);
+    } else if (BW == 4) {
+        *reinterpret_cast<uint2 *>(tile + swz(r, i >> 1) + (i & 1) * 8) = make_uint2(w[0], w[1]);
+    } else {
+        *reinterpret_cast<unsigned *>(tile + swz(r, i >> 2) + (i & 3) * 4) = w[0];
+    }
+}
+
+// One record = 128 * 64/BW block slots, listed as [pruned | dense | unified].  Thread `tid` of
+// the 256 takes flattened entries tid, tid+256, ...: a fixed count, so all loads issue first.
+template <int BW>
 __device__ __forceinline__ void decode_record(unsigned char *tile, const PackedRec r0, const PackedRec r1,
-                                              const Params &p, int tid, int nthr) {
-    constexpr int NBK = BK / BW;                          // blocks per row
+                                              const Params &p, int tid) {
+    constexpr int NBK = BK / BW;
+    constexpr int SLOTS = kTileRows * NBK;
+    constexpr int ENT = SLOTS / NDEC_THREADS;
+    constexpr int WORDS = BW / 2;                           // 32-bit words per block
     const uint2 *ulist = reinterpret_cast<const uint2 *>(p.packed + p.off_ulist);
     const unsigned short *dpos = reinterpret_cast<const unsigned short *>(p.packed + p.off_dpos);
     const unsigned char *dpay = p.packed + p.off_dpay;
     const unsigned short *ppos = reinterpret_cast<const unsigned short *>(p.packed + p.off_ppos);
-    // pruned blocks: zeros
-    for (unsigned e = r0.pbase + tid; e < r1.pbase; e += nthr) {
-        const unsigned pos = __ldg(ppos + e) & (kTileRows * NBK - 1);
-        const unsigned r = pos / NBK, i = pos % NBK;
-        if (BW == 16) {
-            const unsigned a = swz(r, 2 * i);
-            *reinterpret_cast<uint4 *>(tile + a) = make_uint4(0, 0, 0, 0);
-            *reinterpret_cast<uint4 *>(tile + (a ^ 16u)) = make_uint4(0, 0, 0, 0);
-        } else if (BW == 8) {
-            *reinterpret_cast<uint4 *>(tile + swz(r, i)) = make_uint4(0, 0, 0, 0);
-        } else if (BW == 4) {
-            *reinterpret_cast<uint2 *>(tile + swz(r, i >> 1) + (i & 1) * 8) = make_uint2(0, 0);
-        } else {
-            *reinterpret_cast<unsigned *>(tile + swz(r, i >> 2) + (i & 3) * 4) = 0u;
+    const unsigned n_p = r1.pbase - r0.pbase, n_d = r1.dbase - r0.dbase, n_u = r1.ubase - r0.ubase;
+    unsigned meta[ENT], uval[ENT];
+    unsigned pay[ENT][WORDS];
+#pragma unroll
+    for (int k = 0; k < ENT; ++k) {
+        const unsigned f = (unsigned)tid + (unsigned)k * NDEC_THREADS;
+        meta[k] = 0xffffffffu;                              // nothing to write
+        uval[k] = 0;
+#pragma unroll
+        for (int w = 0; w < WORDS; ++w) pay[k][w] = 0;
+        if (f < n_p) {
+            const unsigned e = r0.pbase + f;
+            if (e < p.n_plist) meta[k] = __ldg(ppos + e);
+        } else if (f < n_p + n_d) {
+            const unsigned e = r0.dbase + (f - n_p);
+            if (e < p.n_dense) {
+                meta[k] = __ldg(dpos + e);
+                const unsigned char *src = dpay + (size_t)e * (2 * BW);
+                if (BW == 16) {
+                    const uint4 v0 = __ldg(reinterpret_cast<const uint4 *>(src));
+                    const uint4 v1 = __ldg(reinterpret_cast<const uint4 *>(src + 16));
+                    pay[k][0] = v0.x; pay[k][1] = v0.y; pay[k][2] = v0.z; pay[k][3] = v0.w;
+                    pay[k][4 % WORDS] = v1.x; pay[k][5 % WORDS] = v1.y; pay[k][6 % WORDS] = v1.z; pay[k][7 % WORDS] = v1.w;
+                } else if (BW == 8) {
+                    const uint4 v0 = __ldg(reinterpret_cast<const uint4 *>(src));
+                    pay[k][0] = v0.x; pay[k][1 % WORDS] = v0.y; pay[k][2 % WORDS] = v0.z; pay[k][3 % WORDS] = v0.w;
+                } else if (BW == 4) {
+                    const uint2 v0 = __ldg(reinterpret_cast<const uint2 *>(src));
+                    pay[k][0] = v0.x; pay[k][1 % WORDS] = v0.y;
+                } else {
+                    pay[k][0] = __ldg(reinterpret_cast<const unsigned *>(src));
+                }
+            }
+        } else if (f < n_p + n_d + n_u) {
+            const unsigned e = r0.ubase + (f - n_p - n_d);
+            if (e < p.n_unified) {
+                const uint2 ent = __ldg(ulist + e);
+                meta[k] = ent.x;
+                uval[k] = ent.y;
+            }
         }
     }
-    // dense blocks: copy the stored bf16 values
-    for (unsigned e = r0.dbase + tid; e < r1.dbase; e += nthr) {
-        const unsigned pos = __ldg(dpos + e) & (kTileRows * NBK - 1);
-        const unsigned r = pos / NBK, i = pos % NBK;
-        const unsigned char *src = dpay + (size_t)e * (2 * BW);
-        if (BW == 16) {
-            const uint4 v0 = __ldg(reinterpret_cast<const uint4 *>(src));
-            const uint4 v1 = __ldg(reinterpret_cast<const uint4 *>(src + 16));
-            const unsigned a = swz(r, 2 * i);
-            *reinterpret_cast<uint4 *>(tile + a) = v0;
-            *reinterpret_cast<uint4 *>(tile + (a ^ 16u)) = v1;
-        } else if (BW == 8) {
-            *reinterpret_cast<uint4 *>(tile + swz(r, i)) = __ldg(reinterpret_cast<const uint4 *>(src));
-        } else if (BW == 4) {
-            *reinterpret_cast<uint2 *>(tile + swz(r, i >> 1) + (i & 1) * 8) =
-                __ldg(reinterpret_cast<const uint2 *>(src));
+#pragma unroll
+    for (int k = 0; k < ENT; ++k) {
+        const unsigned f = (unsigned)tid + (unsigned)k * NDEC_THREADS;
+        if (meta[k] == 0xffffffffu) continue;
+        const unsigned pos = meta[k] & (SLOTS - 1);
+        unsigned w[8];
+        if (f >= n_p + n_d) {
+            const unsigned sbits = meta[k] >> 16;
+            const unsigned u1 = (unsigned)__bfloat16_as_ushort(__float2bfloat16_rn(__uint_as_float(uval[k])));
+            const unsigned u2 = u1 | (u1 << 16);
+#pragma unroll
+            for (int q = 0; q < 8; ++q) w[q] = (q < WORDS) ? sign_word(u2, sbits, q) : 0u;
         } else {
-            *reinterpret_cast<unsigned *>(tile + swz(r, i >> 2) + (i & 3) * 4) =
-                __ldg(reinterpret_cast<const unsigned *>(src));
+#pragma unroll
+            for (int q = 0; q < 8; ++q) w[q] = (q < WORDS) ? pay[k][q % WORDS] : 0u;
         }
-    }
-    // unified blocks: sign . bf16(u)
-    for (unsigned e = r0.ubase + tid; e < r1.ubase; e += nthr) {
-        const uint2 ent = __ldg(ulist + e);
-        const unsigned pos = ent.x & (kTileRows * NBK - 1);
-        const unsigned sbits = ent.x >> 16;
-        const unsigned r = pos / NBK, i = pos % NBK;
-        const __nv_bfloat16 ub = __float2bfloat16_rn(__uint_as_float(ent.y));
-        const unsigned u1 = (unsigned)__bfloat16_as_ushort(ub);
-        const unsigned u2 = u1 | (u1 << 16);
-        if (BW == 16) {
-            const unsigned a = swz(r, 2 * i);
-            *reinterpret_cast<uint4 *>(tile + a) = make_uint4(sign_word(u2, sbits, 0), sign_word(u2, sbits, 1),
-                                                              sign_word(u2, sbits, 2), sign_word(u2, sbits, 3));
-            *reinterpret_cast<uint4 *>(tile + (a ^ 16u)) = make_uint4(sign_word(u2, sbits, 4), sign_word(u2, sbits, 5),
-                                                                      sign_word(u2, sbits, 6), sign_word(u2, sbits, 7));
-        } else if (BW == 8) {
-            *reinterpret_cast<uint4 *>(tile + swz(r, i)) = make_uint4(sign_word(u2, sbits, 0), sign_word(u2, sbits, 1),
-                                                                      sign_word(u2, sbits, 2), sign_word(u2, sbits, 3));
-        } else if (BW == 4) {
-            *reinterpret_cast<uint2 *>(tile + swz(r, i >> 1) + (i & 1) * 8) =
-                make_uint2(sign_word(u2, sbits, 0), sign_word(u2, sbits, 1));
-        } else {
-            *reinterpret_cast<unsigned *>(tile + swz(r, i >> 2) + (i & 3) * 4) = sign_word(u2, sbits, 0);
-        }
+        store_block<BW>(tile, pos, w);
     }
 }
 
@@ -232,7 +261,14 @@ struct Smem {
     unsigned long long full_a[STAGES], full_b[STAGES], empty[STAGES], tfull[2], tempty[2], drain;
     unsigned tmem_base;
     int abort;
+    unsigned char live_prod[MAX_STAGES_K];                  // live masks of the producer's tile
+    unsigned char live_mma[MAX_STAGES_K];                   // ... of the MMA issuer's tile
+    unsigned char live_gather[NGATHER_WARPS][MAX_STAGES_K]; // ... of each gather warp's tile
 };
+
+__device__ __forceinline__ void group_bar(int group) {      // the threads of one decode group
+    asm volatile("bar.sync %0, %1;" ::"r"(1 + group), "r"(NDEC_THREADS) : "memory");
+}
 
 template <int MODE, int NREC, int BW>
 __global__ void __launch_bounds__(MODE ? THREADS_CONV : THREADS_GEMM, 1)
@@ -244,7 +280,10 @@ mwu_gemm_kernel(const __grid_constant__ CUtensorMap tmap, const Params p) {
     unsigned char *sB = base + STAGES * A_BYTES;
     constexpr int B_BYTES = NREC * REC_BYTES;
     Smem *sm = reinterpret_cast<Smem *>(sB + STAGES * B_BYTES);
-    int2 *ktab = reinterpret_cast<int2 *>(reinterpret_cast<unsigned char *>(sm) + 256);   // conv only
+    const int n_stages = (int)p.n_stages;
+    // per decode group: the record table of its current tile, [NREC][n_stages + 1]
+    uint4 *srec = reinterpret_cast<uint4 *>(reinterpret_cast<unsigned char *>(sm) + ((sizeof(Smem) + 15) & ~(size_t)15));
+    int2 *ktab = reinterpret_cast<int2 *>(srec + (size_t)NDEC_GROUPS * NREC * (n_stages + 1));   // conv only
     volatile int *abort = &sm->abort;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -252,7 +291,6 @@ mwu_gemm_kernel(const __grid_constant__ CUtensorMap tmap, const Params p) {
     const long long m_tiles = (p.M + BM - 1) / BM;
     const long long n_tiles = (p.n_rec_tiles + NREC - 1) / NREC;
     const long long total_tiles = m_tiles * n_tiles;
-    const int n_stages = (int)p.n_stages;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
@@ -291,17 +329,24 @@ mwu_gemm_kernel(const __grid_constant__ CUtensorMap tmap, const Params p) {
         }
         return live;
     };
+    // one warp copies the live masks of tile nt into its table
+    auto load_live = [&](unsigned char *table, long long nt) {
+        __syncwarp();
+        for (int ks = lane; ks < n_stages; ks += 32) table[ks] = (unsigned char)live_of(nt, ks);
+        __syncwarp();
+    };
 
     if (warp == 0 && MODE == 0) {
         // ---------------- TMA producer ----------------
-        if (lane == 0) {
-            int stage = 0;
-            unsigned phase = 0;
-            bool ok = true;
-            for (long long t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
-                const long long mt = t % m_tiles, nt = t / m_tiles;
+        int stage = 0;
+        unsigned phase = 0;
+        bool ok = true;
+        for (long long t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+            const long long mt = t % m_tiles, nt = t / m_tiles;
+            load_live(sm->live_prod, nt);
+            if (lane == 0) {
                 for (int ks = 0; ks < n_stages; ++ks) {
-                    if (!live_of(nt, ks)) continue;
+                    if (!sm->live_prod[ks]) continue;
                     if (!mbar_wait(smem_u32(&sm->empty[stage]), phase ^ 1u, abort)) { ok = false; break; }
                     const unsigned bar = smem_u32(&sm->full_a[stage]);
                     mbar_expect_tx(bar, A_BYTES);
@@ -309,28 +354,30 @@ mwu_gemm_kernel(const __grid_constant__ CUtensorMap tmap, const Params p) {
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                 }
             }
+            ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
         }
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
-        if (lane == 0) {
-            int stage = 0;
-            unsigned phase = 0;
-            unsigned acc_phase[2] = {0, 0};
-            long long it = 0;
-            bool ok = true;
-            bool issued_any = false;
-            for (long long t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++it) {
-                const long long nt = t / m_tiles;
+        int stage = 0;
+        unsigned phase = 0;
+        unsigned acc_phase[2] = {0, 0};
+        long long it = 0;
+        bool ok = true;
+        bool issued_any = false;
+        for (long long t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++it) {
+            const long long nt = t / m_tiles;
+            load_live(sm->live_mma, nt);
+            if (lane == 0) {
                 const int buf = (int)(it & 1);
                 const int nrec_here = (int)((p.n_rec_tiles - nt * NREC) < NREC ? (p.n_rec_tiles - nt * NREC) : NREC);
                 const unsigned idesc = make_idesc(nrec_here * kTileRows);
-                if (!mbar_wait(smem_u32(&sm->tempty[buf]), acc_phase[buf] ^ 1u, abort)) { ok = false; break; }
+                if (!mbar_wait(smem_u32(&sm->tempty[buf]), acc_phase[buf] ^ 1u, abort)) ok = false;
                 acc_phase[buf] ^= 1u;
                 tc_fence_after();
                 const unsigned d_tmem = tmem_base + (unsigned)(buf * 256);
                 bool first = true;
-                for (int ks = 0; ks < n_stages; ++ks) {
-                    const unsigned live = live_of(nt, ks);
+                for (int ks = 0; ks < n_stages && ok; ++ks) {
+                    const unsigned live = sm->live_mma[ks];
                     if (!live) continue;
                     if (!mbar_wait(smem_u32(&sm->full_a[stage]), phase, abort)) { ok = false; break; }
                     if (!mbar_wait(smem_u32(&sm->full_b[stage]), phase, abort)) { ok = false; break; }
@@ -349,16 +396,19 @@ mwu_gemm_kernel(const __grid_constant__ CUtensorMap tmap, const Params p) {
                     umma_commit(smem_u32(&sm->empty[stage]));
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                 }
-                if (!ok) break;
-                if (!first) umma_commit(smem_u32(&sm->tfull[buf]));
-                else mbar_arrive(smem_u32(&sm->tfull[buf]));
+                if (ok) {
+                    if (!first) umma_commit(smem_u32(&sm->tfull[buf]));
+                    else mbar_arrive(smem_u32(&sm->tfull[buf]));
+                }
             }
-            // everything this thread issued must have retired before tensor memory is freed
-            if (issued_any) {
-                umma_commit(smem_u32(&sm->drain));
-                mbar_wait(smem_u32(&sm->drain), 0, abort);
-            }
+            ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
         }
+        // everything this thread issued must have retired before tensor memory is freed
+        if (lane == 0 && issued_any) {
+            umma_commit(smem_u32(&sm->drain));
+            mbar_wait(smem_u32(&sm->drain), 0, abort);
+        }
+        __syncwarp();
     } else if (warp >= 2 && warp < 6) {
         // ---------------- epilogue ----------------
         const int quarter = warp & 3;                       // TMEM lanes this warp may read
@@ -442,41 +492,63 @@ mwu_gemm_kernel(const __grid_constant__ CUtensorMap tmap, const Params p) {
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&sm->tempty[buf]));
         }
-    } else if (warp >= 6 && warp < 6 + NDEC_WARPS) {
-        // ---------------- weight decode ----------------
-        const int tid = threadIdx.x - 6 * 32;
-        constexpr int NTHR = NDEC_WARPS * 32;
-        int stage = 0;
-        unsigned phase = 0;
+    } else if (warp >= 6 && warp < FIRST_GATHER_WARP) {
+        // ---------------- weight decode: two groups on alternate live stages ----------------
+        const int group = (warp - 6) / NDEC_WARPS;
+        const int tid = threadIdx.x - (6 + group * NDEC_WARPS) * 32;
+        uint4 *my_rec = srec + (size_t)group * NREC * (n_stages + 1);
+        long long seq = 0;                                  // live stages seen so far (all tiles)
         bool ok = true;
+        auto rec_at = [&](int q, int ks, PackedRec *r0, PackedRec *r1) {
+            const uint4 a = my_rec[q * (n_stages + 1) + ks], b = my_rec[q * (n_stages + 1) + ks + 1];
+            r0->ubase = a.x; r0->dbase = a.y; r0->pbase = a.z; r0->live = a.w;
+            r1->ubase = b.x; r1->dbase = b.y; r1->pbase = b.z; r1->live = b.w;
+        };
         for (long long t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
             const long long nt = t / m_tiles;
+            group_bar(group);                               // everyone is done with the previous table
+#pragma unroll
+            for (int q = 0; q < NREC; ++q) {
+                const long long rt = nt * NREC + q;
+                for (int ks = tid; ks <= n_stages; ks += NDEC_THREADS) {
+                    uint4 v = make_uint4(0, 0, 0, 0);
+                    if (rt < p.n_rec_tiles) v = __ldg(reinterpret_cast<const uint4 *>(&recs[rt * n_stages + ks]));
+                    if (ks == n_stages) v.w = 0;
+                    my_rec[q * (n_stages + 1) + ks] = v;
+                }
+            }
+            group_bar(group);
+            auto stage_live = [&](int ks) -> unsigned {
+                unsigned l = my_rec[ks].w;
+                if (NREC == 2) l |= my_rec[(n_stages + 1) + ks].w;
+                return l;
+            };
             for (int ks = 0; ks < n_stages; ++ks) {
-                if (!live_of(nt, ks)) continue;
+                if (!stage_live(ks)) continue;
+                const long long my_seq = seq++;
+                if ((int)(my_seq % NDEC_GROUPS) != group) continue;
+                const int stage = (int)(my_seq % STAGES);
+                const unsigned phase = (unsigned)((my_seq / STAGES) & 1);
                 if (!mbar_wait(smem_u32(&sm->empty[stage]), phase ^ 1u, abort)) ok = false;
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
 #pragma unroll
                 for (int q = 0; q < NREC; ++q) {
-                    const long long rt = nt * NREC + q;
-                    if (rt < p.n_rec_tiles) {
-                        const uint4 a = __ldg(reinterpret_cast<const uint4 *>(&recs[rt * n_stages + ks]));
-                        const uint4 b = __ldg(reinterpret_cast<const uint4 *>(&recs[rt * n_stages + ks + 1]));
+                    if (nt * NREC + q < p.n_rec_tiles) {
                         PackedRec r0, r1;
-                        r0.ubase = a.x; r0.dbase = a.y; r0.pbase = a.z; r0.live = a.w;
-                        r1.ubase = b.x; r1.dbase = b.y; r1.pbase = b.z; r1.live = b.w;
-                        decode_record<BW>(sB + stage * B_BYTES + q * REC_BYTES, r0, r1, p, tid, NTHR);
+                        rec_at(q, ks, &r0, &r1);
+                        decode_record<BW>(sB + stage * B_BYTES + q * REC_BYTES, r0, r1, p, tid);
                     }
                 }
                 fence_proxy_async();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(smem_u32(&sm->full_b[stage]));
-                if (++stage == STAGES) { stage = 0; phase ^= 1u; }
             }
         }
-    } else if (MODE == 1 && warp >= 6 + NDEC_WARPS) {
+    } else if (MODE == 1 && warp >= FIRST_GATHER_WARP) {
         // ---------------- im2col gather of the A tile (convolution) ----------------
-        const int r = threadIdx.x - (6 + NDEC_WARPS) * 32;      // row of the tile, 0..127
+        const int gw = warp - FIRST_GATHER_WARP;
+        const int r = threadIdx.x - FIRST_GATHER_WARP * 32;     // row of the tile, 0..127
         const unsigned short *X = reinterpret_cast<const unsigned short *>(p.X);
         int stage = 0;
         unsigned phase = 0;
@@ -484,13 +556,14 @@ mwu_gemm_kernel(const __grid_constant__ CUtensorMap tmap, const Params p) {
         const long long hw = (long long)p.OH * p.OW;
         for (long long t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
             const long long mt = t % m_tiles, nt = t / m_tiles;
+            load_live(sm->live_gather[gw], nt);
             const long long m = mt * BM + r;
             const bool row_ok = m < p.M;
             const long long img = row_ok ? m / hw : 0, pix = row_ok ? m % hw : 0;
             const int ih0 = (int)(pix / p.OW) * p.stride, iw0 = (int)(pix % p.OW) * p.stride;
             const long long xbase = img * (long long)p.C * p.H * p.W + (long long)ih0 * p.W + iw0;
             for (int ks = 0; ks < n_stages; ++ks) {
-                if (!live_of(nt, ks)) continue;
+                if (!sm->live_gather[gw][ks]) continue;
                 if (!mbar_wait(smem_u32(&sm->empty[stage]), phase ^ 1u, abort)) ok = false;
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
@@ -553,8 +626,9 @@ static EncodeTiledFn get_encode_fn() {
     return fn;
 }
 
-static size_t smem_bytes(int nrec, long long conv_k) {
-    return 1024 + (size_t)STAGES * (A_BYTES + nrec * REC_BYTES) + 256 + (size_t)conv_k * sizeof(int2);
+static size_t smem_bytes(int nrec, long long n_stages, long long conv_k) {
+    return 1024 + (size_t)STAGES * (A_BYTES + nrec * REC_BYTES) + ((sizeof(Smem) + 15) & ~(size_t)15) +
+           (size_t)NDEC_GROUPS * nrec * (n_stages + 1) * 16 + (size_t)conv_k * sizeof(int2);
 }
 
 template <int MODE, int NREC, int BW>
@@ -582,6 +656,7 @@ static void fill_common(Params &p, const mwu_proj_desc *desc, const void *packed
     p.packed = (const unsigned char *)packed;
     p.off_rec = L.off_rec; p.off_ulist = L.off_ulist; p.off_dpos = L.off_dpos;
     p.off_dpay = L.off_dpay; p.off_ppos = L.off_ppos;
+    p.n_unified = (unsigned)L.n_unified; p.n_dense = (unsigned)L.n_dense; p.n_plist = (unsigned)L.n_plist;
     p.n_rec_tiles = L.n_tiles;
     p.n_stages = L.n_stages;
     p.N = desc->rows;
@@ -632,7 +707,8 @@ extern "C" int mwu_gemm(const mwu_proj_desc *desc, const void *packed, const voi
     const int nrec = p.n_rec_tiles >= 2 ? 2 : 1;
     const long long tiles = ((M + BM - 1) / BM) * ((p.n_rec_tiles + nrec - 1) / nrec);
     const int grid = (int)(tiles < sm_count ? tiles : sm_count);
-    const size_t smem = smem_bytes(nrec, 0);
+    const size_t smem = smem_bytes(nrec, p.n_stages, 0);
+    if (p.n_stages > MAX_STAGES_K || smem > 227 * 1024) return MWU_ERR_SHAPE;
     cudaStream_t st = (cudaStream_t)cuda_stream;
     cudaError_t e = (nrec == 2) ? launch_bw<0, 2>(desc->block, tmap, p, grid, smem, st)
                                 : launch_bw<0, 1>(desc->block, tmap, p, grid, smem, st);
@@ -670,8 +746,8 @@ extern "C" int mwu_conv_implicit(const mwu_proj_desc *desc, const void *packed, 
     p.M = (long long)n * p.OH * p.OW;
     p.ldy = 0;
     const int nrec = p.n_rec_tiles >= 2 ? 2 : 1;
-    const size_t smem = smem_bytes(nrec, desc->cols);
-    if (smem > 227 * 1024) return MWU_ERR_SHAPE;
+    const size_t smem = smem_bytes(nrec, p.n_stages, desc->cols);
+    if (p.n_stages > MAX_STAGES_K || smem > 227 * 1024) return MWU_ERR_SHAPE;
     const long long tiles = ((p.M + BM - 1) / BM) * ((p.n_rec_tiles + nrec - 1) / nrec);
     const int grid = (int)(tiles < sm_count ? tiles : sm_count);
     CUtensorMap tmap;
