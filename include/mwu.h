@@ -110,20 +110,24 @@ int mwu_project(const mwu_proj_desc *desc, const float *W, const float *U_dual, 
  *
  * Needs cols % 64 == 0.  Inputs are mwu_project's inputs and outputs for the same desc.
  * `packed` receives exactly mwu_packed_bytes(desc) bytes (256-byte aligned buffer).  A record is
- * a row tile of 128 rows x 64 columns; it has 128 * 64/block block slots with slot code
- * pos = row_in_tile * (64/block) + block_in_record.  Per record the blocks are listed by class,
- * each list in ascending pos order, records in tile-major order:
- *   header  256 B : u64 magic "MWUPACK1", version 2, rows, cols, block, rows_padded, n_tiles,
+ * a row tile of 128 rows x 64 columns; it has 128 * 64/block block slots, numbered
+ * pos = row_in_tile * (64/block) + block_in_record.  A block is addressed by `off`, the byte
+ * offset of its first value in the record's decoded bf16 tile as the GEMM lays it out in shared
+ * memory: row r starts at (r/8)*1024 + (r%8)*128 and its 16-byte chunk c sits at chunk position
+ * c ^ (r%8).  Per record the blocks are listed by class, each list in ascending pos order,
+ * records in tile-major order:
+ *   header  256 B : u64 magic "MWUPACK1", version 3, rows, cols, block, rows_padded, n_tiles,
  *                   n_stages, n_pruned, n_unified, n_dense, n_plist, byte offsets of rec, ulist,
  *                   dpos, dpay, ppos, total bytes
  *   rec     16 B per record plus one closing entry: u32 ubase, dbase, pbase (index of the
  *                   record's first entry in ulist, dpos/dpay, ppos; the closing entry holds the
  *                   totals), u32 live (bit s set if some row has a non-pruned block overlapping
  *                   columns [16s,16s+16) of the record)
- *   ulist   8 B per unified block: u32 (pos | sign bits << 16; bit l = (v_l < 0)), fp32 value
- *   dpos    u16 pos per remaining non-pruned ("dense") block
+ *   ulist   8 B per unified block: u32 sign bits, weight l at bit l/2 + 16*(l%2) (set when
+ *                   v_l < 0); u16 off; u16 bf16(unified value), round to nearest even
+ *   dpos    u16 off per remaining non-pruned ("dense") block
  *   dpay    the dense block's `block` values as bf16 (round to nearest even), same order
- *   ppos    u16 pos per pruned block
+ *   ppos    u16 off per pruned block
  * Rows beyond `rows` up to the next multiple of 128 are padding and are listed as pruned
  * (n_plist = n_pruned + padding blocks).  Sections start on 256-byte boundaries, gaps are
  * zero.  A mismatch between the bitmaps and desc's counts sets MWU_DEV_BOUNDS.

@@ -48,7 +48,7 @@ STAGE_K = 64             # reduction-axis extent per record
 HEADER_BYTES = 256
 SECTION_ALIGN = 256
 MAGIC = b"MWUPACK1"
-VERSION = 2
+VERSION = 3
 
 
 def count_from_permille(n_blocks: int, permille: int) -> int:
@@ -205,6 +205,25 @@ def packed_layout(N: int, K: int, b: int, n_unified: int, n_dense: int, n_pruned
                 total=total)
 
 
+def tile_offset(pos: np.ndarray, b: int) -> np.ndarray:
+    """Byte offset of block slot `pos` in a decoded 128 x 64 bf16 tile: row r = pos // (64/b)
+    starts at (r // 8) * 1024 + (r % 8) * 128; the row's 16-byte chunk c is stored at chunk
+    position c XOR (r % 8); inside a chunk bytes keep their order."""
+    pos = np.asarray(pos, dtype=np.int64)
+    nb = STAGE_K // b
+    r, i = pos // nb, pos % nb
+    byte_in_row = i * 2 * b
+    c, within = byte_in_row // 16, byte_in_row % 16
+    return (r // 8) * 1024 + (r % 8) * 128 + ((c ^ (r % 8)) * 16) + within
+
+
+def tile_offset_inverse(off: int, b: int):
+    r = (off >> 10) * 8 + ((off >> 7) & 7)
+    c = ((off >> 4) & 7) ^ (r & 7)
+    byte_in_row = c * 16 + (off & 15)
+    return r, byte_in_row // (2 * b)
+
+
 HEADER_FIELDS = ["magic", "version", "N", "K", "b", "n_pad", "n_tiles", "n_stages", "n_pruned",
                  "n_unified", "n_dense", "n_plist", "off_rec", "off_ulist", "off_dpos", "off_dpay",
                  "off_ppos", "total"]
@@ -214,11 +233,15 @@ def pack(p: Projection, b: int) -> np.ndarray:
     """Serialise a projection into the packed byte format (uint8 array).
 
     A record is (row tile of 128 rows) x (64 reduction-axis entries) and holds 128 * 64/b
-    block slots; slot code pos = row_in_tile * (64/b) + block_in_stage.  Per record the blocks
-    are listed by class, each list in ascending pos order:
-      ulist  8 B per unified block: u32 (pos | sign bits << 16), fp32 unified value
-      dpos   u16 pos per dense block;  dpay  its b values as bf16 (round to nearest even)
-      ppos   u16 pos per pruned block (rows beyond N are padding and count as pruned)
+    block slots; slot number pos = row_in_tile * (64/b) + block_in_stage.  A block is addressed
+    by the byte offset `off` of its first value inside the record's decoded tile (bf16, rows of
+    128 bytes, 16-byte chunks of a row XOR-permuted by the row number mod 8 -- the layout the
+    tensor-core instruction reads; see tile_offset).  Per record the blocks are listed by
+    class, each list in ascending pos order:
+      ulist  8 B per unified block: u32 spread sign bits (weight l -> bit l//2 + 16*(l%2)),
+             u16 off, u16 bf16(unified value)
+      dpos   u16 off per dense block;  dpay  its b values as bf16 (round to nearest even)
+      ppos   u16 off per pruned block (rows beyond N are padding and count as pruned)
     rec[i] = (u32 ubase, dbase, pbase, live) gives where record i starts in each list; rec has
     one extra entry holding the totals.  live bit s = some row of the record has a non-pruned
     block overlapping columns [16s, 16s+16).
@@ -252,7 +275,9 @@ def pack(p: Projection, b: int) -> np.ndarray:
     rec = np.zeros((n_rec + 1, 4), dtype=np.uint32)
     ulist_w0, ulist_u, dpos, dpay, ppos = [], [], [], [], []
     n_u = n_d = n_p = 0
-    bitw = (np.uint32(1) << np.arange(b, dtype=np.uint32))
+    ell = np.arange(b, dtype=np.uint32)
+    bitw = (np.uint32(1) << (ell // 2 + 16 * (ell % 2)))           # spread sign bit of weight l
+    ubf = bf16_bits_rne(u.reshape(-1)).reshape(u.shape).astype(np.uint32)
     for t in range(n_tiles):
         r0 = t * TILE_ROWS
         for s in range(n_stages):
@@ -272,12 +297,13 @@ def pack(p: Projection, b: int) -> np.ndarray:
             pos_p = np.flatnonzero(P.reshape(-1)).astype(np.uint16)
             sg = sign[r0:r0 + TILE_ROWS, s * STAGE_K:(s + 1) * STAGE_K].reshape(TILE_ROWS * nb, b)
             sbits = (sg.astype(np.uint32) * bitw).sum(axis=1).astype(np.uint32)
-            ulist_w0.append(pos_u | (sbits[pos_u] << np.uint32(16)))
-            ulist_u.append(u[r0:r0 + TILE_ROWS, s * nb:(s + 1) * nb].reshape(-1)[pos_u])
-            dpos.append(pos_d)
+            ulist_w0.append(sbits[pos_u])
+            ub = ubf[r0:r0 + TILE_ROWS, s * nb:(s + 1) * nb].reshape(-1)[pos_u]
+            ulist_u.append(tile_offset(pos_u, b).astype(np.uint32) | (ub << np.uint32(16)))
+            dpos.append(tile_offset(pos_d, b).astype(np.uint16))
             vb = vbf[r0:r0 + TILE_ROWS, s * STAGE_K:(s + 1) * STAGE_K].reshape(TILE_ROWS * nb, b)
             dpay.append(vb[pos_d].reshape(-1))
-            ppos.append(pos_p)
+            ppos.append(tile_offset(pos_p, b).astype(np.uint16))
             n_u += pos_u.shape[0]
             n_d += pos_d.shape[0]
             n_p += pos_p.shape[0]
@@ -292,7 +318,7 @@ def pack(p: Projection, b: int) -> np.ndarray:
     if n_unified:
         ul = np.zeros((n_unified, 2), dtype=np.uint32)
         ul[:, 0] = np.concatenate(ulist_w0)
-        ul[:, 1] = np.concatenate(ulist_u).astype(np.float32).view(np.uint32)
+        ul[:, 1] = np.concatenate(ulist_u)
         put(L["off_ulist"], ul)
     if n_dense:
         put(L["off_dpos"], np.concatenate(dpos).astype(np.uint16))
@@ -330,18 +356,18 @@ def decode(buf: np.ndarray) -> np.ndarray:
         for s in range(n_stages):
             ri = t * n_stages + s
             for e in range(int(rec[ri, 0]), int(rec[ri + 1, 0])):
-                w0 = int(ulist[e, 0])
-                pos, sbits = w0 & 0xFFFF, w0 >> 16
-                uval = float(bf16_bits_to_f64(bf16_bits_rne(ulist[e:e + 1, 1].view(np.float32)))[0])
-                r, i = divmod(pos, nb)
+                sbits, w1 = int(ulist[e, 0]), int(ulist[e, 1])
+                uval = float(bf16_bits_to_f64(np.array([w1 >> 16], dtype=np.uint16))[0])
+                r, i = tile_offset_inverse(w1 & 0xFFFF, b)
                 for l in range(b):
-                    What[t * TILE_ROWS + r, s * STAGE_K + i * b + l] = -uval if (sbits >> l) & 1 else uval
+                    neg = (sbits >> (l // 2 + 16 * (l % 2))) & 1
+                    What[t * TILE_ROWS + r, s * STAGE_K + i * b + l] = -uval if neg else uval
             for e in range(int(rec[ri, 1]), int(rec[ri + 1, 1])):
-                r, i = divmod(int(dpos[e]), nb)
+                r, i = tile_offset_inverse(int(dpos[e]), b)
                 k0 = s * STAGE_K + i * b
                 What[t * TILE_ROWS + r, k0:k0 + b] = bf16_bits_to_f64(dpay[e * b:(e + 1) * b])
             for e in range(int(rec[ri, 2]), int(rec[ri + 1, 2])):
-                r, i = divmod(int(ppos[e]), nb)
+                r, i = tile_offset_inverse(int(ppos[e]), b)
                 k0 = s * STAGE_K + i * b
                 What[t * TILE_ROWS + r, k0:k0 + b] = 0.0
     assert not np.isnan(What).any()

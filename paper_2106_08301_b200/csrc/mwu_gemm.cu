@@ -157,30 +157,9 @@ __device__ __forceinline__ unsigned swz(unsigned r, unsigned c) {
 // ------------------------------------------------------------------------------------------
 // decode of one record's class lists into its 128 x 64 tile
 // ------------------------------------------------------------------------------------------
-__device__ __forceinline__ unsigned sign_word(unsigned u2, unsigned sbits, int w) {
-    const unsigned t = (sbits >> (2 * w)) & 3u;          // signs of weights 2w, 2w+1
-    return ((t * 0x40008000u) & 0x80008000u) ^ u2;        // bit0 -> bit 15, bit1 -> bit 31
-}
-
-template <int BW>
-__device__ __forceinline__ void store_block(unsigned char *tile, unsigned pos, const unsigned (&w)[8]) {
-    constexpr int NBK = BK / BW;
-    const unsigned r = pos / NBK, i = pos % NBK;
-    if (BW == 16) {
-        const unsigned a = swz(r, 2 * i);
-        *reinterpret_cast<uint4 *>(tile + a) = make_uint4(w[0], w[1], w[2], w[3]);
-        *reinterpret_cast<uint4 *>(tile + (a ^ 16u)) = make_uint4(w[4], w[5], w[6], w[7]);
-    } else if (BW == 8) {
-        *reinterpret_cast<uint4 *>(tile + swz(r, i)) = make_uint4(w[0], w[1], w[2], w[3]);
-    } else if (BW == 4) {
-        *reinterpret_cast<uint2 *>(tile + swz(r, i >> 1) + (i & 1) * 8) = make_uint2(w[0], w[1]);
-    } else {
-        *reinterpret_cast<unsigned *>(tile + swz(r, i >> 2) + (i & 3) * 4) = w[0];
-    }
-}
-
-// One record = 128 * 64/BW block slots, listed as [pruned | dense | unified].  Thread `tid` of
-// the 256 takes flattened entries tid, tid+256, ...: a fixed count, so all loads issue first.
+// One record = 128 * 64/BW block slots, listed as [pruned | dense | unified]; every entry names
+// the byte offset of its block in the tile.  Thread `tid` of a decode group takes flattened
+// entries tid, tid+NDEC_THREADS, ...: a fixed count, so all loads issue before the first store.
 template <int BW>
 __device__ __forceinline__ void decode_record(unsigned char *tile, const PackedRec r0, const PackedRec r1,
                                               const Params &p, int tid) {
@@ -188,69 +167,70 @@ __device__ __forceinline__ void decode_record(unsigned char *tile, const PackedR
     constexpr int SLOTS = kTileRows * NBK;
     constexpr int ENT = SLOTS / NDEC_THREADS;
     constexpr int WORDS = BW / 2;                           // 32-bit words per block
+    constexpr unsigned OFF_MASK = (unsigned)(REC_BYTES - 1) & ~(unsigned)((BW >= 8 ? 16 : 2 * BW) - 1);
     const uint2 *ulist = reinterpret_cast<const uint2 *>(p.packed + p.off_ulist);
     const unsigned short *dpos = reinterpret_cast<const unsigned short *>(p.packed + p.off_dpos);
     const unsigned char *dpay = p.packed + p.off_dpay;
     const unsigned short *ppos = reinterpret_cast<const unsigned short *>(p.packed + p.off_ppos);
     const unsigned n_p = r1.pbase - r0.pbase, n_d = r1.dbase - r0.dbase, n_u = r1.ubase - r0.ubase;
-    unsigned meta[ENT], uval[ENT];
-    unsigned pay[ENT][WORDS];
+    unsigned off[ENT];                                      // 0xffffffff: nothing to write
+    unsigned w[ENT][WORDS];
 #pragma unroll
     for (int k = 0; k < ENT; ++k) {
         const unsigned f = (unsigned)tid + (unsigned)k * NDEC_THREADS;
-        meta[k] = 0xffffffffu;                              // nothing to write
-        uval[k] = 0;
+        off[k] = 0xffffffffu;
 #pragma unroll
-        for (int w = 0; w < WORDS; ++w) pay[k][w] = 0;
+        for (int q = 0; q < WORDS; ++q) w[k][q] = 0u;
         if (f < n_p) {
             const unsigned e = r0.pbase + f;
-            if (e < p.n_plist) meta[k] = __ldg(ppos + e);
+            if (e < p.n_plist) off[k] = __ldg(ppos + e);
         } else if (f < n_p + n_d) {
             const unsigned e = r0.dbase + (f - n_p);
             if (e < p.n_dense) {
-                meta[k] = __ldg(dpos + e);
+                off[k] = __ldg(dpos + e);
                 const unsigned char *src = dpay + (size_t)e * (2 * BW);
                 if (BW == 16) {
                     const uint4 v0 = __ldg(reinterpret_cast<const uint4 *>(src));
                     const uint4 v1 = __ldg(reinterpret_cast<const uint4 *>(src + 16));
-                    pay[k][0] = v0.x; pay[k][1] = v0.y; pay[k][2] = v0.z; pay[k][3] = v0.w;
-                    pay[k][4 % WORDS] = v1.x; pay[k][5 % WORDS] = v1.y; pay[k][6 % WORDS] = v1.z; pay[k][7 % WORDS] = v1.w;
+                    w[k][0] = v0.x; w[k][1 % WORDS] = v0.y; w[k][2 % WORDS] = v0.z; w[k][3 % WORDS] = v0.w;
+                    w[k][4 % WORDS] = v1.x; w[k][5 % WORDS] = v1.y; w[k][6 % WORDS] = v1.z; w[k][7 % WORDS] = v1.w;
                 } else if (BW == 8) {
                     const uint4 v0 = __ldg(reinterpret_cast<const uint4 *>(src));
-                    pay[k][0] = v0.x; pay[k][1 % WORDS] = v0.y; pay[k][2 % WORDS] = v0.z; pay[k][3 % WORDS] = v0.w;
+                    w[k][0] = v0.x; w[k][1 % WORDS] = v0.y; w[k][2 % WORDS] = v0.z; w[k][3 % WORDS] = v0.w;
                 } else if (BW == 4) {
                     const uint2 v0 = __ldg(reinterpret_cast<const uint2 *>(src));
-                    pay[k][0] = v0.x; pay[k][1 % WORDS] = v0.y;
+                    w[k][0] = v0.x; w[k][1 % WORDS] = v0.y;
                 } else {
-                    pay[k][0] = __ldg(reinterpret_cast<const unsigned *>(src));
+                    w[k][0] = __ldg(reinterpret_cast<const unsigned *>(src));
                 }
             }
         } else if (f < n_p + n_d + n_u) {
             const unsigned e = r0.ubase + (f - n_p - n_d);
             if (e < p.n_unified) {
-                const uint2 ent = __ldg(ulist + e);
-                meta[k] = ent.x;
-                uval[k] = ent.y;
+                const uint2 ent = __ldg(ulist + e);          // x: spread signs, y: off | bf16(u) << 16
+                off[k] = ent.y & 0xffffu;
+                const unsigned u2 = __byte_perm(ent.y, 0u, 0x3232);      // bf16(u) in both halves
+#pragma unroll
+                for (int q = 0; q < WORDS; ++q)              // weights 2q, 2q+1: sign bits q and 16+q
+                    w[k][q] = ((ent.x << (15 - q)) & 0x80008000u) ^ u2;
             }
         }
     }
 #pragma unroll
     for (int k = 0; k < ENT; ++k) {
-        const unsigned f = (unsigned)tid + (unsigned)k * NDEC_THREADS;
-        if (meta[k] == 0xffffffffu) continue;
-        const unsigned pos = meta[k] & (SLOTS - 1);
-        unsigned w[8];
-        if (f >= n_p + n_d) {
-            const unsigned sbits = meta[k] >> 16;
-            const unsigned u1 = (unsigned)__bfloat16_as_ushort(__float2bfloat16_rn(__uint_as_float(uval[k])));
-            const unsigned u2 = u1 | (u1 << 16);
-#pragma unroll
-            for (int q = 0; q < 8; ++q) w[q] = (q < WORDS) ? sign_word(u2, sbits, q) : 0u;
+        if (off[k] == 0xffffffffu) continue;
+        unsigned char *dst = tile + (off[k] & OFF_MASK);
+        if (BW == 16) {
+            *reinterpret_cast<uint4 *>(dst) = make_uint4(w[k][0], w[k][1 % WORDS], w[k][2 % WORDS], w[k][3 % WORDS]);
+            *reinterpret_cast<uint4 *>(tile + ((off[k] & OFF_MASK) ^ 16u)) =
+                make_uint4(w[k][4 % WORDS], w[k][5 % WORDS], w[k][6 % WORDS], w[k][7 % WORDS]);
+        } else if (BW == 8) {
+            *reinterpret_cast<uint4 *>(dst) = make_uint4(w[k][0], w[k][1 % WORDS], w[k][2 % WORDS], w[k][3 % WORDS]);
+        } else if (BW == 4) {
+            *reinterpret_cast<uint2 *>(dst) = make_uint2(w[k][0], w[k][1 % WORDS]);
         } else {
-#pragma unroll
-            for (int q = 0; q < 8; ++q) w[q] = (q < WORDS) ? pay[k][q % WORDS] : 0u;
+            *reinterpret_cast<unsigned *>(dst) = w[k][0];
         }
-        store_block<BW>(tile, pos, w);
     }
 }
 

@@ -46,6 +46,21 @@ __device__ __forceinline__ void row_masks(const Params &p, long long tile, long 
     }
 }
 
+// byte offset of block i of row r inside the record's decoded tile: rows of 128 bytes, the
+// row's 16-byte chunks XOR-permuted by r % 8 (the layout the tensor-core instruction reads)
+__device__ __forceinline__ unsigned tile_offset(unsigned r, unsigned i, int b) {
+    const unsigned byte_in_row = i * 2u * (unsigned)b;
+    const unsigned c = byte_in_row >> 4, within = byte_in_row & 15u;
+    return (r >> 3) * 1024u + (r & 7u) * 128u + ((c ^ (r & 7u)) << 4) + within;
+}
+
+// sign bits of one block (bit l = weight l) -> bit l/2 + 16 * (l % 2)
+__device__ __forceinline__ unsigned spread_signs(unsigned sb, int b) {
+    unsigned out = 0;
+    for (int l = 0; l < b; ++l) out |= ((sb >> l) & 1u) << (l / 2 + 16 * (l & 1));
+    return out;
+}
+
 __device__ __forceinline__ unsigned live_of(unsigned P, int b) {
     const int nb = kStageK / b;
     const unsigned mask = (nb >= 32) ? 0xffffffffu : ((1u << nb) - 1u);
@@ -127,7 +142,7 @@ __global__ void __launch_bounds__(1024) scan_kernel(Params p) {
         unsigned long long v = 0;
         switch (threadIdx.x) {
             case 0: v = kMagic; break;
-            case 1: v = 2; break;
+            case 1: v = 3; break;
             case 2: v = (unsigned long long)p.rows; break;
             case 3: v = (unsigned long long)p.cols; break;
             case 4: v = (unsigned long long)p.b; break;
@@ -192,20 +207,21 @@ __global__ void __launch_bounds__(128) fill_kernel(Params p) {
         unsigned long long ui = ubase + eu, di = dbase + ed, pi = pbase + ep;
         const unsigned bmask = (b >= 32) ? 0xffffffffu : ((1u << b) - 1u);
         for (int i = 0; i < nb; ++i) {
-            const unsigned pos = (unsigned)(r * nb + i);
+            const unsigned off = tile_offset((unsigned)r, (unsigned)i, b);
             if ((U >> i) & 1u) {
                 const unsigned sb = (unsigned)(sgn >> (i * b)) & bmask;
                 const long long j = n * (p.cols / b) + stage * nb + i;
+                const unsigned ub = (unsigned)__bfloat16_as_ushort(__float2bfloat16_rn(p.u[j]));
                 if (ui < (unsigned long long)p.L.n_unified)
-                    ulist[ui] = make_uint2(pos | (sb << 16), __float_as_uint(p.u[j]));
+                    ulist[ui] = make_uint2(spread_signs(sb, b), off | (ub << 16));
                 else bad = true;
                 ++ui;
             } else if ((D >> i) & 1u) {
-                if (di < (unsigned long long)p.L.n_dense) dpos[di] = (unsigned short)pos;
+                if (di < (unsigned long long)p.L.n_dense) dpos[di] = (unsigned short)off;
                 else bad = true;
                 ++di;
             } else {
-                if (pi < (unsigned long long)p.L.n_plist) ppos[pi] = (unsigned short)pos;
+                if (pi < (unsigned long long)p.L.n_plist) ppos[pi] = (unsigned short)off;
                 else bad = true;
                 ++pi;
             }

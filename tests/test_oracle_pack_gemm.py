@@ -79,8 +79,10 @@ def test_live_mask_and_padding():
     assert h["n_plist"] == kp + 28 * (K // b)                           # padding rows pruned
     ppos = buf[h["off_ppos"]:h["off_ppos"] + 2 * h["n_plist"]].view(np.uint16)
     first = ppos[rec[0, 2]:rec[1, 2]]
-    assert np.all(np.diff(first.astype(int)) > 0)                       # ascending slot codes
-    assert set(range(100 * nb, 128 * nb)) <= set(first.tolist())
+    slots = [O.tile_offset_inverse(int(o), b) for o in first]
+    codes = [r * nb + i for r, i in slots]
+    assert np.all(np.diff(codes) > 0)                                   # ascending slot numbers
+    assert set(range(100 * nb, 128 * nb)) <= set(codes)
     assert rec[2].tolist() == [h["n_unified"], h["n_dense"], h["n_plist"], 0]
     assert O.decode(buf).shape == (N, K)
 
@@ -143,3 +145,19 @@ def test_conv_against_library_and_im2col():
     ref2 = torch.nn.functional.conv2d(torch.from_numpy(x),
                                       torch.from_numpy(What).reshape(Oc, C, 3, 3), stride=2)
     assert np.allclose(y2, ref2.numpy(), rtol=1e-12, atol=1e-14)
+
+
+def test_tile_offset_is_a_bijection_and_matches_the_swizzle():
+    for b in (2, 4, 8, 16):
+        nb = 64 // b
+        pos = np.arange(128 * nb)
+        off = O.tile_offset(pos, b)
+        g = min(2 * b, 16)          # a block wider than a chunk starts on a chunk boundary
+        assert off.min() == 0 and off.max() == 16384 - g
+        assert len(set(off.tolist())) == pos.size and np.all(off % g == 0)
+        back = [O.tile_offset_inverse(int(o), b) for o in off]
+        assert [r * nb + i for r, i in back] == pos.tolist()
+    # row 0 is not permuted; row 1 swaps neighbouring chunks; rows 8.. start 1024 bytes later
+    assert O.tile_offset(np.array([0, 1, 2, 3]), 16).tolist() == [0, 32, 64, 96]
+    assert O.tile_offset(np.array([4, 5]), 16).tolist() == [128 + 16, 128 + 48]
+    assert O.tile_offset(np.array([32]), 16).tolist() == [1024]
