@@ -5,9 +5,9 @@
 //   count_kernel  one CTA per record (128 rows x 64 columns): number of unified / dense / pruned
 //                 blocks and the record's live-slice mask.
 //   scan_kernel   one CTA: exclusive scan of the per-record counts over all records, header.
-//   fill_kernel   one CTA per record: per-row class masks, scan over the rows, then the three
-//                 class lists; the dense payload is written warp-per-row so that every row
-//                 segment (256 contiguous bytes of W) is read with one coalesced request.
+//   fill_kernel   one CTA per record, one thread per row: class masks, scan over the rows, then
+//                 the row's entries of the three class lists; a dense block's values are read
+//                 as whole 64-byte (or shorter) runs of W and written as one bf16 vector.
 #include "mwu_common.cuh"
 
 namespace mwu {
@@ -105,13 +105,21 @@ __global__ void __launch_bounds__(128) count_kernel(Params p) {
 
 __global__ void __launch_bounds__(1024) scan_kernel(Params p) {
     const long long n_rec = p.L.n_tiles * p.L.n_stages;
-    PackedRec *recs = reinterpret_cast<PackedRec *>(p.packed + p.L.off_rec);
+    uint4 *recs = reinterpret_cast<uint4 *>(p.packed + p.L.off_rec);     // ubase, dbase, pbase, live
     __shared__ unsigned long long s_u[1024], s_d[1024], s_p[1024];
     const long long per = (n_rec + 1023) / 1024;
     const long long lo = threadIdx.x * per;
     const long long hi = (lo + per < n_rec) ? lo + per : n_rec;
+    constexpr int KEEP = 8;                                 // records held in registers
+    uint4 held[KEEP];
     unsigned long long su = 0, sd = 0, sp = 0;
-    for (long long i = lo; i < hi; ++i) { su += recs[i].ubase; sd += recs[i].dbase; sp += recs[i].pbase; }
+#pragma unroll
+    for (int k = 0; k < KEEP; ++k) {
+        held[k] = make_uint4(0, 0, 0, 0);
+        if (lo + k < hi) held[k] = recs[lo + k];
+        su += held[k].x; sd += held[k].y; sp += held[k].z;
+    }
+    for (long long i = lo + KEEP; i < hi; ++i) { const uint4 v = recs[i]; su += v.x; sd += v.y; sp += v.z; }
     s_u[threadIdx.x] = su; s_d[threadIdx.x] = sd; s_p[threadIdx.x] = sp;
     __syncthreads();
     for (int off = 1; off < 1024; off <<= 1) {
@@ -124,18 +132,24 @@ __global__ void __launch_bounds__(1024) scan_kernel(Params p) {
         __syncthreads();
     }
     unsigned long long ru = s_u[threadIdx.x] - su, rd = s_d[threadIdx.x] - sd, rp = s_p[threadIdx.x] - sp;
-    for (long long i = lo; i < hi; ++i) {
-        const unsigned cu = recs[i].ubase, cd = recs[i].dbase, cp = recs[i].pbase;
-        recs[i].ubase = (unsigned)ru; recs[i].dbase = (unsigned)rd; recs[i].pbase = (unsigned)rp;
-        ru += cu; rd += cd; rp += cp;
+#pragma unroll
+    for (int k = 0; k < KEEP; ++k) {
+        if (lo + k < hi) {
+            recs[lo + k] = make_uint4((unsigned)ru, (unsigned)rd, (unsigned)rp, held[k].w);
+            ru += held[k].x; rd += held[k].y; rp += held[k].z;
+        }
+    }
+    for (long long i = lo + KEEP; i < hi; ++i) {
+        const uint4 v = recs[i];
+        recs[i] = make_uint4((unsigned)ru, (unsigned)rd, (unsigned)rp, v.w);
+        ru += v.x; rd += v.y; rp += v.z;
     }
     if (threadIdx.x == 1023) {
         const unsigned long long tu = s_u[1023], td = s_d[1023], tp = s_p[1023];
         if (tu != (unsigned long long)p.L.n_unified || td != (unsigned long long)p.L.n_dense ||
             tp != (unsigned long long)p.L.n_plist)
             atomicOr(p.dev_status, (unsigned)MWU_DEV_BOUNDS);
-        recs[n_rec].ubase = (unsigned)tu; recs[n_rec].dbase = (unsigned)td;
-        recs[n_rec].pbase = (unsigned)tp; recs[n_rec].live = 0;
+        recs[n_rec] = make_uint4((unsigned)tu, (unsigned)td, (unsigned)tp, 0u);
     }
     if (threadIdx.x < 32) {
         unsigned long long *h = reinterpret_cast<unsigned long long *>(p.packed);
@@ -165,26 +179,25 @@ __global__ void __launch_bounds__(1024) scan_kernel(Params p) {
     }
 }
 
+template <int B>
 __global__ void __launch_bounds__(128) fill_kernel(Params p) {
+    constexpr int NBK = kStageK / B;
+    constexpr unsigned MASK = (NBK >= 32) ? 0xffffffffu : ((1u << NBK) - 1u);
     const long long rec = blockIdx.x;
     const long long tile = rec / p.L.n_stages, stage = rec % p.L.n_stages;
     const int r = threadIdx.x, lane = r & 31, warp = r >> 5;
-    const int b = p.b;
-    const int nb = kStageK / b;
-    const unsigned mask = (nb >= 32) ? 0xffffffffu : ((1u << nb) - 1u);
     const PackedRec *recs = reinterpret_cast<const PackedRec *>(p.packed + p.L.off_rec);
     uint2 *ulist = reinterpret_cast<uint2 *>(p.packed + p.L.off_ulist);
     unsigned short *dpos = reinterpret_cast<unsigned short *>(p.packed + p.L.off_dpos);
-    __nv_bfloat162 *dpay = reinterpret_cast<__nv_bfloat162 *>(p.packed + p.L.off_dpay);
+    unsigned char *dpay = p.packed + p.L.off_dpay;
     unsigned short *ppos = reinterpret_cast<unsigned short *>(p.packed + p.L.off_ppos);
     const unsigned long long ubase = recs[rec].ubase, dbase = recs[rec].dbase, pbase = recs[rec].pbase;
 
-    __shared__ unsigned s_D[kTileRows], s_doff[kTileRows];
     __shared__ unsigned s_w[3][4];
     unsigned P, U;
     unsigned long long sgn;
     row_masks(p, tile, stage, r, &P, &U, &sgn);
-    const unsigned D = ~P & ~U & mask;
+    const unsigned D = ~P & ~U & MASK;
     const unsigned cu = __popc(U), cd = __popc(D), cp = __popc(P);
     unsigned iu = cu, id = cd, ip = cp;
     for (int off = 1; off < 32; off <<= 1) {
@@ -197,57 +210,68 @@ __global__ void __launch_bounds__(128) fill_kernel(Params p) {
     __syncthreads();
     unsigned bu = 0, bd = 0, bp = 0;
     for (int w = 0; w < warp; ++w) { bu += s_w[0][w]; bd += s_w[1][w]; bp += s_w[2][w]; }
-    const unsigned eu = bu + iu - cu, ed = bd + id - cd, ep = bp + ip - cp;   // exclusive over rows
-    s_D[r] = D;
-    s_doff[r] = ed;
+    unsigned long long ui = ubase + (bu + iu - cu), di = dbase + (bd + id - cd), pi = pbase + (bp + ip - cp);
     bool bad = false;
     const long long n = tile * kTileRows + r;
-    // unified, dense-position and pruned lists: one thread per row, ascending pos
-    {
-        unsigned long long ui = ubase + eu, di = dbase + ed, pi = pbase + ep;
-        const unsigned bmask = (b >= 32) ? 0xffffffffu : ((1u << b) - 1u);
-        for (int i = 0; i < nb; ++i) {
-            const unsigned off = tile_offset((unsigned)r, (unsigned)i, b);
-            if ((U >> i) & 1u) {
-                const unsigned sb = (unsigned)(sgn >> (i * b)) & bmask;
-                const long long j = n * (p.cols / b) + stage * nb + i;
-                const unsigned ub = (unsigned)__bfloat16_as_ushort(__float2bfloat16_rn(p.u[j]));
-                if (ui < (unsigned long long)p.L.n_unified)
-                    ulist[ui] = make_uint2(spread_signs(sb, b), off | (ub << 16));
-                else bad = true;
-                ++ui;
-            } else if ((D >> i) & 1u) {
-                if (di < (unsigned long long)p.L.n_dense) dpos[di] = (unsigned short)off;
-                else bad = true;
-                ++di;
-            } else {
-                if (pi < (unsigned long long)p.L.n_plist) ppos[pi] = (unsigned short)off;
-                else bad = true;
-                ++pi;
-            }
-        }
-    }
-    __syncthreads();
-    // dense payload: each warp walks its 32 rows, lanes cover the 64 columns two at a time
-    for (int rr = 0; rr < 32; ++rr) {
-        const int row = warp * 32 + rr;
-        const long long nn = tile * kTileRows + row;
-        if (nn >= p.rows) break;
-        const unsigned Dr = s_D[row];
-        if (!Dr) continue;
-        const long long f = nn * p.cols + stage * kStageK + 2 * lane;
-        float2 v = __ldg(reinterpret_cast<const float2 *>(p.W + f));
-        if (p.U) {
-            const float2 d = __ldg(reinterpret_cast<const float2 *>(p.U + f));
-            v.x = __fadd_rn(v.x, d.x);
-            v.y = __fadd_rn(v.y, d.y);
-        }
-        const int i = (2 * lane) / b;
-        if ((Dr >> i) & 1u) {
-            const unsigned long long di = dbase + s_doff[row] + __popc(Dr & ((1u << i) - 1u));
-            if (di < (unsigned long long)p.L.n_dense)
-                dpay[(di * b + (2 * lane - i * b)) >> 1] = __floats2bfloat162_rn(v.x, v.y);
+    constexpr unsigned BMASK = (B >= 32) ? 0xffffffffu : ((1u << B) - 1u);
+#pragma unroll 4
+    for (int i = 0; i < NBK; ++i) {
+        const unsigned off = tile_offset((unsigned)r, (unsigned)i, B);
+        if ((U >> i) & 1u) {
+            const unsigned sb = (unsigned)(sgn >> (i * B)) & BMASK;
+            const long long j = n * (p.cols / B) + stage * NBK + i;
+            const unsigned ub = (unsigned)__bfloat16_as_ushort(__float2bfloat16_rn(__ldg(p.u + j)));
+            if (ui < (unsigned long long)p.L.n_unified) ulist[ui] = make_uint2(spread_signs(sb, B), off | (ub << 16));
             else bad = true;
+            ++ui;
+        } else if ((D >> i) & 1u) {
+            if (di < (unsigned long long)p.L.n_dense) {
+                dpos[di] = (unsigned short)off;
+                const long long f = n * p.cols + stage * kStageK + i * B;
+                float v[B];
+                if (B >= 4) {
+#pragma unroll
+                    for (int l = 0; l < B; l += 4) {
+                        float4 a = __ldg(reinterpret_cast<const float4 *>(p.W + f + l));
+                        if (p.U) {
+                            const float4 d = __ldg(reinterpret_cast<const float4 *>(p.U + f + l));
+                            a.x = __fadd_rn(a.x, d.x); a.y = __fadd_rn(a.y, d.y); a.z = __fadd_rn(a.z, d.z); a.w = __fadd_rn(a.w, d.w);
+                        }
+                        v[l] = a.x; v[(l + 1) % B] = a.y; v[(l + 2) % B] = a.z; v[(l + 3) % B] = a.w;
+                    }
+                } else {
+                    float2 a = __ldg(reinterpret_cast<const float2 *>(p.W + f));
+                    if (p.U) {
+                        const float2 d = __ldg(reinterpret_cast<const float2 *>(p.U + f));
+                        a.x = __fadd_rn(a.x, d.x); a.y = __fadd_rn(a.y, d.y);
+                    }
+                    v[0] = a.x; v[1 % B] = a.y;
+                }
+                unsigned w[B / 2];
+#pragma unroll
+                for (int l = 0; l < B / 2; ++l) {
+                    const __nv_bfloat162 h = __floats2bfloat162_rn(v[2 * l], v[2 * l + 1]);
+                    w[l] = *reinterpret_cast<const unsigned *>(&h);
+                }
+                unsigned char *dst = dpay + di * (2 * B);
+                if (B == 16) {
+                    *reinterpret_cast<uint4 *>(dst) = make_uint4(w[0], w[1 % (B / 2)], w[2 % (B / 2)], w[3 % (B / 2)]);
+                    *reinterpret_cast<uint4 *>(dst + 16) = make_uint4(w[4 % (B / 2)], w[5 % (B / 2)], w[6 % (B / 2)], w[7 % (B / 2)]);
+                } else if (B == 8) {
+                    *reinterpret_cast<uint4 *>(dst) = make_uint4(w[0], w[1 % (B / 2)], w[2 % (B / 2)], w[3 % (B / 2)]);
+                } else if (B == 4) {
+                    *reinterpret_cast<uint2 *>(dst) = make_uint2(w[0], w[1 % (B / 2)]);
+                } else {
+                    *reinterpret_cast<unsigned *>(dst) = w[0];
+                }
+            } else {
+                bad = true;
+            }
+            ++di;
+        } else {
+            if (pi < (unsigned long long)p.L.n_plist) ppos[pi] = (unsigned short)off;
+            else bad = true;
+            ++pi;
         }
     }
     if (bad) atomicOr(p.dev_status, (unsigned)MWU_DEV_BOUNDS);
@@ -301,6 +325,11 @@ extern "C" int mwu_pack(const mwu_proj_desc *desc, const float *W, const float *
                 return MWU_ERR_CUDA;
     pack::count_kernel<<<(unsigned)n_rec, 128, 0, st>>>(p);
     pack::scan_kernel<<<1, 1024, 0, st>>>(p);
-    pack::fill_kernel<<<(unsigned)n_rec, 128, 0, st>>>(p);
+    switch (desc->block) {
+        case 2: pack::fill_kernel<2><<<(unsigned)n_rec, 128, 0, st>>>(p); break;
+        case 4: pack::fill_kernel<4><<<(unsigned)n_rec, 128, 0, st>>>(p); break;
+        case 8: pack::fill_kernel<8><<<(unsigned)n_rec, 128, 0, st>>>(p); break;
+        default: pack::fill_kernel<16><<<(unsigned)n_rec, 128, 0, st>>>(p); break;
+    }
     return cudaGetLastError() == cudaSuccess ? MWU_OK : MWU_ERR_CUDA;
 }

@@ -1,30 +1,32 @@
 // mwu_project: Q = Unify(W + U), the Q-step of ADMM (Algorithm 1, Eq. 7) for 1-D micro-blocks.
 //
 // Pipeline (all on the caller's stream, no host synchronisation):
-//   sample_kernel   one CTA looks at <= 4096 evenly spaced blocks and places a narrow window of
+//   sample_kernel   one CTA looks at <= 1024 evenly spaced blocks and places a narrow window of
 //                   8190 bins around the k-th smallest key of each selection (prune key, L_u).
 //                   The window only steers efficiency; any window gives the same result.
-//   stats_kernel    streams W (+U) once with 128-bit loads; per block the fp64 keys
-//                   (Section 3.1: q = mean|v|, L_u = sum(|v|-q)^2, L_p = sum v^2) are reduced with
-//                   warp shuffles; writes a 2x16-bit bin code per block and the prune histogram.
-//   resolve_kernel  (cooperative, once per selection) finds the exact threshold element
-//                   (key, block index): scans the histogram, narrows the range of the composite
-//                   96-bit key until <= 2048 candidates remain, sorts them in shared memory.
+//   stats_kernel    streams W (+U) once; every thread owns 64 contiguous bytes (four 128-bit
+//                   loads in flight) and evaluates the fp64 keys of its blocks (Section 3.1:
+//                   q = mean|v|, L_u = sum(|v|-q)^2, L_p = sum v^2) with the fixed pairwise
+//                   tree; writes a 2x16-bit bin code per block and the prune-key histogram.
+//                   The last CTA to finish locates the bin of the k_prune-th key.
+//   collect_kernel  gathers the blocks of that bin (normally a few dozen) and the last CTA sorts
+//                   them: the result is the exact threshold element (key, block index).
+//   histu_kernel    histogram of L_u over the blocks that were not pruned; last CTA locates the
+//                   bin; then collect_kernel again for the unify threshold.
 //   emit_kernel     streams W again: classifies every block from its bin code (exact key only
-//                   for blocks in the threshold bin), writes Q, u, both bitmaps, the sign plane.
-#include <cooperative_groups.h>
-
+//                   for blocks in a threshold bin), writes Q, u, both bitmaps and the sign plane.
+// When a threshold bin holds more than 2048 blocks (massive ties, e.g. re-projecting an already
+// projected tensor) the last CTA narrows the range of the 96-bit composite key (key, index) by
+// itself, pass by pass, until the candidates fit: slow but exact.
 #include "mwu_common.cuh"
-
-namespace cg = cooperative_groups;
 
 namespace mwu {
 namespace proj {
 
 constexpr int NB = 8192;        // level-0 bins: 0 = below the window, NB-1 = above it
 constexpr int CAP = 2048;       // candidates sorted by the last step
-constexpr int NSAMP = 4096;
-constexpr int RESOLVE_THREADS = 1024;
+constexpr int NSAMP = 1024;
+constexpr int FIN_THREADS = 1024;   // block size of the kernels whose last CTA finalises
 
 typedef unsigned long long u64;
 typedef unsigned __int128 u128;
@@ -45,6 +47,7 @@ struct Sel {
 struct Work {
     Sel sel[2];                 // 0: prune, 1: unify
     unsigned cand_count[2];
+    unsigned ticket[4];         // stats, collect<0>, histu, collect<1>
     unsigned pad[2];
 };
 
@@ -75,44 +78,95 @@ __device__ __forceinline__ unsigned bin_of(u64 key, u64 lo0, u64 hi0, unsigned s
 template <typename T>
 __device__ __forceinline__ T ld_vol(const T *p) { return *reinterpret_cast<const volatile T *>(p); }
 
+__device__ __forceinline__ u64 key_bits(double x) { return (u64)__double_as_longlong(x); }
+
 // ---------------------------------------------------------------------------------------------
-// exact keys of one block by one thread (sampling and the rare threshold-bin paths)
+// fp64 statistics of one block held in registers (fixed pairwise tree, every op rounded alone)
 // ---------------------------------------------------------------------------------------------
+template <int B>
+__device__ __forceinline__ double tree_sum(const double (&x)[B]) {
+    double t[B];
+#pragma unroll
+    for (int l = 0; l < B; ++l) t[l] = x[l];
+#pragma unroll
+    for (int w = 1; w < B; w <<= 1)
+#pragma unroll
+        for (int i = 0; i < B; i += 2 * w) t[i] = __dadd_rn(t[i], t[i + w]);
+    return t[0];
+}
+
+// v: the block's B values.  S = sum|v|, Lu = sum(|v| - S/B)^2, Kp = sum v^2 (or S for the L1 key)
+template <int B>
+__device__ __forceinline__ void block_keys(const float *v, int use_l1, double *S_out, double *Lu_out,
+                                           double *Kp_out) {
+    double a[B], t[B];
+#pragma unroll
+    for (int l = 0; l < B; ++l) a[l] = (double)fabsf(v[l]);
+    const double S = tree_sum<B>(a);
+    const double q = __dmul_rn(S, 1.0 / (double)B);
+#pragma unroll
+    for (int l = 0; l < B; ++l) {
+        const double d = __dsub_rn(a[l], q);
+        t[l] = __dmul_rn(d, d);
+    }
+    *Lu_out = tree_sum<B>(t);
+    *S_out = S;
+    if (use_l1) {
+        *Kp_out = S;
+    } else {
+        // a*a is exact in fp64 for fp32-valued a, so fma(a,a,c) == round(a*a + c): the same
+        // bits as a separately rounded multiply and add.
+        double h[B / 2];
+#pragma unroll
+        for (int l = 0; l < B / 2; ++l) h[l] = __fma_rn(a[2 * l], a[2 * l], __dmul_rn(a[2 * l + 1], a[2 * l + 1]));
+        *Kp_out = tree_sum<B / 2>(h);
+    }
+}
+
 __device__ __forceinline__ float load_v(const float *W, const float *U, long long f) {
     float w = __ldg(W + f);
     if (U) w = __fadd_rn(w, __ldg(U + f));
     return w;
 }
 
-__device__ __noinline__ void block_keys_scalar(const float *W, const float *U, long long j, int b,
-                                               int use_l1, double *S_out, double *Lu_out,
-                                               double *Kp_out) {
-    double a[16], t[16];
-    for (int l = 0; l < b; ++l) a[l] = (double)fabsf(load_v(W, U, j * b + l));
-    for (int l = 0; l < b; ++l) t[l] = a[l];
-    for (int w = 1; w < b; w <<= 1)
-        for (int i = 0; i < b; i += 2 * w) t[i] = __dadd_rn(t[i], t[i + w]);
-    const double S = t[0];
-    const double q = __dmul_rn(S, 1.0 / (double)b);
-    for (int l = 0; l < b; ++l) {
-        const double d = __dsub_rn(a[l], q);
-        t[l] = __dmul_rn(d, d);
-    }
-    for (int w = 1; w < b; w <<= 1)
-        for (int i = 0; i < b; i += 2 * w) t[i] = __dadd_rn(t[i], t[i + w]);
-    *Lu_out = t[0];
-    *S_out = S;
-    if (use_l1) {
-        *Kp_out = S;
-    } else {
-        for (int l = 0; l < b; ++l) t[l] = __dmul_rn(a[l], a[l]);
-        for (int w = 1; w < b; w <<= 1)
-            for (int i = 0; i < b; i += 2 * w) t[i] = __dadd_rn(t[i], t[i + w]);
-        *Kp_out = t[0];
-    }
+// exact keys of block j, read from global memory (sampling and threshold-bin blocks)
+template <int B>
+__device__ __forceinline__ void block_keys_at(const float *W, const float *U, long long j, int use_l1,
+                                              double *S, double *Lu, double *Kp) {
+    float v[B];
+#pragma unroll
+    for (int l = 0; l < B; ++l) v[l] = load_v(W, U, j * B + l);
+    block_keys<B>(v, use_l1, S, Lu, Kp);
 }
 
-__device__ __forceinline__ u64 key_bits(double x) { return (u64)__double_as_longlong(x); }
+// which: 0 -> prune key, 1 -> L_u
+template <int B>
+__device__ __forceinline__ u64 exact_key(const Params &p, long long j, int which) {
+    double S, Lu, Kp;
+    block_keys_at<B>(p.W, p.U, j, p.use_l1, &S, &Lu, &Kp);
+    return key_bits(which ? Lu : Kp);
+}
+
+// 16 consecutive floats starting at f (f % 16 == 0); zero beyond n
+__device__ __forceinline__ void load16(const float *W, const float *U, long long f, long long n, float (&v)[16]) {
+    if (f + 16 <= n) {
+        const float4 *src = reinterpret_cast<const float4 *>(W + f);
+        float4 a0 = __ldg(src), a1 = __ldg(src + 1), a2 = __ldg(src + 2), a3 = __ldg(src + 3);
+        if (U) {
+            const float4 *du = reinterpret_cast<const float4 *>(U + f);
+            const float4 d0 = __ldg(du), d1 = __ldg(du + 1), d2 = __ldg(du + 2), d3 = __ldg(du + 3);
+            a0.x = __fadd_rn(a0.x, d0.x); a0.y = __fadd_rn(a0.y, d0.y); a0.z = __fadd_rn(a0.z, d0.z); a0.w = __fadd_rn(a0.w, d0.w);
+            a1.x = __fadd_rn(a1.x, d1.x); a1.y = __fadd_rn(a1.y, d1.y); a1.z = __fadd_rn(a1.z, d1.z); a1.w = __fadd_rn(a1.w, d1.w);
+            a2.x = __fadd_rn(a2.x, d2.x); a2.y = __fadd_rn(a2.y, d2.y); a2.z = __fadd_rn(a2.z, d2.z); a2.w = __fadd_rn(a2.w, d2.w);
+            a3.x = __fadd_rn(a3.x, d3.x); a3.y = __fadd_rn(a3.y, d3.y); a3.z = __fadd_rn(a3.z, d3.z); a3.w = __fadd_rn(a3.w, d3.w);
+        }
+        v[0] = a0.x; v[1] = a0.y; v[2] = a0.z; v[3] = a0.w; v[4] = a1.x; v[5] = a1.y; v[6] = a1.z; v[7] = a1.w;
+        v[8] = a2.x; v[9] = a2.y; v[10] = a2.z; v[11] = a2.w; v[12] = a3.x; v[13] = a3.y; v[14] = a3.z; v[15] = a3.w;
+    } else {
+#pragma unroll
+        for (int l = 0; l < 16; ++l) v[l] = (f + l < n) ? load_v(W, U, f + l) : 0.f;
+    }
+}
 
 // ---------------------------------------------------------------------------------------------
 // sample_kernel: choose the level-0 windows
@@ -150,34 +204,30 @@ __device__ void window_from_sorted(const u64 *a, int n, double frac, Sel *s) {
     s->shift0 = shift;
 }
 
-__global__ void __launch_bounds__(1024) sample_kernel(Params p, long long k_unify, long long k_prune) {
+template <int B>
+__global__ void __launch_bounds__(NSAMP) sample_kernel(Params p, long long k_unify, long long k_prune) {
     __shared__ u64 skey[NSAMP];
     __shared__ int s_kept;
     __shared__ u64 s_That;
     const long long mb = p.n_blocks;
     const int ns = (int)(mb < (long long)NSAMP ? mb : (long long)NSAMP);
-    const int per = NSAMP / 1024;
-    u64 kp[per], ku[per];
-    if (threadIdx.x == 0) s_kept = 0;
-    for (int t = 0; t < per; ++t) {
-        const int i = threadIdx.x + t * 1024;
-        kp[t] = ~0ull;
-        ku[t] = ~0ull;
-        if (i < ns) {
-            const long long j = (long long)(((u128)(u64)i * (u128)(u64)mb) / (u128)(u64)ns);
-            double S, Lu, Kp;
-            block_keys_scalar(p.W, p.U, j, p.b, p.use_l1, &S, &Lu, &Kp);
-            kp[t] = key_bits(Kp);
-            ku[t] = key_bits(Lu);
-        }
-        skey[i] = kp[t];
+    const int i = threadIdx.x;
+    u64 kp = ~0ull, ku = ~0ull;
+    if (i == 0) s_kept = 0;
+    if (i < ns) {
+        const long long j = (long long)(((u128)(u64)i * (u128)(u64)mb) / (u128)(u64)ns);
+        double S, Lu, Kp;
+        block_keys_at<B>(p.W, p.U, j, p.use_l1, &S, &Lu, &Kp);
+        kp = key_bits(Kp);
+        ku = key_bits(Lu);
     }
+    skey[i] = kp;
     __syncthreads();
     Sel *sp = &p.work->sel[0];
     Sel *su = &p.work->sel[1];
     const long long ksel_u = k_unify - k_prune;
     bitonic_sort_u64(skey, NSAMP);
-    if (threadIdx.x == 0) {
+    if (i == 0) {
         const double fp = (double)k_prune / (double)mb;
         window_from_sorted(skey, ns, fp, sp);
         sp->mode = (k_prune == 0) ? 1u : (k_prune == mb ? 2u : 0u);
@@ -188,19 +238,13 @@ __global__ void __launch_bounds__(1024) sample_kernel(Params p, long long k_unif
     }
     __syncthreads();
     const u64 That = s_That;
-    const bool none_pruned = (k_prune == 0);
     __syncthreads();
-    int kept = 0;
-    for (int t = 0; t < per; ++t) {
-        const int i = threadIdx.x + t * 1024;
-        u64 v = ~0ull;
-        if (i < ns && (none_pruned || kp[t] > That)) { v = ku[t]; ++kept; }
-        skey[i] = v;
-    }
-    atomicAdd(&s_kept, kept);
+    u64 v = ~0ull;
+    if (i < ns && (k_prune == 0 || kp > That)) { v = ku; atomicAdd(&s_kept, 1); }
+    skey[i] = v;
     __syncthreads();
     bitonic_sort_u64(skey, NSAMP);
-    if (threadIdx.x == 0) {
+    if (i == 0) {
         const int nr = s_kept > 0 ? s_kept : 1;
         const long long elig = mb - k_prune;
         const double fu = elig > 0 ? (double)ksel_u / (double)elig : 0.0;
@@ -211,84 +255,114 @@ __global__ void __launch_bounds__(1024) sample_kernel(Params p, long long k_unif
 }
 
 // ---------------------------------------------------------------------------------------------
-// per-thread / per-group fp64 statistics with the fixed pairwise tree
+// finalisation helpers, run by the last CTA of a kernel (FIN_THREADS threads)
 // ---------------------------------------------------------------------------------------------
-__device__ __forceinline__ double shfl_xor_f64(double x, int m) {
-    return __shfl_xor_sync(0xffffffffu, x, m);
+// true in exactly one CTA: the one whose threads arrive last.  Everything the other CTAs wrote
+// before is visible to it afterwards.
+__device__ __forceinline__ bool last_block_done(unsigned *ticket) {
+    __shared__ bool s_last;
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const unsigned t = atomicAdd(ticket, 1u);
+        s_last = (t == gridDim.x - 1);
+    }
+    __syncthreads();
+    if (s_last) __threadfence();
+    return s_last;
 }
 
-// loads 4 consecutive floats starting at f (f % 4 == 0); zero beyond n
-__device__ __forceinline__ float4 load4(const float *W, const float *U, long long f, long long n,
-                                        bool *nonfinite) {
-    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (f + 3 < n) {
-        v = __ldg(reinterpret_cast<const float4 *>(W + f));
-        if (U) {
-            const float4 d = __ldg(reinterpret_cast<const float4 *>(U + f));
-            v.x = __fadd_rn(v.x, d.x); v.y = __fadd_rn(v.y, d.y);
-            v.z = __fadd_rn(v.z, d.z); v.w = __fadd_rn(v.w, d.w);
-        }
-    } else if (f < n) {
-        float t[4] = {0.f, 0.f, 0.f, 0.f};
-        for (int l = 0; l < 4 && f + l < n; ++l) t[l] = load_v(W, U, f + l);
-        v = make_float4(t[0], t[1], t[2], t[3]);
+// find the bin holding the r-th element; hist has NB entries
+__device__ void scan_hist(const unsigned *hist, u64 r, unsigned *bin_out, u64 *r_in_bin, u64 *cnt_out,
+                          unsigned *err) {
+    __shared__ u64 s_part[FIN_THREADS];
+    constexpr int PER = NB / FIN_THREADS;
+    u64 local[PER];
+    u64 sum = 0;
+#pragma unroll
+    for (int i = 0; i < PER; ++i) {
+        local[i] = ld_vol(&hist[threadIdx.x * PER + i]);
+        sum += local[i];
     }
-    const unsigned ex = 0x7f800000u;
-    *nonfinite = ((__float_as_uint(v.x) & ex) == ex) | ((__float_as_uint(v.y) & ex) == ex) |
-                 ((__float_as_uint(v.z) & ex) == ex) | ((__float_as_uint(v.w) & ex) == ex);
+    s_part[threadIdx.x] = sum;
+    __syncthreads();
+    for (int off = 1; off < FIN_THREADS; off <<= 1) {
+        u64 add = 0;
+        if ((int)threadIdx.x >= off) add = s_part[threadIdx.x - off];
+        __syncthreads();
+        s_part[threadIdx.x] += add;
+        __syncthreads();
+    }
+    const u64 incl = s_part[threadIdx.x];
+    u64 run = incl - sum;
+    if (threadIdx.x == FIN_THREADS - 1 && incl < r) *err = 1;
+#pragma unroll
+    for (int i = 0; i < PER; ++i) {
+        if (run < r && r <= run + local[i]) {
+            *bin_out = threadIdx.x * PER + i;
+            *r_in_bin = r - run;
+            *cnt_out = local[i];
+        }
+        run += local[i];
+    }
+    __syncthreads();
+}
+
+// level 0: which bin holds the k-th element; writes the bin and its composite range
+__device__ void select_bin(const Params &p, Sel *s, const unsigned *hist) {
+    __shared__ unsigned s_bin, s_err;
+    __shared__ u64 s_r, s_cnt;
+    if (threadIdx.x == 0) { s_err = 0; s_bin = 0; s_r = 0; s_cnt = 0; }
+    __syncthreads();
+    scan_hist(hist, s->k, &s_bin, &s_r, &s_cnt, &s_err);
+    if (threadIdx.x == 0) {
+        if (s_err) atomicOr(p.dev_status, (unsigned)MWU_DEV_SELECT);
+        const unsigned B = s_bin;
+        u64 klo, khi;
+        if (B == 0) { klo = 0; khi = s->lo0; }
+        else if (B == NB - 1) { klo = s->hi0; khi = ~0ull >> 1; }     // keys are < 2^63
+        else {
+            klo = s->lo0 + ((u64)(B - 1) << s->shift0);
+            khi = s->lo0 + ((u64)B << s->shift0);
+            if (khi > s->hi0) khi = s->hi0;
+        }
+        const u128 lo = make_c(klo, 0), hi = make_c(khi, 0);
+        s->B = B;
+        s->r = s_r;
+        s->cnt = s_cnt;
+        s->lo_hi = (u64)(lo >> 64); s->lo_lo = (u64)lo;
+        s->hi_hi = (u64)(hi >> 64); s->hi_lo = (u64)hi;
+        __threadfence();
+    }
+    __syncthreads();
+}
+
+// ---------------------------------------------------------------------------------------------
+// classification of a block from its bin code
+// ---------------------------------------------------------------------------------------------
+struct SelView {
+    unsigned mode, B;
+    u64 T_key, T_idx;
+};
+
+__device__ __forceinline__ SelView view_of(const Sel *s) {
+    SelView v;
+    v.mode = ld_vol(&s->mode);
+    v.B = ld_vol(&s->B);
+    v.T_key = ld_vol(&s->T_key);
+    v.T_idx = ld_vol(&s->T_idx);
     return v;
 }
 
-// Keys of the block(s) a thread touches.  For B >= 8 the block spans B/4 neighbouring lanes.
-// On return (B >= 8): every lane of the group holds S; even lanes hold L_u in `first`, odd
-// lanes hold the prune key in `first`.  For B == 4: first = L_u, second = prune key.
-// For B == 2: handled by keys_b2.
 template <int B>
-__device__ __forceinline__ void keys_group(const float4 v, int use_l1, double *S_out, double *first,
-                                           double *second) {
-    const double a0 = (double)fabsf(v.x), a1 = (double)fabsf(v.y);
-    const double a2 = (double)fabsf(v.z), a3 = (double)fabsf(v.w);
-    double S = __dadd_rn(__dadd_rn(a0, a1), __dadd_rn(a2, a3));
-    if (B >= 8) S = __dadd_rn(S, shfl_xor_f64(S, 1));
-    if (B >= 16) S = __dadd_rn(S, shfl_xor_f64(S, 2));
-    const double q = __dmul_rn(S, 1.0 / (double)B);
-    const double d0 = __dsub_rn(a0, q), d1 = __dsub_rn(a1, q);
-    const double d2 = __dsub_rn(a2, q), d3 = __dsub_rn(a3, q);
-    double Lu = __dadd_rn(__dadd_rn(__dmul_rn(d0, d0), __dmul_rn(d1, d1)),
-                          __dadd_rn(__dmul_rn(d2, d2), __dmul_rn(d3, d3)));
-    double Kp;
-    if (use_l1) {
-        Kp = 0.0;   // replaced by S below
-    } else {
-        // a*a is exact in fp64 for fp32-valued a, so fma(a,a,c) == round(a*a + c): same bits
-        // as a separately rounded multiply and add.
-        Kp = __dadd_rn(__fma_rn(a0, a0, __dmul_rn(a1, a1)), __fma_rn(a2, a2, __dmul_rn(a3, a3)));
-    }
-    if (B >= 8) {
-        const bool odd = (threadIdx.x & 1) != 0;
-        const double send = odd ? Lu : Kp;
-        const double keep = odd ? Kp : Lu;
-        double res = __dadd_rn(keep, shfl_xor_f64(send, 1));
-        if (B >= 16) res = __dadd_rn(res, shfl_xor_f64(res, 2));
-        if (use_l1 && odd) res = S;
-        *first = res;
-        *second = 0.0;
-    } else {
-        *first = Lu;
-        *second = use_l1 ? S : Kp;
-    }
-    *S_out = S;
-}
-
-__device__ __forceinline__ void keys_b2(float x, float y, int use_l1, double *S_out, double *Lu,
-                                        double *Kp) {
-    const double a0 = (double)fabsf(x), a1 = (double)fabsf(y);
-    const double S = __dadd_rn(a0, a1);
-    const double q = __dmul_rn(S, 0.5);
-    const double d0 = __dsub_rn(a0, q), d1 = __dsub_rn(a1, q);
-    *Lu = __dadd_rn(__dmul_rn(d0, d0), __dmul_rn(d1, d1));
-    *Kp = use_l1 ? S : __fma_rn(a0, a0, __dmul_rn(a1, a1));
-    *S_out = S;
+__device__ __forceinline__ bool selected(const Params &p, const SelView &s, long long j, unsigned bin,
+                                         int which) {
+    if (s.mode == 1u) return false;
+    if (s.mode == 2u) return true;
+    if (bin < s.B) return true;
+    if (bin > s.B) return false;
+    const u64 key = exact_key<B>(p, j, which);
+    return key < s.T_key || (key == s.T_key && (u64)j <= s.T_idx);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -296,81 +370,54 @@ __device__ __forceinline__ void keys_b2(float x, float y, int use_l1, double *S_
 // ---------------------------------------------------------------------------------------------
 template <int B>
 __global__ void __launch_bounds__(256) stats_kernel(Params p, double *loss_u, double *loss_p) {
+    constexpr int NBT = 16 / B;                         // blocks per thread and step
     const Sel *sp = &p.work->sel[0];
     const Sel *su = &p.work->sel[1];
     const u64 plo = sp->lo0, phi = sp->hi0, ulo = su->lo0, uhi = su->hi0;
     const unsigned psh = sp->shift0, ush = su->shift0;
     unsigned cnt_under = 0, cnt_over = 0;
-    bool any_nonfinite = false;
+    unsigned nonfinite = 0;
     const long long n = p.n_floats;
-    const long long n_quads = (n + 3) / 4;
-    // a warp always walks whole groups of 32 quads so that shuffles see all lanes
-    const long long n_iter = (n_quads + 31) / 32 * 32;
-    for (long long qd = (long long)blockIdx.x * blockDim.x + threadIdx.x; qd < n_iter;
-         qd += (long long)gridDim.x * blockDim.x) {
-        const long long f = qd * 4;
-        bool nf;
-        const float4 v = load4(p.W, p.U, f, n, &nf);
-        any_nonfinite |= nf;
-        if (B == 2) {
-            double S, Lu, Kp;
-            unsigned code[2];
+    const long long n_units = (n + 15) / 16;
+    for (long long unit = (long long)blockIdx.x * blockDim.x + threadIdx.x; unit < n_units;
+         unit += (long long)gridDim.x * blockDim.x) {
+        float v[16];
+        load16(p.W, p.U, unit * 16, n, v);
+        unsigned ex = 0;
 #pragma unroll
-            for (int e = 0; e < 2; ++e) {
-                keys_b2(e ? v.z : v.x, e ? v.w : v.y, p.use_l1, &S, &Lu, &Kp);
-                const long long j = f / 2 + e;
-                const unsigned bu = bin_of(key_bits(Lu), ulo, uhi, ush);
-                const unsigned bp = bin_of(key_bits(Kp), plo, phi, psh);
-                code[e] = bp | (bu << 16);
-                if (j < p.n_blocks) {
-                    if (bp == 0) ++cnt_under;
-                    else if (bp == NB - 1) ++cnt_over;
-                    else atomicAdd(&p.hist[bp], 1u);
-                    if (loss_u) loss_u[j] = Lu;
-                    if (loss_p) loss_p[j] = Kp;
-                }
+        for (int l = 0; l < 16; ++l) ex = max(ex, __float_as_uint(v[l]) & 0x7fffffffu);
+        nonfinite |= (ex >= 0x7f800000u) ? 1u : 0u;
+        unsigned code[NBT];
+#pragma unroll
+        for (int e = 0; e < NBT; ++e) {
+            double S, Lu, Kp;
+            block_keys<B>(v + e * B, p.use_l1, &S, &Lu, &Kp);
+            const long long j = unit * NBT + e;
+            const unsigned bu = bin_of(key_bits(Lu), ulo, uhi, ush);
+            const unsigned bp = bin_of(key_bits(Kp), plo, phi, psh);
+            code[e] = bp | (bu << 16);
+            if (j < p.n_blocks) {
+                if (bp == 0) ++cnt_under;
+                else if (bp == NB - 1) ++cnt_over;
+                else atomicAdd(&p.hist[bp], 1u);
+                if (loss_u) loss_u[j] = Lu;
+                if (loss_p) loss_p[j] = Kp;
             }
-            const long long j0 = f / 2;
-            if (j0 + 1 < p.n_blocks) {
-                *reinterpret_cast<uint2 *>(p.bins + j0) = make_uint2(code[0], code[1]);
-            } else if (j0 < p.n_blocks) {
-                p.bins[j0] = code[0];
+        }
+        const long long j0 = unit * NBT;
+        if (j0 + NBT <= p.n_blocks) {
+            if (NBT == 1) p.bins[j0] = code[0];
+            else if (NBT == 2) *reinterpret_cast<uint2 *>(p.bins + j0) = make_uint2(code[0], code[1 % NBT]);
+            else {
+#pragma unroll
+                for (int e = 0; e < NBT; e += 4)
+                    *reinterpret_cast<uint4 *>(p.bins + j0 + e) =
+                        make_uint4(code[e % NBT], code[(e + 1) % NBT], code[(e + 2) % NBT], code[(e + 3) % NBT]);
             }
         } else {
-            constexpr int LPB = (B >= 4) ? B / 4 : 1;      // lanes per block
-            double S, first, second;
-            keys_group<B>(v, p.use_l1, &S, &first, &second);
-            const long long j = f / B;
-            if (B == 4) {
-                const unsigned bu = bin_of(key_bits(first), ulo, uhi, ush);
-                const unsigned bp = bin_of(key_bits(second), plo, phi, psh);
-                if (j < p.n_blocks) {
-                    p.bins[j] = bp | (bu << 16);
-                    if (bp == 0) ++cnt_under;
-                    else if (bp == NB - 1) ++cnt_over;
-                    else atomicAdd(&p.hist[bp], 1u);
-                    if (loss_u) loss_u[j] = first;
-                    if (loss_p) loss_p[j] = second;
-                }
-            } else {
-                const bool odd = (threadIdx.x & 1) != 0;
-                const unsigned mine = odd ? bin_of(key_bits(first), plo, phi, psh)
-                                          : (bin_of(key_bits(first), ulo, uhi, ush) << 16);
-                const unsigned code = mine | __shfl_xor_sync(0xffffffffu, mine, 1);
-                const int sub = threadIdx.x & (LPB - 1);
-                if (j < p.n_blocks) {
-                    if (sub == 0) {
-                        p.bins[j] = code;
-                        if (loss_u) loss_u[j] = first;
-                    } else if (sub == 1) {
-                        const unsigned bp = mine;
-                        if (bp == 0) ++cnt_under;
-                        else if (bp == NB - 1) ++cnt_over;
-                        else atomicAdd(&p.hist[bp], 1u);
-                        if (loss_p) loss_p[j] = first;
-                    }
-                }
-            }
+#pragma unroll
+            for (int e = 0; e < NBT; ++e)
+                if (j0 + e < p.n_blocks) p.bins[j0 + e] = code[e];
         }
     }
     // block-level totals of the two catch-all bins
@@ -385,7 +432,7 @@ __global__ void __launch_bounds__(256) stats_kernel(Params p, double *loss_u, do
         if (cnt_under) atomicAdd(&s_under, cnt_under);
         if (cnt_over) atomicAdd(&s_over, cnt_over);
     }
-    if (any_nonfinite) atomicOr(p.dev_status, (unsigned)MWU_DEV_NONFINITE);
+    if (nonfinite) atomicOr(p.dev_status, (unsigned)MWU_DEV_NONFINITE);
     __syncthreads();
     if (threadIdx.x == 0) {
         if (s_under) atomicAdd(&p.hist[0], s_under);
@@ -393,78 +440,47 @@ __global__ void __launch_bounds__(256) stats_kernel(Params p, double *loss_u, do
     }
 }
 
-// ---------------------------------------------------------------------------------------------
-// classification helpers shared by resolve and emit
-// ---------------------------------------------------------------------------------------------
-struct SelView {            // read-only copy of what classification needs
-    unsigned mode, B;
-    u64 T_key, T_idx;
-};
-
-__device__ __forceinline__ SelView view_of(const Sel *s) {
-    SelView v;
-    v.mode = ld_vol(&s->mode);
-    v.B = ld_vol(&s->B);
-    v.T_key = ld_vol(&s->T_key);
-    v.T_idx = ld_vol(&s->T_idx);
-    return v;
-}
-
-// which: 0 -> prune key, 1 -> L_u
-__device__ __forceinline__ u64 exact_key(const Params &p, long long j, int which) {
-    double S, Lu, Kp;
-    block_keys_scalar(p.W, p.U, j, p.b, p.use_l1, &S, &Lu, &Kp);
-    return key_bits(which ? Lu : Kp);
-}
-
-__device__ __forceinline__ bool selected(const Params &p, const SelView &s, long long j,
-                                         unsigned bin, int which) {
-    if (s.mode == 1u) return false;
-    if (s.mode == 2u) return true;
-    if (bin < s.B) return true;
-    if (bin > s.B) return false;
-    const u64 key = exact_key(p, j, which);
-    return key < s.T_key || (key == s.T_key && (u64)j <= s.T_idx);
+// one CTA: locate the threshold bin of a selection from its finished histogram
+template <int KIND>
+__global__ void __launch_bounds__(FIN_THREADS) bin_kernel(Params p) {
+    Sel *s = &p.work->sel[KIND];
+    if (ld_vol(&s->mode) != 0u) return;
+    select_bin(p, s, p.hist + (size_t)KIND * NB);
 }
 
 // ---------------------------------------------------------------------------------------------
-// resolve_kernel: exact threshold element of one selection
+// histu_kernel: histogram of L_u bins over the blocks that were not pruned
 // ---------------------------------------------------------------------------------------------
-// block 0: find the bin holding the r-th element; hist has NB entries
-__device__ void scan_hist(const unsigned *hist, u64 r, unsigned *bin_out, u64 *r_in_bin,
-                          u64 *cnt_out, unsigned *err) {
-    __shared__ u64 s_part[RESOLVE_THREADS];
-    constexpr int PER = NB / RESOLVE_THREADS;
-    u64 local[PER];
-    u64 sum = 0;
-    for (int i = 0; i < PER; ++i) {
-        local[i] = ld_vol(&hist[threadIdx.x * PER + i]);
-        sum += local[i];
+template <int B>
+__global__ void __launch_bounds__(FIN_THREADS) histu_kernel(Params p) {
+    Sel *s = &p.work->sel[1];
+    if (ld_vol(&s->mode) != 0u) return;
+    unsigned *hist = p.hist + NB;
+    const SelView pv = view_of(&p.work->sel[0]);
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    unsigned under = 0, over = 0;
+    for (long long j = (long long)blockIdx.x * blockDim.x + threadIdx.x; j < p.n_blocks; j += stride) {
+        const unsigned code = __ldg(p.bins + j);
+        if (selected<B>(p, pv, j, code & 0xffffu, 0)) continue;
+        const unsigned bu = code >> 16;
+        if (bu == 0) ++under;
+        else if (bu == NB - 1) ++over;
+        else atomicAdd(&hist[bu], 1u);
     }
-    s_part[threadIdx.x] = sum;
-    __syncthreads();
-    // inclusive scan (Hillis-Steele), 1024 entries
-    for (int off = 1; off < RESOLVE_THREADS; off <<= 1) {
-        u64 add = 0;
-        if ((int)threadIdx.x >= off) add = s_part[threadIdx.x - off];
-        __syncthreads();
-        s_part[threadIdx.x] += add;
-        __syncthreads();
+    for (int m = 16; m > 0; m >>= 1) {
+        under += __shfl_xor_sync(0xffffffffu, under, m);
+        over += __shfl_xor_sync(0xffffffffu, over, m);
     }
-    const u64 incl = s_part[threadIdx.x];
-    u64 run = incl - sum;           // exclusive prefix
-    if (threadIdx.x == RESOLVE_THREADS - 1 && incl < r) *err = 1;
-    for (int i = 0; i < PER; ++i) {
-        if (run < r && r <= run + local[i]) {
-            *bin_out = threadIdx.x * PER + i;
-            *r_in_bin = r - run;
-            *cnt_out = local[i];
-        }
-        run += local[i];
+    if ((threadIdx.x & 31) == 0) {
+        if (under) atomicAdd(&hist[0], under);
+        if (over) atomicAdd(&hist[NB - 1], over);
     }
-    __syncthreads();
+    if (last_block_done(&p.work->ticket[2])) select_bin(p, s, hist);
 }
 
+// ---------------------------------------------------------------------------------------------
+// collect_kernel: exact threshold element of one selection
+// ---------------------------------------------------------------------------------------------
 __device__ void sort_candidates(u64 *key, unsigned *idx, int n_pow2) {
     for (int k = 2; k <= n_pow2; k <<= 1) {
         for (int j = k >> 1; j > 0; j >>= 1) {
@@ -483,89 +499,59 @@ __device__ void sort_candidates(u64 *key, unsigned *idx, int n_pow2) {
     }
 }
 
-template <int KIND>
-__global__ void __launch_bounds__(RESOLVE_THREADS) resolve_kernel(Params p) {
-    cg::grid_group grid = cg::this_grid();
+template <int KIND, int B>
+__global__ void __launch_bounds__(FIN_THREADS) collect_kernel(Params p) {
     Sel *s = &p.work->sel[KIND];
-    unsigned *hist = p.hist + (size_t)KIND * NB;
-    unsigned *rhist = p.hist + (size_t)2 * NB;
-    const long long stride = (long long)gridDim.x * blockDim.x;
-    const long long tid0 = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    __shared__ unsigned s_bin, s_err;
-    __shared__ u64 s_r, s_cnt;
+    if (ld_vol(&s->mode) != 0u) return;
     __shared__ u64 c_key[CAP];
     __shared__ unsigned c_idx[CAP];
+    __shared__ unsigned s_bin, s_err, s_n;
+    __shared__ u64 s_r, s_cnt;
+    const SelView pv = view_of(&p.work->sel[0]);
+    const unsigned Bsel = ld_vol(&s->B);
+    const bool too_many = ld_vol(&s->cnt) > (u64)CAP;
+    const long long stride = (long long)gridDim.x * blockDim.x;
 
-    SelView prune_view;
-    if (KIND == 1) {
-        // histogram of L_u over the blocks that were not pruned
-        prune_view = view_of(&p.work->sel[0]);
-        unsigned under = 0, over = 0;
-        for (long long j = tid0; j < p.n_blocks; j += stride) {
-            const unsigned code = p.bins[j];
-            if (selected(p, prune_view, j, code & 0xffffu, 0)) continue;
-            const unsigned bu = code >> 16;
-            if (bu == 0) ++under;
-            else if (bu == NB - 1) ++over;
-            else atomicAdd(&hist[bu], 1u);
-        }
-        for (int m = 16; m > 0; m >>= 1) {
-            under += __shfl_xor_sync(0xffffffffu, under, m);
-            over += __shfl_xor_sync(0xffffffffu, over, m);
-        }
-        if ((threadIdx.x & 31) == 0) {
-            if (under) atomicAdd(&hist[0], under);
-            if (over) atomicAdd(&hist[NB - 1], over);
-        }
-        grid.sync();
-    }
-
-    // level 0: which bin holds the k-th element
-    if (blockIdx.x == 0) {
-        if (threadIdx.x == 0) { s_err = 0; s_bin = 0; s_r = 0; s_cnt = 0; }
-        __syncthreads();
-        scan_hist(hist, s->k, &s_bin, &s_r, &s_cnt, &s_err);
-        if (threadIdx.x == 0) {
-            if (s_err) atomicOr(p.dev_status, (unsigned)MWU_DEV_SELECT);
-            const unsigned B = s_bin;
-            u64 klo, khi;      // key range of the bin
-            if (B == 0) { klo = 0; khi = s->lo0; }
-            else if (B == NB - 1) { klo = s->hi0; khi = ~0ull >> 1; }     // keys are < 2^63
-            else {
-                klo = s->lo0 + ((u64)(B - 1) << s->shift0);
-                khi = s->lo0 + ((u64)B << s->shift0);
-                if (khi > s->hi0) khi = s->hi0;
-            }
-            const u128 lo = make_c(klo, 0), hi = make_c(khi, 0);
-            s->B = B;
-            s->r = s_r;
-            s->cnt = s_cnt;
-            s->lo_hi = (u64)(lo >> 64); s->lo_lo = (u64)lo;
-            s->hi_hi = (u64)(hi >> 64); s->hi_lo = (u64)hi;
-        }
-    }
-    grid.sync();
-
-    // narrow [lo, hi) until the candidates fit the final sort (normally zero iterations)
-    for (int level = 0; level < 10; ++level) {
-        if (ld_vol(&s->cnt) <= (u64)CAP) break;
-        for (long long i = tid0; i < NB; i += stride) rhist[i] = 0;
-        grid.sync();
-        const unsigned B = ld_vol(&s->B);
+    if (!too_many) {
         const u128 lo = from_halves(ld_vol(&s->lo_hi), ld_vol(&s->lo_lo));
         const u128 hi = from_halves(ld_vol(&s->hi_hi), ld_vol(&s->hi_lo));
-        unsigned shift = 0;
-        while (((hi - lo - 1) >> shift) >= (u128)NB) ++shift;
-        for (long long j = tid0; j < p.n_blocks; j += stride) {
-            const unsigned code = p.bins[j];
+        for (long long j = (long long)blockIdx.x * blockDim.x + threadIdx.x; j < p.n_blocks; j += stride) {
+            const unsigned code = __ldg(p.bins + j);
             const unsigned bin = KIND ? (code >> 16) : (code & 0xffffu);
-            if (bin != B) continue;
-            if (KIND == 1 && selected(p, prune_view, j, code & 0xffffu, 0)) continue;
-            const u128 c = make_c(exact_key(p, j, KIND), (u64)j);
-            if (c >= lo && c < hi) atomicAdd(&rhist[(unsigned)((c - lo) >> shift)], 1u);
+            if (bin != Bsel) continue;
+            if (KIND == 1 && selected<B>(p, pv, j, code & 0xffffu, 0)) continue;
+            const u64 key = exact_key<B>(p, j, KIND);
+            const u128 c = make_c(key, (u64)j);
+            if (c >= lo && c < hi) {
+                const unsigned slot = atomicAdd(&p.work->cand_count[KIND], 1u);
+                if (slot < (unsigned)CAP) { p.cand_key[slot] = key; p.cand_idx[slot] = (unsigned)j; }
+            }
         }
-        grid.sync();
-        if (blockIdx.x == 0) {
+    }
+    if (!last_block_done(&p.work->ticket[KIND ? 3 : 1])) return;
+
+    // ---- last CTA only ----
+    if (too_many) {
+        // massive ties: narrow the composite range pass by pass with this CTA alone
+        unsigned *rhist = p.hist + (size_t)2 * NB;
+        for (int level = 0; level < 10; ++level) {
+            if (ld_vol(&s->cnt) <= (u64)CAP) break;
+            for (int i = threadIdx.x; i < NB; i += blockDim.x) rhist[i] = 0;
+            __syncthreads();
+            const u128 lo = from_halves(ld_vol(&s->lo_hi), ld_vol(&s->lo_lo));
+            const u128 hi = from_halves(ld_vol(&s->hi_hi), ld_vol(&s->hi_lo));
+            unsigned shift = 0;
+            while (((hi - lo - 1) >> shift) >= (u128)NB) ++shift;
+            for (long long j = threadIdx.x; j < p.n_blocks; j += blockDim.x) {
+                const unsigned code = ld_vol(p.bins + j);
+                const unsigned bin = KIND ? (code >> 16) : (code & 0xffffu);
+                if (bin != Bsel) continue;
+                if (KIND == 1 && selected<B>(p, pv, j, code & 0xffffu, 0)) continue;
+                const u128 c = make_c(exact_key<B>(p, j, KIND), (u64)j);
+                if (c >= lo && c < hi) atomicAdd(&rhist[(unsigned)((c - lo) >> shift)], 1u);
+            }
+            __threadfence();
+            __syncthreads();
             if (threadIdx.x == 0) s_err = 0;
             __syncthreads();
             scan_hist(rhist, ld_vol(&s->r), &s_bin, &s_r, &s_cnt, &s_err);
@@ -578,49 +564,50 @@ __global__ void __launch_bounds__(RESOLVE_THREADS) resolve_kernel(Params p) {
                 s->cnt = s_cnt;
                 s->lo_hi = (u64)(nlo >> 64); s->lo_lo = (u64)nlo;
                 s->hi_hi = (u64)(nhi >> 64); s->hi_lo = (u64)nhi;
+                __threadfence();
             }
+            __syncthreads();
         }
-        grid.sync();
-    }
-
-    // collect the candidates
-    {
-        const unsigned B = ld_vol(&s->B);
+        // collect inside the narrowed range
+        if (threadIdx.x == 0) s_n = 0;
+        __syncthreads();
         const u128 lo = from_halves(ld_vol(&s->lo_hi), ld_vol(&s->lo_lo));
         const u128 hi = from_halves(ld_vol(&s->hi_hi), ld_vol(&s->hi_lo));
-        for (long long j = tid0; j < p.n_blocks; j += stride) {
-            const unsigned code = p.bins[j];
+        for (long long j = threadIdx.x; j < p.n_blocks; j += blockDim.x) {
+            const unsigned code = ld_vol(p.bins + j);
             const unsigned bin = KIND ? (code >> 16) : (code & 0xffffu);
-            if (bin != B) continue;
-            if (KIND == 1 && selected(p, prune_view, j, code & 0xffffu, 0)) continue;
-            const u64 key = exact_key(p, j, KIND);
+            if (bin != Bsel) continue;
+            if (KIND == 1 && selected<B>(p, pv, j, code & 0xffffu, 0)) continue;
+            const u64 key = exact_key<B>(p, j, KIND);
             const u128 c = make_c(key, (u64)j);
             if (c >= lo && c < hi) {
-                const unsigned slot = atomicAdd(&p.work->cand_count[KIND], 1u);
+                const unsigned slot = atomicAdd(&s_n, 1u);
                 if (slot < (unsigned)CAP) { p.cand_key[slot] = key; p.cand_idx[slot] = (unsigned)j; }
             }
         }
-    }
-    grid.sync();
-
-    if (blockIdx.x == 0) {
-        const unsigned n = ld_vol(&p.work->cand_count[KIND]);
-        const u64 r = ld_vol(&s->r);
-        const unsigned m = n < (unsigned)CAP ? n : (unsigned)CAP;
-        for (int i = threadIdx.x; i < CAP; i += blockDim.x) {
-            c_key[i] = (i < (int)m) ? ld_vol(&p.cand_key[i]) : ~0ull;
-            c_idx[i] = (i < (int)m) ? ld_vol(&p.cand_idx[i]) : ~0u;
-        }
+        __threadfence();
         __syncthreads();
-        sort_candidates(c_key, c_idx, CAP);
-        if (threadIdx.x == 0) {
-            if (n > (unsigned)CAP || r == 0 || r > (u64)m) {
-                atomicOr(p.dev_status, (unsigned)MWU_DEV_SELECT);
-                s->T_key = 0; s->T_idx = 0;
-            } else {
-                s->T_key = c_key[r - 1];
-                s->T_idx = (u64)c_idx[r - 1];
-            }
+        if (threadIdx.x == 0) p.work->cand_count[KIND] = s_n;
+        __syncthreads();
+    }
+    const unsigned n = ld_vol(&p.work->cand_count[KIND]);
+    const u64 r = ld_vol(&s->r);
+    const unsigned m = n < (unsigned)CAP ? n : (unsigned)CAP;
+    for (int i = threadIdx.x; i < CAP; i += blockDim.x) {
+        c_key[i] = (i < (int)m) ? ld_vol(&p.cand_key[i]) : ~0ull;
+        c_idx[i] = (i < (int)m) ? ld_vol(&p.cand_idx[i]) : ~0u;
+    }
+    __syncthreads();
+    int np2 = 2;
+    while (np2 < (int)m) np2 <<= 1;
+    sort_candidates(c_key, c_idx, np2);
+    if (threadIdx.x == 0) {
+        if (n > (unsigned)CAP || r == 0 || r > (u64)m) {
+            atomicOr(p.dev_status, (unsigned)MWU_DEV_SELECT);
+            s->T_key = 0; s->T_idx = 0;
+        } else {
+            s->T_key = c_key[r - 1];
+            s->T_idx = (u64)c_idx[r - 1];
         }
     }
 }
@@ -632,120 +619,120 @@ template <int B>
 __global__ void __launch_bounds__(256) emit_kernel(Params p, float *Q, float *u_out,
                                                    unsigned *pruned_bitmap, unsigned *unified_bitmap,
                                                    unsigned *sign_bits) {
+    constexpr int NBT = 16 / B;
     const SelView vp = view_of(&p.work->sel[0]);
     const SelView vu = view_of(&p.work->sel[1]);
     const long long n = p.n_floats;
     const int lane = threadIdx.x & 31;
-    constexpr int CPT = (B >= 4) ? B / 4 : 1;                // 128-float chunks per warp task
-    constexpr int BPC = 128 / B;                             // blocks per chunk
-    const long long n_chunks = (n + 127) / 128;
-    const long long n_tasks = (n_chunks + CPT - 1) / CPT;
-    const long long warp0 = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-    const long long n_warps = ((long long)gridDim.x * blockDim.x) >> 5;
+    const long long n_units = (n + 15) / 16;
+    const long long n_iter = (n_units + 31) / 32 * 32;      // whole warps take part in every step
     const long long n_sign_words = (n + 31) / 32;
     const long long n_bm_words = (p.n_blocks + 31) / 32;
 
-    for (long long task = warp0; task < n_tasks; task += n_warps) {
-        unsigned word_p = 0, word_u = 0, word_p2 = 0, word_u2 = 0;
+    for (long long unit = (long long)blockIdx.x * blockDim.x + threadIdx.x; unit < n_iter;
+         unit += (long long)gridDim.x * blockDim.x) {
+        const long long f = unit * 16;
+        float v[16];
+        unsigned code[NBT];
+        if (unit < n_units) load16(p.W, p.U, f, n, v);
+        else {
 #pragma unroll
-        for (int it = 0; it < CPT; ++it) {
-            const long long chunk = task * CPT + it;
-            const long long f = chunk * 128 + lane * 4;
-            bool nf;
-            const float4 v = load4(p.W, p.U, f, n, &nf);
-            float4 q4 = v;
-            unsigned cls = 0;           // bit0 pruned, bit1 unified (B == 2: bits 2,3 second block)
-            if (B == 2) {
+            for (int l = 0; l < 16; ++l) v[l] = 0.f;
+        }
+        const long long j0 = unit * NBT;
+        if (j0 + NBT <= p.n_blocks) {
+            if (NBT == 1) code[0] = __ldg(p.bins + j0);
+            else if (NBT == 2) { const uint2 c = __ldg(reinterpret_cast<const uint2 *>(p.bins + j0)); code[0] = c.x; code[1 % NBT] = c.y; }
+            else {
 #pragma unroll
-                for (int e = 0; e < 2; ++e) {
-                    const long long j = f / 2 + e;
-                    const float x = e ? v.z : v.x, y = e ? v.w : v.y;
-                    if (j < p.n_blocks) {
-                        const unsigned code = p.bins[j];
-                        const bool pr = selected(p, vp, j, code & 0xffffu, 0);
-                        const bool un = !pr && selected(p, vu, j, code >> 16, 1);
-                        float qq = 0.f;
-                        if (un) {
-                            const double S = __dadd_rn((double)fabsf(x), (double)fabsf(y));
-                            qq = __double2float_rn(__dmul_rn(S, 0.5));
-                        }
-                        float ox = x, oy = y;
-                        if (pr) { ox = 0.f; oy = 0.f; }
-                        if (un) { ox = (x >= 0.f) ? qq : -qq; oy = (y >= 0.f) ? qq : -qq; }
-                        if (e) { q4.z = ox; q4.w = oy; } else { q4.x = ox; q4.y = oy; }
-                        u_out[j] = qq;
-                        cls |= ((pr ? 1u : 0u) | (un ? 2u : 0u)) << (2 * e);
-                    }
-                }
-            } else {
-                constexpr int LPB = B / 4;
-                const long long j = f / B;
-                const double a0 = (double)fabsf(v.x), a1 = (double)fabsf(v.y);
-                const double a2 = (double)fabsf(v.z), a3 = (double)fabsf(v.w);
-                double S = __dadd_rn(__dadd_rn(a0, a1), __dadd_rn(a2, a3));
-                if (B >= 8) S = __dadd_rn(S, shfl_xor_f64(S, 1));
-                if (B >= 16) S = __dadd_rn(S, shfl_xor_f64(S, 2));
-                if (j < p.n_blocks) {
-                    const unsigned code = p.bins[j];
-                    const bool pr = selected(p, vp, j, code & 0xffffu, 0);
-                    const bool un = !pr && selected(p, vu, j, code >> 16, 1);
-                    float qq = 0.f;
-                    if (un) qq = __double2float_rn(__dmul_rn(S, 1.0 / (double)B));
-                    if (pr) q4 = make_float4(0.f, 0.f, 0.f, 0.f);
-                    if (un) {
-                        q4.x = (v.x >= 0.f) ? qq : -qq; q4.y = (v.y >= 0.f) ? qq : -qq;
-                        q4.z = (v.z >= 0.f) ? qq : -qq; q4.w = (v.w >= 0.f) ? qq : -qq;
-                    }
-                    if ((lane & (LPB - 1)) == 0) u_out[j] = qq;
-                    cls = (pr ? 1u : 0u) | (un ? 2u : 0u);
+                for (int e = 0; e < NBT; e += 4) {
+                    const uint4 c = __ldg(reinterpret_cast<const uint4 *>(p.bins + j0 + e));
+                    code[e % NBT] = c.x; code[(e + 1) % NBT] = c.y; code[(e + 2) % NBT] = c.z; code[(e + 3) % NBT] = c.w;
                 }
             }
-            // Q
+        } else {
+#pragma unroll
+            for (int e = 0; e < NBT; ++e) code[e] = (j0 + e < p.n_blocks) ? __ldg(p.bins + j0 + e) : 0u;
+        }
+        float q[16];
+        float uo[NBT];
+        unsigned cls_p = 0, cls_u = 0;                       // bit e: block e of this thread
+#pragma unroll
+        for (int e = 0; e < NBT; ++e) {
+            const long long j = j0 + e;
+            bool pr = false, un = false;
+            if (j < p.n_blocks) {
+                pr = selected<B>(p, vp, j, code[e] & 0xffffu, 0);
+                un = !pr && selected<B>(p, vu, j, code[e] >> 16, 1);
+            }
+            float qq = 0.f;
+            if (un) {
+                double a[B];
+#pragma unroll
+                for (int l = 0; l < B; ++l) a[l] = (double)fabsf(v[e * B + l]);
+                qq = __double2float_rn(__dmul_rn(tree_sum<B>(a), 1.0 / (double)B));
+            }
+#pragma unroll
+            for (int l = 0; l < B; ++l) {
+                const float x = v[e * B + l];
+                q[e * B + l] = pr ? 0.f : (un ? ((x >= 0.f) ? qq : -qq) : x);
+            }
+            uo[e] = qq;
+            cls_p |= (pr ? 1u : 0u) << e;
+            cls_u |= (un ? 1u : 0u) << e;
+        }
+        if (unit < n_units) {
             if (Q) {
-                if (f + 3 < n) {
-                    *reinterpret_cast<float4 *>(Q + f) = q4;
-                } else if (f < n) {
-                    const float t[4] = {q4.x, q4.y, q4.z, q4.w};
-                    for (int l = 0; l < 4 && f + l < n; ++l) Q[f + l] = t[l];
+                if (f + 16 <= n) {
+                    float4 *dst = reinterpret_cast<float4 *>(Q + f);
+                    dst[0] = make_float4(q[0], q[1], q[2], q[3]);
+                    dst[1] = make_float4(q[4], q[5], q[6], q[7]);
+                    dst[2] = make_float4(q[8], q[9], q[10], q[11]);
+                    dst[3] = make_float4(q[12], q[13], q[14], q[15]);
+                } else {
+#pragma unroll
+                    for (int l = 0; l < 16; ++l)
+                        if (f + l < n) Q[f + l] = q[l];
                 }
             }
-            // sign plane: 8 lanes make one 32-bit word
-            {
-                unsigned nib = (v.x < 0.f ? 1u : 0u) | (v.y < 0.f ? 2u : 0u) |
-                               (v.z < 0.f ? 4u : 0u) | (v.w < 0.f ? 8u : 0u);
-                nib <<= 4 * (lane & 7);
-                nib |= __shfl_xor_sync(0xffffffffu, nib, 1);
-                nib |= __shfl_xor_sync(0xffffffffu, nib, 2);
-                nib |= __shfl_xor_sync(0xffffffffu, nib, 4);
-                const long long wi = chunk * 4 + (lane >> 3);
-                if ((lane & 7) == 0 && wi < n_sign_words) sign_bits[wi] = nib;
-            }
-            // class bitmaps
-            if (B == 2) {
-                const unsigned c0 = __shfl_sync(0xffffffffu, cls, lane >> 1);
-                const unsigned c1 = __shfl_sync(0xffffffffu, cls, 16 + (lane >> 1));
-                const unsigned sh = 2 * (lane & 1);
-                word_p = __ballot_sync(0xffffffffu, (c0 >> sh) & 1u);
-                word_u = __ballot_sync(0xffffffffu, (c0 >> (sh + 1)) & 1u);
-                word_p2 = __ballot_sync(0xffffffffu, (c1 >> sh) & 1u);
-                word_u2 = __ballot_sync(0xffffffffu, (c1 >> (sh + 1)) & 1u);
+            if (j0 + NBT <= p.n_blocks) {
+                if (NBT == 1) u_out[j0] = uo[0];
+                else if (NBT == 2) *reinterpret_cast<float2 *>(u_out + j0) = make_float2(uo[0], uo[1 % NBT]);
+                else {
+#pragma unroll
+                    for (int e = 0; e < NBT; e += 4)
+                        *reinterpret_cast<float4 *>(u_out + j0 + e) =
+                            make_float4(uo[e % NBT], uo[(e + 1) % NBT], uo[(e + 2) % NBT], uo[(e + 3) % NBT]);
+                }
             } else {
-                constexpr int LPB = B / 4;
-                const unsigned c = __shfl_sync(0xffffffffu, cls, (lane * LPB) & 31);
-                const unsigned valid = (BPC >= 32) ? 0xffffffffu : ((1u << BPC) - 1u);
-                const unsigned bp = __ballot_sync(0xffffffffu, c & 1u) & valid;
-                const unsigned bu = __ballot_sync(0xffffffffu, (c >> 1) & 1u) & valid;
-                word_p |= bp << ((it * BPC) & 31);
-                word_u |= bu << ((it * BPC) & 31);
+#pragma unroll
+                for (int e = 0; e < NBT; ++e)
+                    if (j0 + e < p.n_blocks) u_out[j0 + e] = uo[e];
             }
         }
-        if (lane == 0) {
-            if (B == 2) {
-                const long long w0 = task * 2;
-                if (w0 < n_bm_words) { pruned_bitmap[w0] = word_p; unified_bitmap[w0] = word_u; }
-                if (w0 + 1 < n_bm_words) { pruned_bitmap[w0 + 1] = word_p2; unified_bitmap[w0 + 1] = word_u2; }
-            } else {
-                if (task < n_bm_words) { pruned_bitmap[task] = word_p; unified_bitmap[task] = word_u; }
+        // sign plane: two neighbouring threads make one 32-bit word
+        {
+            unsigned sb = 0;
+#pragma unroll
+            for (int l = 0; l < 16; ++l) sb |= (v[l] < 0.f ? 1u : 0u) << l;
+            const unsigned other = __shfl_xor_sync(0xffffffffu, sb, 1);
+            const long long wi = unit >> 1;
+            if ((lane & 1) == 0 && wi < n_sign_words) sign_bits[wi] = sb | (other << 16);
+        }
+        // class bitmaps: the warp's 32 * NBT blocks make NBT words
+        {
+            const long long word0 = ((unit - lane) * NBT) >> 5;
+#pragma unroll
+            for (int w = 0; w < NBT; ++w) {
+                const int blk = w * 32 + lane;               // block of this warp step that lane reports
+                const unsigned sp = __shfl_sync(0xffffffffu, cls_p, blk / NBT);
+                const unsigned su = __shfl_sync(0xffffffffu, cls_u, blk / NBT);
+                const unsigned wp = __ballot_sync(0xffffffffu, (sp >> (blk % NBT)) & 1u);
+                const unsigned wu = __ballot_sync(0xffffffffu, (su >> (blk % NBT)) & 1u);
+                if (lane == 0 && word0 + w < n_bm_words) {
+                    pruned_bitmap[word0 + w] = wp;
+                    unified_bitmap[word0 + w] = wu;
+                }
             }
         }
     }
@@ -774,37 +761,28 @@ static cudaError_t launch_project(const mwu::proj::Params &p, const mwu_proj_des
                                   float *u, unsigned *pb, unsigned *ub, unsigned *sb, double *loss_u,
                                   double *loss_p, int sm_count, cudaStream_t st) {
     using namespace mwu::proj;
-    const long long n_quads = (p.n_floats + 3) / 4;
-    long long want = (n_quads + 255) / 256;
+    sample_kernel<B><<<1, NSAMP, 0, st>>>(p, desc->k_unify, desc->k_prune);
+    const long long n_units = (p.n_floats + 15) / 16;
+    const long long want = (n_units + 255) / 256;
     const long long cap_blocks = (long long)sm_count * 8;
-    const int grid_stats = (int)(want < cap_blocks ? (want > 0 ? want : 1) : cap_blocks);
-    stats_kernel<B><<<grid_stats, 256, 0, st>>>(p, loss_u, loss_p);
-    cudaError_t e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
+    const int grid_stream = (int)(want < cap_blocks ? (want > 0 ? want : 1) : cap_blocks);
+    stats_kernel<B><<<grid_stream, 256, 0, st>>>(p, loss_u, loss_p);
 
-    Params pp = p;
-    void *args[] = {&pp};
     const long long mb = p.n_blocks;
-    long long rb = (mb + RESOLVE_THREADS - 1) / RESOLVE_THREADS;
-    const int grid_res = (int)(rb < sm_count ? (rb > 0 ? rb : 1) : sm_count);
+    const long long rb = (mb + FIN_THREADS - 1) / FIN_THREADS;
+    const int grid_fin = (int)(rb < 2LL * sm_count ? (rb > 0 ? rb : 1) : 2LL * sm_count);
     const bool need_p = desc->k_prune > 0 && desc->k_prune < mb;
     const long long ksel_u = desc->k_unify - desc->k_prune;
     const bool need_u = ksel_u > 0 && ksel_u < mb - desc->k_prune;
     if (need_p) {
-        e = cudaLaunchCooperativeKernel((void *)resolve_kernel<0>, dim3(grid_res), dim3(RESOLVE_THREADS),
-                                        args, 0, st);
-        if (e != cudaSuccess) return e;
+        bin_kernel<0><<<1, FIN_THREADS, 0, st>>>(p);
+        collect_kernel<0, B><<<grid_fin, FIN_THREADS, 0, st>>>(p);
     }
     if (need_u) {
-        e = cudaLaunchCooperativeKernel((void *)resolve_kernel<1>, dim3(grid_res), dim3(RESOLVE_THREADS),
-                                        args, 0, st);
-        if (e != cudaSuccess) return e;
+        histu_kernel<B><<<grid_fin, FIN_THREADS, 0, st>>>(p);
+        collect_kernel<1, B><<<grid_fin, FIN_THREADS, 0, st>>>(p);
     }
-    constexpr int CPT = (B >= 4) ? B / 4 : 1;
-    const long long n_tasks = ((p.n_floats + 127) / 128 + CPT - 1) / CPT;
-    long long eb = (n_tasks + 7) / 8;
-    const int grid_emit = (int)(eb < cap_blocks ? (eb > 0 ? eb : 1) : cap_blocks);
-    emit_kernel<B><<<grid_emit, 256, 0, st>>>(p, Q, u, pb, ub, sb);
+    emit_kernel<B><<<grid_stream, 256, 0, st>>>(p, Q, u, pb, ub, sb);
     return cudaGetLastError();
 }
 
@@ -844,8 +822,6 @@ extern "C" int mwu_project(const mwu_proj_desc *desc, const float *W, const floa
     p.dev_status = dev_status;
 
     if (cudaMemsetAsync(ws, 0, ws_off_cand_key(), st) != cudaSuccess) return MWU_ERR_CUDA;
-    proj::sample_kernel<<<1, 1024, 0, st>>>(p, desc->k_unify, desc->k_prune);
-    if (cudaGetLastError() != cudaSuccess) return MWU_ERR_CUDA;
     cudaError_t e;
     switch (desc->block) {
         case 2: e = launch_project<2>(p, desc, Q, u, pruned_bitmap, unified_bitmap, sign_bits, loss_u, loss_p, sm_count, st); break;
