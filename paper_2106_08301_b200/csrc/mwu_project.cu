@@ -1,7 +1,7 @@
 // mwu_project: Q = Unify(W + U), the Q-step of ADMM (Algorithm 1, Eq. 7) for 1-D micro-blocks.
 //
 // Pipeline (all on the caller's stream, no host synchronisation):
-//   sample_kernel   one CTA looks at <= 1024 evenly spaced blocks and places a narrow window of
+//   sample_kernel   one CTA ranks <= 256 evenly spaced blocks and places a narrow window of
 //                   8190 bins around the k-th smallest key of each selection (prune key, L_u).
 //                   The window only steers efficiency; any window gives the same result.
 //   stats_kernel    streams W (+U) once; every thread owns 64 contiguous bytes (four 128-bit
@@ -25,7 +25,7 @@ namespace proj {
 
 constexpr int NB = 8192;        // level-0 bins: 0 = below the window, NB-1 = above it
 constexpr int CAP = 2048;       // candidates sorted by the last step
-constexpr int NSAMP = 1024;
+constexpr int NSAMP = 256;
 constexpr int FIN_THREADS = 1024;   // block size of the kernels whose last CTA finalises
 
 typedef unsigned long long u64;
@@ -171,31 +171,19 @@ __device__ __forceinline__ void load16(const float *W, const float *U, long long
 // ---------------------------------------------------------------------------------------------
 // sample_kernel: choose the level-0 windows
 // ---------------------------------------------------------------------------------------------
-__device__ void bitonic_sort_u64(u64 *a, int n_pow2) {
-    for (int k = 2; k <= n_pow2; k <<= 1) {
-        for (int j = k >> 1; j > 0; j >>= 1) {
-            for (int i = threadIdx.x; i < n_pow2; i += blockDim.x) {
-                const int ixj = i ^ j;
-                if (ixj > i) {
-                    const u64 x = a[i], y = a[ixj];
-                    const bool up = ((i & k) == 0);
-                    if ((x > y) == up) { a[i] = y; a[ixj] = x; }
-                }
-            }
-            __syncthreads();
-        }
-    }
-}
-
-__device__ void window_from_sorted(const u64 *a, int n, double frac, Sel *s) {
-    // n sorted sample keys; the target quantile is `frac`; keep +-4 sigma (binomial) around it
+// Window around the `frac` quantile of n sample keys: +-4 sigma (binomial) in rank.  Returns the
+// two ranks whose keys bound the window and the rank of the quantile itself.
+__device__ __forceinline__ void window_ranks(int n, double frac, int *il, int *ih, int *ipos) {
     const double pos = frac * n;
     const double margin = 4.0 * sqrt(fmax(n * frac * (1.0 - frac), 0.0)) + 4.0;
-    long long il = (long long)floor(pos - margin);
-    long long ih = (long long)ceil(pos + margin);
-    if (il < 0) il = 0;
-    if (ih > n - 1) ih = n - 1;
-    u64 lo = a[il], hi = a[ih];
+    long long a = (long long)floor(pos - margin), b = (long long)ceil(pos + margin), c = (long long)pos;
+    if (a < 0) a = 0;
+    if (b > n - 1) b = n - 1;
+    if (c > n - 1) c = n - 1;
+    *il = (int)a; *ih = (int)b; *ipos = (int)c;
+}
+
+__device__ __forceinline__ void set_window(Sel *s, u64 lo, u64 hi) {
     if (hi < lo) hi = lo;
     unsigned shift = 0;
     while (((hi - lo) >> shift) >= (u64)(NB - 2)) ++shift;
@@ -204,11 +192,21 @@ __device__ void window_from_sorted(const u64 *a, int n, double frac, Sel *s) {
     s->shift0 = shift;
 }
 
+// rank of (key, i) among the n keys in shared memory (ties ordered by position)
+__device__ __forceinline__ int rank_of(const u64 *keys, int n, u64 key, int i) {
+    int r = 0;
+    for (int t = 0; t < n; ++t) {
+        const u64 k = keys[t];
+        r += (k < key || (k == key && t < i)) ? 1 : 0;
+    }
+    return r;
+}
+
 template <int B>
 __global__ void __launch_bounds__(NSAMP) sample_kernel(Params p, long long k_unify, long long k_prune) {
     __shared__ u64 skey[NSAMP];
+    __shared__ u64 s_stat[3];                  // keys at the ranks il, ih, ipos
     __shared__ int s_kept;
-    __shared__ u64 s_That;
     const long long mb = p.n_blocks;
     const int ns = (int)(mb < (long long)NSAMP ? mb : (long long)NSAMP);
     const int i = threadIdx.x;
@@ -226,29 +224,38 @@ __global__ void __launch_bounds__(NSAMP) sample_kernel(Params p, long long k_uni
     Sel *sp = &p.work->sel[0];
     Sel *su = &p.work->sel[1];
     const long long ksel_u = k_unify - k_prune;
-    bitonic_sort_u64(skey, NSAMP);
-    if (i == 0) {
-        const double fp = (double)k_prune / (double)mb;
-        window_from_sorted(skey, ns, fp, sp);
-        sp->mode = (k_prune == 0) ? 1u : (k_prune == mb ? 2u : 0u);
-        sp->k = (u64)k_prune;
-        long long pos = (long long)(fp * ns);
-        if (pos > ns - 1) pos = ns - 1;
-        s_That = (k_prune == 0) ? 0ull : skey[pos];
+    int il, ih, ipos;
+    window_ranks(ns, (double)k_prune / (double)mb, &il, &ih, &ipos);
+    if (i < ns) {
+        const int r = rank_of(skey, ns, kp, i);
+        if (r == il) s_stat[0] = kp;
+        if (r == ih) s_stat[1] = kp;
+        if (r == ipos) s_stat[2] = kp;
     }
     __syncthreads();
-    const u64 That = s_That;
-    __syncthreads();
-    u64 v = ~0ull;
-    if (i < ns && (k_prune == 0 || kp > That)) { v = ku; atomicAdd(&s_kept, 1); }
-    skey[i] = v;
-    __syncthreads();
-    bitonic_sort_u64(skey, NSAMP);
+    const u64 That = s_stat[2];
     if (i == 0) {
-        const int nr = s_kept > 0 ? s_kept : 1;
-        const long long elig = mb - k_prune;
-        const double fu = elig > 0 ? (double)ksel_u / (double)elig : 0.0;
-        window_from_sorted(skey, nr, fu, su);
+        set_window(sp, s_stat[0], s_stat[1]);
+        sp->mode = (k_prune == 0) ? 1u : (k_prune == mb ? 2u : 0u);
+        sp->k = (u64)k_prune;
+    }
+    // the sample blocks that survive the (estimated) prune threshold
+    const bool kept = i < ns && (k_prune == 0 || kp > That);
+    __syncthreads();
+    skey[i] = kept ? ku : ~0ull;
+    if (kept) atomicAdd(&s_kept, 1);
+    __syncthreads();
+    const int nr = s_kept > 0 ? s_kept : 1;
+    const long long elig = mb - k_prune;
+    window_ranks(nr, elig > 0 ? (double)ksel_u / (double)elig : 0.0, &il, &ih, &ipos);
+    if (i < ns) {
+        const int r = rank_of(skey, ns, kept ? ku : ~0ull, i);     // dropped samples rank last
+        if (r == il) s_stat[0] = skey[i];
+        if (r == ih) s_stat[1] = skey[i];
+    }
+    __syncthreads();
+    if (i == 0) {
+        set_window(su, s_stat[0], s_stat[1]);
         su->mode = (ksel_u == 0) ? 1u : (ksel_u == elig ? 2u : 0u);
         su->k = (u64)ksel_u;
     }
@@ -451,6 +458,17 @@ __global__ void __launch_bounds__(FIN_THREADS) bin_kernel(Params p) {
 // ---------------------------------------------------------------------------------------------
 // histu_kernel: histogram of L_u bins over the blocks that were not pruned
 // ---------------------------------------------------------------------------------------------
+// four consecutive bin codes starting at j4 (j4 % 4 == 0); codes beyond n read as 0
+__device__ __forceinline__ void load_codes4(const unsigned *bins, long long j4, long long n, unsigned (&c)[4]) {
+    if (j4 + 4 <= n) {
+        const uint4 v = __ldg(reinterpret_cast<const uint4 *>(bins + j4));
+        c[0] = v.x; c[1] = v.y; c[2] = v.z; c[3] = v.w;
+    } else {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) c[e] = (j4 + e < n) ? __ldg(bins + j4 + e) : 0u;
+    }
+}
+
 template <int B>
 __global__ void __launch_bounds__(FIN_THREADS) histu_kernel(Params p) {
     Sel *s = &p.work->sel[1];
@@ -459,13 +477,19 @@ __global__ void __launch_bounds__(FIN_THREADS) histu_kernel(Params p) {
     const SelView pv = view_of(&p.work->sel[0]);
     const long long stride = (long long)gridDim.x * blockDim.x;
     unsigned under = 0, over = 0;
-    for (long long j = (long long)blockIdx.x * blockDim.x + threadIdx.x; j < p.n_blocks; j += stride) {
-        const unsigned code = __ldg(p.bins + j);
-        if (selected<B>(p, pv, j, code & 0xffffu, 0)) continue;
-        const unsigned bu = code >> 16;
-        if (bu == 0) ++under;
-        else if (bu == NB - 1) ++over;
-        else atomicAdd(&hist[bu], 1u);
+    for (long long j4 = ((long long)blockIdx.x * blockDim.x + threadIdx.x) * 4; j4 < p.n_blocks; j4 += stride * 4) {
+        unsigned codes[4];
+        load_codes4(p.bins, j4, p.n_blocks, codes);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const long long j = j4 + e;
+            if (j >= p.n_blocks) break;
+            if (selected<B>(p, pv, j, codes[e] & 0xffffu, 0)) continue;
+            const unsigned bu = codes[e] >> 16;
+            if (bu == 0) ++under;
+            else if (bu == NB - 1) ++over;
+            else atomicAdd(&hist[bu], 1u);
+        }
     }
     for (int m = 16; m > 0; m >>= 1) {
         under += __shfl_xor_sync(0xffffffffu, under, m);
@@ -515,16 +539,22 @@ __global__ void __launch_bounds__(FIN_THREADS) collect_kernel(Params p) {
     if (!too_many) {
         const u128 lo = from_halves(ld_vol(&s->lo_hi), ld_vol(&s->lo_lo));
         const u128 hi = from_halves(ld_vol(&s->hi_hi), ld_vol(&s->hi_lo));
-        for (long long j = (long long)blockIdx.x * blockDim.x + threadIdx.x; j < p.n_blocks; j += stride) {
-            const unsigned code = __ldg(p.bins + j);
-            const unsigned bin = KIND ? (code >> 16) : (code & 0xffffu);
-            if (bin != Bsel) continue;
-            if (KIND == 1 && selected<B>(p, pv, j, code & 0xffffu, 0)) continue;
-            const u64 key = exact_key<B>(p, j, KIND);
-            const u128 c = make_c(key, (u64)j);
-            if (c >= lo && c < hi) {
-                const unsigned slot = atomicAdd(&p.work->cand_count[KIND], 1u);
-                if (slot < (unsigned)CAP) { p.cand_key[slot] = key; p.cand_idx[slot] = (unsigned)j; }
+        for (long long j4 = ((long long)blockIdx.x * blockDim.x + threadIdx.x) * 4; j4 < p.n_blocks; j4 += stride * 4) {
+            unsigned codes[4];
+            load_codes4(p.bins, j4, p.n_blocks, codes);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const long long j = j4 + e;
+                const unsigned code = codes[e];
+                const unsigned bin = KIND ? (code >> 16) : (code & 0xffffu);
+                if (j >= p.n_blocks || bin != Bsel) continue;
+                if (KIND == 1 && selected<B>(p, pv, j, code & 0xffffu, 0)) continue;
+                const u64 key = exact_key<B>(p, j, KIND);
+                const u128 c = make_c(key, (u64)j);
+                if (c >= lo && c < hi) {
+                    const unsigned slot = atomicAdd(&p.work->cand_count[KIND], 1u);
+                    if (slot < (unsigned)CAP) { p.cand_key[slot] = key; p.cand_idx[slot] = (unsigned)j; }
+                }
             }
         }
     }
@@ -616,7 +646,7 @@ __global__ void __launch_bounds__(FIN_THREADS) collect_kernel(Params p) {
 // emit_kernel
 // ---------------------------------------------------------------------------------------------
 template <int B>
-__global__ void __launch_bounds__(256) emit_kernel(Params p, float *Q, float *u_out,
+__global__ void __launch_bounds__(256, 3) emit_kernel(Params p, float *Q, float *u_out,
                                                    unsigned *pruned_bitmap, unsigned *unified_bitmap,
                                                    unsigned *sign_bits) {
     constexpr int NBT = 16 / B;
@@ -769,8 +799,8 @@ static cudaError_t launch_project(const mwu::proj::Params &p, const mwu_proj_des
     stats_kernel<B><<<grid_stream, 256, 0, st>>>(p, loss_u, loss_p);
 
     const long long mb = p.n_blocks;
-    const long long rb = (mb + FIN_THREADS - 1) / FIN_THREADS;
-    const int grid_fin = (int)(rb < 2LL * sm_count ? (rb > 0 ? rb : 1) : 2LL * sm_count);
+    const long long rb = (mb + 4 * FIN_THREADS - 1) / (4 * FIN_THREADS);
+    const int grid_fin = (int)(rb < (long long)sm_count ? (rb > 0 ? rb : 1) : (long long)sm_count);
     const bool need_p = desc->k_prune > 0 && desc->k_prune < mb;
     const long long ksel_u = desc->k_unify - desc->k_prune;
     const bool need_u = ksel_u > 0 && ksel_u < mb - desc->k_prune;
