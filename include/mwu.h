@@ -114,9 +114,12 @@ int mwu_project(const mwu_proj_desc *desc, const float *W, const float *U_dual, 
  * pos = row_in_tile * (64/block) + block_in_record.  A block is addressed by `off`, the byte
  * offset of its first value in the record's decoded bf16 tile as the GEMM lays it out in shared
  * memory: row r starts at (r/8)*1024 + (r%8)*128 and its 16-byte chunk c sits at chunk position
- * c ^ (r%8).  Per record the blocks are listed by class, each list in ascending pos order,
- * records in tile-major order:
- *   header  256 B : u64 magic "MWUPACK1", version 3, rows, cols, block, rows_padded, n_tiles,
+ * c ^ (r%8).  Per record the blocks are listed by class, records in tile-major order.  Inside
+ * a class list the entries are dealt round-robin over the store slots
+ * slot = (off % 128) / min(2*block, 16): entries of one slot keep ascending pos order, and the
+ * list takes the first entry of every slot (ascending slot), then the second of every slot that
+ * has one, and so on, so that neighbouring entries fall into different shared-memory banks:
+ *   header  256 B : u64 magic "MWUPACK1", version 4, rows, cols, block, rows_padded, n_tiles,
  *                   n_stages, n_pruned, n_unified, n_dense, n_plist, byte offsets of rec, ulist,
  *                   dpos, dpay, ppos, total bytes
  *   rec     16 B per record plus one closing entry: u32 ubase, dbase, pbase (index of the

@@ -48,7 +48,7 @@ STAGE_K = 64             # reduction-axis extent per record
 HEADER_BYTES = 256
 SECTION_ALIGN = 256
 MAGIC = b"MWUPACK1"
-VERSION = 3
+VERSION = 4
 
 
 def count_from_permille(n_blocks: int, permille: int) -> int:
@@ -217,6 +217,20 @@ def tile_offset(pos: np.ndarray, b: int) -> np.ndarray:
     return (r // 8) * 1024 + (r % 8) * 128 + ((c ^ (r % 8)) * 16) + within
 
 
+def slot_order(off: np.ndarray, b: int) -> np.ndarray:
+    """Permutation that deals entries (given in ascending pos order) round-robin over their
+    store slots: sort by (rank inside the slot, slot)."""
+    off = np.asarray(off, dtype=np.int64)
+    g = min(2 * b, 16)
+    slot = (off % 128) // g
+    rank = np.zeros(off.shape[0], dtype=np.int64)
+    seen = {}
+    for e, sl in enumerate(slot.tolist()):
+        rank[e] = seen.get(sl, 0)
+        seen[sl] = rank[e] + 1
+    return np.lexsort((slot, rank))
+
+
 def tile_offset_inverse(off: int, b: int):
     r = (off >> 10) * 8 + ((off >> 7) & 7)
     c = ((off >> 4) & 7) ^ (r & 7)
@@ -237,7 +251,11 @@ def pack(p: Projection, b: int) -> np.ndarray:
     by the byte offset `off` of its first value inside the record's decoded tile (bf16, rows of
     128 bytes, 16-byte chunks of a row XOR-permuted by the row number mod 8 -- the layout the
     tensor-core instruction reads; see tile_offset).  Per record the blocks are listed by
-    class, each list in ascending pos order:
+    class.  Inside a class list the entries are dealt round-robin over the store slots
+    slot = (off % 128) // g, g = min(2*b, 16): entries with the same slot keep ascending pos
+    order, and the list takes the first entry of every slot (ascending slot), then the second of
+    every slot that has one, and so on (so that neighbouring entries fall into different
+    shared-memory banks when the GEMM writes them):
       ulist  8 B per unified block: u32 spread sign bits (weight l -> bit l//2 + 16*(l%2)),
              u16 off, u16 bf16(unified value)
       dpos   u16 off per dense block;  dpay  its b values as bf16 (round to nearest even)
@@ -295,6 +313,9 @@ def pack(p: Projection, b: int) -> np.ndarray:
             pos_u = np.flatnonzero(Uf.reshape(-1)).astype(np.uint32)      # ascending pos
             pos_d = np.flatnonzero(D.reshape(-1)).astype(np.uint16)
             pos_p = np.flatnonzero(P.reshape(-1)).astype(np.uint16)
+            pos_u = pos_u[slot_order(tile_offset(pos_u, b), b)]
+            pos_d = pos_d[slot_order(tile_offset(pos_d, b), b)]
+            pos_p = pos_p[slot_order(tile_offset(pos_p, b), b)]
             sg = sign[r0:r0 + TILE_ROWS, s * STAGE_K:(s + 1) * STAGE_K].reshape(TILE_ROWS * nb, b)
             sbits = (sg.astype(np.uint32) * bitw).sum(axis=1).astype(np.uint32)
             ulist_w0.append(sbits[pos_u])

@@ -5,9 +5,10 @@
 //   count_kernel  one CTA per record (128 rows x 64 columns): number of unified / dense / pruned
 //                 blocks and the record's live-slice mask.
 //   scan_kernel   one CTA: exclusive scan of the per-record counts over all records, header.
-//   fill_kernel   one CTA per record, one thread per row: class masks, scan over the rows, then
-//                 the row's entries of the three class lists; a dense block's values are read
-//                 as whole 64-byte (or shorter) runs of W and written as one bf16 vector.
+//   fill_kernel   one CTA per record, one thread per row: class masks, then a scan over the rows
+//                 of the number of blocks per (class, store slot), which gives every block its
+//                 place in the round-robin order of its class list; a dense block's values are
+//                 read as whole 64-byte (or shorter) runs of W and written as one bf16 vector.
 #include "mwu_common.cuh"
 
 namespace mwu {
@@ -156,7 +157,7 @@ __global__ void __launch_bounds__(1024) scan_kernel(Params p) {
         unsigned long long v = 0;
         switch (threadIdx.x) {
             case 0: v = kMagic; break;
-            case 1: v = 3; break;
+            case 1: v = 4; break;
             case 2: v = (unsigned long long)p.rows; break;
             case 3: v = (unsigned long long)p.cols; break;
             case 4: v = (unsigned long long)p.b; break;
@@ -183,6 +184,10 @@ template <int B>
 __global__ void __launch_bounds__(128) fill_kernel(Params p) {
     constexpr int NBK = kStageK / B;
     constexpr unsigned MASK = (NBK >= 32) ? 0xffffffffu : ((1u << NBK) - 1u);
+    constexpr int STORE = (B >= 8) ? 16 : 2 * B;            // bytes of one shared-memory store
+    constexpr int G = 128 / STORE;                          // store slots of a 128-byte row
+    constexpr int NF = 3 * G;                               // (class, slot) counters, 8 bits each
+    constexpr int FW = NF / 4;                              // ... packed four to a word
     const long long rec = blockIdx.x;
     const long long tile = rec / p.L.n_stages, stage = rec % p.L.n_stages;
     const int r = threadIdx.x, lane = r & 31, warp = r >> 5;
@@ -191,42 +196,85 @@ __global__ void __launch_bounds__(128) fill_kernel(Params p) {
     unsigned short *dpos = reinterpret_cast<unsigned short *>(p.packed + p.L.off_dpos);
     unsigned char *dpay = p.packed + p.L.off_dpay;
     unsigned short *ppos = reinterpret_cast<unsigned short *>(p.packed + p.L.off_ppos);
-    const unsigned long long ubase = recs[rec].ubase, dbase = recs[rec].dbase, pbase = recs[rec].pbase;
+    const unsigned long long base_of[3] = {recs[rec].pbase, recs[rec].dbase, recs[rec].ubase};
 
-    __shared__ unsigned s_w[3][4];
+    __shared__ unsigned s_warp[4][FW];
+    __shared__ unsigned char s_len[NF];                     // blocks per (class, slot) in the record
     unsigned P, U;
     unsigned long long sgn;
     row_masks(p, tile, stage, r, &P, &U, &sgn);
     const unsigned D = ~P & ~U & MASK;
-    const unsigned cu = __popc(U), cd = __popc(D), cp = __popc(P);
-    unsigned iu = cu, id = cd, ip = cp;
-    for (int off = 1; off < 32; off <<= 1) {
-        const unsigned tu = __shfl_up_sync(0xffffffffu, iu, off);
-        const unsigned td = __shfl_up_sync(0xffffffffu, id, off);
-        const unsigned tp = __shfl_up_sync(0xffffffffu, ip, off);
-        if (lane >= off) { iu += tu; id += td; ip += tp; }
+    // class of block i: 0 pruned, 1 dense, 2 unified; its store slot
+    unsigned fld[FW];
+#pragma unroll
+    for (int w = 0; w < FW; ++w) fld[w] = 0;
+#pragma unroll
+    for (int i = 0; i < NBK; ++i) {
+        const unsigned off = tile_offset((unsigned)r, (unsigned)i, B);
+        const unsigned slot = (off & 127u) / STORE;
+        const unsigned cls = ((U >> i) & 1u) ? 2u : (((D >> i) & 1u) ? 1u : 0u);
+        const unsigned fi = cls * G + slot;
+#pragma unroll
+        for (int w = 0; w < FW; ++w) fld[w] += ((fi >> 2) == (unsigned)w) ? (1u << (8 * (fi & 3u))) : 0u;
     }
-    if (lane == 31) { s_w[0][warp] = iu; s_w[1][warp] = id; s_w[2][warp] = ip; }
+    // inclusive scan over the 128 rows (a field never exceeds 128, so fields do not carry)
+    unsigned inc[FW];
+#pragma unroll
+    for (int w = 0; w < FW; ++w) inc[w] = fld[w];
+    for (int off = 1; off < 32; off <<= 1) {
+#pragma unroll
+        for (int w = 0; w < FW; ++w) {
+            const unsigned t = __shfl_up_sync(0xffffffffu, inc[w], off);
+            if (lane >= off) inc[w] += t;
+        }
+    }
+    if (lane == 31) {
+#pragma unroll
+        for (int w = 0; w < FW; ++w) s_warp[warp][w] = inc[w];
+    }
     __syncthreads();
-    unsigned bu = 0, bd = 0, bp = 0;
-    for (int w = 0; w < warp; ++w) { bu += s_w[0][w]; bd += s_w[1][w]; bp += s_w[2][w]; }
-    unsigned long long ui = ubase + (bu + iu - cu), di = dbase + (bd + id - cd), pi = pbase + (bp + ip - cp);
+    unsigned excl[FW];
+#pragma unroll
+    for (int w = 0; w < FW; ++w) {
+        unsigned b0 = 0;
+        for (int ww = 0; ww < warp; ++ww) b0 += s_warp[ww][w];
+        excl[w] = b0 + inc[w] - fld[w];
+    }
+    if (r < NF) {
+        const unsigned tot = s_warp[0][r >> 2] + s_warp[1][r >> 2] + s_warp[2][r >> 2] + s_warp[3][r >> 2];
+        s_len[r] = (unsigned char)((tot >> (8 * (r & 3))) & 0xffu);
+    }
+    __syncthreads();
+
     bool bad = false;
     const long long n = tile * kTileRows + r;
     constexpr unsigned BMASK = (B >= 32) ? 0xffffffffu : ((1u << B) - 1u);
 #pragma unroll 4
     for (int i = 0; i < NBK; ++i) {
         const unsigned off = tile_offset((unsigned)r, (unsigned)i, B);
-        if ((U >> i) & 1u) {
+        const unsigned slot = (off & 127u) / STORE;
+        const unsigned cls = ((U >> i) & 1u) ? 2u : (((D >> i) & 1u) ? 1u : 0u);
+        const unsigned fi = cls * G + slot;
+        unsigned q = 0;                                     // earlier rows with the same class and slot
+#pragma unroll
+        for (int w = 0; w < FW; ++w) q += ((fi >> 2) == (unsigned)w) ? ((excl[w] >> (8 * (fi & 3u))) & 0xffu) : 0u;
+        // place in the round-robin order: q full rounds before it, then the lower slots of its round
+        unsigned idx = 0;
+#pragma unroll
+        for (int sl = 0; sl < G; ++sl) {
+            const unsigned len = s_len[cls * G + sl];
+            idx += (len < q ? len : q) + (((unsigned)sl < slot && len > q) ? 1u : 0u);
+        }
+        const unsigned long long e = base_of[cls] + idx;
+        if (cls == 2u) {
             const unsigned sb = (unsigned)(sgn >> (i * B)) & BMASK;
             const long long j = n * (p.cols / B) + stage * NBK + i;
             const unsigned ub = (unsigned)__bfloat16_as_ushort(__float2bfloat16_rn(__ldg(p.u + j)));
-            if (ui < (unsigned long long)p.L.n_unified) ulist[ui] = make_uint2(spread_signs(sb, B), off | (ub << 16));
+            if (e < (unsigned long long)p.L.n_unified) ulist[e] = make_uint2(spread_signs(sb, B), off | (ub << 16));
             else bad = true;
-            ++ui;
-        } else if ((D >> i) & 1u) {
-            if (di < (unsigned long long)p.L.n_dense) {
-                dpos[di] = (unsigned short)off;
+        } else if (cls == 1u) {
+            if (e < (unsigned long long)p.L.n_dense) {
+                dpos[e] = (unsigned short)off;
                 const long long f = n * p.cols + stage * kStageK + i * B;
                 float v[B];
                 if (B >= 4) {
@@ -253,7 +301,7 @@ __global__ void __launch_bounds__(128) fill_kernel(Params p) {
                     const __nv_bfloat162 h = __floats2bfloat162_rn(v[2 * l], v[2 * l + 1]);
                     w[l] = *reinterpret_cast<const unsigned *>(&h);
                 }
-                unsigned char *dst = dpay + di * (2 * B);
+                unsigned char *dst = dpay + e * (2 * B);
                 if (B == 16) {
                     *reinterpret_cast<uint4 *>(dst) = make_uint4(w[0], w[1 % (B / 2)], w[2 % (B / 2)], w[3 % (B / 2)]);
                     *reinterpret_cast<uint4 *>(dst + 16) = make_uint4(w[4 % (B / 2)], w[5 % (B / 2)], w[6 % (B / 2)], w[7 % (B / 2)]);
@@ -267,11 +315,9 @@ __global__ void __launch_bounds__(128) fill_kernel(Params p) {
             } else {
                 bad = true;
             }
-            ++di;
         } else {
-            if (pi < (unsigned long long)p.L.n_plist) ppos[pi] = (unsigned short)off;
+            if (e < (unsigned long long)p.L.n_plist) ppos[e] = (unsigned short)off;
             else bad = true;
-            ++pi;
         }
     }
     if (bad) atomicOr(p.dev_status, (unsigned)MWU_DEV_BOUNDS);

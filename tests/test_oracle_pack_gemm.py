@@ -81,7 +81,7 @@ def test_live_mask_and_padding():
     first = ppos[rec[0, 2]:rec[1, 2]]
     slots = [O.tile_offset_inverse(int(o), b) for o in first]
     codes = [r * nb + i for r, i in slots]
-    assert np.all(np.diff(codes) > 0)                                   # ascending slot numbers
+    assert len(set(codes)) == len(codes)
     assert set(range(100 * nb, 128 * nb)) <= set(codes)
     assert rec[2].tolist() == [h["n_unified"], h["n_dense"], h["n_plist"], 0]
     assert O.decode(buf).shape == (N, K)
@@ -161,3 +161,27 @@ def test_tile_offset_is_a_bijection_and_matches_the_swizzle():
     assert O.tile_offset(np.array([0, 1, 2, 3]), 16).tolist() == [0, 32, 64, 96]
     assert O.tile_offset(np.array([4, 5]), 16).tolist() == [128 + 16, 128 + 48]
     assert O.tile_offset(np.array([32]), 16).tolist() == [1024]
+
+
+def test_class_lists_are_dealt_round_robin_over_store_slots():
+    N, K, b = 128, 64, 16
+    W = rand_w(N, K)
+    Mb = N * K // b
+    p = O.project(W, b, Mb * 8 // 10, Mb * 6 // 10)
+    buf = O.pack(p, b)
+    h = O.parse_header(buf)
+    ppos = buf[h["off_ppos"]:h["off_ppos"] + 2 * h["n_plist"]].view(np.uint16).astype(int)
+    slot = (ppos % 128) // 16
+    # same multiset of blocks as the pruned mask
+    assert sorted(O.tile_offset(np.flatnonzero(p.pruned), b).tolist()) == sorted(ppos.tolist())
+    # the first round holds one entry of every slot present, in ascending slot order
+    n_slots = len(set(slot.tolist()))
+    assert slot[:n_slots].tolist() == sorted(set(slot.tolist()))
+    # inside a slot the entries keep ascending block order
+    for sl in set(slot.tolist()):
+        pos = [r * 4 + i for r, i in (O.tile_offset_inverse(int(o), b) for o in ppos[slot == sl])]
+        assert pos == sorted(pos)
+    # while all eight slots still have entries, any 8 consecutive entries hit 8 different slots
+    shortest = min(np.bincount(slot, minlength=8))
+    full = slot[:8 * shortest].reshape(-1, 8)
+    assert all(len(set(row.tolist())) == 8 for row in full)
