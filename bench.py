@@ -26,11 +26,11 @@ import torch
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
-from paper_2106_08301_b200 import inputs  # noqa: E402
+from paper_2106_08301_b200 import inputs, replicas  # noqa: E402
 
 METRIC = "mwu_hot_path_effective_tflops"
 UNIT = "TFLOP/s"
-KERNELS_PER_STEP = 9      # sample, stats, resolve x2, emit | count, scan, fill | gemm
+KERNELS_PER_STEP = 11     # sample, stats, bin, collect x2, histu, emit | count, scan, fill | gemm
 
 
 def measured_peaks():
@@ -270,11 +270,7 @@ def run_gpu(args):
     t_end.record(stream)
     barrier()
     sampler.stop()
-    total_ms = t_begin.elapsed_time(t_end)
-    if dist is not None:
-        t = torch.tensor([total_ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = replicas.max_over_ranks(t_begin.elapsed_time(t_end), dist, "cuda")
     ms_per_step = total_ms / args.steps
     proj_ms = statistics.mean(e[0].elapsed_time(e[1]) for e in ev)
     pack_ms = statistics.mean(e[1].elapsed_time(e[2]) for e in ev)
@@ -294,18 +290,14 @@ def run_gpu(args):
         Y_host.copy_(Y, non_blocking=True)
     t1.record(stream)
     barrier()
-    e2e_ms = t0.elapsed_time(t1) / e2e_steps
-    if dist is not None:
-        t = torch.tensor([e2e_ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
+    e2e_ms = replicas.max_over_ranks(t0.elapsed_time(t1) / e2e_steps, dist, "cuda")
 
     flops = effective_flops(wl, m, kp)
     dense_flops = 2.0 * m * wl.rows * wl.cols
     abytes = algorithmic_bytes(wl, m, ku, kp)
     peaks = measured_peaks()
-    value = world * flops / (ms_per_step * 1e-3) / 1e12
-    e2e_value = world * flops / (e2e_ms * 1e-3) / 1e12
+    value = replicas.whole_job_rate(flops, world, ms_per_step) / 1e12
+    e2e_value = replicas.whole_job_rate(flops, world, e2e_ms) / 1e12
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
