@@ -104,6 +104,33 @@ int mwu_project(const mwu_proj_desc *desc, const float *W, const float *U_dual, 
                 void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 /*
+ * mwu_project_static -- mwu_project without a caller-supplied workspace.  (The paper has no
+ * counterpart: this is a packaging variant of the same projection, with the same outputs.)
+ *
+ * For callers that cannot allocate device memory where they need the projection -- code running
+ * inside an engine that owns the memory pool, or after a job's memory budget has been frozen,
+ * where a cudaMalloc may fail or stall the device.  The scratch memory is a fixed array inside
+ * the library's device image (about 4.2 MB, held by every GPU that loads the library until the
+ * process exits), so the call allocates nothing.
+ *
+ * Limits and rules:
+ *   - at most MWU_STATIC_MAX_BLOCKS blocks (rows*cols/block); larger tensors return
+ *     MWU_ERR_WORKSPACE and nothing is launched -- use mwu_project with your own workspace;
+ *   - the first call on each device looks up the device address of the built-in array (one
+ *     runtime query, no allocation); make that first call outside any stream capture;
+ *   - all calls on one device share the array: two calls whose kernels can overlap on the GPU
+ *     (different streams without an ordering between them) race and give undefined results;
+ *     calls on one stream, or otherwise ordered, are fine.  Each call clears the part of the
+ *     scratch that must start at zero, so earlier calls leave no trace.
+ * Arguments, outputs and errors are those of mwu_project.
+ */
+#define MWU_STATIC_MAX_BLOCKS 1048576
+int mwu_project_static(const mwu_proj_desc *desc, const float *W, const float *U_dual, float *Q,
+                       float *u, uint32_t *pruned_bitmap, uint32_t *unified_bitmap,
+                       uint32_t *sign_bits, double *loss_u, double *loss_p, uint32_t *dev_status,
+                       void *cuda_stream);
+
+/*
  * mwu_pack -- the storage form of Section 3.1 / Table 1: a unified block keeps one
  * magnitude, a pruned block nothing, every weight one sign bit, the remaining blocks their
  * values (here rounded to bf16, the type the GEMM multiplies in).

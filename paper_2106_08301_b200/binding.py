@@ -16,7 +16,9 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libmwu.so")
 
 EXPORTS = ["mwu_status_string", "mwu_count_from_permille", "mwu_project_workspace_bytes",
-           "mwu_project", "mwu_packed_bytes", "mwu_pack", "mwu_gemm", "mwu_conv_implicit"]
+           "mwu_project", "mwu_project_static", "mwu_packed_bytes", "mwu_pack", "mwu_gemm",
+           "mwu_conv_implicit"]
+MWU_STATIC_MAX_BLOCKS = 1048576
 
 MWU_OK = 0
 MWU_DEV_NONFINITE, MWU_DEV_TIMEOUT, MWU_DEV_BOUNDS, MWU_DEV_SELECT = 1, 2, 4, 8
@@ -55,6 +57,8 @@ def lib() -> ctypes.CDLL:
         L.mwu_project_workspace_bytes.argtypes = [dp]
         L.mwu_project.restype = ctypes.c_int
         L.mwu_project.argtypes = [dp] + [vp] * 11 + [sz, vp]
+        L.mwu_project_static.restype = ctypes.c_int
+        L.mwu_project_static.argtypes = [dp] + [vp] * 10 + [vp]
         L.mwu_packed_bytes.restype = sz
         L.mwu_packed_bytes.argtypes = [dp]
         L.mwu_pack.restype = ctypes.c_int
@@ -105,6 +109,17 @@ def mwu_project(desc, W, U_dual, Q, u, pruned_bitmap, unified_bitmap, sign_bits,
                            _stream(stream))
     if check and rc != MWU_OK:
         raise MwuError(rc, "mwu_project")
+    return rc
+
+
+def mwu_project_static(desc, W, U_dual, Q, u, pruned_bitmap, unified_bitmap, sign_bits, loss_u,
+                       loss_p, dev_status, stream=None, check=True) -> int:
+    """mwu_project on the library's built-in scratch: no workspace argument, no allocation."""
+    rc = lib().mwu_project_static(ctypes.byref(desc), _ptr(W), _ptr(U_dual), _ptr(Q), _ptr(u),
+                                  _ptr(pruned_bitmap), _ptr(unified_bitmap), _ptr(sign_bits),
+                                  _ptr(loss_u), _ptr(loss_p), _ptr(dev_status), _stream(stream))
+    if check and rc != MWU_OK:
+        raise MwuError(rc, "mwu_project_static")
     return rc
 
 
