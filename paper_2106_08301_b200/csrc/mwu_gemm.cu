@@ -1,19 +1,23 @@
 // mwu_gemm / mwu_conv_implicit: Y = X . W_hat^T on the packed weights (Section 3.2).
 //
-// One persistent CTA per SM, warp-specialised:
-//   warp 0        producer of the activation tile (A operand, 128 rows x 64 k, bf16): one thread
-//                 issues a TMA load per stage (GEMM); for the convolution four extra warps gather
-//                 the im2col rows with plain loads instead.
-//   warp 1        allocates tensor memory and issues tcgen05.mma (one thread); fp32 accumulators
-//                 live in TMEM, two buffers so that the epilogue of tile i overlaps tile i+1.
-//   warps 2-5     epilogue: tcgen05.ld -> bf16/fp32 -> global.
-//   warps 6-21    decode the weight tile (B operand) from the packed class lists into the
-//                 128-byte-swizzled K-major layout the MMA reads: pruned blocks -> zeros,
-//                 unified blocks -> sign . bf16(u), dense blocks -> stored bf16 values.  Four
-//                 groups of four warps, one per pipeline slot, take every fourth live stage, so
-//                 a group has four stage times to hide the latency of its list reads; each
-//                 thread reads a fixed number of list entries per stage (all loads first, then
-//                 the stores).
+// One persistent CTA per SM works on tiles of 256 activation rows x 256 weight rows (GEMM; the
+// convolution and narrow problems use 128 activation rows).  A 64-wide k stage of the weight
+// tile is decoded once into shared memory and multiplied with both 128-row halves of the
+// activation tile, which halves decode work, shared-memory stores and slot hand-shakes per FLOP.
+// Warp roles:
+//   warp 0        producer of the activation tile (A operand, bf16, K-major, 128-byte swizzle):
+//                 one thread issues one TMA load per stage (GEMM); for the convolution four extra
+//                 warps gather the im2col rows with plain loads instead.
+//   warp 1        allocates tensor memory and issues tcgen05.mma (one thread), M = 128, N = 256
+//                 per instruction, fp32 accumulators in TMEM (columns [0,256) for the first half
+//                 of the rows, [256,512) for the second).
+//   warps 2-9     epilogue: tcgen05.ld -> bf16/fp32 -> global, one warp per (half, 32 rows).
+//   warps 10-27   decode the weight tile (B operand) from the packed class lists into the
+//                 swizzled K-major layout the MMA reads: pruned blocks -> zeros, unified blocks
+//                 -> sign . bf16(u), dense blocks -> stored bf16 values.  Three groups of six
+//                 warps, one per pipeline slot.  A group reads the small per-entry words of its
+//                 next stage before it waits for the slot; once the slot is free it writes zeros
+//                 and sign . u words with plain stores and moves dense values with cp.async.
 // A 64-wide k stage whose blocks are pruned in every row of the weight tile is skipped by all
 // roles (no load, no decode, no MMA); inside a live stage the MMA skips dead 16-wide slices.
 // Every wait on an mbarrier is bounded; when one runs out the kernel raises MWU_DEV_TIMEOUT,
@@ -25,19 +29,21 @@
 namespace mwu {
 namespace gemm {
 
-constexpr int BM = 128;                 // rows of X per tile
+constexpr int BMH = 128;                // rows of X per MMA (one half of a tile)
 constexpr int BK = kStageK;             // 64
-constexpr int STAGES = 4;
-constexpr int A_BYTES = BM * BK * 2;    // 16 KiB
+constexpr int STAGES = 3;
+constexpr int AH_BYTES = BMH * BK * 2;  // 16 KiB: one 128-row half of the activation stage
 constexpr int REC_BYTES = kTileRows * BK * 2;
-constexpr int NDEC_WARPS = 4;           // warps per decode group
-constexpr int NDEC_GROUPS = 4;          // one group per pipeline slot
+constexpr int NDEC_GROUPS = STAGES;     // one decode group per pipeline slot
+constexpr int NDEC_WARPS = 6;           // warps per decode group
 constexpr int NDEC_THREADS = NDEC_WARPS * 32;
+constexpr int NEPI_WARPS = 8;
+constexpr int FIRST_DEC_WARP = 2 + NEPI_WARPS;
+constexpr int FIRST_GATHER_WARP = FIRST_DEC_WARP + NDEC_WARPS * NDEC_GROUPS;
 constexpr int NGATHER_WARPS = 4;
-constexpr int FIRST_GATHER_WARP = 6 + NDEC_WARPS * NDEC_GROUPS;
 constexpr int THREADS_GEMM = 32 * FIRST_GATHER_WARP;
-constexpr int MAX_STAGES_K = 256;       // cols <= 16384
 constexpr int THREADS_CONV = THREADS_GEMM + 32 * NGATHER_WARPS;
+constexpr int MAX_STAGES_K = 256;       // cols <= 16384
 constexpr long long WAIT_LIMIT_CYCLES = 4000000000ll;   // about two seconds
 
 struct Params {
@@ -80,8 +86,19 @@ __device__ __forceinline__ bool mbar_try_wait(unsigned bar, unsigned parity) {
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
+// non-blocking probe of a phase
+__device__ __forceinline__ bool mbar_test(unsigned bar, unsigned parity) {
+    unsigned ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
 // bounded wait: false when aborted or out of time (then *abort is set)
 __device__ __forceinline__ bool mbar_wait(unsigned bar, unsigned parity, volatile int *abort) {
+    if (mbar_test(bar, parity)) return true;
 #pragma unroll 1
     for (int i = 0; i < 128; ++i)
         if (mbar_try_wait(bar, parity)) return true;
@@ -92,6 +109,14 @@ __device__ __forceinline__ bool mbar_wait(unsigned bar, unsigned parity, volatil
         if (*abort) return false;
         if (clock64() - t0 > WAIT_LIMIT_CYCLES) { *abort = 1; return false; }
     }
+}
+template <int BYTES>
+__device__ __forceinline__ void cp_async_if(unsigned dst, const void *src, unsigned pred) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.u32 p, %2, 0;\n\t"
+        "@p cp.async.ca.shared.global [%0], [%1], %3;\n\t}"
+        ::"r"(dst), "l"(src), "r"(pred), "n"(BYTES) : "memory");
 }
 __device__ __forceinline__ void fence_proxy_async() {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -146,7 +171,7 @@ __device__ __forceinline__ unsigned long long make_desc(unsigned smem_addr) {
 }
 // bf16 x bf16 -> fp32, both operands K-major, M = 128
 __device__ __forceinline__ unsigned make_idesc(int n) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((unsigned)(n >> 3) << 17) | ((unsigned)(BM >> 4) << 24);
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((unsigned)(n >> 3) << 17) | ((unsigned)(BMH >> 4) << 24);
 }
 
 // byte offset of 16-byte chunk c of row r inside a swizzled K-major tile
@@ -158,78 +183,99 @@ __device__ __forceinline__ unsigned swz(unsigned r, unsigned c) {
 // decode of one record's class lists into its 128 x 64 tile
 // ------------------------------------------------------------------------------------------
 // One record = 128 * 64/BW block slots, listed as [pruned | dense | unified]; every entry names
-// the byte offset of its block in the tile.  Thread `tid` of a decode group takes flattened
-// entries tid, tid+NDEC_THREADS, ...: a fixed count, so all loads issue before the first store.
+// the byte offset of its block in the tile.  The three lists are laid end to end, each padded
+// to a multiple of 8 entries, and thread `tid` of a decode group takes entries tid,
+// tid+NDEC_THREADS, ... of that sequence, so the 8 lanes of a quarter warp always hold 8
+// neighbouring entries of one list, which the packer ordered to fall into different banks.
+// The work is split in two: fetch_entries reads the small per-entry words (it can run before the
+// pipeline slot is free), write_entries fills the tile: zeros for pruned blocks, sign . bf16(u)
+// for unified blocks, and an asynchronous global->shared copy of the stored values for dense ones.
 template <int BW>
-__device__ __forceinline__ void decode_record(unsigned char *tile, const PackedRec r0, const PackedRec r1,
-                                              const Params &p, int tid) {
-    constexpr int NBK = BK / BW;
-    constexpr int SLOTS = kTileRows * NBK;
-    constexpr int ENT = SLOTS / NDEC_THREADS;
-    constexpr int WORDS = BW / 2;                           // 32-bit words per block
-    constexpr unsigned OFF_MASK = (unsigned)(REC_BYTES - 1) & ~(unsigned)((BW >= 8 ? 16 : 2 * BW) - 1);
+struct DecodeCfg {
+    static constexpr int NBK = BK / BW;
+    static constexpr int SLOTS = kTileRows * NBK;
+    static constexpr int ENT = (SLOTS + 24 + NDEC_THREADS - 1) / NDEC_THREADS;
+    static constexpr int WORDS = BW / 2;                    // 32-bit words per block
+    static constexpr unsigned OFF_MASK = (unsigned)(REC_BYTES - 1) & ~(unsigned)((BW >= 8 ? 16 : 2 * BW) - 1);
+};
+
+template <int BW>
+__device__ __forceinline__ void fetch_entries(const PackedRec r0, const PackedRec r1, const Params &p, int tid,
+                                              unsigned (&m0)[DecodeCfg<BW>::ENT], unsigned (&m1)[DecodeCfg<BW>::ENT]) {
+    constexpr int ENT = DecodeCfg<BW>::ENT;
     const uint2 *ulist = reinterpret_cast<const uint2 *>(p.packed + p.off_ulist);
     const unsigned short *dpos = reinterpret_cast<const unsigned short *>(p.packed + p.off_dpos);
-    const unsigned char *dpay = p.packed + p.off_dpay;
     const unsigned short *ppos = reinterpret_cast<const unsigned short *>(p.packed + p.off_ppos);
     const unsigned n_p = r1.pbase - r0.pbase, n_d = r1.dbase - r0.dbase, n_u = r1.ubase - r0.ubase;
-    unsigned off[ENT];                                      // 0xffffffff: nothing to write
-    unsigned w[ENT][WORDS];
+    const unsigned p8 = (n_p + 7u) & ~7u, d8 = (n_d + 7u) & ~7u;
 #pragma unroll
     for (int k = 0; k < ENT; ++k) {
         const unsigned f = (unsigned)tid + (unsigned)k * NDEC_THREADS;
-        off[k] = 0xffffffffu;
-#pragma unroll
-        for (int q = 0; q < WORDS; ++q) w[k][q] = 0u;
-        if (f < n_p) {
+        m0[k] = 0xffffffffu;                                // nothing to write
+        m1[k] = 0u;
+        if (f < p8) {
             const unsigned e = r0.pbase + f;
-            if (e < p.n_plist) off[k] = __ldg(ppos + e);
-        } else if (f < n_p + n_d) {
-            const unsigned e = r0.dbase + (f - n_p);
-            if (e < p.n_dense) {
-                off[k] = __ldg(dpos + e);
-                const unsigned char *src = dpay + (size_t)e * (2 * BW);
-                if (BW == 16) {
-                    const uint4 v0 = __ldg(reinterpret_cast<const uint4 *>(src));
-                    const uint4 v1 = __ldg(reinterpret_cast<const uint4 *>(src + 16));
-                    w[k][0] = v0.x; w[k][1 % WORDS] = v0.y; w[k][2 % WORDS] = v0.z; w[k][3 % WORDS] = v0.w;
-                    w[k][4 % WORDS] = v1.x; w[k][5 % WORDS] = v1.y; w[k][6 % WORDS] = v1.z; w[k][7 % WORDS] = v1.w;
-                } else if (BW == 8) {
-                    const uint4 v0 = __ldg(reinterpret_cast<const uint4 *>(src));
-                    w[k][0] = v0.x; w[k][1 % WORDS] = v0.y; w[k][2 % WORDS] = v0.z; w[k][3 % WORDS] = v0.w;
-                } else if (BW == 4) {
-                    const uint2 v0 = __ldg(reinterpret_cast<const uint2 *>(src));
-                    w[k][0] = v0.x; w[k][1 % WORDS] = v0.y;
-                } else {
-                    w[k][0] = __ldg(reinterpret_cast<const unsigned *>(src));
-                }
-            }
-        } else if (f < n_p + n_d + n_u) {
-            const unsigned e = r0.ubase + (f - n_p - n_d);
+            if (f < n_p && e < p.n_plist) m0[k] = __ldg(ppos + e);
+        } else if (f < p8 + d8) {
+            const unsigned e = r0.dbase + (f - p8);
+            if (f - p8 < n_d && e < p.n_dense) m0[k] = __ldg(dpos + e);
+        } else if (f - p8 - d8 < n_u) {
+            const unsigned e = r0.ubase + (f - p8 - d8);
             if (e < p.n_unified) {
                 const uint2 ent = __ldg(ulist + e);          // x: spread signs, y: off | bf16(u) << 16
-                off[k] = ent.y & 0xffffu;
-                const unsigned u2 = __byte_perm(ent.y, 0u, 0x3232);      // bf16(u) in both halves
-#pragma unroll
-                for (int q = 0; q < WORDS; ++q)              // weights 2q, 2q+1: sign bits q and 16+q
-                    w[k][q] = ((ent.x << (15 - q)) & 0x80008000u) ^ u2;
+                m0[k] = ent.y;
+                m1[k] = ent.x;
             }
         }
     }
+}
+
+template <int BW>
+__device__ __forceinline__ void write_entries(unsigned char *tile, const PackedRec r0, const PackedRec r1,
+                                              const Params &p, int tid,
+                                              const unsigned (&m0)[DecodeCfg<BW>::ENT],
+                                              const unsigned (&m1)[DecodeCfg<BW>::ENT]) {
+    constexpr int ENT = DecodeCfg<BW>::ENT;
+    constexpr int WORDS = DecodeCfg<BW>::WORDS;
+    constexpr unsigned OFF_MASK = DecodeCfg<BW>::OFF_MASK;
+    const unsigned char *dpay = p.packed + p.off_dpay;
+    const unsigned n_p = r1.pbase - r0.pbase, n_d = r1.dbase - r0.dbase;
+    const unsigned p8 = (n_p + 7u) & ~7u, d8 = (n_d + 7u) & ~7u;
+    const unsigned tile_s = smem_u32(tile);
+    // no branches per entry: every entry computes its words (zero unless unified), stores them
+    // unless it is dense, and issues its copy if it is dense
 #pragma unroll
     for (int k = 0; k < ENT; ++k) {
-        if (off[k] == 0xffffffffu) continue;
-        unsigned char *dst = tile + (off[k] & OFF_MASK);
+        const unsigned f = (unsigned)tid + (unsigned)k * NDEC_THREADS;
+        const bool valid = m0[k] != 0xffffffffu;
+        const unsigned off = m0[k] & OFF_MASK;
+        const bool is_d = (f - p8) < d8;                    // unsigned: also false for f < p8
+        const bool is_u = f >= p8 + d8;
+        const unsigned umask = is_u ? 0xffffffffu : 0u;
+        const unsigned u2 = __byte_perm(m0[k], 0u, 0x3232);  // bf16(u) in both halves
+        unsigned w[8];
+#pragma unroll
+        for (int q = 0; q < 8; ++q)                          // weights 2q, 2q+1: sign bits q and 16+q
+            w[q] = (q < WORDS) ? ((((m1[k] << (15 - q)) & 0x80008000u) ^ u2) & umask) : 0u;
+        const unsigned char *src = dpay + (size_t)(r0.dbase + (f - p8)) * (2 * BW);
+        const unsigned do_copy = (valid && is_d) ? 1u : 0u;
+        const bool do_store = valid && !is_d;
         if (BW == 16) {
-            *reinterpret_cast<uint4 *>(dst) = make_uint4(w[k][0], w[k][1 % WORDS], w[k][2 % WORDS], w[k][3 % WORDS]);
-            *reinterpret_cast<uint4 *>(tile + ((off[k] & OFF_MASK) ^ 16u)) =
-                make_uint4(w[k][4 % WORDS], w[k][5 % WORDS], w[k][6 % WORDS], w[k][7 % WORDS]);
+            cp_async_if<16>(tile_s + off, src, do_copy);
+            cp_async_if<16>(tile_s + (off ^ 16u), src + 16, do_copy);
+            if (do_store) {
+                *reinterpret_cast<uint4 *>(tile + off) = make_uint4(w[0], w[1], w[2], w[3]);
+                *reinterpret_cast<uint4 *>(tile + (off ^ 16u)) = make_uint4(w[4], w[5], w[6], w[7]);
+            }
         } else if (BW == 8) {
-            *reinterpret_cast<uint4 *>(dst) = make_uint4(w[k][0], w[k][1 % WORDS], w[k][2 % WORDS], w[k][3 % WORDS]);
+            cp_async_if<16>(tile_s + off, src, do_copy);
+            if (do_store) *reinterpret_cast<uint4 *>(tile + off) = make_uint4(w[0], w[1], w[2], w[3]);
         } else if (BW == 4) {
-            *reinterpret_cast<uint2 *>(dst) = make_uint2(w[k][0], w[k][1 % WORDS]);
+            cp_async_if<8>(tile_s + off, src, do_copy);
+            if (do_store) *reinterpret_cast<uint2 *>(tile + off) = make_uint2(w[0], w[1]);
         } else {
-            *reinterpret_cast<unsigned *>(dst) = w[k][0];
+            cp_async_if<4>(tile_s + off, src, do_copy);
+            if (do_store) *reinterpret_cast<unsigned *>(tile + off) = w[0];
         }
     }
 }
@@ -238,27 +284,33 @@ __device__ __forceinline__ void decode_record(unsigned char *tile, const PackedR
 // the kernel
 // ------------------------------------------------------------------------------------------
 struct Smem {
-    unsigned long long full_a[STAGES], full_b[STAGES], empty[STAGES], tfull[2], tempty[2], drain;
+    unsigned long long full[STAGES], empty[STAGES], tfull, tempty, drain;
     unsigned tmem_base;
     int abort;
     unsigned char live_prod[MAX_STAGES_K];                  // live masks of the producer's tile
     unsigned char live_mma[MAX_STAGES_K];                   // ... of the MMA issuer's tile
     unsigned char live_gather[NGATHER_WARPS][MAX_STAGES_K]; // ... of each gather warp's tile
+    unsigned short live_list[NDEC_GROUPS][MAX_STAGES_K];    // live stage numbers of a decode group's tile
+    int n_live[NDEC_GROUPS];
 };
 
 __device__ __forceinline__ void group_bar(int group) {      // the threads of one decode group
     asm volatile("bar.sync %0, %1;" ::"r"(1 + group), "r"(NDEC_THREADS) : "memory");
 }
 
-template <int MODE, int NREC, int BW>
+// MODE 0: GEMM (A by TMA), 1: convolution (A gathered).  NREC: 128-row weight records per tile.
+// MT: 128-row halves of the activation tile (1 or 2).
+template <int MODE, int NREC, int BW, int MT>
 __global__ void __launch_bounds__(MODE ? THREADS_CONV : THREADS_GEMM, 1)
 mwu_gemm_kernel(const __grid_constant__ CUtensorMap tmap, const Params p) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char *base = reinterpret_cast<unsigned char *>(
         (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    constexpr int A_BYTES = MT * AH_BYTES;
+    constexpr int B_BYTES = NREC * REC_BYTES;
+    constexpr int BM = MT * BMH;
     unsigned char *sA = base;
     unsigned char *sB = base + STAGES * A_BYTES;
-    constexpr int B_BYTES = NREC * REC_BYTES;
     Smem *sm = reinterpret_cast<Smem *>(sB + STAGES * B_BYTES);
     const int n_stages = (int)p.n_stages;
     // per decode group: the record table of its current tile, [NREC][n_stages + 1]
@@ -274,14 +326,12 @@ mwu_gemm_kernel(const __grid_constant__ CUtensorMap tmap, const Params p) {
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
-            mbar_init(smem_u32(&sm->full_a[s]), MODE ? NGATHER_WARPS : 1);
-            mbar_init(smem_u32(&sm->full_b[s]), NDEC_WARPS);
+            // one barrier per slot: the A producer(s) and the decode warps of the slot's group
+            mbar_init(smem_u32(&sm->full[s]), (MODE ? NGATHER_WARPS : 1) + NDEC_WARPS);
             mbar_init(smem_u32(&sm->empty[s]), 1);
         }
-        for (int b = 0; b < 2; ++b) {
-            mbar_init(smem_u32(&sm->tfull[b]), 1);
-            mbar_init(smem_u32(&sm->tempty[b]), 4);
-        }
+        mbar_init(smem_u32(&sm->tfull), 1);
+        mbar_init(smem_u32(&sm->tempty), 4 * MT);
         mbar_init(smem_u32(&sm->drain), 1);
         sm->abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -328,7 +378,7 @@ mwu_gemm_kernel(const __grid_constant__ CUtensorMap tmap, const Params p) {
                 for (int ks = 0; ks < n_stages; ++ks) {
                     if (!sm->live_prod[ks]) continue;
                     if (!mbar_wait(smem_u32(&sm->empty[stage]), phase ^ 1u, abort)) { ok = false; break; }
-                    const unsigned bar = smem_u32(&sm->full_a[stage]);
+                    const unsigned bar = smem_u32(&sm->full[stage]);
                     mbar_expect_tx(bar, A_BYTES);
                     tma_load_2d(smem_u32(sA + stage * A_BYTES), &tmap, bar, ks * BK, (int)(mt * BM));
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
@@ -339,46 +389,51 @@ mwu_gemm_kernel(const __grid_constant__ CUtensorMap tmap, const Params p) {
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
         int stage = 0;
-        unsigned phase = 0;
-        unsigned acc_phase[2] = {0, 0};
-        long long it = 0;
+        unsigned phase = 0, acc_phase = 0;
         bool ok = true;
         bool issued_any = false;
-        for (long long t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++it) {
+        bool ready = false;                                 // next slot's full barrier already seen complete
+        for (long long t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
             const long long nt = t / m_tiles;
             load_live(sm->live_mma, nt);
             if (lane == 0) {
-                const int buf = (int)(it & 1);
                 const int nrec_here = (int)((p.n_rec_tiles - nt * NREC) < NREC ? (p.n_rec_tiles - nt * NREC) : NREC);
                 const unsigned idesc = make_idesc(nrec_here * kTileRows);
-                if (!mbar_wait(smem_u32(&sm->tempty[buf]), acc_phase[buf] ^ 1u, abort)) ok = false;
-                acc_phase[buf] ^= 1u;
+                // the epilogue must have read the previous tile's accumulators
+                if (!mbar_wait(smem_u32(&sm->tempty), acc_phase ^ 1u, abort)) ok = false;
+                acc_phase ^= 1u;
                 tc_fence_after();
-                const unsigned d_tmem = tmem_base + (unsigned)(buf * 256);
                 bool first = true;
                 for (int ks = 0; ks < n_stages && ok; ++ks) {
                     const unsigned live = sm->live_mma[ks];
                     if (!live) continue;
-                    if (!mbar_wait(smem_u32(&sm->full_a[stage]), phase, abort)) { ok = false; break; }
-                    if (!mbar_wait(smem_u32(&sm->full_b[stage]), phase, abort)) { ok = false; break; }
+                    // `ready` was probed while the previous stage's MMAs were being issued
+                    if (!ready && !mbar_wait(smem_u32(&sm->full[stage]), phase, abort)) { ok = false; break; }
                     tc_fence_after();
                     const unsigned long long adesc = make_desc(smem_u32(sA + stage * A_BYTES));
                     const unsigned long long bdesc = make_desc(smem_u32(sB + stage * B_BYTES));
+                    const int nstage = (stage + 1 == STAGES) ? 0 : stage + 1;
+                    const unsigned nphase = (stage + 1 == STAGES) ? (phase ^ 1u) : phase;
 #pragma unroll
                     for (int k4 = 0; k4 < 4; ++k4) {
                         if ((live >> k4) & 1u) {
-                            umma_bf16(d_tmem, adesc + (unsigned long long)(k4 * 2), bdesc + (unsigned long long)(k4 * 2),
-                                      idesc, first ? 0u : 1u);
+#pragma unroll
+                            for (int h = 0; h < MT; ++h)
+                                umma_bf16(tmem_base + (unsigned)(h * 256),
+                                          adesc + (unsigned long long)(h * (AH_BYTES >> 4) + k4 * 2),
+                                          bdesc + (unsigned long long)(k4 * 2), idesc, first ? 0u : 1u);
                             first = false;
                             issued_any = true;
                         }
                     }
                     umma_commit(smem_u32(&sm->empty[stage]));
-                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                    ready = mbar_test(smem_u32(&sm->full[nstage]), nphase);
+                    stage = nstage;
+                    phase = nphase;
                 }
                 if (ok) {
-                    if (!first) umma_commit(smem_u32(&sm->tfull[buf]));
-                    else mbar_arrive(smem_u32(&sm->tfull[buf]));
+                    if (!first) umma_commit(smem_u32(&sm->tfull));
+                    else mbar_arrive(smem_u32(&sm->tfull));
                 }
             }
             ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
@@ -389,104 +444,109 @@ mwu_gemm_kernel(const __grid_constant__ CUtensorMap tmap, const Params p) {
             mbar_wait(smem_u32(&sm->drain), 0, abort);
         }
         __syncwarp();
-    } else if (warp >= 2 && warp < 6) {
+    } else if (warp >= 2 && warp < FIRST_DEC_WARP) {
         // ---------------- epilogue ----------------
         const int quarter = warp & 3;                       // TMEM lanes this warp may read
-        unsigned acc_phase[2] = {0, 0};
-        long long it = 0;
-        bool ok = true;
-        for (long long t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++it) {
-            const long long mt = t % m_tiles, nt = t / m_tiles;
-            const int buf = (int)(it & 1);
-            unsigned any = 0;
-            for (int ks = lane; ks < n_stages; ks += 32) any |= live_of(nt, ks);
-            any = __reduce_or_sync(0xffffffffu, any);
-            if (!mbar_wait(smem_u32(&sm->tfull[buf]), acc_phase[buf], abort)) { ok = false; }
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
-            acc_phase[buf] ^= 1u;
-            tc_fence_after();
-            const long long m = mt * BM + quarter * 32 + lane;
-            const int ncols_tile = (int)(((p.n_rec_tiles - nt * NREC) < NREC ? (p.n_rec_tiles - nt * NREC) : NREC) * kTileRows);
-            for (int c0 = 0; c0 < ncols_tile; c0 += 32) {
-                unsigned v[32];
-                if (any) {
-                    tmem_ld32(tmem_base + ((unsigned)(quarter * 32) << 16) + (unsigned)(buf * 256 + c0), v);
-                } else {
+        const int half = (warp - 2) >> 2;                   // which 128-row half of the tile
+        if (half < MT) {
+            unsigned acc_phase = 0;
+            bool ok = true;
+            for (long long t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+                const long long mt = t % m_tiles, nt = t / m_tiles;
+                unsigned any = 0;
+                for (int ks = lane; ks < n_stages; ks += 32) any |= live_of(nt, ks);
+                any = __reduce_or_sync(0xffffffffu, any);
+                if (!mbar_wait(smem_u32(&sm->tfull), acc_phase, abort)) { ok = false; }
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                acc_phase ^= 1u;
+                tc_fence_after();
+                const long long m = mt * BM + half * BMH + quarter * 32 + lane;
+                const int ncols_tile = (int)(((p.n_rec_tiles - nt * NREC) < NREC ? (p.n_rec_tiles - nt * NREC) : NREC) * kTileRows);
+                for (int c0 = 0; c0 < ncols_tile; c0 += 32) {
+                    unsigned v[32];
+                    if (any) {
+                        tmem_ld32(tmem_base + ((unsigned)(quarter * 32) << 16) + (unsigned)(half * 256 + c0), v);
+                    } else {
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) v[j] = 0u;
-                }
-                const long long n0 = nt * (NREC * kTileRows) + c0;
-                if (MODE == 0) {
-                    if (m < p.M) {
-                        if (p.y_fp32) {
-                            float *dst = reinterpret_cast<float *>(p.Y) + m * p.ldy + n0;
-                            if (n0 + 32 <= p.N) {
+                        for (int j = 0; j < 32; ++j) v[j] = 0u;
+                    }
+                    const long long n0 = nt * (NREC * kTileRows) + c0;
+                    if (MODE == 0) {
+                        if (m < p.M) {
+                            if (p.y_fp32) {
+                                float *dst = reinterpret_cast<float *>(p.Y) + m * p.ldy + n0;
+                                if (n0 + 32 <= p.N) {
 #pragma unroll
-                                for (int j = 0; j < 32; j += 4)
-                                    *reinterpret_cast<uint4 *>(dst + j) = make_uint4(v[j], v[j + 1], v[j + 2], v[j + 3]);
-                            } else {
-                                for (int j = 0; j < 32; ++j)
-                                    if (n0 + j < p.N) dst[j] = __uint_as_float(v[j]);
-                            }
-                        } else {
-                            __nv_bfloat16 *dst = reinterpret_cast<__nv_bfloat16 *>(p.Y) + m * p.ldy + n0;
-                            if (n0 + 32 <= p.N) {
-#pragma unroll
-                                for (int j = 0; j < 32; j += 8) {
-                                    uint4 o;
-                                    __nv_bfloat162 h;
-                                    h = __floats2bfloat162_rn(__uint_as_float(v[j]), __uint_as_float(v[j + 1]));
-                                    o.x = *reinterpret_cast<unsigned *>(&h);
-                                    h = __floats2bfloat162_rn(__uint_as_float(v[j + 2]), __uint_as_float(v[j + 3]));
-                                    o.y = *reinterpret_cast<unsigned *>(&h);
-                                    h = __floats2bfloat162_rn(__uint_as_float(v[j + 4]), __uint_as_float(v[j + 5]));
-                                    o.z = *reinterpret_cast<unsigned *>(&h);
-                                    h = __floats2bfloat162_rn(__uint_as_float(v[j + 6]), __uint_as_float(v[j + 7]));
-                                    o.w = *reinterpret_cast<unsigned *>(&h);
-                                    *reinterpret_cast<uint4 *>(dst + j) = o;
+                                    for (int j = 0; j < 32; j += 4)
+                                        *reinterpret_cast<uint4 *>(dst + j) = make_uint4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+                                } else {
+                                    for (int j = 0; j < 32; ++j)
+                                        if (n0 + j < p.N) dst[j] = __uint_as_float(v[j]);
                                 }
                             } else {
-                                for (int j = 0; j < 32; ++j)
-                                    if (n0 + j < p.N) dst[j] = __float2bfloat16_rn(__uint_as_float(v[j]));
+                                __nv_bfloat16 *dst = reinterpret_cast<__nv_bfloat16 *>(p.Y) + m * p.ldy + n0;
+                                if (n0 + 32 <= p.N) {
+#pragma unroll
+                                    for (int j = 0; j < 32; j += 8) {
+                                        uint4 o;
+                                        __nv_bfloat162 h2;
+                                        h2 = __floats2bfloat162_rn(__uint_as_float(v[j]), __uint_as_float(v[j + 1]));
+                                        o.x = *reinterpret_cast<unsigned *>(&h2);
+                                        h2 = __floats2bfloat162_rn(__uint_as_float(v[j + 2]), __uint_as_float(v[j + 3]));
+                                        o.y = *reinterpret_cast<unsigned *>(&h2);
+                                        h2 = __floats2bfloat162_rn(__uint_as_float(v[j + 4]), __uint_as_float(v[j + 5]));
+                                        o.z = *reinterpret_cast<unsigned *>(&h2);
+                                        h2 = __floats2bfloat162_rn(__uint_as_float(v[j + 6]), __uint_as_float(v[j + 7]));
+                                        o.w = *reinterpret_cast<unsigned *>(&h2);
+                                        *reinterpret_cast<uint4 *>(dst + j) = o;
+                                    }
+                                } else {
+                                    for (int j = 0; j < 32; ++j)
+                                        if (n0 + j < p.N) dst[j] = __float2bfloat16_rn(__uint_as_float(v[j]));
+                                }
                             }
                         }
-                    }
-                } else {
-                    // NCHW output: row m = (img, oh, ow); consecutive lanes write consecutive pixels
-                    if (m < p.M) {
-                        const long long hw = (long long)p.OH * p.OW;
-                        const long long img = m / hw, pix = m % hw;
-                        for (int j = 0; j < 32; ++j) {
-                            const long long o = n0 + j;
-                            if (o < p.N) {
-                                const long long idx = (img * p.N + o) * hw + pix;
-                                if (p.y_fp32) reinterpret_cast<float *>(p.Y)[idx] = __uint_as_float(v[j]);
-                                else reinterpret_cast<__nv_bfloat16 *>(p.Y)[idx] = __float2bfloat16_rn(__uint_as_float(v[j]));
+                    } else {
+                        // NCHW output: row m = (img, oh, ow); consecutive lanes write consecutive pixels
+                        if (m < p.M) {
+                            const long long hw = (long long)p.OH * p.OW;
+                            const long long img = m / hw, pix = m % hw;
+                            for (int j = 0; j < 32; ++j) {
+                                const long long o = n0 + j;
+                                if (o < p.N) {
+                                    const long long idx = (img * p.N + o) * hw + pix;
+                                    if (p.y_fp32) reinterpret_cast<float *>(p.Y)[idx] = __uint_as_float(v[j]);
+                                    else reinterpret_cast<__nv_bfloat16 *>(p.Y)[idx] = __float2bfloat16_rn(__uint_as_float(v[j]));
+                                }
                             }
                         }
                     }
                 }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&sm->tempty));
             }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&sm->tempty[buf]));
         }
-    } else if (warp >= 6 && warp < FIRST_GATHER_WARP) {
-        // ---------------- weight decode: two groups on alternate live stages ----------------
-        const int group = (warp - 6) / NDEC_WARPS;
-        const int tid = threadIdx.x - (6 + group * NDEC_WARPS) * 32;
+    } else if (warp >= FIRST_DEC_WARP && warp < FIRST_GATHER_WARP) {
+        // ---------------- weight decode: one group per pipeline slot ----------------
+        const int group = (warp - FIRST_DEC_WARP) / NDEC_WARPS;
+        const int tid = threadIdx.x - (FIRST_DEC_WARP + group * NDEC_WARPS) * 32;
+        const int gwarp = tid >> 5;
         uint4 *my_rec = srec + (size_t)group * NREC * (n_stages + 1);
-        long long seq = 0;                                  // live stages seen so far (all tiles)
+        unsigned short *my_list = sm->live_list[group];
+        long long seq0 = 0;                                 // live stages of all earlier tiles
         bool ok = true;
         auto rec_at = [&](int q, int ks, PackedRec *r0, PackedRec *r1) {
             const uint4 a = my_rec[q * (n_stages + 1) + ks], b = my_rec[q * (n_stages + 1) + ks + 1];
             r0->ubase = a.x; r0->dbase = a.y; r0->pbase = a.z; r0->live = a.w;
             r1->ubase = b.x; r1->dbase = b.y; r1->pbase = b.z; r1->live = b.w;
         };
+        constexpr int ENT = DecodeCfg<BW>::ENT;
+        unsigned m0[NREC][ENT], m1[NREC][ENT];
         for (long long t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
             const long long nt = t / m_tiles;
-            group_bar(group);                               // everyone is done with the previous table
+            group_bar(group);                               // everyone is done with the previous tables
 #pragma unroll
             for (int q = 0; q < NREC; ++q) {
                 const long long rt = nt * NREC + q;
@@ -498,35 +558,60 @@ mwu_gemm_kernel(const __grid_constant__ CUtensorMap tmap, const Params p) {
                 }
             }
             group_bar(group);
-            auto stage_live = [&](int ks) -> unsigned {
-                unsigned l = my_rec[ks].w;
-                if (NREC == 2) l |= my_rec[(n_stages + 1) + ks].w;
-                return l;
+            if (gwarp == 0) {
+                // compact list of the live stages of this tile
+                int n = 0;
+                for (int k0 = 0; k0 < n_stages; k0 += 32) {
+                    const int ks = k0 + lane;
+                    unsigned l = 0;
+                    if (ks < n_stages) {
+                        l = my_rec[ks].w;
+                        if (NREC == 2) l |= my_rec[(n_stages + 1) + ks].w;
+                    }
+                    const unsigned m = __ballot_sync(0xffffffffu, l != 0);
+                    if (l) my_list[n + __popc(m & ((1u << lane) - 1u))] = (unsigned short)ks;
+                    n += __popc(m);
+                }
+                if (lane == 0) sm->n_live[group] = n;
+            }
+            group_bar(group);
+            const int n_live = sm->n_live[group];
+            auto fetch_stage = [&](int ks) {
+#pragma unroll
+                for (int q = 0; q < NREC; ++q) {
+                    PackedRec r0, r1;
+                    rec_at(q, ks, &r0, &r1);
+                    fetch_entries<BW>(r0, r1, p, tid, m0[q], m1[q]);
+                }
             };
-            for (int ks = 0; ks < n_stages; ++ks) {
-                if (!stage_live(ks)) continue;
-                const long long my_seq = seq++;
-                if ((int)(my_seq % NDEC_GROUPS) != group) continue;
-                const int stage = (int)(my_seq % STAGES);
+            // this group owns the live stages whose running number is congruent to `group`
+            int i = (int)((group + NDEC_GROUPS - (seq0 % NDEC_GROUPS)) % NDEC_GROUPS);
+            if (i < n_live) fetch_stage(my_list[i]);
+            for (; i < n_live; i += NDEC_GROUPS) {
+                const int ks = my_list[i];
+                const long long my_seq = seq0 + i;
+                const int stage = group;                    // = my_seq % STAGES
                 const unsigned phase = (unsigned)((my_seq / STAGES) & 1);
                 if (!mbar_wait(smem_u32(&sm->empty[stage]), phase ^ 1u, abort)) ok = false;
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
 #pragma unroll
                 for (int q = 0; q < NREC; ++q) {
-                    if (nt * NREC + q < p.n_rec_tiles) {
-                        PackedRec r0, r1;
-                        rec_at(q, ks, &r0, &r1);
-                        decode_record<BW>(sB + stage * B_BYTES + q * REC_BYTES, r0, r1, p, tid);
-                    }
+                    PackedRec r0, r1;
+                    rec_at(q, ks, &r0, &r1);
+                    write_entries<BW>(sB + stage * B_BYTES + q * REC_BYTES, r0, r1, p, tid, m0[q], m1[q]);
                 }
+                // the entry words of this group's next stage travel while the copies above land
+                if (i + NDEC_GROUPS < n_live) fetch_stage(my_list[i + NDEC_GROUPS]);
+                asm volatile("cp.async.wait_all;" ::: "memory");
                 fence_proxy_async();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&sm->full_b[stage]));
+                if (lane == 0) mbar_arrive(smem_u32(&sm->full[stage]));
             }
+            seq0 += n_live;
         }
     } else if (MODE == 1 && warp >= FIRST_GATHER_WARP) {
-        // ---------------- im2col gather of the A tile (convolution) ----------------
+        // ---------------- im2col gather of the A tile (convolution, MT == 1) ----------------
         const int gw = warp - FIRST_GATHER_WARP;
         const int r = threadIdx.x - FIRST_GATHER_WARP * 32;     // row of the tile, 0..127
         const unsigned short *X = reinterpret_cast<const unsigned short *>(p.X);
@@ -569,7 +654,7 @@ mwu_gemm_kernel(const __grid_constant__ CUtensorMap tmap, const Params p) {
                 }
                 fence_proxy_async();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&sm->full_a[stage]));
+                if (lane == 0) mbar_arrive(smem_u32(&sm->full[stage]));
                 if (++stage == STAGES) { stage = 0; phase ^= 1u; }
             }
         }
@@ -606,27 +691,27 @@ static EncodeTiledFn get_encode_fn() {
     return fn;
 }
 
-static size_t smem_bytes(int nrec, long long n_stages, long long conv_k) {
-    return 1024 + (size_t)STAGES * (A_BYTES + nrec * REC_BYTES) + ((sizeof(Smem) + 15) & ~(size_t)15) +
+static size_t smem_bytes(int nrec, int mt, long long n_stages, long long conv_k) {
+    return 1024 + (size_t)STAGES * (mt * AH_BYTES + nrec * REC_BYTES) + ((sizeof(Smem) + 15) & ~(size_t)15) +
            (size_t)NDEC_GROUPS * nrec * (n_stages + 1) * 16 + (size_t)conv_k * sizeof(int2);
 }
 
-template <int MODE, int NREC, int BW>
+template <int MODE, int NREC, int BW, int MT>
 static cudaError_t launch(const CUtensorMap &tmap, const Params &p, int grid, size_t smem, cudaStream_t st) {
-    auto kern = mwu_gemm_kernel<MODE, NREC, BW>;
+    auto kern = mwu_gemm_kernel<MODE, NREC, BW, MT>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     kern<<<grid, MODE ? THREADS_CONV : THREADS_GEMM, smem, st>>>(tmap, p);
     return cudaGetLastError();
 }
 
-template <int MODE, int NREC>
+template <int MODE, int NREC, int MT>
 static cudaError_t launch_bw(int bw, const CUtensorMap &tmap, const Params &p, int grid, size_t smem, cudaStream_t st) {
     switch (bw) {
-        case 2: return launch<MODE, NREC, 2>(tmap, p, grid, smem, st);
-        case 4: return launch<MODE, NREC, 4>(tmap, p, grid, smem, st);
-        case 8: return launch<MODE, NREC, 8>(tmap, p, grid, smem, st);
-        default: return launch<MODE, NREC, 16>(tmap, p, grid, smem, st);
+        case 2: return launch<MODE, NREC, 2, MT>(tmap, p, grid, smem, st);
+        case 4: return launch<MODE, NREC, 4, MT>(tmap, p, grid, smem, st);
+        case 8: return launch<MODE, NREC, 8, MT>(tmap, p, grid, smem, st);
+        default: return launch<MODE, NREC, 16, MT>(tmap, p, grid, smem, st);
     }
 }
 
@@ -670,10 +755,13 @@ extern "C" int mwu_gemm(const mwu_proj_desc *desc, const void *packed, const voi
     EncodeTiledFn encode = get_encode_fn();
     if (!encode) return MWU_ERR_CUDA;
 
+    // tiles of 256 activation rows unless the problem has no second half to fill
+    const int mt = (M > BMH) ? 2 : 1;
+    const int bm = mt * BMH;
     CUtensorMap tmap;
     const cuuint64_t gdim[2] = {(cuuint64_t)desc->cols, (cuuint64_t)M};
     const cuuint64_t gstride[1] = {(cuuint64_t)ldx * 2};
-    const cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)BM};
+    const cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)bm};
     const cuuint32_t estr[2] = {1, 1};
     if (encode(&tmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(X), gdim, gstride, box, estr,
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -685,13 +773,16 @@ extern "C" int mwu_gemm(const mwu_proj_desc *desc, const void *packed, const voi
     p.M = M;
     p.ldy = ldy;
     const int nrec = p.n_rec_tiles >= 2 ? 2 : 1;
-    const long long tiles = ((M + BM - 1) / BM) * ((p.n_rec_tiles + nrec - 1) / nrec);
+    const long long tiles = ((M + bm - 1) / bm) * ((p.n_rec_tiles + nrec - 1) / nrec);
     const int grid = (int)(tiles < sm_count ? tiles : sm_count);
-    const size_t smem = smem_bytes(nrec, p.n_stages, 0);
+    const size_t smem = smem_bytes(nrec, mt, p.n_stages, 0);
     if (p.n_stages > MAX_STAGES_K || smem > 227 * 1024) return MWU_ERR_SHAPE;
     cudaStream_t st = (cudaStream_t)cuda_stream;
-    cudaError_t e = (nrec == 2) ? launch_bw<0, 2>(desc->block, tmap, p, grid, smem, st)
-                                : launch_bw<0, 1>(desc->block, tmap, p, grid, smem, st);
+    cudaError_t e;
+    if (mt == 2) e = (nrec == 2) ? launch_bw<0, 2, 2>(desc->block, tmap, p, grid, smem, st)
+                                 : launch_bw<0, 1, 2>(desc->block, tmap, p, grid, smem, st);
+    else e = (nrec == 2) ? launch_bw<0, 2, 1>(desc->block, tmap, p, grid, smem, st)
+                         : launch_bw<0, 1, 1>(desc->block, tmap, p, grid, smem, st);
     return e == cudaSuccess ? MWU_OK : MWU_ERR_CUDA;
 }
 
@@ -726,14 +817,14 @@ extern "C" int mwu_conv_implicit(const mwu_proj_desc *desc, const void *packed, 
     p.M = (long long)n * p.OH * p.OW;
     p.ldy = 0;
     const int nrec = p.n_rec_tiles >= 2 ? 2 : 1;
-    const size_t smem = smem_bytes(nrec, p.n_stages, desc->cols);
+    const size_t smem = smem_bytes(nrec, 1, p.n_stages, desc->cols);
     if (p.n_stages > MAX_STAGES_K || smem > 227 * 1024) return MWU_ERR_SHAPE;
-    const long long tiles = ((p.M + BM - 1) / BM) * ((p.n_rec_tiles + nrec - 1) / nrec);
+    const long long tiles = ((p.M + BMH - 1) / BMH) * ((p.n_rec_tiles + nrec - 1) / nrec);
     const int grid = (int)(tiles < sm_count ? tiles : sm_count);
     CUtensorMap tmap;
     memset(&tmap, 0, sizeof(tmap));
     cudaStream_t st = (cudaStream_t)cuda_stream;
-    cudaError_t e = (nrec == 2) ? launch_bw<1, 2>(desc->block, tmap, p, grid, smem, st)
-                                : launch_bw<1, 1>(desc->block, tmap, p, grid, smem, st);
+    cudaError_t e = (nrec == 2) ? launch_bw<1, 2, 1>(desc->block, tmap, p, grid, smem, st)
+                                : launch_bw<1, 1, 1>(desc->block, tmap, p, grid, smem, st);
     return e == cudaSuccess ? MWU_OK : MWU_ERR_CUDA;
 }
