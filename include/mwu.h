@@ -110,7 +110,7 @@ int mwu_project(const mwu_proj_desc *desc, const float *W, const float *U_dual, 
  * For callers that cannot allocate device memory where they need the projection -- code running
  * inside an engine that owns the memory pool, or after a job's memory budget has been frozen,
  * where a cudaMalloc may fail or stall the device.  The scratch memory is a fixed array inside
- * the library's device image (about 4.2 MB, held by every GPU that loads the library until the
+ * the library's device image (about 5.2 MB, held by every GPU that loads the library until the
  * process exits), so the call allocates nothing.
  *
  * Limits and rules:

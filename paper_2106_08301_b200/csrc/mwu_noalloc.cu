@@ -14,8 +14,8 @@
 namespace {
 
 // Enough for MWU_STATIC_MAX_BLOCKS blocks: 4 bytes of bin codes per block plus the fixed
-// selection state (histograms, candidate lists) of mwu_project, which is under 128 KiB.
-constexpr size_t kScratchBytes = (size_t)128 * 1024 + 4 * ((size_t)MWU_STATIC_MAX_BLOCKS + 8) + 256;
+// selection state (histograms, candidate lists) of mwu_project, which is under 1 MiB.
+constexpr size_t kScratchBytes = (size_t)1024 * 1024 + 4 * ((size_t)MWU_STATIC_MAX_BLOCKS + 8) + 256;
 
 static __device__ __align__(256) unsigned char g_scratch[kScratchBytes];
 

@@ -2,7 +2,7 @@
 //
 // Pipeline (all on the caller's stream, no host synchronisation):
 //   sample_kernel   one CTA ranks <= 256 evenly spaced blocks and places a narrow window of
-//                   8190 bins around the k-th smallest key of each selection (prune key, L_u).
+//                   8190 bins (65534 above 8M blocks) around the k-th smallest key of each selection (prune key, L_u).
 //                   The window only steers efficiency; any window gives the same result.
 //   stats_kernel    streams W (+U) once; every thread owns 64 contiguous bytes (four 128-bit
 //                   loads in flight) and evaluates the fp64 keys of its blocks (Section 3.1:
@@ -23,7 +23,8 @@
 namespace mwu {
 namespace proj {
 
-constexpr int NB = 8192;        // level-0 bins: 0 = below the window, NB-1 = above it
+constexpr int NB_MAX = 65536;   // level-0 bins (codes fit 16 bits): bin 0 = below the window, nb-1 = above it
+constexpr int NB_SMALL = 8192;  // used up to 8M blocks: fewer bins to clear and scan
 constexpr int CAP = 2048;       // candidates sorted by the last step
 constexpr int NSAMP = 256;
 constexpr int FIN_THREADS = 1024;   // block size of the kernels whose last CTA finalises
@@ -59,7 +60,8 @@ struct Params {
     int b;
     int use_l1;
     Work *work;
-    unsigned *hist;             // [3][NB]: prune, unify, refine scratch
+    int nb;                     // level-0 bins in use (NB_SMALL or NB_MAX)
+    unsigned *hist;             // [3][nb]: prune, unify, refine scratch
     u64 *cand_key;              // [CAP]
     unsigned *cand_idx;         // [CAP]
     unsigned *bins;             // [n_blocks]
@@ -69,9 +71,9 @@ struct Params {
 __device__ __forceinline__ u128 make_c(u64 key, u64 idx) { return ((u128)key << 32) | (u128)idx; }
 __device__ __forceinline__ u128 from_halves(u64 hi, u64 lo) { return ((u128)hi << 64) | (u128)lo; }
 
-__device__ __forceinline__ unsigned bin_of(u64 key, u64 lo0, u64 hi0, unsigned shift0) {
+__device__ __forceinline__ unsigned bin_of(u64 key, u64 lo0, u64 hi0, unsigned shift0, unsigned nb) {
     if (key < lo0) return 0u;
-    if (key >= hi0) return (unsigned)(NB - 1);
+    if (key >= hi0) return nb - 1u;
     return 1u + (unsigned)((key - lo0) >> shift0);
 }
 
@@ -183,10 +185,10 @@ __device__ __forceinline__ void window_ranks(int n, double frac, int *il, int *i
     *il = (int)a; *ih = (int)b; *ipos = (int)c;
 }
 
-__device__ __forceinline__ void set_window(Sel *s, u64 lo, u64 hi) {
+__device__ __forceinline__ void set_window(Sel *s, u64 lo, u64 hi, int nb) {
     if (hi < lo) hi = lo;
     unsigned shift = 0;
-    while (((hi - lo) >> shift) >= (u64)(NB - 2)) ++shift;
+    while (((hi - lo) >> shift) >= (u64)(nb - 2)) ++shift;
     s->lo0 = lo;
     s->hi0 = hi;
     s->shift0 = shift;
@@ -235,7 +237,7 @@ __global__ void __launch_bounds__(NSAMP) sample_kernel(Params p, long long k_uni
     __syncthreads();
     const u64 That = s_stat[2];
     if (i == 0) {
-        set_window(sp, s_stat[0], s_stat[1]);
+        set_window(sp, s_stat[0], s_stat[1], p.nb);
         sp->mode = (k_prune == 0) ? 1u : (k_prune == mb ? 2u : 0u);
         sp->k = (u64)k_prune;
     }
@@ -255,7 +257,7 @@ __global__ void __launch_bounds__(NSAMP) sample_kernel(Params p, long long k_uni
     }
     __syncthreads();
     if (i == 0) {
-        set_window(su, s_stat[0], s_stat[1]);
+        set_window(su, s_stat[0], s_stat[1], p.nb);
         su->mode = (ksel_u == 0) ? 1u : (ksel_u == elig ? 2u : 0u);
         su->k = (u64)ksel_u;
     }
@@ -279,18 +281,14 @@ __device__ __forceinline__ bool last_block_done(unsigned *ticket) {
     return s_last;
 }
 
-// find the bin holding the r-th element; hist has NB entries
-__device__ void scan_hist(const unsigned *hist, u64 r, unsigned *bin_out, u64 *r_in_bin, u64 *cnt_out,
+// find the bin holding the r-th element; hist has nb entries
+__device__ void scan_hist(const unsigned *hist, int nb, u64 r, unsigned *bin_out, u64 *r_in_bin, u64 *cnt_out,
                           unsigned *err) {
     __shared__ u64 s_part[FIN_THREADS];
-    constexpr int PER = NB / FIN_THREADS;
-    u64 local[PER];
+    const int PER = nb / FIN_THREADS;
     u64 sum = 0;
-#pragma unroll
-    for (int i = 0; i < PER; ++i) {
-        local[i] = ld_vol(&hist[threadIdx.x * PER + i]);
-        sum += local[i];
-    }
+#pragma unroll 8
+    for (int i = 0; i < PER; ++i) sum += ld_vol(&hist[threadIdx.x * PER + i]);
     s_part[threadIdx.x] = sum;
     __syncthreads();
     for (int off = 1; off < FIN_THREADS; off <<= 1) {
@@ -303,14 +301,16 @@ __device__ void scan_hist(const unsigned *hist, u64 r, unsigned *bin_out, u64 *r
     const u64 incl = s_part[threadIdx.x];
     u64 run = incl - sum;
     if (threadIdx.x == FIN_THREADS - 1 && incl < r) *err = 1;
-#pragma unroll
-    for (int i = 0; i < PER; ++i) {
-        if (run < r && r <= run + local[i]) {
-            *bin_out = threadIdx.x * PER + i;
-            *r_in_bin = r - run;
-            *cnt_out = local[i];
+    if (run < r && r <= incl) {                              // the bin is in this thread's range
+        for (int i = 0; i < PER; ++i) {
+            const u64 c = ld_vol(&hist[threadIdx.x * PER + i]);
+            if (run < r && r <= run + c) {
+                *bin_out = threadIdx.x * PER + i;
+                *r_in_bin = r - run;
+                *cnt_out = c;
+            }
+            run += c;
         }
-        run += local[i];
     }
     __syncthreads();
 }
@@ -321,13 +321,13 @@ __device__ void select_bin(const Params &p, Sel *s, const unsigned *hist) {
     __shared__ u64 s_r, s_cnt;
     if (threadIdx.x == 0) { s_err = 0; s_bin = 0; s_r = 0; s_cnt = 0; }
     __syncthreads();
-    scan_hist(hist, s->k, &s_bin, &s_r, &s_cnt, &s_err);
+    scan_hist(hist, p.nb, s->k, &s_bin, &s_r, &s_cnt, &s_err);
     if (threadIdx.x == 0) {
         if (s_err) atomicOr(p.dev_status, (unsigned)MWU_DEV_SELECT);
         const unsigned B = s_bin;
         u64 klo, khi;
         if (B == 0) { klo = 0; khi = s->lo0; }
-        else if (B == NB - 1) { klo = s->hi0; khi = ~0ull >> 1; }     // keys are < 2^63
+        else if (B == (unsigned)p.nb - 1u) { klo = s->hi0; khi = ~0ull >> 1; }     // keys are < 2^63
         else {
             klo = s->lo0 + ((u64)(B - 1) << s->shift0);
             khi = s->lo0 + ((u64)B << s->shift0);
@@ -382,6 +382,7 @@ __global__ void __launch_bounds__(256) stats_kernel(Params p, double *loss_u, do
     const Sel *su = &p.work->sel[1];
     const u64 plo = sp->lo0, phi = sp->hi0, ulo = su->lo0, uhi = su->hi0;
     const unsigned psh = sp->shift0, ush = su->shift0;
+    const unsigned nb = (unsigned)p.nb;
     unsigned cnt_under = 0, cnt_over = 0;
     unsigned nonfinite = 0;
     const long long n = p.n_floats;
@@ -400,12 +401,12 @@ __global__ void __launch_bounds__(256) stats_kernel(Params p, double *loss_u, do
             double S, Lu, Kp;
             block_keys<B>(v + e * B, p.use_l1, &S, &Lu, &Kp);
             const long long j = unit * NBT + e;
-            const unsigned bu = bin_of(key_bits(Lu), ulo, uhi, ush);
-            const unsigned bp = bin_of(key_bits(Kp), plo, phi, psh);
+            const unsigned bu = bin_of(key_bits(Lu), ulo, uhi, ush, nb);
+            const unsigned bp = bin_of(key_bits(Kp), plo, phi, psh, nb);
             code[e] = bp | (bu << 16);
             if (j < p.n_blocks) {
                 if (bp == 0) ++cnt_under;
-                else if (bp == NB - 1) ++cnt_over;
+                else if (bp == nb - 1u) ++cnt_over;
                 else atomicAdd(&p.hist[bp], 1u);
                 if (loss_u) loss_u[j] = Lu;
                 if (loss_p) loss_p[j] = Kp;
@@ -443,7 +444,7 @@ __global__ void __launch_bounds__(256) stats_kernel(Params p, double *loss_u, do
     __syncthreads();
     if (threadIdx.x == 0) {
         if (s_under) atomicAdd(&p.hist[0], s_under);
-        if (s_over) atomicAdd(&p.hist[NB - 1], s_over);
+        if (s_over) atomicAdd(&p.hist[nb - 1u], s_over);
     }
 }
 
@@ -452,7 +453,7 @@ template <int KIND>
 __global__ void __launch_bounds__(FIN_THREADS) bin_kernel(Params p) {
     Sel *s = &p.work->sel[KIND];
     if (ld_vol(&s->mode) != 0u) return;
-    select_bin(p, s, p.hist + (size_t)KIND * NB);
+    select_bin(p, s, p.hist + (size_t)KIND * p.nb);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -473,7 +474,7 @@ template <int B>
 __global__ void __launch_bounds__(FIN_THREADS) histu_kernel(Params p) {
     Sel *s = &p.work->sel[1];
     if (ld_vol(&s->mode) != 0u) return;
-    unsigned *hist = p.hist + NB;
+    unsigned *hist = p.hist + p.nb;
     const SelView pv = view_of(&p.work->sel[0]);
     const long long stride = (long long)gridDim.x * blockDim.x;
     unsigned under = 0, over = 0;
@@ -487,7 +488,7 @@ __global__ void __launch_bounds__(FIN_THREADS) histu_kernel(Params p) {
             if (selected<B>(p, pv, j, codes[e] & 0xffffu, 0)) continue;
             const unsigned bu = codes[e] >> 16;
             if (bu == 0) ++under;
-            else if (bu == NB - 1) ++over;
+            else if (bu == (unsigned)p.nb - 1u) ++over;
             else atomicAdd(&hist[bu], 1u);
         }
     }
@@ -497,7 +498,7 @@ __global__ void __launch_bounds__(FIN_THREADS) histu_kernel(Params p) {
     }
     if ((threadIdx.x & 31) == 0) {
         if (under) atomicAdd(&hist[0], under);
-        if (over) atomicAdd(&hist[NB - 1], over);
+        if (over) atomicAdd(&hist[p.nb - 1], over);
     }
     if (last_block_done(&p.work->ticket[2])) select_bin(p, s, hist);
 }
@@ -563,15 +564,15 @@ __global__ void __launch_bounds__(FIN_THREADS) collect_kernel(Params p) {
     // ---- last CTA only ----
     if (too_many) {
         // massive ties: narrow the composite range pass by pass with this CTA alone
-        unsigned *rhist = p.hist + (size_t)2 * NB;
+        unsigned *rhist = p.hist + (size_t)2 * p.nb;
         for (int level = 0; level < 10; ++level) {
             if (ld_vol(&s->cnt) <= (u64)CAP) break;
-            for (int i = threadIdx.x; i < NB; i += blockDim.x) rhist[i] = 0;
+            for (int i = threadIdx.x; i < p.nb; i += blockDim.x) rhist[i] = 0;
             __syncthreads();
             const u128 lo = from_halves(ld_vol(&s->lo_hi), ld_vol(&s->lo_lo));
             const u128 hi = from_halves(ld_vol(&s->hi_hi), ld_vol(&s->hi_lo));
             unsigned shift = 0;
-            while (((hi - lo - 1) >> shift) >= (u128)NB) ++shift;
+            while (((hi - lo - 1) >> shift) >= (u128)p.nb) ++shift;
             for (long long j = threadIdx.x; j < p.n_blocks; j += blockDim.x) {
                 const unsigned code = ld_vol(p.bins + j);
                 const unsigned bin = KIND ? (code >> 16) : (code & 0xffffu);
@@ -584,7 +585,7 @@ __global__ void __launch_bounds__(FIN_THREADS) collect_kernel(Params p) {
             __syncthreads();
             if (threadIdx.x == 0) s_err = 0;
             __syncthreads();
-            scan_hist(rhist, ld_vol(&s->r), &s_bin, &s_r, &s_cnt, &s_err);
+            scan_hist(rhist, p.nb, ld_vol(&s->r), &s_bin, &s_r, &s_cnt, &s_err);
             if (threadIdx.x == 0) {
                 if (s_err) atomicOr(p.dev_status, (unsigned)MWU_DEV_SELECT);
                 u128 nlo = lo + ((u128)s_bin << shift);
@@ -774,7 +775,7 @@ __global__ void __launch_bounds__(256, 3) emit_kernel(Params p, float *Q, float 
 // host side
 // ---------------------------------------------------------------------------------------------
 static size_t ws_off_hist() { return align_up(sizeof(proj::Work)); }
-static size_t ws_off_cand_key() { return align_up(ws_off_hist() + 3 * proj::NB * sizeof(unsigned)); }
+static size_t ws_off_cand_key() { return align_up(ws_off_hist() + 3 * proj::NB_MAX * sizeof(unsigned)); }
 static size_t ws_off_cand_idx() { return align_up(ws_off_cand_key() + proj::CAP * sizeof(proj::u64)); }
 static size_t ws_off_bins() { return align_up(ws_off_cand_idx() + proj::CAP * sizeof(unsigned)); }
 
@@ -851,7 +852,9 @@ extern "C" int mwu_project(const mwu_proj_desc *desc, const float *W, const floa
     p.bins = (unsigned *)(ws + ws_off_bins());
     p.dev_status = dev_status;
 
-    if (cudaMemsetAsync(ws, 0, ws_off_cand_key(), st) != cudaSuccess) return MWU_ERR_CUDA;
+    p.nb = p.n_blocks <= (8ll << 20) ? proj::NB_SMALL : proj::NB_MAX;
+    if (cudaMemsetAsync(ws, 0, ws_off_hist() + 3 * (size_t)p.nb * sizeof(unsigned), st) != cudaSuccess)
+        return MWU_ERR_CUDA;
     cudaError_t e;
     switch (desc->block) {
         case 2: e = launch_project<2>(p, desc, Q, u, pruned_bitmap, unified_bitmap, sign_bits, loss_u, loss_p, sm_count, st); break;
