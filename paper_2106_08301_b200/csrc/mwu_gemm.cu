@@ -1,21 +1,21 @@
 // mwu_gemm / mwu_conv_implicit: Y = X . W_hat^T on the packed weights (Section 3.2).
 //
-// One persistent CTA per SM works on tiles of 256 activation rows x 256 weight rows (GEMM; the
-// convolution and narrow problems use 128 activation rows).  A 64-wide k stage of the weight
+// One persistent CTA per SM works on tiles of 256 activation rows x 256 weight rows (128
+// activation rows when the problem has no more).  A 64-wide k stage of the weight
 // tile is decoded once into shared memory and multiplied with both 128-row halves of the
 // activation tile, which halves decode work, shared-memory stores and slot hand-shakes per FLOP.
 // Warp roles:
 //   warp 0        producer of the activation tile (A operand, bf16, K-major, 128-byte swizzle):
-//                 one thread issues one TMA load per stage (GEMM); for the convolution four extra
-//                 warps gather the im2col rows with plain loads instead.
+//                 one thread issues one TMA load per stage (GEMM); for the convolution one extra
+//                 warp per 32 tile rows gathers the im2col rows with plain loads instead.
 //   warp 1        allocates tensor memory and issues tcgen05.mma (one thread), M = 128, N = 256
 //                 per instruction, fp32 accumulators in TMEM (columns [0,256) for the first half
 //                 of the rows, [256,512) for the second).
 //   warps 2-9     epilogue: tcgen05.ld -> bf16/fp32 -> global, one warp per (half, 32 rows).
-//   warps 10-27   decode the weight tile (B operand) from the packed class lists into the
+//   warps 10-..   decode the weight tile (B operand) from the packed class lists into the
 //                 swizzled K-major layout the MMA reads: pruned blocks -> zeros, unified blocks
 //                 -> sign . bf16(u), dense blocks -> stored bf16 values.  Three groups of six
-//                 warps, one per pipeline slot.  A group reads the small per-entry words of its
+//                 warps (four for the convolution), one per pipeline slot.  A group reads the small per-entry words of its
 //                 next stage before it waits for the slot; once the slot is free it writes zeros
 //                 and sign . u words with plain stores and moves dense values with cp.async.
 // A 64-wide k stage whose blocks are pruned in every row of the weight tile is skipped by all
@@ -35,14 +35,17 @@ constexpr int STAGES = 3;
 constexpr int AH_BYTES = BMH * BK * 2;  // 16 KiB: one 128-row half of the activation stage
 constexpr int REC_BYTES = kTileRows * BK * 2;
 constexpr int NDEC_GROUPS = STAGES;     // one decode group per pipeline slot
-constexpr int NDEC_WARPS = 6;           // warps per decode group
-constexpr int NDEC_THREADS = NDEC_WARPS * 32;
 constexpr int NEPI_WARPS = 8;
 constexpr int FIRST_DEC_WARP = 2 + NEPI_WARPS;
-constexpr int FIRST_GATHER_WARP = FIRST_DEC_WARP + NDEC_WARPS * NDEC_GROUPS;
-constexpr int NGATHER_WARPS = 4;
-constexpr int THREADS_GEMM = 32 * FIRST_GATHER_WARP;
-constexpr int THREADS_CONV = THREADS_GEMM + 32 * NGATHER_WARPS;
+constexpr int MAX_GATHER_WARPS = 8;
+// warps per decode group: six for the GEMM, four for the convolution (whose gather warps also
+// need room inside the 1024-thread limit)
+__host__ __device__ constexpr int dec_warps(int mode) { return mode ? 4 : 6; }
+__host__ __device__ constexpr int first_gather_warp(int mode) { return FIRST_DEC_WARP + dec_warps(mode) * NDEC_GROUPS; }
+__host__ __device__ constexpr int gather_warps(int mode, int mt) { return mode ? 4 * mt : 0; }
+__host__ __device__ constexpr int cta_threads(int mode, int mt) {
+    return 32 * (first_gather_warp(mode) + gather_warps(mode, mt));
+}
 constexpr int MAX_STAGES_K = 256;       // cols <= 16384
 constexpr long long WAIT_LIMIT_CYCLES = 4000000000ll;   // about two seconds
 
@@ -59,7 +62,9 @@ struct Params {
     unsigned *dev_status;
     // convolution only
     const __nv_bfloat16 *X;
-    int C, H, W, KH, KW, stride, pad, OH, OW;
+    int C, H, W, KH, KW, stride, pad, OH, OW, NIMG;
+    // staged gather (0 rows: gather straight from global memory instead)
+    int patch_rows, patch_pitch, patch_nch;   // input rows per tile, row pitch (elements), channels per stage
 };
 
 // ------------------------------------------------------------------------------------------
@@ -190,7 +195,7 @@ __device__ __forceinline__ unsigned swz(unsigned r, unsigned c) {
 // The work is split in two: fetch_entries reads the small per-entry words (it can run before the
 // pipeline slot is free), write_entries fills the tile: zeros for pruned blocks, sign . bf16(u)
 // for unified blocks, and an asynchronous global->shared copy of the stored values for dense ones.
-template <int BW>
+template <int BW, int NDEC_THREADS>
 struct DecodeCfg {
     static constexpr int NBK = BK / BW;
     static constexpr int SLOTS = kTileRows * NBK;
@@ -199,10 +204,11 @@ struct DecodeCfg {
     static constexpr unsigned OFF_MASK = (unsigned)(REC_BYTES - 1) & ~(unsigned)((BW >= 8 ? 16 : 2 * BW) - 1);
 };
 
-template <int BW>
+template <int BW, int NDEC_THREADS>
 __device__ __forceinline__ void fetch_entries(const PackedRec r0, const PackedRec r1, const Params &p, int tid,
-                                              unsigned (&m0)[DecodeCfg<BW>::ENT], unsigned (&m1)[DecodeCfg<BW>::ENT]) {
-    constexpr int ENT = DecodeCfg<BW>::ENT;
+                                              unsigned (&m0)[DecodeCfg<BW, NDEC_THREADS>::ENT],
+                                              unsigned (&m1)[DecodeCfg<BW, NDEC_THREADS>::ENT]) {
+    constexpr int ENT = DecodeCfg<BW, NDEC_THREADS>::ENT;
     const uint2 *ulist = reinterpret_cast<const uint2 *>(p.packed + p.off_ulist);
     const unsigned short *dpos = reinterpret_cast<const unsigned short *>(p.packed + p.off_dpos);
     const unsigned short *ppos = reinterpret_cast<const unsigned short *>(p.packed + p.off_ppos);
@@ -230,14 +236,14 @@ __device__ __forceinline__ void fetch_entries(const PackedRec r0, const PackedRe
     }
 }
 
-template <int BW>
+template <int BW, int NDEC_THREADS>
 __device__ __forceinline__ void write_entries(unsigned char *tile, const PackedRec r0, const PackedRec r1,
                                               const Params &p, int tid,
-                                              const unsigned (&m0)[DecodeCfg<BW>::ENT],
-                                              const unsigned (&m1)[DecodeCfg<BW>::ENT]) {
-    constexpr int ENT = DecodeCfg<BW>::ENT;
-    constexpr int WORDS = DecodeCfg<BW>::WORDS;
-    constexpr unsigned OFF_MASK = DecodeCfg<BW>::OFF_MASK;
+                                              const unsigned (&m0)[DecodeCfg<BW, NDEC_THREADS>::ENT],
+                                              const unsigned (&m1)[DecodeCfg<BW, NDEC_THREADS>::ENT]) {
+    constexpr int ENT = DecodeCfg<BW, NDEC_THREADS>::ENT;
+    constexpr int WORDS = DecodeCfg<BW, NDEC_THREADS>::WORDS;
+    constexpr unsigned OFF_MASK = DecodeCfg<BW, NDEC_THREADS>::OFF_MASK;
     const unsigned char *dpay = p.packed + p.off_dpay;
     const unsigned n_p = r1.pbase - r0.pbase, n_d = r1.dbase - r0.dbase;
     const unsigned p8 = (n_p + 7u) & ~7u, d8 = (n_d + 7u) & ~7u;
@@ -289,20 +295,24 @@ struct Smem {
     int abort;
     unsigned char live_prod[MAX_STAGES_K];                  // live masks of the producer's tile
     unsigned char live_mma[MAX_STAGES_K];                   // ... of the MMA issuer's tile
-    unsigned char live_gather[NGATHER_WARPS][MAX_STAGES_K]; // ... of each gather warp's tile
+    unsigned char live_gather[MAX_GATHER_WARPS][MAX_STAGES_K]; // ... of each gather warp's tile
     unsigned short live_list[NDEC_GROUPS][MAX_STAGES_K];    // live stage numbers of a decode group's tile
     int n_live[NDEC_GROUPS];
 };
 
-__device__ __forceinline__ void group_bar(int group) {      // the threads of one decode group
-    asm volatile("bar.sync %0, %1;" ::"r"(1 + group), "r"(NDEC_THREADS) : "memory");
+__device__ __forceinline__ void group_bar(int group, int nthreads) {   // the threads of one decode group
+    asm volatile("bar.sync %0, %1;" ::"r"(1 + group), "r"(nthreads) : "memory");
 }
 
 // MODE 0: GEMM (A by TMA), 1: convolution (A gathered).  NREC: 128-row weight records per tile.
 // MT: 128-row halves of the activation tile (1 or 2).
 template <int MODE, int NREC, int BW, int MT>
-__global__ void __launch_bounds__(MODE ? THREADS_CONV : THREADS_GEMM, 1)
+__global__ void __launch_bounds__(cta_threads(MODE, MT), 1)
 mwu_gemm_kernel(const __grid_constant__ CUtensorMap tmap, const Params p) {
+    constexpr int NDEC_WARPS = dec_warps(MODE);
+    constexpr int NDEC_THREADS = NDEC_WARPS * 32;
+    constexpr int FIRST_GATHER_WARP = first_gather_warp(MODE);
+    constexpr int NGATHER_WARPS = gather_warps(MODE, MT);
     extern __shared__ unsigned char smem_raw[];
     unsigned char *base = reinterpret_cast<unsigned char *>(
         (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -316,6 +326,8 @@ mwu_gemm_kernel(const __grid_constant__ CUtensorMap tmap, const Params p) {
     // per decode group: the record table of its current tile, [NREC][n_stages + 1]
     uint4 *srec = reinterpret_cast<uint4 *>(reinterpret_cast<unsigned char *>(sm) + ((sizeof(Smem) + 15) & ~(size_t)15));
     int2 *ktab = reinterpret_cast<int2 *>(srec + (size_t)NDEC_GROUPS * NREC * (n_stages + 1));   // conv only
+    int2 *ptab = ktab + (MODE ? p.K : 0);                                                        // conv, staged
+    unsigned char *patch = reinterpret_cast<unsigned char *>(ptab + ((MODE && p.patch_rows) ? p.K : 0));
     volatile int *abort = &sm->abort;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -341,6 +353,11 @@ mwu_gemm_kernel(const __grid_constant__ CUtensorMap tmap, const Params p) {
             const int c = k / (p.KH * p.KW), rem = k % (p.KH * p.KW);
             const int di = rem / p.KW - p.pad, dj = rem % p.KW - p.pad;
             ktab[k] = make_int2(c * p.H * p.W + di * p.W + dj, (di & 0xffff) | (dj << 16));
+            if (p.patch_rows) {
+                const int c_lo = ((k / BK) * BK) / (p.KH * p.KW);      // first channel of k's stage
+                ptab[k] = make_int2((c - c_lo) * p.patch_rows * p.patch_pitch + (rem / p.KW) * p.patch_pitch + dj,
+                                    rem % p.KW);
+            }
         }
     }
     if (warp == 1) tmem_alloc(smem_u32(&sm->tmem_base), 512);
@@ -542,11 +559,11 @@ mwu_gemm_kernel(const __grid_constant__ CUtensorMap tmap, const Params p) {
             r0->ubase = a.x; r0->dbase = a.y; r0->pbase = a.z; r0->live = a.w;
             r1->ubase = b.x; r1->dbase = b.y; r1->pbase = b.z; r1->live = b.w;
         };
-        constexpr int ENT = DecodeCfg<BW>::ENT;
+        constexpr int ENT = DecodeCfg<BW, NDEC_THREADS>::ENT;
         unsigned m0[NREC][ENT], m1[NREC][ENT];
         for (long long t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
             const long long nt = t / m_tiles;
-            group_bar(group);                               // everyone is done with the previous tables
+            group_bar(group, NDEC_THREADS);                               // everyone is done with the previous tables
 #pragma unroll
             for (int q = 0; q < NREC; ++q) {
                 const long long rt = nt * NREC + q;
@@ -557,7 +574,7 @@ mwu_gemm_kernel(const __grid_constant__ CUtensorMap tmap, const Params p) {
                     my_rec[q * (n_stages + 1) + ks] = v;
                 }
             }
-            group_bar(group);
+            group_bar(group, NDEC_THREADS);
             if (gwarp == 0) {
                 // compact list of the live stages of this tile
                 int n = 0;
@@ -574,14 +591,14 @@ mwu_gemm_kernel(const __grid_constant__ CUtensorMap tmap, const Params p) {
                 }
                 if (lane == 0) sm->n_live[group] = n;
             }
-            group_bar(group);
+            group_bar(group, NDEC_THREADS);
             const int n_live = sm->n_live[group];
             auto fetch_stage = [&](int ks) {
 #pragma unroll
                 for (int q = 0; q < NREC; ++q) {
                     PackedRec r0, r1;
                     rec_at(q, ks, &r0, &r1);
-                    fetch_entries<BW>(r0, r1, p, tid, m0[q], m1[q]);
+                    fetch_entries<BW, NDEC_THREADS>(r0, r1, p, tid, m0[q], m1[q]);
                 }
             };
             // this group owns the live stages whose running number is congruent to `group`
@@ -599,7 +616,7 @@ mwu_gemm_kernel(const __grid_constant__ CUtensorMap tmap, const Params p) {
                 for (int q = 0; q < NREC; ++q) {
                     PackedRec r0, r1;
                     rec_at(q, ks, &r0, &r1);
-                    write_entries<BW>(sB + stage * B_BYTES + q * REC_BYTES, r0, r1, p, tid, m0[q], m1[q]);
+                    write_entries<BW, NDEC_THREADS>(sB + stage * B_BYTES + q * REC_BYTES, r0, r1, p, tid, m0[q], m1[q]);
                 }
                 // the entry words of this group's next stage travel while the copies above land
                 if (i + NDEC_GROUPS < n_live) fetch_stage(my_list[i + NDEC_GROUPS]);
@@ -611,12 +628,13 @@ mwu_gemm_kernel(const __grid_constant__ CUtensorMap tmap, const Params p) {
             seq0 += n_live;
         }
     } else if (MODE == 1 && warp >= FIRST_GATHER_WARP) {
-        // ---------------- im2col gather of the A tile (convolution, MT == 1) ----------------
+        // ---------------- im2col gather of the A tile (convolution) ----------------
         const int gw = warp - FIRST_GATHER_WARP;
-        const int r = threadIdx.x - FIRST_GATHER_WARP * 32;     // row of the tile, 0..127
+        const int r = threadIdx.x - FIRST_GATHER_WARP * 32;     // row of the tile, 0 .. BM-1
         const unsigned short *X = reinterpret_cast<const unsigned short *>(p.X);
         int stage = 0;
         unsigned phase = 0;
+        unsigned pcount = 0;                                     // patch buffers used so far
         bool ok = true;
         const long long hw = (long long)p.OH * p.OW;
         for (long long t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
@@ -626,31 +644,104 @@ mwu_gemm_kernel(const __grid_constant__ CUtensorMap tmap, const Params p) {
             const bool row_ok = m < p.M;
             const long long img = row_ok ? m / hw : 0, pix = row_ok ? m % hw : 0;
             const int ih0 = (int)(pix / p.OW) * p.stride, iw0 = (int)(pix % p.OW) * p.stride;
-            const long long xbase = img * (long long)p.C * p.H * p.W + (long long)ih0 * p.W + iw0;
+            const unsigned short *xrow = X + img * (long long)p.C * p.H * p.W + (long long)ih0 * p.W + iw0;
+            unsigned char *row_base = sA + (r >> 7) * AH_BYTES;  // which 128-row half
+            const unsigned rr = (unsigned)(r & 127);
+            if (p.patch_rows) {
+                // ---- staged: copy the needed input rows of the stage's channels into shared memory
+                // once (8-byte loads), then assemble the im2col rows from there.  Rows and columns are
+                // addressed in padded coordinates: padded row = oh*stride + i, padded col = ow*stride + j.
+                const int HP = p.H + 2 * p.pad;
+                const long long m_first = mt * BM;
+                const long long prow0 = (m_first / hw) * HP + ((m_first % hw) / p.OW) * p.stride;
+                const int PR = p.patch_rows, PW = p.patch_pitch, QW = PW / 4;
+                const int prow_r = (int)(img * HP + ih0 - prow0);
+                const int tbase = prow_r * PW + iw0;
+                unsigned colmask = 0;                                    // tap column j stays inside the image
+                for (int j = 0; j < p.KW; ++j)
+                    if ((unsigned)(iw0 + j - p.pad) < (unsigned)p.W) colmask |= 1u << j;
+                if (!row_ok) colmask = 0;
+                for (int ks = 0; ks < n_stages; ++ks) {
+                    if (!sm->live_gather[gw][ks]) continue;
+                    const int c_lo = (ks * BK) / (p.KH * p.KW);
+                    int c_hi = (ks * BK + BK - 1) / (p.KH * p.KW);
+                    if (c_hi > p.C - 1) c_hi = p.C - 1;
+                    unsigned char *buf = patch + (size_t)(pcount & 1) * ((size_t)p.patch_nch * PR * PW * 2);
+                    ++pcount;
+                    for (int idx = r; idx < PR * QW; idx += NGATHER_WARPS * 32) {
+                        const int pr = idx / QW, q4 = (idx % QW) * 4;
+                        const long long pabs = prow0 + pr;
+                        const long long pimg = pabs / HP;
+                        const int ih = (int)(pabs % HP) - p.pad;
+                        const bool inside = pimg < p.NIMG && (unsigned)ih < (unsigned)p.H && q4 < p.W;
+                        const unsigned short *src = X + ((pimg * p.C + c_lo) * p.H + ih) * (long long)p.W + q4;
+                        unsigned char *dst = buf + ((size_t)pr * PW + q4) * 2;
+                        for (int c = c_lo; c <= c_hi; ++c) {
+                            uint2 v = make_uint2(0, 0);
+                            if (inside) v = __ldg(reinterpret_cast<const uint2 *>(src));
+                            *reinterpret_cast<uint2 *>(dst) = v;
+                            src += (long long)p.H * p.W;
+                            dst += (size_t)PR * PW * 2;
+                        }
+                    }
+                    asm volatile("bar.sync %0, %1;" ::"r"(1 + NDEC_GROUPS), "r"(NGATHER_WARPS * 32) : "memory");
+                    if (!mbar_wait(smem_u32(&sm->empty[stage]), phase ^ 1u, abort)) ok = false;
+                    ok = __all_sync(0xffffffffu, ok);
+                    if (!ok) break;
+                    unsigned char *tile = row_base + stage * A_BYTES;
+                    const int2 *tab = ptab + ks * BK;
+                    const unsigned short *pb = reinterpret_cast<const unsigned short *>(buf) + tbase;
+#pragma unroll 2
+                    for (int c = 0; c < 8; ++c) {
+                        unsigned short v[8];
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) {
+                            const int2 tb = tab[c * 8 + e];
+                            v[e] = 0;
+                            if ((colmask >> tb.y) & 1u) v[e] = pb[tb.x];
+                        }
+                        uint4 o;
+                        o.x = (unsigned)v[0] | ((unsigned)v[1] << 16);
+                        o.y = (unsigned)v[2] | ((unsigned)v[3] << 16);
+                        o.z = (unsigned)v[4] | ((unsigned)v[5] << 16);
+                        o.w = (unsigned)v[6] | ((unsigned)v[7] << 16);
+                        *reinterpret_cast<uint4 *>(tile + swz(rr, (unsigned)c)) = o;
+                    }
+                    fence_proxy_async();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&sm->full[stage]));
+                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                }
+                continue;
+            }
             for (int ks = 0; ks < n_stages; ++ks) {
                 if (!sm->live_gather[gw][ks]) continue;
                 if (!mbar_wait(smem_u32(&sm->empty[stage]), phase ^ 1u, abort)) ok = false;
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
-                unsigned char *tile = sA + stage * A_BYTES;
-#pragma unroll 1
-                for (int c = 0; c < 8; ++c) {
-                    unsigned w[4];
+                unsigned char *tile = row_base + stage * A_BYTES;
+                const int2 *tab = ktab + ks * BK;
+#pragma unroll 2
+                for (int c = 0; c < 8; c += 2) {
+                    // sixteen loads in flight, then two 16-byte stores
+                    unsigned short v[16];
 #pragma unroll
-                    for (int h = 0; h < 4; ++h) {
-                        unsigned pair = 0;
-#pragma unroll
-                        for (int e = 0; e < 2; ++e) {
-                            const int2 tb = ktab[ks * BK + c * 8 + h * 2 + e];
-                            const int ih = ih0 + (int)(short)(tb.y & 0xffff), iw = iw0 + (tb.y >> 16);
-                            unsigned val = 0;
-                            if (row_ok && (unsigned)ih < (unsigned)p.H && (unsigned)iw < (unsigned)p.W)
-                                val = __ldg(X + xbase + tb.x);
-                            pair |= val << (16 * e);
-                        }
-                        w[h] = pair;
+                    for (int e = 0; e < 16; ++e) {
+                        const int2 tb = tab[c * 8 + e];
+                        const int ih = ih0 + (int)(short)(tb.y & 0xffff), iw = iw0 + (tb.y >> 16);
+                        v[e] = 0;
+                        if (row_ok && (unsigned)ih < (unsigned)p.H && (unsigned)iw < (unsigned)p.W)
+                            v[e] = __ldg(xrow + tb.x);
                     }
-                    *reinterpret_cast<uint4 *>(tile + swz((unsigned)r, (unsigned)c)) = make_uint4(w[0], w[1], w[2], w[3]);
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        uint4 o;
+                        o.x = (unsigned)v[h * 8 + 0] | ((unsigned)v[h * 8 + 1] << 16);
+                        o.y = (unsigned)v[h * 8 + 2] | ((unsigned)v[h * 8 + 3] << 16);
+                        o.z = (unsigned)v[h * 8 + 4] | ((unsigned)v[h * 8 + 5] << 16);
+                        o.w = (unsigned)v[h * 8 + 6] | ((unsigned)v[h * 8 + 7] << 16);
+                        *reinterpret_cast<uint4 *>(tile + swz(rr, (unsigned)(c + h))) = o;
+                    }
                 }
                 fence_proxy_async();
                 __syncwarp();
@@ -691,9 +782,10 @@ static EncodeTiledFn get_encode_fn() {
     return fn;
 }
 
-static size_t smem_bytes(int nrec, int mt, long long n_stages, long long conv_k) {
+static size_t smem_bytes(int nrec, int mt, long long n_stages, long long conv_k, size_t patch_bytes = 0) {
     return 1024 + (size_t)STAGES * (mt * AH_BYTES + nrec * REC_BYTES) + ((sizeof(Smem) + 15) & ~(size_t)15) +
-           (size_t)NDEC_GROUPS * nrec * (n_stages + 1) * 16 + (size_t)conv_k * sizeof(int2);
+           (size_t)NDEC_GROUPS * nrec * (n_stages + 1) * 16 + (size_t)conv_k * sizeof(int2) +
+           (patch_bytes ? (size_t)conv_k * sizeof(int2) + patch_bytes : 0);
 }
 
 template <int MODE, int NREC, int BW, int MT>
@@ -701,7 +793,7 @@ static cudaError_t launch(const CUtensorMap &tmap, const Params &p, int grid, si
     auto kern = mwu_gemm_kernel<MODE, NREC, BW, MT>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    kern<<<grid, MODE ? THREADS_CONV : THREADS_GEMM, smem, st>>>(tmap, p);
+    kern<<<grid, cta_threads(MODE, MT), smem, st>>>(tmap, p);
     return cudaGetLastError();
 }
 
@@ -817,14 +909,46 @@ extern "C" int mwu_conv_implicit(const mwu_proj_desc *desc, const void *packed, 
     p.M = (long long)n * p.OH * p.OW;
     p.ldy = 0;
     const int nrec = p.n_rec_tiles >= 2 ? 2 : 1;
-    const size_t smem = smem_bytes(nrec, 1, p.n_stages, desc->cols);
+    const int mt = (p.M > BMH) ? 2 : 1;
+    p.NIMG = n;
+    // staged gather: possible when image rows are 8-byte multiples and two patches fit beside the ring
+    size_t patch_bytes = 0;
+    if (w % 4 == 0) {
+        const long long hwo = (long long)p.OH * p.OW, hp = h + 2 * pad, bm = (long long)mt * BMH;
+        long long pr_max = 0;
+        for (long long m0 = 0; m0 < p.M; m0 += bm) {
+            const long long m1 = (m0 + bm < p.M ? m0 + bm : p.M) - 1;
+            const long long r0 = (m0 / hwo) * hp + ((m0 % hwo) / p.OW) * stride;
+            const long long r1 = (m1 / hwo) * hp + ((m1 % hwo) / p.OW) * stride + kh - 1;
+            if (r1 - r0 + 1 > pr_max) pr_max = r1 - r0 + 1;
+        }
+        const int khkw = kh * kw;
+        int nch = 1;
+        for (long long ks = 0; ks < p.n_stages; ++ks) {
+            const int c_lo = (int)(ks * BK) / khkw;
+            int c_hi = (int)(ks * BK + BK - 1) / khkw;
+            if (c_hi > c - 1) c_hi = c - 1;
+            if (c_hi - c_lo + 1 > nch) nch = c_hi - c_lo + 1;
+        }
+        const size_t one = (size_t)nch * pr_max * w * 2;
+        if (smem_bytes(nrec, mt, p.n_stages, desc->cols, 2 * one + 16) <= 227 * 1024 && pr_max < 32768) {
+            p.patch_rows = (int)pr_max;
+            p.patch_pitch = w;
+            p.patch_nch = nch;
+            patch_bytes = 2 * one + 16;
+        }
+    }
+    const size_t smem = smem_bytes(nrec, mt, p.n_stages, desc->cols, patch_bytes);
     if (p.n_stages > MAX_STAGES_K || smem > 227 * 1024) return MWU_ERR_SHAPE;
-    const long long tiles = ((p.M + BMH - 1) / BMH) * ((p.n_rec_tiles + nrec - 1) / nrec);
+    const long long tiles = ((p.M + mt * BMH - 1) / (mt * BMH)) * ((p.n_rec_tiles + nrec - 1) / nrec);
     const int grid = (int)(tiles < sm_count ? tiles : sm_count);
     CUtensorMap tmap;
     memset(&tmap, 0, sizeof(tmap));
     cudaStream_t st = (cudaStream_t)cuda_stream;
-    cudaError_t e = (nrec == 2) ? launch_bw<1, 2, 1>(desc->block, tmap, p, grid, smem, st)
-                                : launch_bw<1, 1, 1>(desc->block, tmap, p, grid, smem, st);
+    cudaError_t e;
+    if (mt == 2) e = (nrec == 2) ? launch_bw<1, 2, 2>(desc->block, tmap, p, grid, smem, st)
+                                 : launch_bw<1, 1, 2>(desc->block, tmap, p, grid, smem, st);
+    else e = (nrec == 2) ? launch_bw<1, 2, 1>(desc->block, tmap, p, grid, smem, st)
+                         : launch_bw<1, 1, 1>(desc->block, tmap, p, grid, smem, st);
     return e == cudaSuccess ? MWU_OK : MWU_ERR_CUDA;
 }

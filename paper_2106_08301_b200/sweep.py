@@ -146,11 +146,12 @@ def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--set", default="main", choices=["main", "blocks", "projection", "all"])
     ap.add_argument("--reps", type=int, default=10)
+    ap.add_argument("--only", default="", help="run just this workload of the main set")
     args = ap.parse_args()
     B.lib()
     timer = Timer()
     if args.set in ("main", "all"):
-        for name in ["c1_linear", "c2_conv3x3", "c3_conv1x1", "c4_ffn"]:
+        for name in ([args.only] if args.only else ["c1_linear", "c2_conv3x3", "c3_conv1x1", "c4_ffn"]):
             print(json.dumps(run_workload(inputs.WORKLOADS[name], timer, args.reps)), flush=True)
     if args.set in ("blocks", "all"):
         for b in (2, 4, 8, 16):
