@@ -334,6 +334,8 @@ mwu_gemm_kernel(const __grid_constant__ CUtensorMap tmap, const Params p) {
     const PackedRec *recs = reinterpret_cast<const PackedRec *>(p.packed + p.off_rec);
     const long long m_tiles = (p.M + BM - 1) / BM;
     const long long n_tiles = (p.n_rec_tiles + NREC - 1) / NREC;
+    // tile t -> (mt, nt) with nt fastest: the CTAs of a wave share a few activation row blocks and
+    // sweep the packed weights, which are the smaller operand and stay resident in L2
     const long long total_tiles = m_tiles * n_tiles;
 
     if (threadIdx.x == 0) {
@@ -389,7 +391,7 @@ mwu_gemm_kernel(const __grid_constant__ CUtensorMap tmap, const Params p) {
         unsigned phase = 0;
         bool ok = true;
         for (long long t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
-            const long long mt = t % m_tiles, nt = t / m_tiles;
+            const long long mt = t / n_tiles, nt = t % n_tiles;
             load_live(sm->live_prod, nt);
             if (lane == 0) {
                 for (int ks = 0; ks < n_stages; ++ks) {
@@ -411,7 +413,7 @@ mwu_gemm_kernel(const __grid_constant__ CUtensorMap tmap, const Params p) {
         bool issued_any = false;
         bool ready = false;                                 // next slot's full barrier already seen complete
         for (long long t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
-            const long long nt = t / m_tiles;
+            const long long nt = t % n_tiles;
             load_live(sm->live_mma, nt);
             if (lane == 0) {
                 const int nrec_here = (int)((p.n_rec_tiles - nt * NREC) < NREC ? (p.n_rec_tiles - nt * NREC) : NREC);
@@ -469,7 +471,7 @@ mwu_gemm_kernel(const __grid_constant__ CUtensorMap tmap, const Params p) {
             unsigned acc_phase = 0;
             bool ok = true;
             for (long long t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
-                const long long mt = t % m_tiles, nt = t / m_tiles;
+                const long long mt = t / n_tiles, nt = t % n_tiles;
                 unsigned any = 0;
                 for (int ks = lane; ks < n_stages; ks += 32) any |= live_of(nt, ks);
                 any = __reduce_or_sync(0xffffffffu, any);
@@ -561,8 +563,9 @@ mwu_gemm_kernel(const __grid_constant__ CUtensorMap tmap, const Params p) {
         };
         constexpr int ENT = DecodeCfg<BW, NDEC_THREADS>::ENT;
         unsigned m0[NREC][ENT], m1[NREC][ENT];
+        PackedRec fr0[NREC], fr1[NREC];                     // record entries of the fetched stage
         for (long long t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
-            const long long nt = t / m_tiles;
+            const long long nt = t % n_tiles;
             group_bar(group, NDEC_THREADS);                               // everyone is done with the previous tables
 #pragma unroll
             for (int q = 0; q < NREC; ++q) {
@@ -596,16 +599,14 @@ mwu_gemm_kernel(const __grid_constant__ CUtensorMap tmap, const Params p) {
             auto fetch_stage = [&](int ks) {
 #pragma unroll
                 for (int q = 0; q < NREC; ++q) {
-                    PackedRec r0, r1;
-                    rec_at(q, ks, &r0, &r1);
-                    fetch_entries<BW, NDEC_THREADS>(r0, r1, p, tid, m0[q], m1[q]);
+                    rec_at(q, ks, &fr0[q], &fr1[q]);
+                    fetch_entries<BW, NDEC_THREADS>(fr0[q], fr1[q], p, tid, m0[q], m1[q]);
                 }
             };
             // this group owns the live stages whose running number is congruent to `group`
             int i = (int)((group + NDEC_GROUPS - (seq0 % NDEC_GROUPS)) % NDEC_GROUPS);
             if (i < n_live) fetch_stage(my_list[i]);
             for (; i < n_live; i += NDEC_GROUPS) {
-                const int ks = my_list[i];
                 const long long my_seq = seq0 + i;
                 const int stage = group;                    // = my_seq % STAGES
                 const unsigned phase = (unsigned)((my_seq / STAGES) & 1);
@@ -613,11 +614,9 @@ mwu_gemm_kernel(const __grid_constant__ CUtensorMap tmap, const Params p) {
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
 #pragma unroll
-                for (int q = 0; q < NREC; ++q) {
-                    PackedRec r0, r1;
-                    rec_at(q, ks, &r0, &r1);
-                    write_entries<BW, NDEC_THREADS>(sB + stage * B_BYTES + q * REC_BYTES, r0, r1, p, tid, m0[q], m1[q]);
-                }
+                for (int q = 0; q < NREC; ++q)
+                    write_entries<BW, NDEC_THREADS>(sB + stage * B_BYTES + q * REC_BYTES, fr0[q], fr1[q], p, tid,
+                                                    m0[q], m1[q]);
                 // the entry words of this group's next stage travel while the copies above land
                 if (i + NDEC_GROUPS < n_live) fetch_stage(my_list[i + NDEC_GROUPS]);
                 asm volatile("cp.async.wait_all;" ::: "memory");
@@ -638,7 +637,7 @@ mwu_gemm_kernel(const __grid_constant__ CUtensorMap tmap, const Params p) {
         bool ok = true;
         const long long hw = (long long)p.OH * p.OW;
         for (long long t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
-            const long long mt = t % m_tiles, nt = t / m_tiles;
+            const long long mt = t / n_tiles, nt = t % n_tiles;
             load_live(sm->live_gather[gw], nt);
             const long long m = mt * BM + r;
             const bool row_ok = m < p.M;
