@@ -387,10 +387,16 @@ __global__ void __launch_bounds__(256) stats_kernel(Params p, double *loss_u, do
     unsigned nonfinite = 0;
     const long long n = p.n_floats;
     const long long n_units = (n + 15) / 16;
-    for (long long unit = (long long)blockIdx.x * blockDim.x + threadIdx.x; unit < n_units;
-         unit += (long long)gridDim.x * blockDim.x) {
+    const long long ustride = (long long)gridDim.x * blockDim.x;
+    long long unit = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    float nxt[16];
+    if (unit < n_units) load16(p.W, p.U, unit * 16, n, nxt);
+    for (; unit < n_units; unit += ustride) {
         float v[16];
-        load16(p.W, p.U, unit * 16, n, v);
+#pragma unroll
+        for (int l = 0; l < 16; ++l) v[l] = nxt[l];
+        // the next unit's 64 bytes travel while this one is evaluated
+        if (unit + ustride < n_units) load16(p.W, p.U, (unit + ustride) * 16, n, nxt);
         unsigned ex = 0;
 #pragma unroll
         for (int l = 0; l < 16; ++l) ex = max(ex, __float_as_uint(v[l]) & 0x7fffffffu);
