@@ -160,8 +160,8 @@ def cpu_threads():
 
 
 def oracle_sample_sizes(wl):
-    # about 10-30 s of CPU work: 1/16 of the weight rows, 128 activation rows
-    return max(128, wl.rows // 16), 128
+    # about 10-30 s of CPU work on the default workload: half of the weight rows, 1024 activation rows
+    return max(128, wl.rows // 2), min(1024, max(1, wl.m))
 
 
 def run_reference(args):
