@@ -180,3 +180,25 @@ def test_conv_config2():
     n, c, h, w, kh, kw, stride, pad = wl.conv
     conv_case(wl.weights(), wl.block, B.mwu_count_from_permille(Mb, wl.unified_permille),
               B.mwu_count_from_permille(Mb, wl.pruned_permille), x, kh, kw, stride, pad)
+
+
+@pytest.mark.parametrize("b", [2, 4, 8, 16])
+def test_gemm_pair_tiles(b):
+    """Shapes that take the two-CTA path: M > 256, an even number of 128-row weight tiles, N a
+    multiple of 256; M = 900 leaves a ragged last 512-row tile, K = 320 gives five stages (more
+    than the four pipeline slots)."""
+    W = inputs.normal_weights(512, 320, 0.02, 80 + b)
+    Mb = W.numel() // b
+    check_gemm(W, b, Mb * 7 // 10, Mb * 4 // 10, 900, seed=20 + b)
+
+
+def test_gemm_pair_tiles_dead_stages_and_all_pruned():
+    W = inputs.normal_weights(512, 512, 0.02, 90)
+    W[:, 128:256] = 0.0                 # stages 2 and 3 dead in every record
+    W[:256, 448:464] = 0.0              # one dead slice in the first pair tile only
+    b = 16
+    Mb = W.numel() // b
+    n_zero = int((W.reshape(-1, b).abs().sum(dim=1) == 0).sum())
+    check_gemm(W, b, n_zero + 700, n_zero, 1030)
+    check_gemm(W, b, Mb, Mb, 600)       # everything pruned: zeros, no MMA issued at all
+    check_gemm(W, b, 0, 0, 513)         # everything dense
