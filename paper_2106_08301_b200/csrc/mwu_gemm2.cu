@@ -108,6 +108,20 @@ mwu_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap, const Params p) {
     const long long n_tiles = p.n_rec_tiles / 2;        // the host only takes this path for even counts
     const long long total_tiles = m_tiles * n_tiles;
     const long long pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+    // k-th tile of this CTA pair.  Normally tiles are dealt round-robin with the weight tile
+    // fastest.  In resident mode (the whole reduction fits the pipeline slots) a pair keeps one
+    // weight tile and walks the activation tiles, so the decoded weights stay in shared memory.
+    auto tile_of = [&](long long k, long long &mt, long long &nt) -> bool {
+        if (p.resident) {
+            nt = pair % n_tiles;
+            mt = pair / n_tiles + k * (n_pairs / n_tiles);
+            return mt < m_tiles;
+        }
+        const long long t = pair + k * n_pairs;
+        mt = t / n_tiles;
+        nt = t % n_tiles;
+        return t < total_tiles;
+    };
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < P_STAGES; ++s) {
@@ -144,8 +158,8 @@ mwu_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap, const Params p) {
         int stage = 0;
         unsigned phase = 0;
         bool ok = true;
-        for (long long t = pair; t < total_tiles && ok; t += n_pairs) {
-            const long long mt = t / n_tiles, nt = t % n_tiles;
+        long long mt = 0, nt = 0;
+        for (long long kt = 0; ok && tile_of(kt, mt, nt); ++kt) {
             load_live(sm->live_prod, nt);
             if (lane == 0) {
                 for (int ks = 0; ks < n_stages; ++ks) {
@@ -167,8 +181,8 @@ mwu_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap, const Params p) {
         unsigned phase = 0, acc_phase = 0;
         bool ok = true, issued_any = false, ready = false;
         const unsigned idesc = make_idesc_pair(256);
-        for (long long t = pair; t < total_tiles && ok; t += n_pairs) {
-            const long long nt = t % n_tiles;
+        long long mt = 0, nt = 0;
+        for (long long kt = 0; ok && tile_of(kt, mt, nt); ++kt) {
             load_live(sm->live_mma, nt);
             if (lane == 0) {
                 if (!mbar_wait(smem_u32(&sm->tempty), acc_phase ^ 1u, abort)) ok = false;
@@ -222,8 +236,8 @@ mwu_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap, const Params p) {
         int stage = 0;
         unsigned phase = 0;
         bool ok = true;
-        for (long long t = pair; t < total_tiles && ok; t += n_pairs) {
-            const long long nt = t % n_tiles;
+        long long mt = 0, nt = 0;
+        for (long long kt = 0; ok && tile_of(kt, mt, nt); ++kt) {
             load_live(sm->live_mma, nt);
             if (lane == 0) {
                 for (int ks = 0; ks < n_stages; ++ks) {
@@ -241,8 +255,8 @@ mwu_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap, const Params p) {
         const int half = (warp - 2) >> 2;
         unsigned acc_phase = 0;
         bool ok = true;
-        for (long long t = pair; t < total_tiles && ok; t += n_pairs) {
-            const long long mt = t / n_tiles, nt = t % n_tiles;
+        long long mt = 0, nt = 0;
+        for (long long kt = 0; ok && tile_of(kt, mt, nt); ++kt) {
             unsigned any = 0;
             for (int ks = lane; ks < n_stages; ks += 32) any |= live_of(nt, ks);
             any = __reduce_or_sync(0xffffffffu, any);
@@ -310,7 +324,8 @@ mwu_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap, const Params p) {
         const int gwarp = tid >> 5;
         uint4 *my_rec = srec + (size_t)group * 2 * (n_stages + 1);   // [own | other][n_stages + 1]
         unsigned short *my_list = sm->live_list[group];
-        long long seq0 = 0;
+        long long seq0 = 0, prev_nt = -1;
+        int prev_live = -1;
         bool ok = true;
         constexpr int ENT = DecodeCfg<BW, P_DEC_THREADS>::ENT;
         unsigned m0[ENT], m1[ENT];
@@ -320,8 +335,25 @@ mwu_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap, const Params p) {
             r0->ubase = a.x; r0->dbase = a.y; r0->pbase = a.z; r0->live = a.w;
             r1->ubase = b.x; r1->dbase = b.y; r1->pbase = b.z; r1->live = b.w;
         };
-        for (long long t = pair; t < total_tiles && ok; t += n_pairs) {
-            const long long nt = t % n_tiles;
+        long long mt = 0, nt = 0;
+        for (long long kt = 0; ok && tile_of(kt, mt, nt); ++kt) {
+            if (p.resident && nt == prev_nt && prev_live == P_STAGES) {
+                // the slots already hold this weight tile's stages (stage i sits in slot i):
+                // only keep the barrier phases moving
+                const int i = group;
+                const long long my_seq = seq0 + i;
+                const unsigned phase = (unsigned)((my_seq / P_STAGES) & 1);
+                if (!mbar_wait(smem_u32(&sm->empty[group]), phase ^ 1u, abort)) ok = false;
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                __syncwarp();
+                if (lane == 0) {
+                    if (rank == 0) mbar_arrive(smem_u32(&sm->full[group]));
+                    else mbar_arrive_cluster(smem_u32(&sm->full[group]), 0);
+                }
+                seq0 += P_STAGES;
+                continue;
+            }
             pair_group_bar(group);
             for (int q = 0; q < 2; ++q) {
                 const long long rt = nt * 2 + (q == 0 ? rank : 1 - rank);
@@ -346,6 +378,8 @@ mwu_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap, const Params p) {
             }
             pair_group_bar(group);
             const int n_live = sm->n_live[group];
+            prev_nt = nt;
+            prev_live = n_live;
             int i = (int)((group + P_GROUPS - (seq0 % P_GROUPS)) % P_GROUPS);
             if (i < n_live) { rec_at(my_list[i], &fr0, &fr1); fetch_entries<BW, P_DEC_THREADS>(fr0, fr1, p, tid, m0, m1); }
             for (; i < n_live; i += P_GROUPS) {
@@ -399,9 +433,17 @@ static cudaError_t launch_pair_bw(const CUtensorMap &tmap, const Params &p, int 
     const size_t smem = pair_smem_bytes(p.n_stages);
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    const long long tiles = ((p.M + 511) / 512) * (p.n_rec_tiles / 2);
+    const long long n_tiles = p.n_rec_tiles / 2;
+    const long long tiles = ((p.M + 511) / 512) * n_tiles;
     long long pairs = sm_count / 2;
     if (tiles < pairs) pairs = tiles;
+    Params q = p;
+    // resident weights: the whole reduction fits the slots and every pair can own one weight tile
+    q.resident = 0;
+    if (p.n_stages <= P_STAGES && n_tiles <= pairs && tiles >= 4 * pairs) {
+        q.resident = 1;
+        pairs = pairs / n_tiles * n_tiles;
+    }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(2 * pairs));
     cfg.blockDim = dim3(P_THREADS);
@@ -414,7 +456,7 @@ static cudaError_t launch_pair_bw(const CUtensorMap &tmap, const Params &p, int 
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, kern, tmap, p);
+    return cudaLaunchKernelEx(&cfg, kern, tmap, q);
 }
 
 cudaError_t launch_pair(int bw, const CUtensorMap &tmap, const Params &p, int sm_count, cudaStream_t st) {

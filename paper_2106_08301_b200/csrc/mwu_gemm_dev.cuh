@@ -40,6 +40,7 @@ struct Params {
     void *Y;
     long long ldy;
     int y_fp32;
+    int resident;                       // pair kernel: a CTA pair keeps one weight tile (see mwu_gemm2.cu)
     unsigned *dev_status;
     // convolution only
     const __nv_bfloat16 *X;

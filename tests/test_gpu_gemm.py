@@ -202,3 +202,13 @@ def test_gemm_pair_tiles_dead_stages_and_all_pruned():
     check_gemm(W, b, n_zero + 700, n_zero, 1030)
     check_gemm(W, b, Mb, Mb, 600)       # everything pruned: zeros, no MMA issued at all
     check_gemm(W, b, 0, 0, 513)         # everything dense
+
+
+@pytest.mark.parametrize("K,b", [(256, 8), (192, 16)])
+def test_gemm_pair_tiles_resident_weights(K, b):
+    """Small reduction, many activation rows: a CTA pair keeps one weight tile in shared memory and
+    walks the activation tiles (K = 256 fills the four slots exactly, so decode is skipped after
+    the first tile; K = 192 takes the same tile order but re-decodes)."""
+    W = inputs.normal_weights(512, K, 0.02, 95 + b)
+    Mb = W.numel() // b
+    check_gemm(W, b, Mb * 3 // 4, Mb // 2, 77000 + 37, seed=31 + b)
