@@ -237,40 +237,11 @@ mwu_gemm_kernel(const __grid_constant__ CUtensorMap tmap, const Params p) {
                     }
                     const long long n0 = nt * (NREC * kTileRows) + c0;
                     if (MODE == 0) {
-                        if (m < p.M) {
-                            if (p.y_fp32) {
-                                float *dst = reinterpret_cast<float *>(p.Y) + m * p.ldy + n0;
-                                if (n0 + 32 <= p.N) {
-#pragma unroll
-                                    for (int j = 0; j < 32; j += 4)
-                                        *reinterpret_cast<uint4 *>(dst + j) = make_uint4(v[j], v[j + 1], v[j + 2], v[j + 3]);
-                                } else {
-                                    for (int j = 0; j < 32; ++j)
-                                        if (n0 + j < p.N) dst[j] = __uint_as_float(v[j]);
-                                }
-                            } else {
-                                __nv_bfloat16 *dst = reinterpret_cast<__nv_bfloat16 *>(p.Y) + m * p.ldy + n0;
-                                if (n0 + 32 <= p.N) {
-#pragma unroll
-                                    for (int j = 0; j < 32; j += 8) {
-                                        uint4 o;
-                                        __nv_bfloat162 h2;
-                                        h2 = __floats2bfloat162_rn(__uint_as_float(v[j]), __uint_as_float(v[j + 1]));
-                                        o.x = *reinterpret_cast<unsigned *>(&h2);
-                                        h2 = __floats2bfloat162_rn(__uint_as_float(v[j + 2]), __uint_as_float(v[j + 3]));
-                                        o.y = *reinterpret_cast<unsigned *>(&h2);
-                                        h2 = __floats2bfloat162_rn(__uint_as_float(v[j + 4]), __uint_as_float(v[j + 5]));
-                                        o.z = *reinterpret_cast<unsigned *>(&h2);
-                                        h2 = __floats2bfloat162_rn(__uint_as_float(v[j + 6]), __uint_as_float(v[j + 7]));
-                                        o.w = *reinterpret_cast<unsigned *>(&h2);
-                                        *reinterpret_cast<uint4 *>(dst + j) = o;
-                                    }
-                                } else {
-                                    for (int j = 0; j < 32; ++j)
-                                        if (n0 + j < p.N) dst[j] = __float2bfloat16_rn(__uint_as_float(v[j]));
-                                }
-                            }
-                        }
+                        if (p.stage_epi && !p.y_fp32 && n0 + 32 <= p.N)
+                            store_chunk_staged(p, m - lane, lane, n0, v,
+                                               reinterpret_cast<unsigned char *>(ktab) + (warp - 2) * 2048);
+                        else
+                            store_row_chunk<32>(p, m, n0, v);
                     } else {
                         // NCHW output: row m = (img, oh, ow); consecutive lanes write consecutive pixels
                         if (m < p.M) {
@@ -611,10 +582,15 @@ extern "C" int mwu_gemm(const mwu_proj_desc *desc, const void *packed, const voi
     const int nrec = p.n_rec_tiles >= 2 ? 2 : 1;
     const long long tiles = ((M + bm - 1) / bm) * ((p.n_rec_tiles + nrec - 1) / nrec);
     const int grid = (int)(tiles < sm_count ? tiles : sm_count);
-    const size_t smem = smem_bytes(nrec, mt, p.n_stages, 0);
+    size_t smem = smem_bytes(nrec, mt, p.n_stages, 0);
     if (p.n_stages > MAX_STAGES_K || smem > 227 * 1024) return MWU_ERR_SHAPE;
     cudaStream_t st = (cudaStream_t)cuda_stream;
     cudaError_t e;
+    // bf16 rows are 16-byte aligned (checked above), which the staged epilogue stores need
+    if (!y_dtype && smem + NEPI_WARPS * 2048 <= 227 * 1024) {
+        p.stage_epi = 1;
+        smem += NEPI_WARPS * 2048;
+    }
     if (mt == 2 && pair_eligible(p))
         return launch_pair(desc->block, tmap, p, sm_count, st) == cudaSuccess ? MWU_OK : MWU_ERR_CUDA;
     if (mt == 2) e = (nrec == 2) ? launch_bw<0, 2, 2>(desc->block, tmap, p, grid, smem, st)

@@ -99,6 +99,7 @@ mwu_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap, const Params p) {
     PairSmem *sm = reinterpret_cast<PairSmem *>(sB + P_STAGES * P_B_BYTES);
     const int n_stages = (int)p.n_stages;
     uint4 *srec = reinterpret_cast<uint4 *>(reinterpret_cast<unsigned char *>(sm) + ((sizeof(PairSmem) + 15) & ~(size_t)15));
+    unsigned char *stage_buf = reinterpret_cast<unsigned char *>(srec + (size_t)P_GROUPS * 2 * (n_stages + 1));  // epilogue
     volatile int *abort = &sm->abort;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -266,49 +267,22 @@ mwu_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap, const Params p) {
             acc_phase ^= 1u;
             tc_fence_after();
             const long long m = mt * 512 + rank * 256 + half * BMH + quarter * 32 + lane;
+            const unsigned trow = tmem_base + ((unsigned)(quarter * 32) << 16) + (unsigned)(half * 256);
+            const long long ncol0 = nt * 256;
+            unsigned char *stg = stage_buf + (warp - 2) * 2048;        // this warp's 32 x 64-byte buffer
             for (int c0 = 0; c0 < 256; c0 += 32) {
                 unsigned v[32];
                 if (any) {
-                    tmem_ld32(tmem_base + ((unsigned)(quarter * 32) << 16) + (unsigned)(half * 256 + c0), v);
+                    tmem_ld32(trow + (unsigned)c0, v);
                 } else {
 #pragma unroll
                     for (int j = 0; j < 32; ++j) v[j] = 0u;
                 }
-                const long long n0 = nt * 256 + c0;
-                if (m < p.M) {
-                    if (p.y_fp32) {
-                        float *dst = reinterpret_cast<float *>(p.Y) + m * p.ldy + n0;
-                        if (n0 + 32 <= p.N) {
-#pragma unroll
-                            for (int j = 0; j < 32; j += 4)
-                                *reinterpret_cast<uint4 *>(dst + j) = make_uint4(v[j], v[j + 1], v[j + 2], v[j + 3]);
-                        } else {
-                            for (int j = 0; j < 32; ++j)
-                                if (n0 + j < p.N) dst[j] = __uint_as_float(v[j]);
-                        }
-                    } else {
-                        __nv_bfloat16 *dst = reinterpret_cast<__nv_bfloat16 *>(p.Y) + m * p.ldy + n0;
-                        if (n0 + 32 <= p.N) {
-#pragma unroll
-                            for (int j = 0; j < 32; j += 8) {
-                                uint4 o;
-                                __nv_bfloat162 h2;
-                                h2 = __floats2bfloat162_rn(__uint_as_float(v[j]), __uint_as_float(v[j + 1]));
-                                o.x = *reinterpret_cast<unsigned *>(&h2);
-                                h2 = __floats2bfloat162_rn(__uint_as_float(v[j + 2]), __uint_as_float(v[j + 3]));
-                                o.y = *reinterpret_cast<unsigned *>(&h2);
-                                h2 = __floats2bfloat162_rn(__uint_as_float(v[j + 4]), __uint_as_float(v[j + 5]));
-                                o.z = *reinterpret_cast<unsigned *>(&h2);
-                                h2 = __floats2bfloat162_rn(__uint_as_float(v[j + 6]), __uint_as_float(v[j + 7]));
-                                o.w = *reinterpret_cast<unsigned *>(&h2);
-                                *reinterpret_cast<uint4 *>(dst + j) = o;
-                            }
-                        } else {
-                            for (int j = 0; j < 32; ++j)
-                                if (n0 + j < p.N) dst[j] = __float2bfloat16_rn(__uint_as_float(v[j]));
-                        }
-                    }
+                if (p.y_fp32 || ncol0 + c0 + 32 > p.N) {
+                    store_row_chunk<32>(p, m, ncol0 + c0, v);
+                    continue;
                 }
+                store_chunk_staged(p, m - lane, lane, ncol0 + c0, v, stg);
             }
             tc_fence_before();
             __syncwarp();
@@ -419,7 +393,7 @@ mwu_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap, const Params p) {
 
 static size_t pair_smem_bytes(long long n_stages) {
     return 1024 + (size_t)P_STAGES * (P_A_BYTES + P_B_BYTES) + ((sizeof(PairSmem) + 15) & ~(size_t)15) +
-           (size_t)P_GROUPS * 2 * (n_stages + 1) * 16;
+           (size_t)P_GROUPS * 2 * (n_stages + 1) * 16 + (size_t)NEPI_WARPS * 2048;
 }
 
 bool pair_eligible(const Params &p) {

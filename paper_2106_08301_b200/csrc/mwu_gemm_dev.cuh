@@ -41,6 +41,7 @@ struct Params {
     long long ldy;
     int y_fp32;
     int resident;                       // pair kernel: a CTA pair keeps one weight tile (see mwu_gemm2.cu)
+    int stage_epi;                      // single-CTA GEMM: 16 KB of shared memory is there for store_chunk_staged
     unsigned *dev_status;
     // convolution only
     const __nv_bfloat16 *X;
@@ -134,7 +135,8 @@ __device__ __forceinline__ void umma_bf16(unsigned d_tmem, unsigned long long ad
 __device__ __forceinline__ void umma_commit(unsigned bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
-__device__ __forceinline__ void tmem_ld32(unsigned taddr, unsigned (&r)[32]) {
+// issue a 32-lane x 32-column load from tensor memory; the registers are valid after tmem_ld_wait
+__device__ __forceinline__ void tmem_ld32_issue(unsigned taddr, unsigned (&r)[32]) {
     asm volatile(
         "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
         "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
@@ -143,7 +145,91 @@ __device__ __forceinline__ void tmem_ld32(unsigned taddr, unsigned (&r)[32]) {
           "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
           "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
         : "r"(taddr) : "memory");
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+// wait for all tensor-memory loads of this thread; the registers are passed through so that the
+// compiler orders every later use of them after the wait
+__device__ __forceinline__ void tmem_ld_wait(unsigned (&r)[32]) {
+    asm volatile(
+        "tcgen05.wait::ld.sync.aligned;"
+        : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
+          "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]),
+          "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]),
+          "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
+        :: "memory");
+}
+__device__ __forceinline__ void tmem_ld32(unsigned taddr, unsigned (&r)[32]) {
+    tmem_ld32_issue(taddr, r);
+    tmem_ld_wait(r);
+}
+
+// a chunk of NC (16 or 32) columns of an output row: fp32 accumulators -> bf16 or fp32 -> global
+template <int NC>
+__device__ __forceinline__ void store_row_chunk(const Params &p, long long m, long long n0, const unsigned (&v)[NC]) {
+    if (m >= p.M) return;
+    if (p.y_fp32) {
+        float *dst = reinterpret_cast<float *>(p.Y) + m * p.ldy + n0;
+        if (n0 + NC <= p.N) {
+#pragma unroll
+            for (int j = 0; j < NC; j += 4)
+                *reinterpret_cast<uint4 *>(dst + j) = make_uint4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+        } else {
+            for (int j = 0; j < NC; ++j)
+                if (n0 + j < p.N) dst[j] = __uint_as_float(v[j]);
+        }
+    } else {
+        __nv_bfloat16 *dst = reinterpret_cast<__nv_bfloat16 *>(p.Y) + m * p.ldy + n0;
+        if (n0 + NC <= p.N) {
+#pragma unroll
+            for (int j = 0; j < NC; j += 8) {
+                uint4 o;
+                __nv_bfloat162 h2;
+                h2 = __floats2bfloat162_rn(__uint_as_float(v[j]), __uint_as_float(v[j + 1]));
+                o.x = *reinterpret_cast<unsigned *>(&h2);
+                h2 = __floats2bfloat162_rn(__uint_as_float(v[j + 2]), __uint_as_float(v[j + 3]));
+                o.y = *reinterpret_cast<unsigned *>(&h2);
+                h2 = __floats2bfloat162_rn(__uint_as_float(v[j + 4]), __uint_as_float(v[j + 5]));
+                o.z = *reinterpret_cast<unsigned *>(&h2);
+                h2 = __floats2bfloat162_rn(__uint_as_float(v[j + 6]), __uint_as_float(v[j + 7]));
+                o.w = *reinterpret_cast<unsigned *>(&h2);
+                *reinterpret_cast<uint4 *>(dst + j) = o;
+            }
+        } else {
+            for (int j = 0; j < NC; ++j)
+                if (n0 + j < p.N) dst[j] = __float2bfloat16_rn(__uint_as_float(v[j]));
+        }
+    }
+}
+
+// A 32-row x 32-column chunk of bf16 output, transposed through a 2 KB per-warp buffer so that four
+// lanes write one 64-byte run of a row (whole 32-byte sectors) instead of 32 lanes writing 16 bytes
+// to 32 different rows.  Lane l holds row mrow0 + l in v[]; row r keeps its four 16-byte pieces at
+// positions j ^ ((r >> 1) & 3), which makes both the writes and the transposed reads conflict-free.
+// All 32 lanes must call it; the caller guarantees n0 + 32 <= N and 16-byte aligned rows.
+__device__ __forceinline__ void store_chunk_staged(const Params &p, long long mrow0, int lane, long long n0,
+                                                   const unsigned (&v)[32], unsigned char *stg) {
+    __syncwarp();
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        uint4 o;
+        __nv_bfloat162 h2;
+        h2 = __floats2bfloat162_rn(__uint_as_float(v[8 * j]), __uint_as_float(v[8 * j + 1]));
+        o.x = *reinterpret_cast<unsigned *>(&h2);
+        h2 = __floats2bfloat162_rn(__uint_as_float(v[8 * j + 2]), __uint_as_float(v[8 * j + 3]));
+        o.y = *reinterpret_cast<unsigned *>(&h2);
+        h2 = __floats2bfloat162_rn(__uint_as_float(v[8 * j + 4]), __uint_as_float(v[8 * j + 5]));
+        o.z = *reinterpret_cast<unsigned *>(&h2);
+        h2 = __floats2bfloat162_rn(__uint_as_float(v[8 * j + 6]), __uint_as_float(v[8 * j + 7]));
+        o.w = *reinterpret_cast<unsigned *>(&h2);
+        *reinterpret_cast<uint4 *>(stg + lane * 64 + ((j ^ ((lane >> 1) & 3)) << 4)) = o;
+    }
+    __syncwarp();
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int r = (lane >> 2) + 8 * i, pc = lane & 3;
+        const uint4 o = *reinterpret_cast<const uint4 *>(stg + r * 64 + ((pc ^ ((r >> 1) & 3)) << 4));
+        if (mrow0 + r < p.M)
+            *reinterpret_cast<uint4 *>(reinterpret_cast<__nv_bfloat16 *>(p.Y) + (mrow0 + r) * p.ldy + n0 + pc * 8) = o;
+    }
 }
 
 // K-major operand, 128-byte swizzle: rows of 128 bytes, 8-row groups 1024 bytes apart
