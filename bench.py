@@ -31,6 +31,7 @@ from paper_2106_08301_b200 import inputs, replicas  # noqa: E402
 METRIC = "mwu_hot_path_effective_tflops"
 UNIT = "TFLOP/s"
 KERNELS_PER_STEP = 11     # sample, stats, bin, collect x2, histu, emit | count, scan, fill | gemm
+KERNELS_PER_STEP_WS = 12  # ... | decode, dense gemm (with a workspace and enough activation rows)
 
 
 def measured_peaks():
@@ -233,6 +234,8 @@ def run_gpu(args):
     Y = torch.empty((m, wl.rows), dtype=torch.bfloat16, device="cuda")
     Y_host = torch.empty((m, wl.rows), dtype=torch.bfloat16).pin_memory()
     stream = torch.cuda.current_stream()
+    ws_bytes = 0 if args.fused else B.mwu_gemm_workspace_bytes(desc, m)
+    workspace = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda") if ws_bytes else None
 
     def step(events=None):
         if events is not None:
@@ -243,7 +246,7 @@ def run_gpu(args):
         bufs.pack(W, packed=packed)
         if events is not None:
             events[2].record(stream)
-        B.mwu_gemm(desc, packed, X, m, wl.cols, Y, wl.rows, 0, bufs.dev_status)
+        B.mwu_gemm_ws(desc, packed, X, m, wl.cols, Y, wl.rows, 0, workspace, bufs.dev_status)
         if events is not None:
             events[3].record(stream)
 
@@ -305,9 +308,11 @@ def run_gpu(args):
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": wl.name, "rows": wl.rows, "cols": wl.cols, "block": wl.block,
                    "k_unify": ku, "k_prune": kp, "m": m, "parallelism": "replicas only",
+                   "gemm_path": "decode once + two-operand GEMM (workspace %.0f MB)" % (ws_bytes / 1e6)
+                   if ws_bytes else "decode fused into the GEMM",
                    "l2": "inputs larger than L2 (W %.0f MB, X %.0f MB, Y %.0f MB)" % (
                        W.numel() * 4 / 1e6, X.numel() * 2 / 1e6, Y.numel() * 2 / 1e6)},
-        "gpu_launches": KERNELS_PER_STEP * args.steps,
+        "gpu_launches": (KERNELS_PER_STEP_WS if ws_bytes else KERNELS_PER_STEP) * args.steps,
         "device_status": status,
     }
     if rank == 0:
@@ -335,7 +340,8 @@ def run_gpu(args):
         peak_tf = peaks["bf16_tflops_sustained"]
         ach = flops / (gemm_ms * 1e-3) / 1e12
         line["roofline"] = {
-            "kernel": "mwu_gemm_kernel", "bound": "tensor", "achieved": ach, "peak": peak_tf,
+            "kernel": "mwu_decode_kernel + mwu_dense_pair_kernel" if ws_bytes else "mwu_gemm_pair_kernel",
+            "bound": "tensor", "achieved": ach, "peak": peak_tf,
             "unit": "TFLOP/s", "frac": ach / peak_tf,
             "peak_source": peaks["source"] + " (sustained cuBLAS bf16)",
             "algorithmic_flops_per_launch": flops, "traffic": None,
@@ -369,6 +375,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default="c4_ffn")
     ap.add_argument("--m", type=int, default=0, help="override the number of activation rows")
+    ap.add_argument("--fused", action="store_true",
+                    help="no workspace: the GEMM decodes the packed weights inside its main loop")
     ap.add_argument("--impl", default="mwu", choices=["mwu", "reference"])
     args = ap.parse_args()
     if args.impl == "reference":

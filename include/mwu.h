@@ -184,6 +184,35 @@ int mwu_gemm(const mwu_proj_desc *desc, const void *packed, const void *X, int64
              void *cuda_stream);
 
 /*
+ * mwu_decode -- the compressed weights expanded to a dense matrix (Section 3.2, the layer's
+ * weight as the GEMM sees it): Wd[r][c] = W_hat[r][c] in bf16, i.e. 0 for pruned blocks,
+ * +-bf16(u) by sign bit for unified blocks, the stored bf16 value otherwise.
+ *
+ *   Wd   out  device, bf16 [n_pad][ldw] with n_pad = rows rounded up to a multiple of 128,
+ *             ldw >= cols, ldw % 8 == 0, 16-byte aligned; rows past `rows` are written as zeros.
+ * Every element of the n_pad x cols region is written; the caller owns the buffer.
+ */
+int mwu_decode(const mwu_proj_desc *desc, const void *packed, void *Wd, int64_t ldw,
+               uint32_t *dev_status, void *cuda_stream);
+
+/*
+ * mwu_gemm_ws -- mwu_gemm with a caller-owned scratch buffer.  With many activation rows the
+ * fused kernel would decode every weight record once per 512-row activation tile; given
+ * `workspace` of at least mwu_gemm_workspace_bytes(desc, M) bytes (device memory, 256-byte
+ * aligned) the weights are expanded once per call as by mwu_decode and a two-operand
+ * tensor-core GEMM reads them, still skipping the column slices that are pruned in every row
+ * of a weight tile.  The result is the same contraction with the same rounding of operands
+ * (bf16 x bf16, fp32 accumulation); only the summation order inside the tensor cores may differ.
+ * mwu_gemm_workspace_bytes returns 0 when M is too small for this to pay (or desc is invalid);
+ * with workspace == NULL, or fewer bytes than that, the call behaves exactly like mwu_gemm.
+ * The workspace holds nothing between calls and may be shared by calls on the same stream.
+ */
+size_t mwu_gemm_workspace_bytes(const mwu_proj_desc *desc, int64_t M);
+int mwu_gemm_ws(const mwu_proj_desc *desc, const void *packed, const void *X, int64_t M,
+                int64_t ldx, void *Y, int64_t ldy, int32_t y_dtype, void *workspace,
+                size_t workspace_bytes, uint32_t *dev_status, void *cuda_stream);
+
+/*
  * mwu_conv_implicit -- the same contraction for a convolution lowered to GEMM without
  * materialising the lowered matrix (Section 3.2: "convolution ... implemented by GEMM"):
  *   A[(n,oh,ow)][(c,i,j)] = x[n][c][oh*stride+i-pad][ow*stride+j-pad]  (0 outside),

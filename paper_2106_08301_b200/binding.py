@@ -16,7 +16,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libmwu.so")
 
 EXPORTS = ["mwu_status_string", "mwu_count_from_permille", "mwu_project_workspace_bytes",
-           "mwu_project", "mwu_project_static", "mwu_packed_bytes", "mwu_pack", "mwu_gemm",
+           "mwu_project", "mwu_project_static", "mwu_packed_bytes", "mwu_pack", "mwu_gemm", "mwu_decode", "mwu_gemm_workspace_bytes", "mwu_gemm_ws",
            "mwu_conv_implicit"]
 MWU_STATIC_MAX_BLOCKS = 1048576
 
@@ -65,6 +65,12 @@ def lib() -> ctypes.CDLL:
         L.mwu_pack.argtypes = [dp] + [vp] * 7 + [sz, vp, vp]
         L.mwu_gemm.restype = ctypes.c_int
         L.mwu_gemm.argtypes = [dp, vp, vp, i64, i64, vp, i64, i32, vp, vp]
+        L.mwu_decode.restype = ctypes.c_int
+        L.mwu_decode.argtypes = [dp, vp, vp, i64, vp, vp]
+        L.mwu_gemm_workspace_bytes.restype = ctypes.c_size_t
+        L.mwu_gemm_workspace_bytes.argtypes = [dp, i64]
+        L.mwu_gemm_ws.restype = ctypes.c_int
+        L.mwu_gemm_ws.argtypes = [dp, vp, vp, i64, i64, vp, i64, i32, vp, ctypes.c_size_t, vp, vp]
         L.mwu_conv_implicit.restype = ctypes.c_int
         L.mwu_conv_implicit.argtypes = [dp, vp, vp] + [i32] * 8 + [vp, i32, vp, vp]
         _lib = L
@@ -143,6 +149,27 @@ def mwu_gemm(desc, packed, X, M, ldx, Y, ldy, y_dtype, dev_status, stream=None, 
                         int(ldy), int(y_dtype), _ptr(dev_status), _stream(stream))
     if check and rc != MWU_OK:
         raise MwuError(rc, "mwu_gemm")
+    return rc
+
+
+def mwu_decode(desc, packed, Wd, ldw, dev_status, stream=None, check=True) -> int:
+    rc = lib().mwu_decode(ctypes.byref(desc), _ptr(packed), _ptr(Wd), int(ldw), _ptr(dev_status), _stream(stream))
+    if check and rc != MWU_OK:
+        raise MwuError(rc, "mwu_decode")
+    return rc
+
+
+def mwu_gemm_workspace_bytes(desc, M) -> int:
+    return int(lib().mwu_gemm_workspace_bytes(ctypes.byref(desc), int(M)))
+
+
+def mwu_gemm_ws(desc, packed, X, M, ldx, Y, ldy, y_dtype, workspace, dev_status, stream=None, check=True) -> int:
+    """mwu_gemm with a scratch tensor (uint8, or None); its size is taken from the tensor."""
+    nbytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    rc = lib().mwu_gemm_ws(ctypes.byref(desc), _ptr(packed), _ptr(X), int(M), int(ldx), _ptr(Y), int(ldy),
+                           int(y_dtype), _ptr(workspace), nbytes, _ptr(dev_status), _stream(stream))
+    if check and rc != MWU_OK:
+        raise MwuError(rc, "mwu_gemm_ws")
     return rc
 
 

@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 LIB = os.path.join(HERE, "libmwu.so")
-SOURCES = ["mwu_api.cu", "mwu_project.cu", "mwu_pack.cu", "mwu_gemm.cu", "mwu_gemm2.cu", "mwu_noalloc.cu"]
+SOURCES = ["mwu_api.cu", "mwu_project.cu", "mwu_pack.cu", "mwu_gemm.cu", "mwu_gemm2.cu", "mwu_gemm3.cu", "mwu_noalloc.cu"]
 
 
 def _sources():

@@ -30,6 +30,10 @@ namespace gemm {
 // pair kernel (two CTAs per tile), defined in mwu_gemm2.cu
 bool pair_eligible(const Params &p);
 cudaError_t launch_pair(int bw, const CUtensorMap &tmap, const Params &p, int sm_count, cudaStream_t st);
+// decode-once path, defined in mwu_gemm3.cu
+cudaError_t launch_decode(int bw, const Params &p, __nv_bfloat16 *Wd, long long ldw, cudaStream_t st);
+cudaError_t launch_dense(const CUtensorMap &tmap_x, const CUtensorMap &tmap_w, const Params &p, int sm_count,
+                         cudaStream_t st);
 
 // ------------------------------------------------------------------------------------------
 // the kernel
@@ -157,27 +161,34 @@ mwu_gemm_kernel(const __grid_constant__ CUtensorMap tmap, const Params p) {
         bool ok = true;
         bool issued_any = false;
         bool ready = false;                                 // next slot's full barrier already seen complete
+        // All 32 lanes run the loop and one elected lane issues the MMAs and commits: in a
+        // lane-0 branch the issue of one tcgen05.mma took about 100 cycles.
         for (long long t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
             const long long nt = t % n_tiles;
             load_live(sm->live_mma, nt);
-            if (lane == 0) {
-                const int nrec_here = (int)((p.n_rec_tiles - nt * NREC) < NREC ? (p.n_rec_tiles - nt * NREC) : NREC);
-                const unsigned idesc = make_idesc(nrec_here * kTileRows);
-                // the epilogue must have read the previous tile's accumulators
-                if (!mbar_wait(smem_u32(&sm->tempty), acc_phase ^ 1u, abort)) ok = false;
-                acc_phase ^= 1u;
+            const int nrec_here = (int)((p.n_rec_tiles - nt * NREC) < NREC ? (p.n_rec_tiles - nt * NREC) : NREC);
+            const unsigned idesc = make_idesc(nrec_here * kTileRows);
+            // the epilogue must have read the previous tile's accumulators
+            if (!mbar_wait(smem_u32(&sm->tempty), acc_phase ^ 1u, abort)) ok = false;
+            if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
+            acc_phase ^= 1u;
+            tc_fence_after();
+            bool first = true;
+            for (int ks = 0; ks < n_stages; ++ks) {
+                const unsigned live = sm->live_mma[ks];
+                if (!live) continue;
+                // `ready` was probed before the previous stage's MMAs were issued
+                if (!ready) {
+                    if (!mbar_wait_spin(smem_u32(&sm->full[stage]), phase, abort)) ok = false;
+                    if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
+                }
                 tc_fence_after();
-                bool first = true;
-                for (int ks = 0; ks < n_stages && ok; ++ks) {
-                    const unsigned live = sm->live_mma[ks];
-                    if (!live) continue;
-                    // `ready` was probed while the previous stage's MMAs were being issued
-                    if (!ready && !mbar_wait(smem_u32(&sm->full[stage]), phase, abort)) { ok = false; break; }
-                    tc_fence_after();
-                    const unsigned long long adesc = make_desc(smem_u32(sA + stage * A_BYTES));
-                    const unsigned long long bdesc = make_desc(smem_u32(sB + stage * B_BYTES));
-                    const int nstage = (stage + 1 == STAGES) ? 0 : stage + 1;
-                    const unsigned nphase = (stage + 1 == STAGES) ? (phase ^ 1u) : phase;
+                const unsigned long long adesc = make_desc(smem_u32(sA + stage * A_BYTES));
+                const unsigned long long bdesc = make_desc(smem_u32(sB + stage * B_BYTES));
+                const int nstage = (stage + 1 == STAGES) ? 0 : stage + 1;
+                const unsigned nphase = (stage + 1 == STAGES) ? (phase ^ 1u) : phase;
+                ready = __all_sync(0xffffffffu, mbar_test(smem_u32(&sm->full[nstage]), nphase));
+                if (elect_one()) {
 #pragma unroll
                     for (int k4 = 0; k4 < 4; ++k4) {
                         if ((live >> k4) & 1u) {
@@ -187,20 +198,22 @@ mwu_gemm_kernel(const __grid_constant__ CUtensorMap tmap, const Params p) {
                                           adesc + (unsigned long long)(h * (AH_BYTES >> 4) + k4 * 2),
                                           bdesc + (unsigned long long)(k4 * 2), idesc, first ? 0u : 1u);
                             first = false;
-                            issued_any = true;
                         }
                     }
                     umma_commit(smem_u32(&sm->empty[stage]));
-                    ready = mbar_test(smem_u32(&sm->full[nstage]), nphase);
-                    stage = nstage;
-                    phase = nphase;
                 }
-                if (ok) {
-                    if (!first) umma_commit(smem_u32(&sm->tfull));
-                    else mbar_arrive(smem_u32(&sm->tfull));
-                }
+                first = false;
+                issued_any = true;
+                __syncwarp();
+                stage = nstage;
+                phase = nphase;
             }
-            ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+            if (!ok) break;
+            if (elect_one()) {
+                if (!first) umma_commit(smem_u32(&sm->tfull));
+                else mbar_arrive(smem_u32(&sm->tfull));
+            }
+            __syncwarp();
         }
         // everything this thread issued must have retired before tensor memory is freed
         if (lane == 0 && issued_any) {
@@ -541,9 +554,48 @@ static void fill_common(Params &p, const mwu_proj_desc *desc, const void *packed
 }  // namespace gemm
 }  // namespace mwu
 
-extern "C" int mwu_gemm(const mwu_proj_desc *desc, const void *packed, const void *X, int64_t M,
-                        int64_t ldx, void *Y, int64_t ldy, int32_t y_dtype, uint32_t *dev_status,
-                        void *cuda_stream) {
+// Activation rows from which expanding the weights once per call beats decoding them again for
+// every 512-row activation tile.
+static const int64_t kDecodeOnceMinRows = 1024;
+
+static bool encode_bf16_2d(mwu::gemm::EncodeTiledFn encode, CUtensorMap *tmap, const void *ptr, int64_t inner,
+                           int64_t outer, int64_t ld, int box_rows) {
+    const cuuint64_t gdim[2] = {(cuuint64_t)inner, (cuuint64_t)outer};
+    const cuuint64_t gstride[1] = {(cuuint64_t)ld * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)mwu::gemm::BK, (cuuint32_t)box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    return encode(tmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(ptr), gdim, gstride, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+extern "C" size_t mwu_gemm_workspace_bytes(const mwu_proj_desc *desc, int64_t M) {
+    if (mwu::validate_desc(desc, true) != MWU_OK || M < kDecodeOnceMinRows) return 0;
+    const mwu::PackedLayout L = mwu::packed_layout(desc);
+    return (size_t)L.n_pad * (size_t)desc->cols * 2;
+}
+
+extern "C" int mwu_decode(const mwu_proj_desc *desc, const void *packed, void *Wd, int64_t ldw,
+                          uint32_t *dev_status, void *cuda_stream) {
+    using namespace mwu;
+    using namespace mwu::gemm;
+    int rc = validate_desc(desc, true);
+    if (rc != MWU_OK) return rc;
+    if (!packed || !Wd || !dev_status) return MWU_ERR_INVALID_ARG;
+    if (ldw < desc->cols) return MWU_ERR_SHAPE;
+    if (!aligned_to(packed, 256) || !aligned_to(Wd, 16) || ldw % 8 != 0 || !aligned_to(dev_status, 4))
+        return MWU_ERR_ALIGNMENT;
+    rc = check_device(nullptr);
+    if (rc != MWU_OK) return rc;
+    Params p = {};
+    fill_common(p, desc, packed, nullptr, 0, dev_status);
+    return launch_decode(desc->block, p, (__nv_bfloat16 *)Wd, ldw, (cudaStream_t)cuda_stream) == cudaSuccess
+               ? MWU_OK : MWU_ERR_CUDA;
+}
+
+extern "C" int mwu_gemm_ws(const mwu_proj_desc *desc, const void *packed, const void *X, int64_t M,
+                           int64_t ldx, void *Y, int64_t ldy, int32_t y_dtype, void *workspace,
+                           size_t workspace_bytes, uint32_t *dev_status, void *cuda_stream) {
     using namespace mwu;
     using namespace mwu::gemm;
     int rc = validate_desc(desc, true);
@@ -555,36 +607,44 @@ extern "C" int mwu_gemm(const mwu_proj_desc *desc, const void *packed, const voi
     if (!aligned_to(packed, 256) || !aligned_to(X, 16) || !aligned_to(Y, 16) || ldx % 8 != 0 ||
         ldy % (y_dtype ? 4 : 8) != 0 || !aligned_to(dev_status, 4))
         return MWU_ERR_ALIGNMENT;
+    if (workspace && !aligned_to(workspace, 256)) return MWU_ERR_ALIGNMENT;
     if (M == 0) return MWU_OK;
     int sm_count = 0;
     rc = check_device(&sm_count);
     if (rc != MWU_OK) return rc;
     EncodeTiledFn encode = get_encode_fn();
     if (!encode) return MWU_ERR_CUDA;
-
-    // tiles of 256 activation rows unless the problem has no second half to fill
-    const int mt = (M > BMH) ? 2 : 1;
-    const int bm = mt * BMH;
-    CUtensorMap tmap;
-    const cuuint64_t gdim[2] = {(cuuint64_t)desc->cols, (cuuint64_t)M};
-    const cuuint64_t gstride[1] = {(cuuint64_t)ldx * 2};
-    const cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)bm};
-    const cuuint32_t estr[2] = {1, 1};
-    if (encode(&tmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(X), gdim, gstride, box, estr,
-               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-        return MWU_ERR_CUDA;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
 
     Params p = {};
     fill_common(p, desc, packed, Y, y_dtype, dev_status);
     p.M = M;
     p.ldy = ldy;
+    if (p.n_stages > MAX_STAGES_K) return MWU_ERR_SHAPE;
+
+    // decode once into the caller's workspace, then a two-operand GEMM over it
+    const size_t need = mwu_gemm_workspace_bytes(desc, M);
+    if (workspace && need && workspace_bytes >= need) {
+        const int64_t n_pad = p.n_rec_tiles * kTileRows;
+        CUtensorMap tmap_x, tmap_w;
+        if (!encode_bf16_2d(encode, &tmap_x, X, desc->cols, M, ldx, BMH) ||
+            !encode_bf16_2d(encode, &tmap_w, workspace, desc->cols, n_pad, desc->cols, kTileRows))
+            return MWU_ERR_CUDA;
+        if (launch_decode(desc->block, p, (__nv_bfloat16 *)workspace, desc->cols, st) != cudaSuccess)
+            return MWU_ERR_CUDA;
+        return launch_dense(tmap_x, tmap_w, p, sm_count, st) == cudaSuccess ? MWU_OK : MWU_ERR_CUDA;
+    }
+
+    // tiles of 256 activation rows unless the problem has no second half to fill
+    const int mt = (M > BMH) ? 2 : 1;
+    const int bm = mt * BMH;
+    CUtensorMap tmap;
+    if (!encode_bf16_2d(encode, &tmap, X, desc->cols, M, ldx, bm)) return MWU_ERR_CUDA;
     const int nrec = p.n_rec_tiles >= 2 ? 2 : 1;
     const long long tiles = ((M + bm - 1) / bm) * ((p.n_rec_tiles + nrec - 1) / nrec);
     const int grid = (int)(tiles < sm_count ? tiles : sm_count);
     size_t smem = smem_bytes(nrec, mt, p.n_stages, 0);
-    if (p.n_stages > MAX_STAGES_K || smem > 227 * 1024) return MWU_ERR_SHAPE;
-    cudaStream_t st = (cudaStream_t)cuda_stream;
+    if (smem > 227 * 1024) return MWU_ERR_SHAPE;
     cudaError_t e;
     // bf16 rows are 16-byte aligned (checked above), which the staged epilogue stores need
     if (!y_dtype && smem + NEPI_WARPS * 2048 <= 227 * 1024) {
@@ -598,6 +658,12 @@ extern "C" int mwu_gemm(const mwu_proj_desc *desc, const void *packed, const voi
     else e = (nrec == 2) ? launch_bw<0, 2, 1>(desc->block, tmap, p, grid, smem, st)
                          : launch_bw<0, 1, 1>(desc->block, tmap, p, grid, smem, st);
     return e == cudaSuccess ? MWU_OK : MWU_ERR_CUDA;
+}
+
+extern "C" int mwu_gemm(const mwu_proj_desc *desc, const void *packed, const void *X, int64_t M,
+                        int64_t ldx, void *Y, int64_t ldy, int32_t y_dtype, uint32_t *dev_status,
+                        void *cuda_stream) {
+    return mwu_gemm_ws(desc, packed, X, M, ldx, Y, ldy, y_dtype, nullptr, 0, dev_status, cuda_stream);
 }
 
 extern "C" int mwu_conv_implicit(const mwu_proj_desc *desc, const void *packed, const void *X_nchw,

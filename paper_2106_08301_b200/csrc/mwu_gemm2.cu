@@ -39,51 +39,6 @@ struct PairSmem {
     int n_live[P_GROUPS];
 };
 
-__device__ __forceinline__ unsigned cluster_rank() {
-    unsigned r;
-    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
-    return r;
-}
-__device__ __forceinline__ void cluster_sync_all() {
-    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
-    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-// arrive on the barrier at the same shared-memory offset in CTA `cta` of the cluster
-__device__ __forceinline__ void mbar_arrive_cluster(unsigned local_bar, unsigned cta) {
-    unsigned remote;
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_bar), "r"(cta));
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(remote) : "memory");
-}
-__device__ __forceinline__ void tmem_alloc2(unsigned dst_smem, unsigned ncols) {
-    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void tmem_dealloc2(unsigned taddr, unsigned ncols) {
-    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
-}
-__device__ __forceinline__ void umma2_bf16(unsigned d_tmem, unsigned long long adesc, unsigned long long bdesc,
-                                           unsigned idesc, unsigned accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
-}
-// completion of all MMAs issued so far arrives on the barrier at this offset in both CTAs
-__device__ __forceinline__ void umma2_commit_both(unsigned bar) {
-    asm volatile(
-        "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
-        ::"r"(bar), "h"((unsigned short)3) : "memory");
-}
-// ... on the issuing CTA's barrier only
-__device__ __forceinline__ void umma2_commit_local(unsigned bar) {
-    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-// bf16 x bf16 -> fp32, both operands K-major, M = 256 over the CTA pair
-__device__ __forceinline__ unsigned make_idesc_pair(int n) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((unsigned)(n >> 3) << 17) | ((unsigned)(256 >> 4) << 24);
-}
-
 __device__ __forceinline__ void pair_group_bar(int group) {
     asm volatile("bar.sync %0, %1;" ::"r"(1 + group), "r"(P_DEC_THREADS) : "memory");
 }
@@ -183,22 +138,29 @@ mwu_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap, const Params p) {
         bool ok = true, issued_any = false, ready = false;
         const unsigned idesc = make_idesc_pair(256);
         long long mt = 0, nt = 0;
+        // All 32 lanes run the loop and one elected lane issues the MMAs and commits: in a
+        // lane-0 branch the issue of one tcgen05.mma took about 100 cycles.
         for (long long kt = 0; ok && tile_of(kt, mt, nt); ++kt) {
             load_live(sm->live_mma, nt);
-            if (lane == 0) {
-                if (!mbar_wait(smem_u32(&sm->tempty), acc_phase ^ 1u, abort)) ok = false;
-                acc_phase ^= 1u;
+            if (!mbar_wait(smem_u32(&sm->tempty), acc_phase ^ 1u, abort)) ok = false;
+            if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
+            acc_phase ^= 1u;
+            tc_fence_after();
+            bool first = true;
+            for (int ks = 0; ks < n_stages; ++ks) {
+                const unsigned live = sm->live_mma[ks];
+                if (!live) continue;
+                if (!ready) {
+                    if (!mbar_wait_spin(smem_u32(&sm->full[stage]), phase, abort)) ok = false;
+                    if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
+                }
                 tc_fence_after();
-                bool first = true;
-                for (int ks = 0; ks < n_stages && ok; ++ks) {
-                    const unsigned live = sm->live_mma[ks];
-                    if (!live) continue;
-                    if (!ready && !mbar_wait(smem_u32(&sm->full[stage]), phase, abort)) { ok = false; break; }
-                    tc_fence_after();
-                    const unsigned long long adesc = make_desc(smem_u32(sA + stage * P_A_BYTES));
-                    const unsigned long long bdesc = make_desc(smem_u32(sB + stage * P_B_BYTES));
-                    const int nstage = (stage + 1 == P_STAGES) ? 0 : stage + 1;
-                    const unsigned nphase = (stage + 1 == P_STAGES) ? (phase ^ 1u) : phase;
+                const unsigned long long adesc = make_desc(smem_u32(sA + stage * P_A_BYTES));
+                const unsigned long long bdesc = make_desc(smem_u32(sB + stage * P_B_BYTES));
+                const int nstage = (stage + 1 == P_STAGES) ? 0 : stage + 1;
+                const unsigned nphase = (stage + 1 == P_STAGES) ? (phase ^ 1u) : phase;
+                ready = __all_sync(0xffffffffu, mbar_test(smem_u32(&sm->full[nstage]), nphase));
+                if (elect_one()) {
 #pragma unroll
                     for (int k4 = 0; k4 < 4; ++k4) {
                         if ((live >> k4) & 1u) {
@@ -208,24 +170,26 @@ mwu_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap, const Params p) {
                                            adesc + (unsigned long long)(h * (AH_BYTES >> 4) + k4 * 2),
                                            bdesc + (unsigned long long)(k4 * 2), idesc, first ? 0u : 1u);
                             first = false;
-                            issued_any = true;
                         }
                     }
                     umma2_commit_both(smem_u32(&sm->empty[stage]));
-                    ready = mbar_test(smem_u32(&sm->full[nstage]), nphase);
-                    stage = nstage;
-                    phase = nphase;
                 }
-                if (ok) {
-                    if (!first) {
-                        umma2_commit_both(smem_u32(&sm->tfull));
-                    } else {
-                        mbar_arrive(smem_u32(&sm->tfull));
-                        mbar_arrive_cluster(smem_u32(&sm->tfull), 1);
-                    }
+                first = false;
+                issued_any = true;
+                __syncwarp();
+                stage = nstage;
+                phase = nphase;
+            }
+            if (!ok) break;
+            if (elect_one()) {
+                if (!first) {
+                    umma2_commit_both(smem_u32(&sm->tfull));
+                } else {
+                    mbar_arrive(smem_u32(&sm->tfull));
+                    mbar_arrive_cluster(smem_u32(&sm->tfull), 1);
                 }
             }
-            ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+            __syncwarp();
         }
         if (lane == 0 && issued_any) {
             umma2_commit_local(smem_u32(&sm->drain));

@@ -98,6 +98,14 @@ __device__ __forceinline__ bool mbar_wait(unsigned bar, unsigned parity, volatil
         if (clock64() - t0 > WAIT_LIMIT_CYCLES) { *abort = 1; return false; }
     }
 }
+// the same for a single latency-critical thread: probe in a tight loop first (a suspended try_wait
+// wakes up a few hundred cycles late), then fall back to the bounded wait
+__device__ __forceinline__ bool mbar_wait_spin(unsigned bar, unsigned parity, volatile int *abort) {
+#pragma unroll 1
+    for (int i = 0; i < 2048; ++i)
+        if (mbar_test(bar, parity)) return true;
+    return mbar_wait(bar, parity, abort);
+}
 template <int BYTES>
 __device__ __forceinline__ void cp_async_if(unsigned dst, const void *src, unsigned pred) {
     asm volatile(
@@ -105,6 +113,12 @@ __device__ __forceinline__ void cp_async_if(unsigned dst, const void *src, unsig
         "setp.ne.u32 p, %2, 0;\n\t"
         "@p cp.async.ca.shared.global [%0], [%1], %3;\n\t}"
         ::"r"(dst), "l"(src), "r"(pred), "n"(BYTES) : "memory");
+}
+// true in exactly one lane of a converged warp
+__device__ __forceinline__ bool elect_one() {
+    unsigned pred;
+    asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(pred));
+    return pred != 0;
 }
 __device__ __forceinline__ void fence_proxy_async() {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -135,6 +149,68 @@ __device__ __forceinline__ void umma_bf16(unsigned d_tmem, unsigned long long ad
 __device__ __forceinline__ void umma_commit(unsigned bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
+// ---- CTA pairs (clusters of two, tcgen05 cta_group::2) ----
+__device__ __forceinline__ unsigned cluster_rank() {
+    unsigned r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// arrive on the barrier at the same shared-memory offset in CTA `cta` of the cluster
+__device__ __forceinline__ void mbar_arrive_cluster(unsigned local_bar, unsigned cta) {
+    unsigned remote;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_bar), "r"(cta));
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(remote) : "memory");
+}
+// address of the barrier at the same shared-memory offset in CTA `cta` of the cluster
+__device__ __forceinline__ unsigned mbar_addr_in_cta(unsigned local_bar, unsigned cta) {
+    unsigned remote;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_bar), "r"(cta));
+    return remote;
+}
+// TMA load of a CTA pair: the data lands in this CTA's shared memory, the bytes are reported to a
+// barrier that may live in either CTA of the pair (`bar_cluster` is a shared::cluster address).
+// No multicast: each CTA fetches its own box.
+__device__ __forceinline__ void tma_load_2d_pair(unsigned dst, const CUtensorMap *map, unsigned bar_cluster,
+                                                 int x, int y) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.cta_group::2 "
+        "[%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar_cluster), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void tmem_alloc2(unsigned dst_smem, unsigned ncols) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc2(unsigned taddr, unsigned ncols) {
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void umma2_bf16(unsigned d_tmem, unsigned long long adesc, unsigned long long bdesc,
+                                           unsigned idesc, unsigned accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// completion of all MMAs issued so far arrives on the barrier at this offset in both CTAs
+__device__ __forceinline__ void umma2_commit_both(unsigned bar) {
+    asm volatile(
+        "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+        ::"r"(bar), "h"((unsigned short)3) : "memory");
+}
+// ... on the issuing CTA's barrier only
+__device__ __forceinline__ void umma2_commit_local(unsigned bar) {
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// bf16 x bf16 -> fp32, both operands K-major, M = 256 over the CTA pair
+__device__ __forceinline__ unsigned make_idesc_pair(int n) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((unsigned)(n >> 3) << 17) | ((unsigned)(256 >> 4) << 24);
+}
+
 // issue a 32-lane x 32-column load from tensor memory; the registers are valid after tmem_ld_wait
 __device__ __forceinline__ void tmem_ld32_issue(unsigned taddr, unsigned (&r)[32]) {
     asm volatile(

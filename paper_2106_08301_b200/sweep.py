@@ -5,7 +5,7 @@ events on the launching stream, L2 is flushed between repetitions (a 256 MB buff
 and the dense bf16 library routine (torch.matmul / conv2d on the decoded weights) is timed beside
 them.  Roofline time = max(surviving-block FLOPs / tensor peak, algorithmic bytes / HBM peak).
 
-  python -m paper_2106_08301_b200.sweep [--set main|blocks|projection|all] [--reps 10]
+  python -m paper_2106_08301_b200.sweep [--set main|blocks|projection|all] [--reps 10] [--m M] [--fused]
 """
 from __future__ import annotations
 
@@ -57,7 +57,7 @@ def packed_algorithmic_bytes(wl, ku, kp):
     return (2 * kp + n_u * (32 + wl.block + 2) + n_d * (16 * wl.block + 2)) / 8.0
 
 
-def run_workload(wl, timer, reps, m_override=None):
+def run_workload(wl, timer, reps, m_override=None, fused=False):
     hbm, tf, src = peaks()
     ku = B.mwu_count_from_permille(wl.n_blocks, wl.unified_permille)
     kp = B.mwu_count_from_permille(wl.n_blocks, wl.pruned_permille)
@@ -96,9 +96,12 @@ def run_workload(wl, timer, reps, m_override=None):
         m = m_override or wl.m
         X = wl.activations(m=m).cuda()
         Y = torch.empty((m, wl.rows), dtype=torch.bfloat16, device="cuda")
+        ws_bytes = 0 if fused else B.mwu_gemm_workspace_bytes(desc, m)
+        ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda") if ws_bytes else None
+        res["gemm_path"] = "decode once" if ws_bytes else "fused decode"
 
         def call():
-            B.mwu_gemm(desc, packed, X, m, wl.cols, Y, wl.rows, 0, bufs.dev_status)
+            B.mwu_gemm_ws(desc, packed, X, m, wl.cols, Y, wl.rows, 0, ws, bufs.dev_status)
 
         def lib():
             torch.matmul(X, Wd.T)
@@ -147,16 +150,20 @@ def main():
     ap.add_argument("--set", default="main", choices=["main", "blocks", "projection", "all"])
     ap.add_argument("--reps", type=int, default=10)
     ap.add_argument("--only", default="", help="run just this workload of the main set")
+    ap.add_argument("--m", type=int, default=0, help="override the activation rows of linear workloads")
+    ap.add_argument("--fused", action="store_true", help="never use the decode-once workspace path")
     args = ap.parse_args()
     B.lib()
     timer = Timer()
     if args.set in ("main", "all"):
         for name in ([args.only] if args.only else ["c1_linear", "c2_conv3x3", "c3_conv1x1", "c4_ffn"]):
-            print(json.dumps(run_workload(inputs.WORKLOADS[name], timer, args.reps)), flush=True)
+            print(json.dumps(run_workload(inputs.WORKLOADS[name], timer, args.reps, args.m or None, args.fused)),
+                  flush=True)
     if args.set in ("blocks", "all"):
         for b in (2, 4, 8, 16):
             for pr in (0, 250, 500, 750, 900):
-                print(json.dumps(run_workload(inputs.sweep_workload(b, pr), timer, args.reps)), flush=True)
+                print(json.dumps(run_workload(inputs.sweep_workload(b, pr), timer, args.reps, None, args.fused)),
+                      flush=True)
     if args.set in ("projection", "all"):
         for lg in (20, 22, 24, 26, 28):
             for b in (4, 16):
