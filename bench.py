@@ -344,7 +344,11 @@ def run_gpu(args):
             "bound": "tensor", "achieved": ach, "peak": peak_tf,
             "unit": "TFLOP/s", "frac": ach / peak_tf,
             "peak_source": peaks["source"] + " (sustained cuBLAS bf16)",
-            "algorithmic_flops_per_launch": flops, "traffic": None,
+            "algorithmic_flops_per_launch": flops,
+            # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the two-operand GEMM kernel
+            # (615.2 MB + 252.9 MB, ncu capture of this workload; see profiles/step_kernels_c4_ffn.md);
+            # not taken for other workloads or for the fused path
+            "traffic": 868.1e6 if (ws_bytes and wl.name == "c4_ffn" and m == wl.m) else None,
             "projection": {"bound": "hbm", "achieved": abytes["projection"] / (proj_ms * 1e-3) / 1e9,
                            "peak": peaks["hbm_gbs"], "unit": "GB/s",
                            "frac": abytes["projection"] / (proj_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]},
