@@ -30,8 +30,8 @@ from paper_2106_08301_b200 import inputs, replicas  # noqa: E402
 
 METRIC = "mwu_hot_path_effective_tflops"
 UNIT = "TFLOP/s"
-KERNELS_PER_STEP = 11     # sample, stats, bin, collect x2, histu, emit | count, scan, fill | gemm
-KERNELS_PER_STEP_WS = 12  # ... | decode, dense gemm (with a workspace and enough activation rows)
+KERNELS_PER_STEP = 9      # sample, stats, prune_select, collect, emit | count, scan, fill | gemm
+KERNELS_PER_STEP_WS = 10  # ... | decode, dense gemm (with a workspace and enough activation rows)
 
 
 def measured_peaks():

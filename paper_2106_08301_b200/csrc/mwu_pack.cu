@@ -107,7 +107,7 @@ __global__ void __launch_bounds__(128) count_kernel(Params p) {
 __global__ void __launch_bounds__(1024) scan_kernel(Params p) {
     const long long n_rec = p.L.n_tiles * p.L.n_stages;
     uint4 *recs = reinterpret_cast<uint4 *>(p.packed + p.L.off_rec);     // ubase, dbase, pbase, live
-    __shared__ unsigned long long s_u[1024], s_d[1024], s_p[1024];
+    __shared__ unsigned long long s_u[64], s_d[64], s_p[64];
     const long long per = (n_rec + 1023) / 1024;
     const long long lo = threadIdx.x * per;
     const long long hi = (lo + per < n_rec) ? lo + per : n_rec;
@@ -121,18 +121,32 @@ __global__ void __launch_bounds__(1024) scan_kernel(Params p) {
         su += held[k].x; sd += held[k].y; sp += held[k].z;
     }
     for (long long i = lo + KEEP; i < hi; ++i) { const uint4 v = recs[i]; su += v.x; sd += v.y; sp += v.z; }
-    s_u[threadIdx.x] = su; s_d[threadIdx.x] = sd; s_p[threadIdx.x] = sp;
-    __syncthreads();
-    for (int off = 1; off < 1024; off <<= 1) {
-        unsigned long long au = 0, ad = 0, ap = 0;
-        if ((int)threadIdx.x >= off) {
-            au = s_u[threadIdx.x - off]; ad = s_d[threadIdx.x - off]; ap = s_p[threadIdx.x - off];
-        }
-        __syncthreads();
-        s_u[threadIdx.x] += au; s_d[threadIdx.x] += ad; s_p[threadIdx.x] += ap;
-        __syncthreads();
+    // inclusive scan over the 1024 threads: shuffles inside a warp, then the 32 warp totals
+    unsigned long long iu = su, id = sd, ip = sp;
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const unsigned long long au = __shfl_up_sync(0xffffffffu, iu, off);
+        const unsigned long long ad = __shfl_up_sync(0xffffffffu, id, off);
+        const unsigned long long ap = __shfl_up_sync(0xffffffffu, ip, off);
+        if (lane >= off) { iu += au; id += ad; ip += ap; }
     }
-    unsigned long long ru = s_u[threadIdx.x] - su, rd = s_d[threadIdx.x] - sd, rp = s_p[threadIdx.x] - sp;
+    if (lane == 31) { s_u[wid] = iu; s_d[wid] = id; s_p[wid] = ip; }
+    __syncthreads();
+    if (wid == 0) {
+        unsigned long long wu = s_u[lane], wd = s_d[lane], wp = s_p[lane];
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const unsigned long long au = __shfl_up_sync(0xffffffffu, wu, off);
+            const unsigned long long ad = __shfl_up_sync(0xffffffffu, wd, off);
+            const unsigned long long ap = __shfl_up_sync(0xffffffffu, wp, off);
+            if (lane >= off) { wu += au; wd += ad; wp += ap; }
+        }
+        s_u[32 + lane] = wu; s_d[32 + lane] = wd; s_p[32 + lane] = wp;     // inclusive warp totals
+    }
+    __syncthreads();
+    if (wid > 0) { iu += s_u[32 + wid - 1]; id += s_d[32 + wid - 1]; ip += s_p[32 + wid - 1]; }
+    unsigned long long ru = iu - su, rd = id - sd, rp = ip - sp;
 #pragma unroll
     for (int k = 0; k < KEEP; ++k) {
         if (lo + k < hi) {
@@ -146,7 +160,7 @@ __global__ void __launch_bounds__(1024) scan_kernel(Params p) {
         ru += v.x; rd += v.y; rp += v.z;
     }
     if (threadIdx.x == 1023) {
-        const unsigned long long tu = s_u[1023], td = s_d[1023], tp = s_p[1023];
+        const unsigned long long tu = iu, td = id, tp = ip;
         if (tu != (unsigned long long)p.L.n_unified || td != (unsigned long long)p.L.n_dense ||
             tp != (unsigned long long)p.L.n_plist)
             atomicOr(p.dev_status, (unsigned)MWU_DEV_BOUNDS);

@@ -7,14 +7,19 @@
 //   stats_kernel    streams W (+U) once; every thread owns 64 contiguous bytes (four 128-bit
 //                   loads in flight) and evaluates the fp64 keys of its blocks (Section 3.1:
 //                   q = mean|v|, L_u = sum(|v|-q)^2, L_p = sum v^2) with the fixed pairwise
-//                   tree; writes a 2x16-bit bin code per block and the prune-key histogram.
-//                   The last CTA to finish locates the bin of the k_prune-th key.
-//   collect_kernel  gathers the blocks of that bin (normally a few dozen) and the last CTA sorts
-//                   them: the result is the exact threshold element (key, block index).
-//   histu_kernel    histogram of L_u over the blocks that were not pruned; last CTA locates the
-//                   bin; then collect_kernel again for the unify threshold.
-//   emit_kernel     streams W again: classifies every block from its bin code (exact key only
-//                   for blocks in a threshold bin), writes Q, u, both bitmaps and the sign plane.
+//                   tree; writes a 2x16-bit bin code per block, the prune-key histogram, the
+//                   sign plane and q of every block (into u).
+//   prune_select_kernel  locates the bin of the k_prune-th key, then one pass over the bin codes:
+//                   blocks of that bin become candidates (normally a few dozen to a few hundred),
+//                   blocks above it are counted in the L_u histogram.  The last CTA sorts the
+//                   candidates: the result is the exact threshold element (key, block index); it
+//                   adds the surviving candidates to the L_u histogram and locates the bin of the
+//                   unify threshold.
+//   collect_kernel  gathers the blocks of that bin that were not pruned; the last CTA sorts them.
+//   emit_kernel     classifies every block from its bin code (exact key only for blocks in a
+//                   threshold bin), writes Q, both bitmaps and the final u (0 unless unified).  W
+//                   is read again only for the 64-byte units that hold a block keeping its values:
+//                   unified blocks are rebuilt from q and the sign plane, pruned ones are zeros.
 // When a threshold bin holds more than 2048 blocks (massive ties, e.g. re-projecting an already
 // projected tensor) the last CTA narrows the range of the 96-bit composite key (key, index) by
 // itself, pass by pass, until the candidates fit: slow but exact.
@@ -27,6 +32,7 @@ constexpr int NB_MAX = 65536;   // level-0 bins (codes fit 16 bits): bin 0 = bel
 constexpr int NB_SMALL = 8192;  // used up to 8M blocks: fewer bins to clear and scan
 constexpr int CAP = 2048;       // candidates sorted by the last step
 constexpr int NSAMP = 256;
+constexpr int PASS_LOADS = 4;      // 16-byte loads of bin codes a thread keeps in flight in the selection passes
 constexpr int FIN_THREADS = 1024;   // block size of the kernels whose last CTA finalises
 
 typedef unsigned long long u64;
@@ -48,7 +54,7 @@ struct Sel {
 struct Work {
     Sel sel[2];                 // 0: prune, 1: unify
     unsigned cand_count[2];
-    unsigned ticket[4];         // stats, collect<0>, histu, collect<1>
+    unsigned ticket[4];         // [1]: prune_select, [3]: collect<1>
     unsigned pad[2];
 };
 
@@ -376,7 +382,8 @@ __device__ __forceinline__ bool selected(const Params &p, const SelView &s, long
 // stats_kernel
 // ---------------------------------------------------------------------------------------------
 template <int B>
-__global__ void __launch_bounds__(256) stats_kernel(Params p, double *loss_u, double *loss_p) {
+__global__ void __launch_bounds__(256) stats_kernel(Params p, double *loss_u, double *loss_p, float *u_out,
+                                                    unsigned *sign_bits) {
     constexpr int NBT = 16 / B;                         // blocks per thread and step
     const Sel *sp = &p.work->sel[0];
     const Sel *su = &p.work->sel[1];
@@ -401,11 +408,22 @@ __global__ void __launch_bounds__(256) stats_kernel(Params p, double *loss_u, do
 #pragma unroll
         for (int l = 0; l < 16; ++l) ex = max(ex, __float_as_uint(v[l]) & 0x7fffffffu);
         nonfinite |= (ex >= 0x7f800000u) ? 1u : 0u;
+        // sign plane (final): bit l of this unit's half word = (v[l] < 0)
+        {
+            unsigned sb = 0;
+#pragma unroll
+            for (int l = 0; l < 16; ++l) sb |= (v[l] < 0.f ? 1u : 0u) << l;
+            unsigned short *halves = reinterpret_cast<unsigned short *>(sign_bits);
+            halves[unit] = (unsigned short)sb;
+            if (unit == n_units - 1 && (n_units & 1)) halves[unit + 1] = 0;
+        }
         unsigned code[NBT];
+        float qv[NBT];                                   // q = mean|v| of every block; emit keeps the unified ones
 #pragma unroll
         for (int e = 0; e < NBT; ++e) {
             double S, Lu, Kp;
             block_keys<B>(v + e * B, p.use_l1, &S, &Lu, &Kp);
+            qv[e] = __double2float_rn(__dmul_rn(S, 1.0 / (double)B));
             const long long j = unit * NBT + e;
             const unsigned bu = bin_of(key_bits(Lu), ulo, uhi, ush, nb);
             const unsigned bp = bin_of(key_bits(Kp), plo, phi, psh, nb);
@@ -420,18 +438,23 @@ __global__ void __launch_bounds__(256) stats_kernel(Params p, double *loss_u, do
         }
         const long long j0 = unit * NBT;
         if (j0 + NBT <= p.n_blocks) {
-            if (NBT == 1) p.bins[j0] = code[0];
-            else if (NBT == 2) *reinterpret_cast<uint2 *>(p.bins + j0) = make_uint2(code[0], code[1 % NBT]);
-            else {
+            if (NBT == 1) { p.bins[j0] = code[0]; u_out[j0] = qv[0]; }
+            else if (NBT == 2) {
+                *reinterpret_cast<uint2 *>(p.bins + j0) = make_uint2(code[0], code[1 % NBT]);
+                *reinterpret_cast<float2 *>(u_out + j0) = make_float2(qv[0], qv[1 % NBT]);
+            } else {
 #pragma unroll
-                for (int e = 0; e < NBT; e += 4)
+                for (int e = 0; e < NBT; e += 4) {
                     *reinterpret_cast<uint4 *>(p.bins + j0 + e) =
                         make_uint4(code[e % NBT], code[(e + 1) % NBT], code[(e + 2) % NBT], code[(e + 3) % NBT]);
+                    *reinterpret_cast<float4 *>(u_out + j0 + e) =
+                        make_float4(qv[e % NBT], qv[(e + 1) % NBT], qv[(e + 2) % NBT], qv[(e + 3) % NBT]);
+                }
             }
         } else {
 #pragma unroll
             for (int e = 0; e < NBT; ++e)
-                if (j0 + e < p.n_blocks) p.bins[j0 + e] = code[e];
+                if (j0 + e < p.n_blocks) { p.bins[j0 + e] = code[e]; u_out[j0 + e] = qv[e]; }
         }
     }
     // block-level totals of the two catch-all bins
@@ -454,17 +477,6 @@ __global__ void __launch_bounds__(256) stats_kernel(Params p, double *loss_u, do
     }
 }
 
-// one CTA: locate the threshold bin of a selection from its finished histogram
-template <int KIND>
-__global__ void __launch_bounds__(FIN_THREADS) bin_kernel(Params p) {
-    Sel *s = &p.work->sel[KIND];
-    if (ld_vol(&s->mode) != 0u) return;
-    select_bin(p, s, p.hist + (size_t)KIND * p.nb);
-}
-
-// ---------------------------------------------------------------------------------------------
-// histu_kernel: histogram of L_u bins over the blocks that were not pruned
-// ---------------------------------------------------------------------------------------------
 // four consecutive bin codes starting at j4 (j4 % 4 == 0); codes beyond n read as 0
 __device__ __forceinline__ void load_codes4(const unsigned *bins, long long j4, long long n, unsigned (&c)[4]) {
     if (j4 + 4 <= n) {
@@ -474,39 +486,6 @@ __device__ __forceinline__ void load_codes4(const unsigned *bins, long long j4, 
 #pragma unroll
         for (int e = 0; e < 4; ++e) c[e] = (j4 + e < n) ? __ldg(bins + j4 + e) : 0u;
     }
-}
-
-template <int B>
-__global__ void __launch_bounds__(FIN_THREADS) histu_kernel(Params p) {
-    Sel *s = &p.work->sel[1];
-    if (ld_vol(&s->mode) != 0u) return;
-    unsigned *hist = p.hist + p.nb;
-    const SelView pv = view_of(&p.work->sel[0]);
-    const long long stride = (long long)gridDim.x * blockDim.x;
-    unsigned under = 0, over = 0;
-    for (long long j4 = ((long long)blockIdx.x * blockDim.x + threadIdx.x) * 4; j4 < p.n_blocks; j4 += stride * 4) {
-        unsigned codes[4];
-        load_codes4(p.bins, j4, p.n_blocks, codes);
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            const long long j = j4 + e;
-            if (j >= p.n_blocks) break;
-            if (selected<B>(p, pv, j, codes[e] & 0xffffu, 0)) continue;
-            const unsigned bu = codes[e] >> 16;
-            if (bu == 0) ++under;
-            else if (bu == (unsigned)p.nb - 1u) ++over;
-            else atomicAdd(&hist[bu], 1u);
-        }
-    }
-    for (int m = 16; m > 0; m >>= 1) {
-        under += __shfl_xor_sync(0xffffffffu, under, m);
-        over += __shfl_xor_sync(0xffffffffu, over, m);
-    }
-    if ((threadIdx.x & 31) == 0) {
-        if (under) atomicAdd(&hist[0], under);
-        if (over) atomicAdd(&hist[p.nb - 1], over);
-    }
-    if (last_block_done(&p.work->ticket[2])) select_bin(p, s, hist);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -546,21 +525,26 @@ __global__ void __launch_bounds__(FIN_THREADS) collect_kernel(Params p) {
     if (!too_many) {
         const u128 lo = from_halves(ld_vol(&s->lo_hi), ld_vol(&s->lo_lo));
         const u128 hi = from_halves(ld_vol(&s->hi_hi), ld_vol(&s->hi_lo));
-        for (long long j4 = ((long long)blockIdx.x * blockDim.x + threadIdx.x) * 4; j4 < p.n_blocks; j4 += stride * 4) {
-            unsigned codes[4];
-            load_codes4(p.bins, j4, p.n_blocks, codes);
+        for (long long j0 = ((long long)blockIdx.x * blockDim.x + threadIdx.x) * 4; j0 < p.n_blocks;
+             j0 += stride * 4 * PASS_LOADS) {
+            unsigned codes[PASS_LOADS][4];
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const long long j = j4 + e;
-                const unsigned code = codes[e];
-                const unsigned bin = KIND ? (code >> 16) : (code & 0xffffu);
-                if (j >= p.n_blocks || bin != Bsel) continue;
-                if (KIND == 1 && selected<B>(p, pv, j, code & 0xffffu, 0)) continue;
-                const u64 key = exact_key<B>(p, j, KIND);
-                const u128 c = make_c(key, (u64)j);
-                if (c >= lo && c < hi) {
-                    const unsigned slot = atomicAdd(&p.work->cand_count[KIND], 1u);
-                    if (slot < (unsigned)CAP) { p.cand_key[slot] = key; p.cand_idx[slot] = (unsigned)j; }
+            for (int q = 0; q < PASS_LOADS; ++q) load_codes4(p.bins, j0 + q * stride * 4, p.n_blocks, codes[q]);
+#pragma unroll
+            for (int q = 0; q < PASS_LOADS; ++q) {
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const long long j = j0 + q * stride * 4 + e;
+                    const unsigned code = codes[q][e];
+                    const unsigned bin = KIND ? (code >> 16) : (code & 0xffffu);
+                    if (j >= p.n_blocks || bin != Bsel) continue;
+                    if (KIND == 1 && selected<B>(p, pv, j, code & 0xffffu, 0)) continue;
+                    const u64 key = exact_key<B>(p, j, KIND);
+                    const u128 c = make_c(key, (u64)j);
+                    if (c >= lo && c < hi) {
+                        const unsigned slot = atomicAdd(&p.work->cand_count[KIND], 1u);
+                        if (slot < (unsigned)CAP) { p.cand_key[slot] = key; p.cand_idx[slot] = (unsigned)j; }
+                    }
                 }
             }
         }
@@ -650,6 +634,175 @@ __global__ void __launch_bounds__(FIN_THREADS) collect_kernel(Params p) {
 }
 
 // ---------------------------------------------------------------------------------------------
+// prune_select_kernel: exact prune threshold and the L_u histogram of the survivors in one pass
+// ---------------------------------------------------------------------------------------------
+// Every CTA first locates the prune threshold bin from the finished histogram (all write the same
+// values).  The pass over the bin codes then needs no exact key outside that bin: blocks below it
+// are pruned, blocks above it survive and are counted in the L_u histogram, blocks inside it become
+// candidates.  The last CTA sorts the candidates, which fixes the threshold element, counts the
+// L_u bins of the candidates that survive, and locates the unify threshold bin.
+template <int B>
+__global__ void __launch_bounds__(FIN_THREADS) prune_select_kernel(Params p) {
+    Sel *sp = &p.work->sel[0];
+    Sel *su = &p.work->sel[1];
+    const unsigned mode_p = ld_vol(&sp->mode), mode_u = ld_vol(&su->mode);
+    if (mode_p != 0u && mode_u != 0u) return;
+    __shared__ u64 c_key[CAP];
+    __shared__ unsigned c_idx[CAP];
+    __shared__ unsigned s_bin, s_err, s_n;
+    __shared__ u64 s_r, s_cnt;
+    unsigned *hist_u = p.hist + p.nb;
+    if (mode_p == 0u) select_bin(p, sp, p.hist);
+    const unsigned Bp = ld_vol(&sp->B);
+    const bool too_many = mode_p == 0u && ld_vol(&sp->cnt) > (u64)CAP;
+    const u128 lo0 = from_halves(ld_vol(&sp->lo_hi), ld_vol(&sp->lo_lo));
+    const u128 hi0 = from_halves(ld_vol(&sp->hi_hi), ld_vol(&sp->hi_lo));
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    unsigned under = 0, over = 0;
+    if (mode_p != 2u) {                                   // mode 2: everything is pruned, nothing survives
+        // PASS_LOADS 16-byte loads are in flight per thread before their codes are looked at
+        for (long long j0 = ((long long)blockIdx.x * blockDim.x + threadIdx.x) * 4; j0 < p.n_blocks;
+             j0 += stride * 4 * PASS_LOADS) {
+            unsigned codes[PASS_LOADS][4];
+#pragma unroll
+            for (int q = 0; q < PASS_LOADS; ++q) load_codes4(p.bins, j0 + q * stride * 4, p.n_blocks, codes[q]);
+#pragma unroll
+            for (int q = 0; q < PASS_LOADS; ++q) {
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const long long j = j0 + q * stride * 4 + e;
+                    if (j >= p.n_blocks) break;
+                    const unsigned bp = codes[q][e] & 0xffffu, bu = codes[q][e] >> 16;
+                    if (mode_p == 0u) {
+                        if (bp < Bp) continue;                // pruned
+                        if (bp == Bp) {                       // decided by the last CTA
+                            if (!too_many) {
+                                const u64 key = exact_key<B>(p, j, 0);
+                                const u128 c = make_c(key, (u64)j);
+                                if (c >= lo0 && c < hi0) {
+                                    const unsigned slot = atomicAdd(&p.work->cand_count[0], 1u);
+                                    if (slot < (unsigned)CAP) { p.cand_key[slot] = key; p.cand_idx[slot] = (unsigned)j; }
+                                }
+                            }
+                            continue;
+                        }
+                    }
+                    if (mode_u != 0u) continue;
+                    if (bu == 0) ++under;
+                    else if (bu == (unsigned)p.nb - 1u) ++over;
+                    else atomicAdd(&hist_u[bu], 1u);
+                }
+            }
+        }
+    }
+    for (int m = 16; m > 0; m >>= 1) {
+        under += __shfl_xor_sync(0xffffffffu, under, m);
+        over += __shfl_xor_sync(0xffffffffu, over, m);
+    }
+    if ((threadIdx.x & 31) == 0) {
+        if (under) atomicAdd(&hist_u[0], under);
+        if (over) atomicAdd(&hist_u[p.nb - 1], over);
+    }
+    if (!last_block_done(&p.work->ticket[1])) return;
+
+    // ---- last CTA only ----
+    if (mode_p == 0u) {
+        if (too_many) {
+            // massive ties: narrow the composite range pass by pass with this CTA alone
+            unsigned *rhist = p.hist + (size_t)2 * p.nb;
+            for (int level = 0; level < 10; ++level) {
+                if (ld_vol(&sp->cnt) <= (u64)CAP) break;
+                for (int i = threadIdx.x; i < p.nb; i += blockDim.x) rhist[i] = 0;
+                __syncthreads();
+                const u128 lo = from_halves(ld_vol(&sp->lo_hi), ld_vol(&sp->lo_lo));
+                const u128 hi = from_halves(ld_vol(&sp->hi_hi), ld_vol(&sp->hi_lo));
+                unsigned shift = 0;
+                while (((hi - lo - 1) >> shift) >= (u128)p.nb) ++shift;
+                for (long long j = threadIdx.x; j < p.n_blocks; j += blockDim.x) {
+                    if ((ld_vol(p.bins + j) & 0xffffu) != Bp) continue;
+                    const u128 c = make_c(exact_key<B>(p, j, 0), (u64)j);
+                    if (c >= lo && c < hi) atomicAdd(&rhist[(unsigned)((c - lo) >> shift)], 1u);
+                }
+                __threadfence();
+                __syncthreads();
+                if (threadIdx.x == 0) s_err = 0;
+                __syncthreads();
+                scan_hist(rhist, p.nb, ld_vol(&sp->r), &s_bin, &s_r, &s_cnt, &s_err);
+                if (threadIdx.x == 0) {
+                    if (s_err) atomicOr(p.dev_status, (unsigned)MWU_DEV_SELECT);
+                    u128 nlo = lo + ((u128)s_bin << shift);
+                    u128 nhi = nlo + ((u128)1 << shift);
+                    if (nhi > hi) nhi = hi;
+                    sp->r = s_r;
+                    sp->cnt = s_cnt;
+                    sp->lo_hi = (u64)(nlo >> 64); sp->lo_lo = (u64)nlo;
+                    sp->hi_hi = (u64)(nhi >> 64); sp->hi_lo = (u64)nhi;
+                    __threadfence();
+                }
+                __syncthreads();
+            }
+            if (threadIdx.x == 0) s_n = 0;
+            __syncthreads();
+            const u128 lo = from_halves(ld_vol(&sp->lo_hi), ld_vol(&sp->lo_lo));
+            const u128 hi = from_halves(ld_vol(&sp->hi_hi), ld_vol(&sp->hi_lo));
+            for (long long j = threadIdx.x; j < p.n_blocks; j += blockDim.x) {
+                if ((ld_vol(p.bins + j) & 0xffffu) != Bp) continue;
+                const u64 key = exact_key<B>(p, j, 0);
+                const u128 c = make_c(key, (u64)j);
+                if (c >= lo && c < hi) {
+                    const unsigned slot = atomicAdd(&s_n, 1u);
+                    if (slot < (unsigned)CAP) { p.cand_key[slot] = key; p.cand_idx[slot] = (unsigned)j; }
+                }
+            }
+            __threadfence();
+            __syncthreads();
+            if (threadIdx.x == 0) p.work->cand_count[0] = s_n;
+            __syncthreads();
+        }
+        const unsigned n = ld_vol(&p.work->cand_count[0]);
+        const u64 r = ld_vol(&sp->r);
+        const unsigned m = n < (unsigned)CAP ? n : (unsigned)CAP;
+        for (int i = threadIdx.x; i < CAP; i += blockDim.x) {
+            c_key[i] = (i < (int)m) ? ld_vol(&p.cand_key[i]) : ~0ull;
+            c_idx[i] = (i < (int)m) ? ld_vol(&p.cand_idx[i]) : ~0u;
+        }
+        __syncthreads();
+        int np2 = 2;
+        while (np2 < (int)m) np2 <<= 1;
+        sort_candidates(c_key, c_idx, np2);
+        const bool bad = n > (unsigned)CAP || r == 0 || r > (u64)m;
+        if (threadIdx.x == 0) {
+            if (bad) {
+                atomicOr(p.dev_status, (unsigned)MWU_DEV_SELECT);
+                sp->T_key = 0; sp->T_idx = 0;
+            } else {
+                sp->T_key = c_key[r - 1];
+                sp->T_idx = (u64)c_idx[r - 1];
+            }
+            __threadfence();
+        }
+        __syncthreads();
+        // the blocks of the threshold bin that survive join the L_u histogram
+        if (mode_u == 0u && !bad) {
+            if (!too_many) {
+                for (unsigned i = (unsigned)r + threadIdx.x; i < m; i += blockDim.x)
+                    atomicAdd(&hist_u[ld_vol(p.bins + c_idx[i]) >> 16], 1u);
+            } else {
+                const SelView pv = view_of(sp);
+                for (long long j = threadIdx.x; j < p.n_blocks; j += blockDim.x) {
+                    const unsigned code = ld_vol(p.bins + j);
+                    if ((code & 0xffffu) != Bp) continue;
+                    if (!selected<B>(p, pv, j, Bp, 0)) atomicAdd(&hist_u[code >> 16], 1u);
+                }
+            }
+        }
+        __threadfence();
+        __syncthreads();
+    }
+    if (mode_u == 0u) select_bin(p, su, hist_u);
+}
+
+// ---------------------------------------------------------------------------------------------
 // emit_kernel
 // ---------------------------------------------------------------------------------------------
 template <int B>
@@ -663,19 +816,15 @@ __global__ void __launch_bounds__(256, 3) emit_kernel(Params p, float *Q, float 
     const int lane = threadIdx.x & 31;
     const long long n_units = (n + 15) / 16;
     const long long n_iter = (n_units + 31) / 32 * 32;      // whole warps take part in every step
-    const long long n_sign_words = (n + 31) / 32;
     const long long n_bm_words = (p.n_blocks + 31) / 32;
+    __shared__ float4 s_stage[8][128];                       // one warp step of Q per warp
+    float4 *ws = s_stage[threadIdx.x >> 5];
 
     for (long long unit = (long long)blockIdx.x * blockDim.x + threadIdx.x; unit < n_iter;
          unit += (long long)gridDim.x * blockDim.x) {
         const long long f = unit * 16;
-        float v[16];
+        const bool warp_full = (unit - lane + 32) * 16 <= n;      // all 512 floats of this warp step exist
         unsigned code[NBT];
-        if (unit < n_units) load16(p.W, p.U, f, n, v);
-        else {
-#pragma unroll
-            for (int l = 0; l < 16; ++l) v[l] = 0.f;
-        }
         const long long j0 = unit * NBT;
         if (j0 + NBT <= p.n_blocks) {
             if (NBT == 1) code[0] = __ldg(p.bins + j0);
@@ -691,45 +840,68 @@ __global__ void __launch_bounds__(256, 3) emit_kernel(Params p, float *Q, float 
 #pragma unroll
             for (int e = 0; e < NBT; ++e) code[e] = (j0 + e < p.n_blocks) ? __ldg(p.bins + j0 + e) : 0u;
         }
-        float q[16];
-        float uo[NBT];
         unsigned cls_p = 0, cls_u = 0;                       // bit e: block e of this thread
+        constexpr unsigned ALL = (1u << NBT) - 1u;
+        unsigned valid = 0;
 #pragma unroll
         for (int e = 0; e < NBT; ++e) {
             const long long j = j0 + e;
             bool pr = false, un = false;
             if (j < p.n_blocks) {
+                valid |= 1u << e;
                 pr = selected<B>(p, vp, j, code[e] & 0xffffu, 0);
                 un = !pr && selected<B>(p, vu, j, code[e] >> 16, 1);
             }
-            float qq = 0.f;
-            if (un) {
-                double a[B];
-#pragma unroll
-                for (int l = 0; l < B; ++l) a[l] = (double)fabsf(v[e * B + l]);
-                qq = __double2float_rn(__dmul_rn(tree_sum<B>(a), 1.0 / (double)B));
-            }
-#pragma unroll
-            for (int l = 0; l < B; ++l) {
-                const float x = v[e * B + l];
-                q[e * B + l] = pr ? 0.f : (un ? ((x >= 0.f) ? qq : -qq) : x);
-            }
-            uo[e] = qq;
             cls_p |= (pr ? 1u : 0u) << e;
             cls_u |= (un ? 1u : 0u) << e;
         }
+        // q of the unified blocks and the sign plane come from stats_kernel; W is read again
+        // only where a block keeps its own values
+        float uo[NBT];
+#pragma unroll
+        for (int e = 0; e < NBT; ++e) uo[e] = 0.f;
+        if (cls_u) {
+#pragma unroll
+            for (int e = 0; e < NBT; ++e)
+                if ((cls_u >> e) & 1u) uo[e] = u_out[j0 + e];
+        }
         if (unit < n_units) {
             if (Q) {
-                if (f + 16 <= n) {
-                    float4 *dst = reinterpret_cast<float4 *>(Q + f);
-                    dst[0] = make_float4(q[0], q[1], q[2], q[3]);
-                    dst[1] = make_float4(q[4], q[5], q[6], q[7]);
-                    dst[2] = make_float4(q[8], q[9], q[10], q[11]);
-                    dst[3] = make_float4(q[12], q[13], q[14], q[15]);
+                float v[16];
+                const bool need_v = ((~cls_p & ~cls_u) & valid & ALL) != 0u;
+                if (need_v) load16(p.W, p.U, f, n, v);
+                else {
+#pragma unroll
+                    for (int l = 0; l < 16; ++l) v[l] = 0.f;
+                }
+                unsigned sb = 0;
+                if (cls_u) sb = reinterpret_cast<const unsigned short *>(sign_bits)[unit];
+                float q[16];
+#pragma unroll
+                for (int e = 0; e < NBT; ++e) {
+                    const bool pr = (cls_p >> e) & 1u, un = (cls_u >> e) & 1u;
+#pragma unroll
+                    for (int l = 0; l < B; ++l) {
+                        const bool neg = (sb >> (e * B + l)) & 1u;
+                        q[e * B + l] = pr ? 0.f : (un ? (neg ? -uo[e] : uo[e]) : v[e * B + l]);
+                    }
+                }
+                if (!warp_full) {
+                    if (f + 16 <= n) {
+                        float4 *dst = reinterpret_cast<float4 *>(Q + f);
+                        dst[0] = make_float4(q[0], q[1], q[2], q[3]);
+                        dst[1] = make_float4(q[4], q[5], q[6], q[7]);
+                        dst[2] = make_float4(q[8], q[9], q[10], q[11]);
+                        dst[3] = make_float4(q[12], q[13], q[14], q[15]);
+                    } else {
+#pragma unroll
+                        for (int l = 0; l < 16; ++l)
+                            if (f + l < n) Q[f + l] = q[l];
+                    }
                 } else {
 #pragma unroll
-                    for (int l = 0; l < 16; ++l)
-                        if (f + l < n) Q[f + l] = q[l];
+                    for (int c = 0; c < 4; ++c)
+                        ws[lane * 4 + (c ^ ((lane >> 1) & 3))] = make_float4(q[4 * c], q[4 * c + 1], q[4 * c + 2], q[4 * c + 3]);
                 }
             }
             if (j0 + NBT <= p.n_blocks) {
@@ -747,14 +919,18 @@ __global__ void __launch_bounds__(256, 3) emit_kernel(Params p, float *Q, float 
                     if (j0 + e < p.n_blocks) u_out[j0 + e] = uo[e];
             }
         }
-        // sign plane: two neighbouring threads make one 32-bit word
-        {
-            unsigned sb = 0;
+        // Q of a whole warp step (2 KB): 16-byte stores at a 64-byte stride reach L2 as four partial
+        // writes per 64 bytes, so the step goes through shared memory and leaves as four stores of
+        // 512 contiguous bytes.  Thread t keeps piece c at slot c ^ ((t >> 1) & 3): no bank conflicts.
+        if (Q && warp_full) {
+            __syncwarp();
+            float4 *dst = reinterpret_cast<float4 *>(Q + (unit - lane) * 16);
 #pragma unroll
-            for (int l = 0; l < 16; ++l) sb |= (v[l] < 0.f ? 1u : 0u) << l;
-            const unsigned other = __shfl_xor_sync(0xffffffffu, sb, 1);
-            const long long wi = unit >> 1;
-            if ((lane & 1) == 0 && wi < n_sign_words) sign_bits[wi] = sb | (other << 16);
+            for (int k = 0; k < 4; ++k) {
+                const int t = 8 * k + (lane >> 2), c = lane & 3;
+                dst[k * 32 + lane] = ws[t * 4 + (c ^ ((t >> 1) & 3))];
+            }
+            __syncwarp();
         }
         // class bitmaps: the warp's 32 * NBT blocks make NBT words
         {
@@ -803,7 +979,7 @@ static cudaError_t launch_project(const mwu::proj::Params &p, const mwu_proj_des
     const long long want = (n_units + 255) / 256;
     const long long cap_blocks = (long long)sm_count * 8;
     const int grid_stream = (int)(want < cap_blocks ? (want > 0 ? want : 1) : cap_blocks);
-    stats_kernel<B><<<grid_stream, 256, 0, st>>>(p, loss_u, loss_p);
+    stats_kernel<B><<<grid_stream, 256, 0, st>>>(p, loss_u, loss_p, u, sb);
 
     const long long mb = p.n_blocks;
     const long long rb = (mb + 4 * FIN_THREADS - 1) / (4 * FIN_THREADS);
@@ -811,14 +987,8 @@ static cudaError_t launch_project(const mwu::proj::Params &p, const mwu_proj_des
     const bool need_p = desc->k_prune > 0 && desc->k_prune < mb;
     const long long ksel_u = desc->k_unify - desc->k_prune;
     const bool need_u = ksel_u > 0 && ksel_u < mb - desc->k_prune;
-    if (need_p) {
-        bin_kernel<0><<<1, FIN_THREADS, 0, st>>>(p);
-        collect_kernel<0, B><<<grid_fin, FIN_THREADS, 0, st>>>(p);
-    }
-    if (need_u) {
-        histu_kernel<B><<<grid_fin, FIN_THREADS, 0, st>>>(p);
-        collect_kernel<1, B><<<grid_fin, FIN_THREADS, 0, st>>>(p);
-    }
+    if (need_p || need_u) prune_select_kernel<B><<<grid_fin, FIN_THREADS, 0, st>>>(p);
+    if (need_u) collect_kernel<1, B><<<grid_fin, FIN_THREADS, 0, st>>>(p);
     emit_kernel<B><<<grid_stream, 256, 0, st>>>(p, Q, u, pb, ub, sb);
     return cudaGetLastError();
 }
