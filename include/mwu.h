@@ -54,12 +54,22 @@ typedef enum {
     MWU_PRUNE_KEY_L1 = 1    /* sum |v|: the norm Section 3.1's pruning example names          */
 } mwu_prune_key;
 
+/* How mwu_project organises its kernels.  Every choice gives the same bits. */
+typedef enum {
+    MWU_ALGO_AUTO = 0,       /* one pass from 32768 blocks on, multi pass below                */
+    MWU_ALGO_ONE_PASS = 1,   /* outputs written in one sweep over W with thresholds estimated
+                                from a sample, then the few blocks near a threshold corrected */
+    MWU_ALGO_MULTI_PASS = 2  /* statistics pass, exact thresholds, emit pass                  */
+} mwu_proj_algo;
+
 typedef struct {
     int64_t rows, cols;     /* W[rows][cols], row-major, cols % block == 0                    */
     int32_t block;          /* micro-block width along cols: 2, 4, 8 or 16                    */
     int32_t prune_key;      /* mwu_prune_key                                                  */
     int64_t k_unify;        /* number of blocks unified OR pruned (0 <= k_prune <= k_unify)   */
     int64_t k_prune;        /* number of blocks pruned to zero                                */
+    int32_t algo;           /* mwu_proj_algo; only mwu_project reads it                       */
+    int32_t reserved;       /* 0                                                              */
 } mwu_proj_desc;
 
 const char *mwu_status_string(int status);
@@ -110,7 +120,7 @@ int mwu_project(const mwu_proj_desc *desc, const float *W, const float *U_dual, 
  * For callers that cannot allocate device memory where they need the projection -- code running
  * inside an engine that owns the memory pool, or after a job's memory budget has been frozen,
  * where a cudaMalloc may fail or stall the device.  The scratch memory is a fixed array inside
- * the library's device image (about 5.2 MB, held by every GPU that loads the library until the
+ * the library's device image (about 8 MB, held by every GPU that loads the library until the
  * process exits), so the call allocates nothing.
  *
  * Limits and rules:

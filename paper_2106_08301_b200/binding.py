@@ -23,6 +23,7 @@ MWU_STATIC_MAX_BLOCKS = 1048576
 MWU_OK = 0
 MWU_DEV_NONFINITE, MWU_DEV_TIMEOUT, MWU_DEV_BOUNDS, MWU_DEV_SELECT = 1, 2, 4, 8
 MWU_PRUNE_KEY_L2SQ, MWU_PRUNE_KEY_L1 = 0, 1
+MWU_ALGO_AUTO, MWU_ALGO_ONE_PASS, MWU_ALGO_MULTI_PASS = 0, 1, 2
 
 
 class MwuError(RuntimeError):
@@ -34,7 +35,7 @@ class MwuError(RuntimeError):
 class ProjDesc(ctypes.Structure):
     _fields_ = [("rows", ctypes.c_int64), ("cols", ctypes.c_int64), ("block", ctypes.c_int32),
                 ("prune_key", ctypes.c_int32), ("k_unify", ctypes.c_int64),
-                ("k_prune", ctypes.c_int64)]
+                ("k_prune", ctypes.c_int64), ("algo", ctypes.c_int32), ("reserved", ctypes.c_int32)]
 
 
 _lib = None
@@ -94,8 +95,9 @@ def status_string(status: int) -> str:
 
 
 def make_desc(rows: int, cols: int, block: int, k_unify: int, k_prune: int,
-              prune_key: int = MWU_PRUNE_KEY_L2SQ) -> ProjDesc:
-    return ProjDesc(int(rows), int(cols), int(block), int(prune_key), int(k_unify), int(k_prune))
+              prune_key: int = MWU_PRUNE_KEY_L2SQ, algo: int = MWU_ALGO_AUTO) -> ProjDesc:
+    return ProjDesc(int(rows), int(cols), int(block), int(prune_key), int(k_unify), int(k_prune),
+                    int(algo), 0)
 
 
 def mwu_count_from_permille(n_blocks: int, permille: int) -> int:

@@ -55,6 +55,8 @@ inline int validate_desc(const mwu_proj_desc *d, bool need_stage_multiple) {
     if (need_stage_multiple && d->cols % kStageK != 0) return MWU_ERR_SHAPE;
     if (d->prune_key != MWU_PRUNE_KEY_L2SQ && d->prune_key != MWU_PRUNE_KEY_L1)
         return MWU_ERR_INVALID_ARG;
+    if (d->algo != MWU_ALGO_AUTO && d->algo != MWU_ALGO_ONE_PASS && d->algo != MWU_ALGO_MULTI_PASS)
+        return MWU_ERR_INVALID_ARG;
     const int64_t mb = d->rows * d->cols / d->block;
     if (mb >= (int64_t(1) << 31)) return MWU_ERR_SHAPE;
     if (d->k_prune < 0 || d->k_prune > d->k_unify || d->k_unify > mb) return MWU_ERR_SHAPE;

@@ -13,9 +13,11 @@
 
 namespace {
 
-// Enough for MWU_STATIC_MAX_BLOCKS blocks: 4 bytes of bin codes per block plus the fixed
-// selection state (histograms, candidate lists) of mwu_project, which is under 1 MiB.
-constexpr size_t kScratchBytes = (size_t)1024 * 1024 + 4 * ((size_t)MWU_STATIC_MAX_BLOCKS + 8) + 256;
+// Enough for MWU_STATIC_MAX_BLOCKS blocks: 4 bytes of bin codes per block, 8 bytes per entry of
+// the candidate list (a quarter of the blocks) and the fixed selection state (histograms, sort
+// buffers) of mwu_project, which is under 1.5 MiB.
+constexpr size_t kScratchBytes = (size_t)1536 * 1024 + 4 * ((size_t)MWU_STATIC_MAX_BLOCKS + 8) +
+                                 8 * ((size_t)MWU_STATIC_MAX_BLOCKS / 4 + 4096) + 1024;
 
 static __device__ __align__(256) unsigned char g_scratch[kScratchBytes];
 

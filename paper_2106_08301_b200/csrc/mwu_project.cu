@@ -1,9 +1,29 @@
 // mwu_project: Q = Unify(W + U), the Q-step of ADMM (Algorithm 1, Eq. 7) for 1-D micro-blocks.
 //
-// Pipeline (all on the caller's stream, no host synchronisation):
-//   sample_kernel   one CTA ranks <= 256 evenly spaced blocks and places a narrow window of
-//                   8190 bins (65534 above 8M blocks) around the k-th smallest key of each selection (prune key, L_u).
-//                   The window only steers efficiency; any window gives the same result.
+// Two pipelines give the same bits (all on the caller's stream, no host synchronisation).
+//
+// One-pass pipeline (MWU_ALGO_ONE_PASS; the default from ONE_PASS_MIN_BLOCKS blocks on):
+//   sample_kernel   one CTA sorts the keys of <= 4096 evenly spaced blocks; for each selection
+//                   (prune key, L_u of the survivors) it takes the sample quantile as a provisional
+//                   threshold and the sample keys 4 sigma of rank to either side as a window.
+//   pass_kernel     streams W (+U) once, evaluates the fp64 keys of every block (Section 3.1) and
+//                   writes every output -- Q, u, sign plane, bitmaps -- with the class the
+//                   provisional thresholds give.  A block whose key lies outside the window has
+//                   its final class (as long as the exact threshold lies inside, which the counts
+//                   prove afterwards); the few per cent inside go to a candidate list with their
+//                   bin codes and into the window histograms.
+//   list_select_kernel
+//                   exact prune threshold (key, block index) from the window histogram and the
+//                   list; the listed survivors complete the L_u histogram.
+//   list_finish_kernel
+//                   exact unify threshold; rewrites the outputs of the listed blocks whose
+//                   class changed.
+//   If a count shows that a threshold lies outside its window (or a tie group overflows the
+//   sort buffer, or the list overflows) a flag is set and the multi-pass kernels, which are
+//   always enqueued behind and otherwise return at once, redo the projection.
+//
+// Multi-pass pipeline (MWU_ALGO_MULTI_PASS; small tensors, and the fallback):
+//   sample_kernel   as above.  The window only steers efficiency; any window gives the same result.
 //   stats_kernel    streams W (+U) once; every thread owns 64 contiguous bytes (four 128-bit
 //                   loads in flight) and evaluates the fp64 keys of its blocks (Section 3.1:
 //                   q = mean|v|, L_u = sum(|v|-q)^2, L_p = sum v^2) with the fixed pairwise
@@ -31,9 +51,15 @@ namespace proj {
 constexpr int NB_MAX = 65536;   // level-0 bins (codes fit 16 bits): bin 0 = below the window, nb-1 = above it
 constexpr int NB_SMALL = 8192;  // used up to 8M blocks: fewer bins to clear and scan
 constexpr int CAP = 2048;       // candidates sorted by the last step
-constexpr int NSAMP = 256;
+constexpr int NSAMP = 4096;        // sample blocks ranked by sample_kernel
+constexpr int SAMP_THREADS = 1024;
+constexpr int SAMP_PER = NSAMP / SAMP_THREADS;
+static_assert(SAMP_PER == 4, "sample_select ranks one level-A key with the four threads that hold 16 samples");
+constexpr int STAGE_ENTRIES = 64;  // per-warp staging of candidate-list entries in pass_kernel
+constexpr long long ONE_PASS_MIN_BLOCKS = 32768;   // below: launch latency decides, multi-pass has fewer launches
 constexpr int PASS_LOADS = 4;      // 16-byte loads of bin codes a thread keeps in flight in the selection passes
 constexpr int FIN_THREADS = 1024;   // block size of the kernels whose last CTA finalises
+static_assert(NB_MAX / FIN_THREADS <= 64, "scan_hist searches one thread's bins with one warp, two per lane");
 
 typedef unsigned long long u64;
 typedef unsigned __int128 u128;
@@ -55,7 +81,12 @@ struct Work {
     Sel sel[2];                 // 0: prune, 1: unify
     unsigned cand_count[2];
     unsigned ticket[4];         // [1]: prune_select, [3]: collect<1>
-    unsigned pad[2];
+    // one-pass pipeline
+    unsigned fcand_count[2];    // threshold-bin candidates of list_select / list_collect
+    unsigned fticket[2];
+    unsigned list_count;        // entries appended to the candidate list
+    unsigned failed;            // != 0: the one-pass result is void, the multi-pass kernels run
+    u64 That[2];                // provisional thresholds (key bit patterns)
 };
 
 struct Params {
@@ -67,7 +98,11 @@ struct Params {
     int use_l1;
     Work *work;
     int nb;                     // level-0 bins in use (NB_SMALL or NB_MAX)
-    unsigned *hist;             // [3][nb]: prune, unify, refine scratch
+    unsigned *hist;             // [3][nb]: prune, unify, refine scratch (multi-pass kernels)
+    unsigned *fhist;            // [2][nb]: prune, unify (one-pass kernels)
+    uint2 *list;                // [list_cap] candidate list: (block index, bin codes)
+    unsigned list_cap;
+    int gated;                  // multi-pass kernels return at once unless work->failed is set
     u64 *cand_key;              // [CAP]
     unsigned *cand_idx;         // [CAP]
     unsigned *bins;             // [n_blocks]
@@ -137,13 +172,36 @@ __device__ __forceinline__ float load_v(const float *W, const float *U, long lon
     return w;
 }
 
+// the B values of block j with the widest loads its alignment allows (a block starts at a
+// multiple of 4*B bytes): scalar loads of scattered blocks cost one cache-line lookup per value
+template <int B>
+__device__ __forceinline__ void load_block(const float *W, const float *U, long long j, float (&v)[B]) {
+    if (B == 2) {
+        float2 a = __ldg(reinterpret_cast<const float2 *>(W) + j);
+        if (U) {
+            const float2 d = __ldg(reinterpret_cast<const float2 *>(U) + j);
+            a.x = __fadd_rn(a.x, d.x); a.y = __fadd_rn(a.y, d.y);
+        }
+        v[0] = a.x; v[1 % B] = a.y;
+    } else {
+#pragma unroll
+        for (int c = 0; c < B / 4; ++c) {
+            float4 a = __ldg(reinterpret_cast<const float4 *>(W) + j * (B / 4) + c);
+            if (U) {
+                const float4 d = __ldg(reinterpret_cast<const float4 *>(U) + j * (B / 4) + c);
+                a.x = __fadd_rn(a.x, d.x); a.y = __fadd_rn(a.y, d.y); a.z = __fadd_rn(a.z, d.z); a.w = __fadd_rn(a.w, d.w);
+            }
+            v[(4 * c) % B] = a.x; v[(4 * c + 1) % B] = a.y; v[(4 * c + 2) % B] = a.z; v[(4 * c + 3) % B] = a.w;
+        }
+    }
+}
+
 // exact keys of block j, read from global memory (sampling and threshold-bin blocks)
 template <int B>
 __device__ __forceinline__ void block_keys_at(const float *W, const float *U, long long j, int use_l1,
                                               double *S, double *Lu, double *Kp) {
     float v[B];
-#pragma unroll
-    for (int l = 0; l < B; ++l) v[l] = load_v(W, U, j * B + l);
+    load_block<B>(W, U, j, v);
     block_keys<B>(v, use_l1, S, Lu, Kp);
 }
 
@@ -179,18 +237,6 @@ __device__ __forceinline__ void load16(const float *W, const float *U, long long
 // ---------------------------------------------------------------------------------------------
 // sample_kernel: choose the level-0 windows
 // ---------------------------------------------------------------------------------------------
-// Window around the `frac` quantile of n sample keys: +-4 sigma (binomial) in rank.  Returns the
-// two ranks whose keys bound the window and the rank of the quantile itself.
-__device__ __forceinline__ void window_ranks(int n, double frac, int *il, int *ih, int *ipos) {
-    const double pos = frac * n;
-    const double margin = 4.0 * sqrt(fmax(n * frac * (1.0 - frac), 0.0)) + 4.0;
-    long long a = (long long)floor(pos - margin), b = (long long)ceil(pos + margin), c = (long long)pos;
-    if (a < 0) a = 0;
-    if (b > n - 1) b = n - 1;
-    if (c > n - 1) c = n - 1;
-    *il = (int)a; *ih = (int)b; *ipos = (int)c;
-}
-
 __device__ __forceinline__ void set_window(Sel *s, u64 lo, u64 hi, int nb) {
     if (hi < lo) hi = lo;
     unsigned shift = 0;
@@ -200,72 +246,192 @@ __device__ __forceinline__ void set_window(Sel *s, u64 lo, u64 hi, int nb) {
     s->shift0 = shift;
 }
 
-// rank of (key, i) among the n keys in shared memory (ties ordered by position)
-__device__ __forceinline__ int rank_of(const u64 *keys, int n, u64 key, int i) {
-    int r = 0;
-    for (int t = 0; t < n; ++t) {
-        const u64 k = keys[t];
-        r += (k < key || (k == key && t < i)) ? 1 : 0;
+// inclusive prefix sum over the CTA's SAMP_THREADS values (one per thread)
+__device__ __forceinline__ unsigned block_scan_incl(unsigned x, unsigned *s_warp) {
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    for (int m = 1; m < 32; m <<= 1) {
+        const unsigned y = __shfl_up_sync(0xffffffffu, x, m);
+        if (lane >= m) x += y;
     }
-    return r;
+    if (lane == 31) s_warp[w] = x;
+    __syncthreads();
+    if (w == 0) {
+        unsigned t = s_warp[lane];
+        for (int m = 1; m < 32; m <<= 1) {
+            const unsigned y = __shfl_up_sync(0xffffffffu, t, m);
+            if (lane >= m) t += y;
+        }
+        s_warp[lane] = t;
+    }
+    __syncthreads();
+    const unsigned add = w ? s_warp[w - 1] : 0u;
+    __syncthreads();
+    return x + add;
+}
+
+// Window around the `frac` quantile of n sample keys: +-4 sigma (binomial) in rank.  Returns the
+// two ranks whose keys bound the window and the rank of the quantile itself.
+__device__ __forceinline__ void window_ranks_f(int n, float frac, int *il, int *ih, int *ipos) {
+    const float pos = frac * (float)n;
+    const float margin = 4.f * sqrtf(fmaxf((float)n * frac * (1.f - frac), 0.f)) + 4.f;
+    int a = (int)floorf(pos - margin), b = (int)ceilf(pos + margin), c = (int)pos;
+    if (a < 0) a = 0;
+    if (b > n - 1) b = n - 1;
+    if (c > n - 1) c = n - 1;
+    if (c < 0) c = 0;
+    *il = a; *ih = b; *ipos = c;
+}
+
+// One selection of sample_kernel.  key[t] / valid[t]: this thread's sample keys; `frac` of the
+// valid ones are to be selected.  Level A ranks a 1-in-16 subsample (<= 256 keys) to get a coarse
+// window; level B counts all valid samples in SAMP_THREADS bins across that window and reads the
+// final window [lo, hi) and the provisional threshold from the bin edges.
+__device__ void sample_select(const u64 (&key)[SAMP_PER], const bool (&valid)[SAMP_PER], float frac,
+                              u64 *lo_out, u64 *hi_out, u64 *t_out) {
+    constexpr int NA = NSAMP / 16;
+    // level-A keys, shortened to the top 24 bits below the (clear) sign bit, with the key's index in
+    // the low byte: distinct words, one 32-bit compare per pair; invalid keys rank last
+    __shared__ __align__(16) unsigned s_a[NA];
+    __shared__ unsigned s_edge[2];                    // shortened keys at the coarse window's ranks
+    __shared__ unsigned s_hist[SAMP_THREADS + 2];     // [0] under, [1 .. SAMP_THREADS] window, [+1] over
+    __shared__ unsigned s_warp[32];
+    __shared__ unsigned s_nvalid;
+    __shared__ u64 s_res[3];
+    static_assert(NA == 256, "the index of a level-A key fills the low byte of its shortened form");
+    const int tid = threadIdx.x;
+    if (tid == 0) s_nvalid = 0;
+    for (int i = tid; i < SAMP_THREADS + 2; i += SAMP_THREADS) s_hist[i] = 0;
+    // level A: sample index 16 * a is slot 0 of thread 4 * a
+    const bool is_a = (tid % 4) == 0;
+    const int a = tid / 4;
+    const bool a_valid = is_a && valid[0];
+    if (is_a) s_a[a] = a_valid ? ((unsigned)(key[0] >> 39) << 8) | (unsigned)a : 0xffffffffu;
+    int nv = 0;
+#pragma unroll
+    for (int t = 0; t < SAMP_PER; ++t) nv += valid[t] ? 1 : 0;
+    for (int m = 16; m > 0; m >>= 1) nv += __shfl_xor_sync(0xffffffffu, nv, m);
+    const int na_raw = __syncthreads_count(a_valid);           // also orders the stores above
+    if ((tid & 31) == 0 && nv) atomicAdd(&s_nvalid, (unsigned)nv);
+    const int na = na_raw > 0 ? na_raw : 1;
+    int il, ih, ipos;
+    window_ranks_f(na, frac, &il, &ih, &ipos);
+    {
+        // four threads rank one level-A key, each against a quarter of the keys
+        const int part = tid % 4;
+        const unsigned k = s_a[a];
+        int r = 0;
+        const uint4 *q = reinterpret_cast<const uint4 *>(s_a + part * (NA / 4));
+#pragma unroll 4
+        for (int t = 0; t < NA / 16; ++t) {
+            const uint4 x = q[t];
+            r += (x.x < k ? 1 : 0) + (x.y < k ? 1 : 0) + (x.z < k ? 1 : 0) + (x.w < k ? 1 : 0);
+        }
+        r += __shfl_xor_sync(0xffffffffu, r, 1);
+        r += __shfl_xor_sync(0xffffffffu, r, 2);
+        if (is_a) {
+            if (r == il) s_edge[0] = k;
+            if (r == ih) s_edge[1] = k;
+        }
+    }
+    __syncthreads();
+    const int n_valid = (int)s_nvalid > 0 ? (int)s_nvalid : 1;
+    // back to full keys: the low 39 bits of the edges are zero (any window is a valid window)
+    u64 clo = (u64)(s_edge[0] >> 8) << 39;
+    u64 chi = (u64)(s_edge[1] >> 8) << 39;
+    if (s_edge[0] == 0xffffffffu) clo = ~0ull >> 1;
+    if (s_edge[1] == 0xffffffffu) chi = ~0ull >> 1;
+    if (chi < clo) chi = clo;
+    unsigned shift = 0;
+    while (((chi - clo) >> shift) >= (u64)SAMP_THREADS) ++shift;
+    // level B
+    unsigned n_under = 0, n_over = 0;                 // the two catch-all counts stay in registers
+#pragma unroll
+    for (int t = 0; t < SAMP_PER; ++t) {
+        if (!valid[t]) continue;
+        const u64 k = key[t];
+        if (k < clo) ++n_under;
+        else if (k >= chi) ++n_over;
+        else atomicAdd(&s_hist[1u + (unsigned)((k - clo) >> shift)], 1u);
+    }
+    for (int m = 16; m > 0; m >>= 1) {
+        n_under += __shfl_xor_sync(0xffffffffu, n_under, m);
+        n_over += __shfl_xor_sync(0xffffffffu, n_over, m);
+    }
+    if ((tid & 31) == 0) {
+        if (n_under) atomicAdd(&s_hist[0], n_under);
+        if (n_over) atomicAdd(&s_hist[SAMP_THREADS + 1], n_over);
+    }
+    __syncthreads();
+    const unsigned mine = s_hist[1 + tid];
+    const unsigned incl = block_scan_incl(mine, s_warp) + s_hist[0];
+    const unsigned excl = incl - mine;
+    window_ranks_f(n_valid, frac, &il, &ih, &ipos);
+    if (tid == 0) {
+        // ranks outside the coarse window keep its edge
+        s_res[0] = clo;
+        s_res[1] = chi;
+        s_res[2] = clo;
+    }
+    __syncthreads();
+    const u64 edge_lo = clo + ((u64)tid << shift);
+    u64 edge_hi = clo + ((u64)(tid + 1) << shift);
+    if (edge_hi > chi) edge_hi = chi;
+    if (mine) {
+        if (excl <= (unsigned)il && (unsigned)il < incl) s_res[0] = edge_lo < chi ? edge_lo : chi;
+        if (excl <= (unsigned)ih && (unsigned)ih < incl) s_res[1] = edge_hi;
+        if (excl <= (unsigned)ipos && (unsigned)ipos < incl) s_res[2] = edge_lo < chi ? edge_lo : chi;
+    }
+    __syncthreads();
+    u64 lo = s_res[0], hi = s_res[1], That = s_res[2];
+    if (That < lo) That = lo;
+    if (hi > lo && That >= hi) That = hi - 1;         // the provisional threshold lies inside [lo, hi)
+    *lo_out = lo;
+    *hi_out = hi;
+    *t_out = That;
+    __syncthreads();
 }
 
 template <int B>
-__global__ void __launch_bounds__(NSAMP) sample_kernel(Params p, long long k_unify, long long k_prune) {
-    __shared__ u64 skey[NSAMP];
-    __shared__ u64 s_stat[3];                  // keys at the ranks il, ih, ipos
-    __shared__ int s_kept;
+__global__ void __launch_bounds__(SAMP_THREADS) sample_kernel(Params p, long long k_unify, long long k_prune) {
     const long long mb = p.n_blocks;
     const int ns = (int)(mb < (long long)NSAMP ? mb : (long long)NSAMP);
-    const int i = threadIdx.x;
-    u64 kp = ~0ull, ku = ~0ull;
-    if (i == 0) s_kept = 0;
-    if (i < ns) {
-        const long long j = (long long)(((u128)(u64)i * (u128)(u64)mb) / (u128)(u64)ns);
-        double S, Lu, Kp;
-        block_keys_at<B>(p.W, p.U, j, p.use_l1, &S, &Lu, &Kp);
-        kp = key_bits(Kp);
-        ku = key_bits(Lu);
+    u64 kp[SAMP_PER], ku[SAMP_PER];
+    bool valid[SAMP_PER];
+#pragma unroll
+    for (int t = 0; t < SAMP_PER; ++t) {
+        const int i = threadIdx.x * SAMP_PER + t;
+        kp[t] = ~0ull;
+        ku[t] = ~0ull;
+        valid[t] = i < ns;
+        if (i < ns) {
+            const long long j = (long long)(((u64)i * (u64)mb) / (u64)ns);     // i < 2^12, mb < 2^31
+            double S, Lu, Kp;
+            block_keys_at<B>(p.W, p.U, j, p.use_l1, &S, &Lu, &Kp);
+            kp[t] = key_bits(Kp);
+            ku[t] = key_bits(Lu);
+        }
     }
-    skey[i] = kp;
-    __syncthreads();
     Sel *sp = &p.work->sel[0];
     Sel *su = &p.work->sel[1];
     const long long ksel_u = k_unify - k_prune;
-    int il, ih, ipos;
-    window_ranks(ns, (double)k_prune / (double)mb, &il, &ih, &ipos);
-    if (i < ns) {
-        const int r = rank_of(skey, ns, kp, i);
-        if (r == il) s_stat[0] = kp;
-        if (r == ih) s_stat[1] = kp;
-        if (r == ipos) s_stat[2] = kp;
-    }
-    __syncthreads();
-    const u64 That = s_stat[2];
-    if (i == 0) {
-        set_window(sp, s_stat[0], s_stat[1], p.nb);
+    u64 lo, hi, That;
+    sample_select(kp, valid, (float)((double)k_prune / (double)mb), &lo, &hi, &That);
+    if (threadIdx.x == 0) {
+        set_window(sp, lo, hi, p.nb);
         sp->mode = (k_prune == 0) ? 1u : (k_prune == mb ? 2u : 0u);
         sp->k = (u64)k_prune;
+        p.work->That[0] = That;
     }
     // the sample blocks that survive the (estimated) prune threshold
-    const bool kept = i < ns && (k_prune == 0 || kp > That);
-    __syncthreads();
-    skey[i] = kept ? ku : ~0ull;
-    if (kept) atomicAdd(&s_kept, 1);
-    __syncthreads();
-    const int nr = s_kept > 0 ? s_kept : 1;
+#pragma unroll
+    for (int t = 0; t < SAMP_PER; ++t) valid[t] = valid[t] && (k_prune == 0 || kp[t] > That);
     const long long elig = mb - k_prune;
-    window_ranks(nr, elig > 0 ? (double)ksel_u / (double)elig : 0.0, &il, &ih, &ipos);
-    if (i < ns) {
-        const int r = rank_of(skey, ns, kept ? ku : ~0ull, i);     // dropped samples rank last
-        if (r == il) s_stat[0] = skey[i];
-        if (r == ih) s_stat[1] = skey[i];
-    }
-    __syncthreads();
-    if (i == 0) {
-        set_window(su, s_stat[0], s_stat[1], p.nb);
+    sample_select(ku, valid, elig > 0 ? (float)((double)ksel_u / (double)elig) : 0.f, &lo, &hi, &That);
+    if (threadIdx.x == 0) {
+        set_window(su, lo, hi, p.nb);
         su->mode = (ksel_u == 0) ? 1u : (ksel_u == elig ? 2u : 0u);
         su->k = (u64)ksel_u;
+        p.work->That[1] = That;
     }
 }
 
@@ -276,53 +442,86 @@ __global__ void __launch_bounds__(NSAMP) sample_kernel(Params p, long long k_uni
 // before is visible to it afterwards.
 __device__ __forceinline__ bool last_block_done(unsigned *ticket) {
     __shared__ bool s_last;
-    __threadfence();
-    __syncthreads();
+    __syncthreads();                       // every write of this CTA happens before thread 0's fence
     if (threadIdx.x == 0) {
+        __threadfence();                   // cumulative: publishes what the barrier made visible to thread 0
         const unsigned t = atomicAdd(ticket, 1u);
         s_last = (t == gridDim.x - 1);
+        if (s_last) __threadfence();
     }
     __syncthreads();
-    if (s_last) __threadfence();
     return s_last;
 }
 
 // find the bin holding the r-th element; hist has nb entries
 __device__ void scan_hist(const unsigned *hist, int nb, u64 r, unsigned *bin_out, u64 *r_in_bin, u64 *cnt_out,
                           unsigned *err) {
-    __shared__ u64 s_part[FIN_THREADS];
+    __shared__ u64 s_part[32];
     const int PER = nb / FIN_THREADS;
     u64 sum = 0;
 #pragma unroll 8
     for (int i = 0; i < PER; ++i) sum += ld_vol(&hist[threadIdx.x * PER + i]);
-    s_part[threadIdx.x] = sum;
-    __syncthreads();
-    for (int off = 1; off < FIN_THREADS; off <<= 1) {
-        u64 add = 0;
-        if ((int)threadIdx.x >= off) add = s_part[threadIdx.x - off];
-        __syncthreads();
-        s_part[threadIdx.x] += add;
-        __syncthreads();
+    // inclusive scan of the per-thread sums: shuffles inside a warp, then over the 32 warp totals
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    u64 incl = sum;
+    for (int m = 1; m < 32; m <<= 1) {
+        const u64 y = __shfl_up_sync(0xffffffffu, incl, m);
+        if (lane >= m) incl += y;
     }
-    const u64 incl = s_part[threadIdx.x];
-    u64 run = incl - sum;
-    if (threadIdx.x == FIN_THREADS - 1 && incl < r) *err = 1;
-    if (run < r && r <= incl) {                              // the bin is in this thread's range
-        for (int i = 0; i < PER; ++i) {
-            const u64 c = ld_vol(&hist[threadIdx.x * PER + i]);
-            if (run < r && r <= run + c) {
-                *bin_out = threadIdx.x * PER + i;
-                *r_in_bin = r - run;
-                *cnt_out = c;
-            }
-            run += c;
+    __syncthreads();                                         // s_part may still be read by an earlier call
+    if (lane == 31) s_part[wid] = incl;
+    __syncthreads();
+    if (wid == 0) {
+        u64 t = s_part[lane];
+        for (int m = 1; m < 32; m <<= 1) {
+            const u64 y = __shfl_up_sync(0xffffffffu, t, m);
+            if (lane >= m) t += y;
         }
+        s_part[lane] = t;
+    }
+    __syncthreads();
+    if (wid) incl += s_part[wid - 1];
+    const u64 run = incl - sum;
+    if (threadIdx.x == FIN_THREADS - 1 && incl < r) *err = 1;
+    __shared__ int s_owner;
+    __shared__ u64 s_run;
+    if (threadIdx.x == 0) s_owner = -1;
+    __syncthreads();
+    if (run < r && r <= incl) { s_owner = threadIdx.x; s_run = run; }     // the bin is in this thread's range
+    __syncthreads();
+    // warp 0 scans the owner's PER (<= 64) bins together
+    if (wid == 0 && s_owner >= 0) {
+        const int base = s_owner * PER;
+        const u64 c0 = lane < PER ? (u64)ld_vol(&hist[base + lane]) : 0ull;
+        const u64 c1 = lane + 32 < PER ? (u64)ld_vol(&hist[base + lane + 32]) : 0ull;
+        u64 i0 = c0;                                   // inclusive scan over bins 0..31, then 32..63
+        for (int m = 1; m < 32; m <<= 1) {
+            const u64 y = __shfl_up_sync(0xffffffffu, i0, m);
+            if (lane >= m) i0 += y;
+        }
+        const u64 tot0 = __shfl_sync(0xffffffffu, i0, 31);
+        u64 i1 = c1;
+        for (int m = 1; m < 32; m <<= 1) {
+            const u64 y = __shfl_up_sync(0xffffffffu, i1, m);
+            if (lane >= m) i1 += y;
+        }
+        i1 += tot0;
+        const u64 before0 = s_run + i0 - c0, before1 = s_run + i1 - c1;
+        if (c0 && before0 < r && r <= before0 + c0) { *bin_out = base + lane; *r_in_bin = r - before0; *cnt_out = c0; }
+        if (c1 && before1 < r && r <= before1 + c1) { *bin_out = base + lane + 32; *r_in_bin = r - before1; *cnt_out = c1; }
     }
     __syncthreads();
 }
 
+// what select_bin found, kept in shared memory for the CTA that ran it
+struct BinSel {
+    unsigned B;
+    u64 r, cnt;
+    u64 lo_hi, lo_lo, hi_hi, hi_lo;
+};
+
 // level 0: which bin holds the k-th element; writes the bin and its composite range
-__device__ void select_bin(const Params &p, Sel *s, const unsigned *hist) {
+__device__ void select_bin(const Params &p, Sel *s, const unsigned *hist, BinSel *out, bool publish) {
     __shared__ unsigned s_bin, s_err;
     __shared__ u64 s_r, s_cnt;
     if (threadIdx.x == 0) { s_err = 0; s_bin = 0; s_r = 0; s_cnt = 0; }
@@ -340,12 +539,16 @@ __device__ void select_bin(const Params &p, Sel *s, const unsigned *hist) {
             if (khi > s->hi0) khi = s->hi0;
         }
         const u128 lo = make_c(klo, 0), hi = make_c(khi, 0);
-        s->B = B;
-        s->r = s_r;
-        s->cnt = s_cnt;
-        s->lo_hi = (u64)(lo >> 64); s->lo_lo = (u64)lo;
-        s->hi_hi = (u64)(hi >> 64); s->hi_lo = (u64)hi;
-        __threadfence();
+        if (publish) {                                   // for the kernels that follow
+            s->B = B;
+            s->r = s_r;
+            s->cnt = s_cnt;
+            s->lo_hi = (u64)(lo >> 64); s->lo_lo = (u64)lo;
+            s->hi_hi = (u64)(hi >> 64); s->hi_lo = (u64)hi;
+        }
+        out->B = B; out->r = s_r; out->cnt = s_cnt;
+        out->lo_hi = (u64)(lo >> 64); out->lo_lo = (u64)lo;
+        out->hi_hi = (u64)(hi >> 64); out->hi_lo = (u64)hi;
     }
     __syncthreads();
 }
@@ -358,7 +561,19 @@ struct SelView {
     u64 T_key, T_idx;
 };
 
+// Selection state written by an EARLIER kernel: plain (L1-cached) loads.  Volatile loads of one
+// address by every warp of a large grid all queue at one L2 slice -- tens of microseconds.
 __device__ __forceinline__ SelView view_of(const Sel *s) {
+    SelView v;
+    v.mode = s->mode;
+    v.B = s->B;
+    v.T_key = s->T_key;
+    v.T_idx = s->T_idx;
+    return v;
+}
+
+// the same, for state written earlier in the running kernel (read by one CTA only)
+__device__ __forceinline__ SelView view_vol(const Sel *s) {
     SelView v;
     v.mode = ld_vol(&s->mode);
     v.B = ld_vol(&s->B);
@@ -366,6 +581,7 @@ __device__ __forceinline__ SelView view_of(const Sel *s) {
     v.T_idx = ld_vol(&s->T_idx);
     return v;
 }
+
 
 template <int B>
 __device__ __forceinline__ bool selected(const Params &p, const SelView &s, long long j, unsigned bin,
@@ -384,6 +600,7 @@ __device__ __forceinline__ bool selected(const Params &p, const SelView &s, long
 template <int B>
 __global__ void __launch_bounds__(256) stats_kernel(Params p, double *loss_u, double *loss_p, float *u_out,
                                                     unsigned *sign_bits) {
+    if (p.gated && p.work->failed == 0u) return;     // the one-pass result stands
     constexpr int NBT = 16 / B;                         // blocks per thread and step
     const Sel *sp = &p.work->sel[0];
     const Sel *su = &p.work->sel[1];
@@ -511,20 +728,22 @@ __device__ void sort_candidates(u64 *key, unsigned *idx, int n_pow2) {
 
 template <int KIND, int B>
 __global__ void __launch_bounds__(FIN_THREADS) collect_kernel(Params p) {
+    if (p.gated && p.work->failed == 0u) return;     // the one-pass result stands
     Sel *s = &p.work->sel[KIND];
-    if (ld_vol(&s->mode) != 0u) return;
+    if (s->mode != 0u) return;
     __shared__ u64 c_key[CAP];
     __shared__ unsigned c_idx[CAP];
     __shared__ unsigned s_bin, s_err, s_n;
     __shared__ u64 s_r, s_cnt;
+    // the selection state comes from the previous kernel: plain loads
     const SelView pv = view_of(&p.work->sel[0]);
-    const unsigned Bsel = ld_vol(&s->B);
-    const bool too_many = ld_vol(&s->cnt) > (u64)CAP;
+    const unsigned Bsel = s->B;
+    const bool too_many = s->cnt > (u64)CAP;
     const long long stride = (long long)gridDim.x * blockDim.x;
 
     if (!too_many) {
-        const u128 lo = from_halves(ld_vol(&s->lo_hi), ld_vol(&s->lo_lo));
-        const u128 hi = from_halves(ld_vol(&s->hi_hi), ld_vol(&s->hi_lo));
+        const u128 lo = from_halves(s->lo_hi, s->lo_lo);
+        const u128 hi = from_halves(s->hi_hi, s->hi_lo);
         for (long long j0 = ((long long)blockIdx.x * blockDim.x + threadIdx.x) * 4; j0 < p.n_blocks;
              j0 += stride * 4 * PASS_LOADS) {
             unsigned codes[PASS_LOADS][4];
@@ -643,20 +862,24 @@ __global__ void __launch_bounds__(FIN_THREADS) collect_kernel(Params p) {
 // L_u bins of the candidates that survive, and locates the unify threshold bin.
 template <int B>
 __global__ void __launch_bounds__(FIN_THREADS) prune_select_kernel(Params p) {
+    if (p.gated && p.work->failed == 0u) return;     // the one-pass result stands
     Sel *sp = &p.work->sel[0];
     Sel *su = &p.work->sel[1];
-    const unsigned mode_p = ld_vol(&sp->mode), mode_u = ld_vol(&su->mode);
+    const unsigned mode_p = sp->mode, mode_u = su->mode;
     if (mode_p != 0u && mode_u != 0u) return;
     __shared__ u64 c_key[CAP];
     __shared__ unsigned c_idx[CAP];
     __shared__ unsigned s_bin, s_err, s_n;
     __shared__ u64 s_r, s_cnt;
+    __shared__ BinSel s_sel;
     unsigned *hist_u = p.hist + p.nb;
-    if (mode_p == 0u) select_bin(p, sp, p.hist);
-    const unsigned Bp = ld_vol(&sp->B);
-    const bool too_many = mode_p == 0u && ld_vol(&sp->cnt) > (u64)CAP;
-    const u128 lo0 = from_halves(ld_vol(&sp->lo_hi), ld_vol(&sp->lo_lo));
-    const u128 hi0 = from_halves(ld_vol(&sp->hi_hi), ld_vol(&sp->hi_lo));
+    if (threadIdx.x == 0) { s_sel.B = 0; s_sel.r = 0; s_sel.cnt = 0; s_sel.lo_hi = s_sel.lo_lo = s_sel.hi_hi = s_sel.hi_lo = 0; }
+    __syncthreads();
+    if (mode_p == 0u) select_bin(p, sp, p.hist, &s_sel, true);
+    const unsigned Bp = s_sel.B;
+    const bool too_many = mode_p == 0u && s_sel.cnt > (u64)CAP;
+    const u128 lo0 = from_halves(s_sel.lo_hi, s_sel.lo_lo);
+    const u128 hi0 = from_halves(s_sel.hi_hi, s_sel.hi_lo);
     const long long stride = (long long)gridDim.x * blockDim.x;
     unsigned under = 0, over = 0;
     if (mode_p != 2u) {                                   // mode 2: everything is pruned, nothing survives
@@ -788,7 +1011,7 @@ __global__ void __launch_bounds__(FIN_THREADS) prune_select_kernel(Params p) {
                 for (unsigned i = (unsigned)r + threadIdx.x; i < m; i += blockDim.x)
                     atomicAdd(&hist_u[ld_vol(p.bins + c_idx[i]) >> 16], 1u);
             } else {
-                const SelView pv = view_of(sp);
+                const SelView pv = view_vol(sp);
                 for (long long j = threadIdx.x; j < p.n_blocks; j += blockDim.x) {
                     const unsigned code = ld_vol(p.bins + j);
                     if ((code & 0xffffu) != Bp) continue;
@@ -799,7 +1022,7 @@ __global__ void __launch_bounds__(FIN_THREADS) prune_select_kernel(Params p) {
         __threadfence();
         __syncthreads();
     }
-    if (mode_u == 0u) select_bin(p, su, hist_u);
+    if (mode_u == 0u) select_bin(p, su, hist_u, &s_sel, true);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -809,6 +1032,7 @@ template <int B>
 __global__ void __launch_bounds__(256, 3) emit_kernel(Params p, float *Q, float *u_out,
                                                    unsigned *pruned_bitmap, unsigned *unified_bitmap,
                                                    unsigned *sign_bits) {
+    if (p.gated && p.work->failed == 0u) return;     // the one-pass result stands
     constexpr int NBT = 16 / B;
     const SelView vp = view_of(&p.work->sel[0]);
     const SelView vu = view_of(&p.work->sel[1]);
@@ -951,42 +1175,506 @@ __global__ void __launch_bounds__(256, 3) emit_kernel(Params p, float *Q, float 
     }
 }
 
+// ---------------------------------------------------------------------------------------------
+// one-pass pipeline
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ void one_pass_fail(const Params &p) { atomicExch(&p.work->failed, 1u); }
+
+// pass_kernel: keys, provisional classes and every output in one sweep over W (+U).
+// A block is a candidate when its final class is still open: its prune key lies inside the prune
+// window, or it certainly survives pruning and its L_u lies inside the unify window.
+template <int B>
+__global__ void __launch_bounds__(256) pass_kernel(Params p, float *Q, double *loss_u, double *loss_p,
+                                                   float *u_out, unsigned *pruned_bitmap,
+                                                   unsigned *unified_bitmap, unsigned *sign_bits) {
+    constexpr int NBT = 16 / B;
+    const Sel *sp = &p.work->sel[0];
+    const Sel *su = &p.work->sel[1];
+    const u64 plo = sp->lo0, phi = sp->hi0, ulo = su->lo0, uhi = su->hi0;
+    const unsigned psh = sp->shift0, ush = su->shift0;
+    const unsigned mode_p = sp->mode, mode_u = su->mode;
+    const u64 Tp = p.work->That[0], Tu = p.work->That[1];
+    const unsigned nb = (unsigned)p.nb, top = nb - 1u;
+    unsigned *hist_p = p.fhist, *hist_u = p.fhist + p.nb;
+    __shared__ float4 s_q[8][128];                       // one warp step of Q per warp
+    __shared__ uint2 s_cand[8][STAGE_ENTRIES];           // list entries waiting for a full 32-entry flush
+    const int lane = threadIdx.x & 31;
+    float4 *wq = s_q[threadIdx.x >> 5];
+    uint2 *wc = s_cand[threadIdx.x >> 5];
+    const unsigned lt_mask = (1u << lane) - 1u;
+    unsigned fill = 0;                                   // warp-uniform
+    unsigned under_p = 0, over_p = 0, under_u = 0, over_u = 0, nonfinite = 0;
+    const long long n = p.n_floats;
+    const long long n_units = (n + 15) / 16;
+    const long long n_iter = (n_units + 31) / 32 * 32;   // whole warps take part in every step
+    const long long n_bm_words = (p.n_blocks + 31) / 32;
+    const long long ustride = (long long)gridDim.x * blockDim.x;
+    long long unit = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    float nxt[16];
+#pragma unroll
+    for (int l = 0; l < 16; ++l) nxt[l] = 0.f;
+    if (unit < n_units) load16(p.W, p.U, unit * 16, n, nxt);
+    for (; unit < n_iter; unit += ustride) {
+        float v[16];
+#pragma unroll
+        for (int l = 0; l < 16; ++l) v[l] = nxt[l];
+        // the next unit's 64 bytes travel while this one is evaluated
+        if (unit + ustride < n_units) load16(p.W, p.U, (unit + ustride) * 16, n, nxt);
+        else {
+#pragma unroll
+            for (int l = 0; l < 16; ++l) nxt[l] = 0.f;
+        }
+        const bool live = unit < n_units;
+        const bool warp_full = (unit - lane + 32) * 16 <= n;      // all 512 floats of this warp step exist
+        unsigned ex = 0, sb = 0;
+#pragma unroll
+        for (int l = 0; l < 16; ++l) {
+            ex = max(ex, __float_as_uint(v[l]) & 0x7fffffffu);
+            sb |= (v[l] < 0.f ? 1u : 0u) << l;
+        }
+        nonfinite |= (ex >= 0x7f800000u) ? 1u : 0u;
+        if (live) {
+            unsigned short *halves = reinterpret_cast<unsigned short *>(sign_bits);
+            halves[unit] = (unsigned short)sb;
+            if (unit == n_units - 1 && (n_units & 1)) halves[unit + 1] = 0;
+        }
+        unsigned cls_p = 0, cls_u = 0, cand = 0;             // bit e: block e of this thread
+        unsigned code[NBT];
+        float uo[NBT];
+        const long long j0 = unit * NBT;
+#pragma unroll
+        for (int e = 0; e < NBT; ++e) {
+            double S, Lu, Kp;
+            block_keys<B>(v + e * B, p.use_l1, &S, &Lu, &Kp);
+            const float qf = __double2float_rn(__dmul_rn(S, 1.0 / (double)B));
+            const u64 kpb = key_bits(Kp), kub = key_bits(Lu);
+            const unsigned bp = bin_of(kpb, plo, phi, psh, nb);
+            const unsigned bu = bin_of(kub, ulo, uhi, ush, nb);
+            code[e] = bp | (bu << 16);
+            uo[e] = 0.f;
+            const long long j = j0 + e;
+            if (j < p.n_blocks) {
+                if (loss_u) loss_u[j] = Lu;
+                if (loss_p) loss_p[j] = Kp;
+                bool pr, survives, open = false;
+                if (mode_p == 0u) {
+                    pr = kpb <= Tp;
+                    survives = bp == top;
+                    if (bp == 0u) ++under_p;
+                    else if (bp == top) ++over_p;
+                    else { atomicAdd(&hist_p[bp], 1u); open = true; }
+                } else {
+                    pr = mode_p == 2u;
+                    survives = mode_p == 1u;
+                }
+                const bool un = !pr && (mode_u == 2u || (mode_u == 0u && kub <= Tu));
+                if (survives && mode_u == 0u) {
+                    if (bu == 0u) ++under_u;
+                    else if (bu == top) ++over_u;
+                    else { atomicAdd(&hist_u[bu], 1u); open = true; }
+                }
+                cls_p |= (pr ? 1u : 0u) << e;
+                cls_u |= (un ? 1u : 0u) << e;
+                cand |= (open ? 1u : 0u) << e;
+                if (un) uo[e] = qf;
+            }
+        }
+        if (live) {
+            if (j0 + NBT <= p.n_blocks) {
+                if (NBT == 1) u_out[j0] = uo[0];
+                else if (NBT == 2) *reinterpret_cast<float2 *>(u_out + j0) = make_float2(uo[0], uo[1 % NBT]);
+                else {
+#pragma unroll
+                    for (int e = 0; e < NBT; e += 4)
+                        *reinterpret_cast<float4 *>(u_out + j0 + e) =
+                            make_float4(uo[e % NBT], uo[(e + 1) % NBT], uo[(e + 2) % NBT], uo[(e + 3) % NBT]);
+                }
+            } else {
+#pragma unroll
+                for (int e = 0; e < NBT; ++e)
+                    if (j0 + e < p.n_blocks) u_out[j0 + e] = uo[e];
+            }
+            if (Q) {
+                float q[16];
+#pragma unroll
+                for (int e = 0; e < NBT; ++e) {
+                    const bool pr = (cls_p >> e) & 1u, un = (cls_u >> e) & 1u;
+#pragma unroll
+                    for (int l = 0; l < B; ++l) {
+                        const float x = v[e * B + l];
+                        q[e * B + l] = pr ? 0.f : (un ? (x < 0.f ? -uo[e] : uo[e]) : x);
+                    }
+                }
+                const long long f = unit * 16;
+                if (!warp_full) {
+                    if (f + 16 <= n) {
+                        float4 *dst = reinterpret_cast<float4 *>(Q + f);
+                        dst[0] = make_float4(q[0], q[1], q[2], q[3]);
+                        dst[1] = make_float4(q[4], q[5], q[6], q[7]);
+                        dst[2] = make_float4(q[8], q[9], q[10], q[11]);
+                        dst[3] = make_float4(q[12], q[13], q[14], q[15]);
+                    } else {
+#pragma unroll
+                        for (int l = 0; l < 16; ++l)
+                            if (f + l < n) Q[f + l] = q[l];
+                    }
+                } else {
+#pragma unroll
+                    for (int c = 0; c < 4; ++c)
+                        wq[lane * 4 + (c ^ ((lane >> 1) & 3))] = make_float4(q[4 * c], q[4 * c + 1], q[4 * c + 2], q[4 * c + 3]);
+                }
+            }
+        }
+        // Q of a whole warp step (2 KB) leaves as four stores of 512 contiguous bytes: thread t keeps
+        // piece c at slot c ^ ((t >> 1) & 3), so neither side has bank conflicts.
+        if (Q && warp_full) {
+            __syncwarp();
+            float4 *dst = reinterpret_cast<float4 *>(Q + (unit - lane) * 16);
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const int t = 8 * k + (lane >> 2), c = lane & 3;
+                dst[k * 32 + lane] = wq[t * 4 + (c ^ ((t >> 1) & 3))];
+            }
+            __syncwarp();
+        }
+        // class bitmaps: the warp's 32 * NBT blocks make NBT words
+        {
+            const long long word0 = ((unit - lane) * NBT) >> 5;
+#pragma unroll
+            for (int w = 0; w < NBT; ++w) {
+                const int blk = w * 32 + lane;               // block of this warp step that lane reports
+                const unsigned xp = __shfl_sync(0xffffffffu, cls_p, blk / NBT);
+                const unsigned xu = __shfl_sync(0xffffffffu, cls_u, blk / NBT);
+                const unsigned wp = __ballot_sync(0xffffffffu, (xp >> (blk % NBT)) & 1u);
+                const unsigned wu = __ballot_sync(0xffffffffu, (xu >> (blk % NBT)) & 1u);
+                if (lane == 0 && word0 + w < n_bm_words) {
+                    pruned_bitmap[word0 + w] = wp;
+                    unified_bitmap[word0 + w] = wu;
+                }
+            }
+        }
+        // candidate list: entries gather in the warp's staging buffer and leave 32 at a time
+#pragma unroll
+        for (int e = 0; e < NBT; ++e) {
+            const bool c = (cand >> e) & 1u;
+            const unsigned bal = __ballot_sync(0xffffffffu, c);
+            if (bal == 0u) continue;
+            if (c) wc[fill + __popc(bal & lt_mask)] = make_uint2((unsigned)(j0 + e), code[e]);
+            fill += __popc(bal);
+            __syncwarp();
+            if (fill >= 32u) {
+                unsigned base = 0;
+                if (lane == 0) base = atomicAdd(&p.work->list_count, 32u);
+                base = __shfl_sync(0xffffffffu, base, 0);
+                fill -= 32u;
+                if (base + 32u <= p.list_cap) p.list[base + lane] = wc[fill + lane];
+                else if (lane == 0) one_pass_fail(p);
+                __syncwarp();
+            }
+        }
+    }
+    if (fill > 0u) {
+        unsigned base = 0;
+        if (lane == 0) base = atomicAdd(&p.work->list_count, fill);
+        base = __shfl_sync(0xffffffffu, base, 0);
+        if (base + fill <= p.list_cap) {
+            if ((unsigned)lane < fill) p.list[base + lane] = wc[lane];
+        } else if (lane == 0) one_pass_fail(p);
+    }
+    // block-level totals of the catch-all bins
+    __shared__ unsigned s_tot[4];
+    if (threadIdx.x < 4) s_tot[threadIdx.x] = 0;
+    __syncthreads();
+    for (int m = 16; m > 0; m >>= 1) {
+        under_p += __shfl_xor_sync(0xffffffffu, under_p, m);
+        over_p += __shfl_xor_sync(0xffffffffu, over_p, m);
+        under_u += __shfl_xor_sync(0xffffffffu, under_u, m);
+        over_u += __shfl_xor_sync(0xffffffffu, over_u, m);
+    }
+    if (lane == 0) {
+        if (under_p) atomicAdd(&s_tot[0], under_p);
+        if (over_p) atomicAdd(&s_tot[1], over_p);
+        if (under_u) atomicAdd(&s_tot[2], under_u);
+        if (over_u) atomicAdd(&s_tot[3], over_u);
+    }
+    if (nonfinite) atomicOr(p.dev_status, (unsigned)MWU_DEV_NONFINITE);
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        if (s_tot[0]) atomicAdd(&hist_p[0], s_tot[0]);
+        if (s_tot[1]) atomicAdd(&hist_p[top], s_tot[1]);
+        if (s_tot[2]) atomicAdd(&hist_u[0], s_tot[2]);
+        if (s_tot[3]) atomicAdd(&hist_u[top], s_tot[3]);
+    }
+}
+
+// Sort the n candidates (global cand_key / cand_idx) and write the threshold element, the r-th
+// smallest (key, index), into the selection.  Run by one whole CTA; false when the counts do
+// not fit (the caller then gives the one-pass result up).
+__device__ bool pick_threshold(const Params &p, Sel *s, u64 r, unsigned n, u64 *c_key, unsigned *c_idx) {
+    const unsigned m = n < (unsigned)CAP ? n : (unsigned)CAP;
+    if (m <= blockDim.x) {
+        // the usual case, a few dozen candidates: every thread ranks its own by counting
+        u64 k = ~0ull;
+        unsigned ix = ~0u;
+        if (threadIdx.x < m) {
+            k = ld_vol(&p.cand_key[threadIdx.x]);
+            ix = ld_vol(&p.cand_idx[threadIdx.x]);
+            c_key[threadIdx.x] = k;
+            c_idx[threadIdx.x] = ix;
+        }
+        __syncthreads();
+        unsigned rank = 0;
+        if (threadIdx.x < m) {
+            for (unsigned t = 0; t < m; ++t) {
+                const u64 x = c_key[t];
+                const unsigned y = c_idx[t];
+                rank += (x < k || (x == k && y < ix)) ? 1u : 0u;
+            }
+        }
+        __syncthreads();
+        if (threadIdx.x < m) { c_key[rank] = k; c_idx[rank] = ix; }
+        __syncthreads();
+    } else {
+        for (int i = threadIdx.x; i < CAP; i += blockDim.x) {
+            c_key[i] = (i < (int)m) ? ld_vol(&p.cand_key[i]) : ~0ull;
+            c_idx[i] = (i < (int)m) ? ld_vol(&p.cand_idx[i]) : ~0u;
+        }
+        __syncthreads();
+        int np2 = 2;
+        while (np2 < (int)m) np2 <<= 1;
+        sort_candidates(c_key, c_idx, np2);
+    }
+    const bool ok = n <= (unsigned)CAP && r >= 1 && r <= (u64)m;
+    if (threadIdx.x == 0 && ok) {
+        s->T_key = c_key[r - 1];
+        s->T_idx = (u64)c_idx[r - 1];
+    }
+    return ok;
+}
+
+// list_select_kernel: exact prune threshold; the L_u histogram gains the listed blocks that
+// survive pruning; the unify threshold bin.
+template <int B>
+__global__ void __launch_bounds__(FIN_THREADS) list_select_kernel(Params p) {
+    if (p.work->failed != 0u) return;
+    Sel *sp = &p.work->sel[0];
+    Sel *su = &p.work->sel[1];
+    const unsigned mode_p = sp->mode, mode_u = su->mode;
+    if (mode_p != 0u && mode_u != 0u) return;
+    __shared__ u64 c_key[CAP];
+    __shared__ unsigned c_idx[CAP];
+    __shared__ BinSel s_sel;
+    const unsigned nb = (unsigned)p.nb, top = nb - 1u;
+    unsigned *hist_u = p.fhist + p.nb;
+    const u64 ulo = su->lo0, uhi = su->hi0;
+    const unsigned ush = su->shift0;
+    if (threadIdx.x == 0) { s_sel.B = 0; s_sel.r = 0; s_sel.cnt = 0; s_sel.lo_hi = s_sel.lo_lo = s_sel.hi_hi = s_sel.hi_lo = 0; }
+    __syncthreads();
+    if (mode_p == 0u) select_bin(p, sp, p.fhist, &s_sel, blockIdx.x == 0);   // every CTA computes the same values
+    const unsigned Bp = s_sel.B;
+    const u64 r_p = s_sel.r;
+    // the threshold bin must be a real bin of the window and small enough to sort
+    const bool hit_p = mode_p != 0u || (Bp >= 1u && Bp <= nb - 2u && s_sel.cnt <= (u64)CAP);
+    unsigned under = 0, over = 0;
+    if (mode_p == 0u && hit_p) {
+        const u128 lo0 = from_halves(s_sel.lo_hi, s_sel.lo_lo);
+        const u128 hi0 = from_halves(s_sel.hi_hi, s_sel.hi_lo);
+        const unsigned n_list = min(p.work->list_count, p.list_cap);
+        for (unsigned i = blockIdx.x * blockDim.x + threadIdx.x; i < n_list; i += gridDim.x * blockDim.x) {
+            const uint2 e = __ldg(&p.list[i]);
+            const unsigned bp = e.y & 0xffffu, bu = e.y >> 16;
+            if (bp == 0u || bp == top) continue;          // not in the prune window: counted by pass_kernel
+            if (bp < Bp) continue;                        // pruned
+            if (bp == Bp) {                               // decided by the last CTA
+                const u64 key = exact_key<B>(p, (long long)e.x, 0);
+                const u128 c = make_c(key, (u64)e.x);
+                if (c >= lo0 && c < hi0) {
+                    const unsigned slot = atomicAdd(&p.work->fcand_count[0], 1u);
+                    if (slot < (unsigned)CAP) { p.cand_key[slot] = key; p.cand_idx[slot] = e.x; }
+                }
+                continue;
+            }
+            if (mode_u != 0u) continue;
+            if (bu == 0u) ++under;
+            else if (bu == top) ++over;
+            else atomicAdd(&hist_u[bu], 1u);
+        }
+    }
+    for (int m = 16; m > 0; m >>= 1) {
+        under += __shfl_xor_sync(0xffffffffu, under, m);
+        over += __shfl_xor_sync(0xffffffffu, over, m);
+    }
+    if ((threadIdx.x & 31) == 0) {
+        if (under) atomicAdd(&hist_u[0], under);
+        if (over) atomicAdd(&hist_u[top], over);
+    }
+    if (!last_block_done(&p.work->fticket[0])) return;
+
+    // ---- last CTA only ----
+    if (mode_p == 0u) {
+        bool ok = hit_p;
+        const unsigned m = ld_vol(&p.work->fcand_count[0]);
+        if (ok) ok = pick_threshold(p, sp, r_p, m, c_key, c_idx);
+        if (!ok) {
+            if (threadIdx.x == 0) one_pass_fail(p);
+            return;
+        }
+        // the blocks of the threshold bin that survive join the L_u histogram
+        if (mode_u == 0u) {
+            for (unsigned i = (unsigned)r_p + threadIdx.x; i < m; i += blockDim.x) {
+                const u64 ku = exact_key<B>(p, (long long)c_idx[i], 1);
+                atomicAdd(&hist_u[bin_of(ku, ulo, uhi, ush, nb)], 1u);
+            }
+        }
+        __threadfence();
+        __syncthreads();
+    }
+    if (mode_u == 0u) {
+        select_bin(p, su, hist_u, &s_sel, true);
+        if (threadIdx.x == 0 && !(s_sel.B >= 1u && s_sel.B <= nb - 2u && s_sel.cnt <= (u64)CAP)) one_pass_fail(p);
+    }
+}
+
+// Final class of block j against what pass_kernel wrote (read back from the bitmaps); the
+// block's outputs are rewritten where they differ.
+template <int B>
+__device__ __forceinline__ void apply_class(const Params &p, float *Q, float *u_out, unsigned *pruned_bitmap,
+                                            unsigned *unified_bitmap, unsigned idx, bool pr, bool un) {
+    const unsigned bit = 1u << (idx & 31u);
+    unsigned *wp = pruned_bitmap + (idx >> 5), *wu = unified_bitmap + (idx >> 5);
+    const bool pr0 = (ld_vol(wp) & bit) != 0u, un0 = (ld_vol(wu) & bit) != 0u;
+    if (pr == pr0 && un == un0) return;
+    if (pr != pr0) { if (pr) atomicOr(wp, bit); else atomicAnd(wp, ~bit); }
+    if (un != un0) { if (un) atomicOr(wu, bit); else atomicAnd(wu, ~bit); }
+    const long long j = (long long)idx;
+    float v[B];
+    load_block<B>(p.W, p.U, j, v);
+    double S, Lu, Kp;
+    block_keys<B>(v, p.use_l1, &S, &Lu, &Kp);
+    const float qf = __double2float_rn(__dmul_rn(S, 1.0 / (double)B));
+    u_out[j] = un ? qf : 0.f;
+    if (Q) {
+#pragma unroll
+        for (int l = 0; l < B; ++l) Q[j * B + l] = pr ? 0.f : (un ? (v[l] < 0.f ? -qf : qf) : v[l]);
+    }
+}
+
+// list_finish_kernel: every listed block outside the unify threshold bin gets its final class at
+// once; the blocks inside it are sorted by the last CTA, which fixes the threshold element and
+// their classes.
+template <int B>
+__global__ void __launch_bounds__(FIN_THREADS) list_finish_kernel(Params p, float *Q, float *u_out,
+                                                                  unsigned *pruned_bitmap,
+                                                                  unsigned *unified_bitmap) {
+    // everything read here was written by earlier kernels: plain loads
+    if (p.work->failed != 0u) return;
+    Sel *su = &p.work->sel[1];
+    __shared__ u64 c_key[CAP];
+    __shared__ unsigned c_idx[CAP];
+    const SelView vp = view_of(&p.work->sel[0]);
+    const unsigned mode_u = su->mode;
+    const unsigned Bu = su->B;
+    const u64 r_u = su->r;
+    const u128 lo = from_halves(su->lo_hi, su->lo_lo);
+    const u128 hi = from_halves(su->hi_hi, su->hi_lo);
+    const unsigned n_list = min(p.work->list_count, p.list_cap);
+    for (unsigned i = blockIdx.x * blockDim.x + threadIdx.x; i < n_list; i += gridDim.x * blockDim.x) {
+        const uint2 e = __ldg(&p.list[i]);
+        const unsigned bu = e.y >> 16;
+        const bool pr = selected<B>(p, vp, (long long)e.x, e.y & 0xffffu, 0);
+        bool un = false;
+        if (!pr) {
+            if (mode_u == 2u) un = true;
+            else if (mode_u == 0u) {
+                if (bu == Bu) {                            // decided by the last CTA
+                    const u64 key = exact_key<B>(p, (long long)e.x, 1);
+                    const u128 c = make_c(key, (u64)e.x);
+                    if (c >= lo && c < hi) {
+                        const unsigned slot = atomicAdd(&p.work->fcand_count[1], 1u);
+                        if (slot < (unsigned)CAP) { p.cand_key[slot] = key; p.cand_idx[slot] = e.x; }
+                        continue;
+                    }
+                    un = c < lo;
+                } else un = bu < Bu;
+            }
+        }
+        apply_class<B>(p, Q, u_out, pruned_bitmap, unified_bitmap, e.x, pr, un);
+    }
+    if (mode_u != 0u) return;
+    if (!last_block_done(&p.work->fticket[1])) return;
+
+    // ---- last CTA only ----
+    const unsigned m = ld_vol(&p.work->fcand_count[1]);
+    if (!pick_threshold(p, su, r_u, m, c_key, c_idx)) {
+        if (threadIdx.x == 0) one_pass_fail(p);
+        return;
+    }
+    const unsigned r = (unsigned)r_u;
+    for (unsigned i = threadIdx.x; i < m; i += blockDim.x)
+        apply_class<B>(p, Q, u_out, pruned_bitmap, unified_bitmap, c_idx[i], false, i < r);
+}
+
 }  // namespace proj
 
 // ---------------------------------------------------------------------------------------------
 // host side
 // ---------------------------------------------------------------------------------------------
 static size_t ws_off_hist() { return align_up(sizeof(proj::Work)); }
-static size_t ws_off_cand_key() { return align_up(ws_off_hist() + 3 * proj::NB_MAX * sizeof(unsigned)); }
+static size_t ws_off_cand_key() { return align_up(ws_off_hist() + 5 * proj::NB_MAX * sizeof(unsigned)); }
 static size_t ws_off_cand_idx() { return align_up(ws_off_cand_key() + proj::CAP * sizeof(proj::u64)); }
 static size_t ws_off_bins() { return align_up(ws_off_cand_idx() + proj::CAP * sizeof(unsigned)); }
+static size_t ws_off_list(size_t mb) { return align_up(ws_off_bins() + (mb + 8) * sizeof(unsigned)); }
+// candidate list of the one-pass pipeline: a quarter of the blocks (the windows hold a few per cent)
+static size_t list_capacity(size_t mb) { return mb / 4 + 4096; }
+
+static bool use_one_pass(const mwu_proj_desc *desc) {
+    if (desc->algo == MWU_ALGO_ONE_PASS) return true;
+    if (desc->algo == MWU_ALGO_MULTI_PASS) return false;
+    return desc->rows * desc->cols / desc->block >= proj::ONE_PASS_MIN_BLOCKS;
+}
 
 }  // namespace mwu
 
 extern "C" size_t mwu_project_workspace_bytes(const mwu_proj_desc *desc) {
     if (mwu::validate_desc(desc, false) != MWU_OK) return 0;
     const size_t mb = (size_t)(desc->rows * desc->cols / desc->block);
-    return mwu::align_up(mwu::ws_off_bins() + (mb + 8) * sizeof(unsigned));
+    return mwu::align_up(mwu::ws_off_list(mb) + mwu::list_capacity(mb) * sizeof(uint2));
 }
 
 template <int B>
 static cudaError_t launch_project(const mwu::proj::Params &p, const mwu_proj_desc *desc, float *Q,
                                   float *u, unsigned *pb, unsigned *ub, unsigned *sb, double *loss_u,
-                                  double *loss_p, int sm_count, cudaStream_t st) {
+                                  double *loss_p, int sm_count, bool one_pass, cudaStream_t st) {
     using namespace mwu::proj;
-    sample_kernel<B><<<1, NSAMP, 0, st>>>(p, desc->k_unify, desc->k_prune);
+    sample_kernel<B><<<1, SAMP_THREADS, 0, st>>>(p, desc->k_unify, desc->k_prune);
     const long long n_units = (p.n_floats + 15) / 16;
     const long long want = (n_units + 255) / 256;
     const long long cap_blocks = (long long)sm_count * 8;
-    const int grid_stream = (int)(want < cap_blocks ? (want > 0 ? want : 1) : cap_blocks);
-    stats_kernel<B><<<grid_stream, 256, 0, st>>>(p, loss_u, loss_p, u, sb);
-
+    int grid_stream = (int)(want < cap_blocks ? (want > 0 ? want : 1) : cap_blocks);
     const long long mb = p.n_blocks;
-    const long long rb = (mb + 4 * FIN_THREADS - 1) / (4 * FIN_THREADS);
-    const int grid_fin = (int)(rb < (long long)sm_count ? (rb > 0 ? rb : 1) : (long long)sm_count);
     const bool need_p = desc->k_prune > 0 && desc->k_prune < mb;
     const long long ksel_u = desc->k_unify - desc->k_prune;
     const bool need_u = ksel_u > 0 && ksel_u < mb - desc->k_prune;
+
+    if (one_pass) {
+        pass_kernel<B><<<grid_stream, 256, 0, st>>>(p, Q, loss_u, loss_p, u, pb, ub, sb);
+        if (!need_p && !need_u) return cudaGetLastError();       // no threshold: every class is final
+        // the list holds a few per cent of the blocks
+        const long long lb = (mb / 8 + FIN_THREADS - 1) / FIN_THREADS;      // a thread per expected entry
+        // one CTA per SM at most: 1024 threads of 64 registers fill an SM's register file, a second
+        // CTA would only start when the first has ended
+        const int grid_list = (int)(lb < (long long)sm_count ? (lb > 0 ? lb : 1) : (long long)sm_count);
+        list_select_kernel<B><<<grid_list, FIN_THREADS, 0, st>>>(p);
+        list_finish_kernel<B><<<grid_list, FIN_THREADS, 0, st>>>(p, Q, u, pb, ub);
+    }
+    // multi-pass kernels: the whole projection, or (gated) the fallback of the one-pass pipeline.
+    // As a fallback they are needed once in thousands of calls and normally return at once, so
+    // they get one small wave of CTAs (every loop is grid-strided).
+    const int grid_fb = (int)(grid_stream < 2 * sm_count ? grid_stream : 2 * sm_count);
+    if (one_pass) grid_stream = grid_fb;
+    stats_kernel<B><<<grid_stream, 256, 0, st>>>(p, loss_u, loss_p, u, sb);
+    const long long rb = (mb + 4 * FIN_THREADS - 1) / (4 * FIN_THREADS);
+    const int grid_fin = (int)(rb < (long long)sm_count ? (rb > 0 ? rb : 1) : (long long)sm_count);
     if (need_p || need_u) prune_select_kernel<B><<<grid_fin, FIN_THREADS, 0, st>>>(p);
     if (need_u) collect_kernel<1, B><<<grid_fin, FIN_THREADS, 0, st>>>(p);
     emit_kernel<B><<<grid_stream, 256, 0, st>>>(p, Q, u, pb, ub, sb);
@@ -1014,6 +1702,7 @@ extern "C" int mwu_project(const mwu_proj_desc *desc, const float *W, const floa
 
     cudaStream_t st = (cudaStream_t)cuda_stream;
     char *ws = (char *)workspace;
+    const bool one_pass = use_one_pass(desc);
     proj::Params p;
     p.W = W;
     p.U = U_dual;
@@ -1022,21 +1711,25 @@ extern "C" int mwu_project(const mwu_proj_desc *desc, const float *W, const floa
     p.b = desc->block;
     p.use_l1 = desc->prune_key == MWU_PRUNE_KEY_L1;
     p.work = (proj::Work *)ws;
+    p.nb = p.n_blocks <= (8ll << 20) ? proj::NB_SMALL : proj::NB_MAX;
     p.hist = (unsigned *)(ws + ws_off_hist());
+    p.fhist = p.hist + 3 * (size_t)p.nb;
     p.cand_key = (proj::u64 *)(ws + ws_off_cand_key());
     p.cand_idx = (unsigned *)(ws + ws_off_cand_idx());
     p.bins = (unsigned *)(ws + ws_off_bins());
+    p.list = (uint2 *)(ws + ws_off_list((size_t)p.n_blocks));
+    p.list_cap = (unsigned)list_capacity((size_t)p.n_blocks);
+    p.gated = one_pass ? 1 : 0;
     p.dev_status = dev_status;
 
-    p.nb = p.n_blocks <= (8ll << 20) ? proj::NB_SMALL : proj::NB_MAX;
-    if (cudaMemsetAsync(ws, 0, ws_off_hist() + 3 * (size_t)p.nb * sizeof(unsigned), st) != cudaSuccess)
+    if (cudaMemsetAsync(ws, 0, ws_off_hist() + 5 * (size_t)p.nb * sizeof(unsigned), st) != cudaSuccess)
         return MWU_ERR_CUDA;
     cudaError_t e;
     switch (desc->block) {
-        case 2: e = launch_project<2>(p, desc, Q, u, pruned_bitmap, unified_bitmap, sign_bits, loss_u, loss_p, sm_count, st); break;
-        case 4: e = launch_project<4>(p, desc, Q, u, pruned_bitmap, unified_bitmap, sign_bits, loss_u, loss_p, sm_count, st); break;
-        case 8: e = launch_project<8>(p, desc, Q, u, pruned_bitmap, unified_bitmap, sign_bits, loss_u, loss_p, sm_count, st); break;
-        default: e = launch_project<16>(p, desc, Q, u, pruned_bitmap, unified_bitmap, sign_bits, loss_u, loss_p, sm_count, st); break;
+        case 2: e = launch_project<2>(p, desc, Q, u, pruned_bitmap, unified_bitmap, sign_bits, loss_u, loss_p, sm_count, one_pass, st); break;
+        case 4: e = launch_project<4>(p, desc, Q, u, pruned_bitmap, unified_bitmap, sign_bits, loss_u, loss_p, sm_count, one_pass, st); break;
+        case 8: e = launch_project<8>(p, desc, Q, u, pruned_bitmap, unified_bitmap, sign_bits, loss_u, loss_p, sm_count, one_pass, st); break;
+        default: e = launch_project<16>(p, desc, Q, u, pruned_bitmap, unified_bitmap, sign_bits, loss_u, loss_p, sm_count, one_pass, st); break;
     }
     return e == cudaSuccess ? MWU_OK : MWU_ERR_CUDA;
 }

@@ -10,9 +10,9 @@ from paper_2106_08301_b200 import inputs
 pytestmark = pytest.mark.gpu
 
 
-def run_project(W, b, ku, kp, U=None, prune_key=0, want_loss=True):
+def run_project(W, b, ku, kp, U=None, prune_key=0, want_loss=True, algo=B.MWU_ALGO_AUTO):
     rows, cols = W.shape
-    desc = B.make_desc(rows, cols, b, ku, kp, prune_key)
+    desc = B.make_desc(rows, cols, b, ku, kp, prune_key, algo)
     bufs = B.ProjectionBuffers(desc, want_q=True, want_loss=want_loss)
     Wd = W.cuda().contiguous()
     Ud = U.cuda().contiguous() if U is not None else None
@@ -21,11 +21,20 @@ def run_project(W, b, ku, kp, U=None, prune_key=0, want_loss=True):
     return desc, bufs, Wd, Ud
 
 
-def check_against_oracle(W, b, ku, kp, U=None, prune_key=0):
-    desc, bufs, Wd, Ud = run_project(W, b, ku, kp, U, prune_key)
-    assert int(bufs.dev_status.item()) == 0
+def check_against_oracle(W, b, ku, kp, U=None, prune_key=0, algos=None):
+    """Both kernel pipelines of mwu_project (one pass with correction, multi pass) against the
+    CPU checker; returns the buffers of the last one."""
     p = O.project(W.numpy(), b, ku, kp, U=None if U is None else U.numpy(),
                   prune_key="l1" if prune_key else "l2sq")
+    out = None
+    for algo in (algos or (B.MWU_ALGO_MULTI_PASS, B.MWU_ALGO_ONE_PASS)):
+        out = compare_with(p, W, b, ku, kp, U, prune_key, algo)
+    return out + (p,)
+
+
+def compare_with(p, W, b, ku, kp, U, prune_key, algo):
+    desc, bufs, Wd, Ud = run_project(W, b, ku, kp, U, prune_key, algo=algo)
+    assert int(bufs.dev_status.item()) == 0
     # keys: bit-exact fp64
     lu = bufs.loss_u.cpu().numpy()
     lp = bufs.loss_p.cpu().numpy()
@@ -45,7 +54,7 @@ def check_against_oracle(W, b, ku, kp, U=None, prune_key=0):
     assert np.array_equal(u, p.u)
     Q = bufs.Q.cpu().numpy().reshape(W.shape)
     assert np.array_equal(Q.view(np.uint32), p.Q.view(np.uint32))
-    return desc, bufs, Wd, Ud, p
+    return desc, bufs, Wd, Ud
 
 
 @pytest.mark.parametrize("b", [2, 4, 8, 16])
@@ -156,3 +165,37 @@ def test_pack_with_dual_and_structured_pruning():
     rec = ref[h["off_rec"]:h["off_rec"] + 16 * 9].view(np.uint32).reshape(-1, 4)
     assert rec[1, 3] == 0 and rec[5, 3] == 0          # stage 1 of both row tiles is dead
     assert rec[0, 3] == 0xF
+
+
+@pytest.mark.parametrize("b,rows,cols,permille", [(16, 1000, 4112, (800, 600)), (4, 517, 1028, (500, 250)),
+                                                  (2, 300, 1002, (350, 250)), (8, 2048, 1024, (1000, 900)),
+                                                  (8, 640, 1032, (100, 0)), (16, 777, 2064, (700, 700))])
+def test_projection_parity_medium_auto(b, rows, cols, permille):
+    """Sizes above the switch to the one-pass pipeline (default algo), ragged against every tile."""
+    W = inputs.normal_weights(rows, cols, 0.02, 4321 + b)
+    Mb = rows * cols // b
+    assert Mb >= 32768
+    check_against_oracle(W, b, O.count_from_permille(Mb, permille[0]), O.count_from_permille(Mb, permille[1]),
+                         algos=(B.MWU_ALGO_AUTO,))
+
+
+def test_projection_medium_reprojection_falls_back():
+    """Projecting a projected tensor: thousands of exactly equal keys (0 for pruned blocks and for
+    the L_u of unified ones), so no sample window can isolate the threshold and the one-pass
+    pipeline must hand over to the multi-pass kernels."""
+    W = inputs.normal_weights(512, 2048, 0.02, 17)
+    b = 16
+    Mb = W.numel() // b
+    ku, kp = Mb * 8 // 10, Mb * 6 // 10
+    desc, bufs, Wd, _, p = check_against_oracle(W, b, ku, kp, algos=(B.MWU_ALGO_AUTO,))
+    Q1 = bufs.Q.clone().reshape(512, 2048).cpu()
+    desc2, bufs2, _, _, p2 = check_against_oracle(Q1, b, ku, kp, algos=(B.MWU_ALGO_AUTO,))
+    assert torch.equal(bufs2.Q.cpu().view(torch.int32), Q1.reshape(-1).view(torch.int32))
+
+
+def test_projection_one_pass_with_dual_and_l1():
+    W = inputs.normal_weights(512, 1024, 0.02, 31)
+    U = inputs.normal_weights(512, 1024, 0.004, 32)
+    Mb = 512 * 1024 // 4
+    check_against_oracle(W, 4, Mb * 6 // 10, Mb * 3 // 10, U=U, algos=(B.MWU_ALGO_AUTO,))
+    check_against_oracle(W, 4, Mb * 6 // 10, Mb * 3 // 10, prune_key=1, algos=(B.MWU_ALGO_AUTO,))
