@@ -239,7 +239,8 @@ __device__ __forceinline__ void load16(const float *W, const float *U, long long
 // ---------------------------------------------------------------------------------------------
 __device__ __forceinline__ void set_window(Sel *s, u64 lo, u64 hi, int nb) {
     if (hi < lo) hi = lo;
-    unsigned shift = 0;
+    const int width = 64 - __clzll((long long)(hi - lo));
+    unsigned shift = width > 16 ? (unsigned)(width - 16) : 0u;         // nb - 2 < 2^16: start just below
     while (((hi - lo) >> shift) >= (u64)(nb - 2)) ++shift;
     s->lo0 = lo;
     s->hi0 = hi;
@@ -316,14 +317,15 @@ __device__ void sample_select(const u64 (&key)[SAMP_PER], const bool (&valid)[SA
     int il, ih, ipos;
     window_ranks_f(na, frac, &il, &ih, &ipos);
     {
-        // four threads rank one level-A key, each against a quarter of the keys
+        // four threads rank one level-A key, each against a quarter of the keys (every fourth
+        // group of four: the four threads read 64 contiguous bytes, no bank conflict)
         const int part = tid % 4;
         const unsigned k = s_a[a];
         int r = 0;
-        const uint4 *q = reinterpret_cast<const uint4 *>(s_a + part * (NA / 4));
+        const uint4 *q = reinterpret_cast<const uint4 *>(s_a) + part;
 #pragma unroll 4
         for (int t = 0; t < NA / 16; ++t) {
-            const uint4 x = q[t];
+            const uint4 x = q[4 * t];
             r += (x.x < k ? 1 : 0) + (x.y < k ? 1 : 0) + (x.z < k ? 1 : 0) + (x.w < k ? 1 : 0);
         }
         r += __shfl_xor_sync(0xffffffffu, r, 1);
@@ -341,8 +343,10 @@ __device__ void sample_select(const u64 (&key)[SAMP_PER], const bool (&valid)[SA
     if (s_edge[0] == 0xffffffffu) clo = ~0ull >> 1;
     if (s_edge[1] == 0xffffffffu) chi = ~0ull >> 1;
     if (chi < clo) chi = clo;
-    unsigned shift = 0;
-    while (((chi - clo) >> shift) >= (u64)SAMP_THREADS) ++shift;
+    // smallest shift with ((chi - clo) >> shift) < SAMP_THREADS (a power of two)
+    const int width = 64 - __clzll((long long)(chi - clo));            // bits of chi - clo
+    const unsigned shift = width > 10 ? (unsigned)(width - 10) : 0u;
+    static_assert(SAMP_THREADS == 1024, "ten bits of bin index");
     // level B
     unsigned n_under = 0, n_over = 0;                 // the two catch-all counts stay in registers
 #pragma unroll
@@ -1204,35 +1208,33 @@ __global__ void __launch_bounds__(256) pass_kernel(Params p, float *Q, double *l
     const unsigned lt_mask = (1u << lane) - 1u;
     unsigned fill = 0;                                   // warp-uniform
     unsigned under_p = 0, over_p = 0, under_u = 0, over_u = 0, nonfinite = 0;
+    // fewer than 2^31 blocks of at least two values: units (16 values) and blocks count in 32 bits
     const long long n = p.n_floats;
-    const long long n_units = (n + 15) / 16;
-    const long long n_iter = (n_units + 31) / 32 * 32;   // whole warps take part in every step
-    const long long n_bm_words = (p.n_blocks + 31) / 32;
-    const long long ustride = (long long)gridDim.x * blockDim.x;
-    long long unit = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    const unsigned n_units = (unsigned)((n + 15) / 16);
+    const unsigned n_iter = (n_units + 31u) / 32u * 32u;  // whole warps take part in every step
+    const unsigned n_blocks = (unsigned)p.n_blocks;
+    const unsigned n_bm_words = (n_blocks + 31u) / 32u;
+    const unsigned ustride = gridDim.x * blockDim.x;
+    unsigned unit = blockIdx.x * blockDim.x + threadIdx.x;
     float nxt[16];
 #pragma unroll
     for (int l = 0; l < 16; ++l) nxt[l] = 0.f;
-    if (unit < n_units) load16(p.W, p.U, unit * 16, n, nxt);
+    if (unit < n_units) load16(p.W, p.U, (long long)unit * 16, n, nxt);
     for (; unit < n_iter; unit += ustride) {
         float v[16];
 #pragma unroll
         for (int l = 0; l < 16; ++l) v[l] = nxt[l];
         // the next unit's 64 bytes travel while this one is evaluated
-        if (unit + ustride < n_units) load16(p.W, p.U, (unit + ustride) * 16, n, nxt);
+        if (unit + ustride < n_units) load16(p.W, p.U, (long long)(unit + ustride) * 16, n, nxt);
         else {
 #pragma unroll
             for (int l = 0; l < 16; ++l) nxt[l] = 0.f;
         }
         const bool live = unit < n_units;
-        const bool warp_full = (unit - lane + 32) * 16 <= n;      // all 512 floats of this warp step exist
-        unsigned ex = 0, sb = 0;
+        const bool warp_full = (long long)(unit - lane + 32u) * 16 <= n;      // all 512 floats of this warp step exist
+        unsigned sb = 0;
 #pragma unroll
-        for (int l = 0; l < 16; ++l) {
-            ex = max(ex, __float_as_uint(v[l]) & 0x7fffffffu);
-            sb |= (v[l] < 0.f ? 1u : 0u) << l;
-        }
-        nonfinite |= (ex >= 0x7f800000u) ? 1u : 0u;
+        for (int l = 0; l < 16; ++l) sb |= (v[l] < 0.f ? 1u : 0u) << l;
         if (live) {
             unsigned short *halves = reinterpret_cast<unsigned short *>(sign_bits);
             halves[unit] = (unsigned short)sb;
@@ -1241,19 +1243,21 @@ __global__ void __launch_bounds__(256) pass_kernel(Params p, float *Q, double *l
         unsigned cls_p = 0, cls_u = 0, cand = 0;             // bit e: block e of this thread
         unsigned code[NBT];
         float uo[NBT];
-        const long long j0 = unit * NBT;
+        const unsigned j0 = unit * NBT;
 #pragma unroll
         for (int e = 0; e < NBT; ++e) {
             double S, Lu, Kp;
             block_keys<B>(v + e * B, p.use_l1, &S, &Lu, &Kp);
             const float qf = __double2float_rn(__dmul_rn(S, 1.0 / (double)B));
+            // S = sum |v| is Inf or NaN exactly when some value of the block is
+            nonfinite |= ((unsigned)__double2hiint(S) >= 0x7ff00000u) ? 1u : 0u;
             const u64 kpb = key_bits(Kp), kub = key_bits(Lu);
             const unsigned bp = bin_of(kpb, plo, phi, psh, nb);
             const unsigned bu = bin_of(kub, ulo, uhi, ush, nb);
             code[e] = bp | (bu << 16);
             uo[e] = 0.f;
-            const long long j = j0 + e;
-            if (j < p.n_blocks) {
+            const unsigned j = j0 + e;
+            if (j < n_blocks) {
                 if (loss_u) loss_u[j] = Lu;
                 if (loss_p) loss_p[j] = Kp;
                 bool pr, survives, open = false;
@@ -1280,7 +1284,7 @@ __global__ void __launch_bounds__(256) pass_kernel(Params p, float *Q, double *l
             }
         }
         if (live) {
-            if (j0 + NBT <= p.n_blocks) {
+            if (j0 + NBT <= n_blocks) {
                 if (NBT == 1) u_out[j0] = uo[0];
                 else if (NBT == 2) *reinterpret_cast<float2 *>(u_out + j0) = make_float2(uo[0], uo[1 % NBT]);
                 else {
@@ -1292,20 +1296,24 @@ __global__ void __launch_bounds__(256) pass_kernel(Params p, float *Q, double *l
             } else {
 #pragma unroll
                 for (int e = 0; e < NBT; ++e)
-                    if (j0 + e < p.n_blocks) u_out[j0 + e] = uo[e];
+                    if (j0 + e < n_blocks) u_out[j0 + e] = uo[e];
             }
             if (Q) {
+                // q = v (kept), +-u (unified: magnitude u, sign from the sign plane bits), or +0
                 float q[16];
 #pragma unroll
                 for (int e = 0; e < NBT; ++e) {
                     const bool pr = (cls_p >> e) & 1u, un = (cls_u >> e) & 1u;
+                    const unsigned keep = (pr || un) ? 0u : 0xffffffffu;
+                    const unsigned mag = un ? __float_as_uint(uo[e]) : 0u;
+                    const unsigned sgn = un ? 0x80000000u : 0u;
 #pragma unroll
                     for (int l = 0; l < B; ++l) {
-                        const float x = v[e * B + l];
-                        q[e * B + l] = pr ? 0.f : (un ? (x < 0.f ? -uo[e] : uo[e]) : x);
+                        const int k = e * B + l;
+                        q[k] = __uint_as_float((__float_as_uint(v[k]) & keep) | mag | ((sb << (31 - k)) & sgn));
                     }
                 }
-                const long long f = unit * 16;
+                const long long f = (long long)unit * 16;
                 if (!warp_full) {
                     if (f + 16 <= n) {
                         float4 *dst = reinterpret_cast<float4 *>(Q + f);
@@ -1329,7 +1337,7 @@ __global__ void __launch_bounds__(256) pass_kernel(Params p, float *Q, double *l
         // piece c at slot c ^ ((t >> 1) & 3), so neither side has bank conflicts.
         if (Q && warp_full) {
             __syncwarp();
-            float4 *dst = reinterpret_cast<float4 *>(Q + (unit - lane) * 16);
+            float4 *dst = reinterpret_cast<float4 *>(Q + (long long)(unit - lane) * 16);
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
                 const int t = 8 * k + (lane >> 2), c = lane & 3;
@@ -1339,7 +1347,7 @@ __global__ void __launch_bounds__(256) pass_kernel(Params p, float *Q, double *l
         }
         // class bitmaps: the warp's 32 * NBT blocks make NBT words
         {
-            const long long word0 = ((unit - lane) * NBT) >> 5;
+            const unsigned word0 = ((unit - lane) * NBT) >> 5;
 #pragma unroll
             for (int w = 0; w < NBT; ++w) {
                 const int blk = w * 32 + lane;               // block of this warp step that lane reports
@@ -1359,7 +1367,7 @@ __global__ void __launch_bounds__(256) pass_kernel(Params p, float *Q, double *l
             const bool c = (cand >> e) & 1u;
             const unsigned bal = __ballot_sync(0xffffffffu, c);
             if (bal == 0u) continue;
-            if (c) wc[fill + __popc(bal & lt_mask)] = make_uint2((unsigned)(j0 + e), code[e]);
+            if (c) wc[fill + __popc(bal & lt_mask)] = make_uint2(j0 + e, code[e]);
             fill += __popc(bal);
             __syncwarp();
             if (fill >= 32u) {
