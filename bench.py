@@ -30,8 +30,11 @@ from paper_2106_08301_b200 import inputs, replicas  # noqa: E402
 
 METRIC = "mwu_hot_path_effective_tflops"
 UNIT = "TFLOP/s"
-KERNELS_PER_STEP = 9      # sample, stats, prune_select, collect, emit | count, scan, fill | gemm
-KERNELS_PER_STEP_WS = 10  # ... | decode, dense gemm (with a workspace and enough activation rows)
+# launches per step: sample, pass, list_select, list_finish, then the four multi-pass kernels that
+# return at once unless the one-pass result was given up (stats, prune_select, collect, emit)
+# | count, scan, fill | gemm
+KERNELS_PER_STEP = 12
+KERNELS_PER_STEP_WS = 13  # ... | decode, dense gemm (with a workspace and enough activation rows)
 
 
 def measured_peaks():
@@ -161,8 +164,8 @@ def cpu_threads():
 
 
 def oracle_sample_sizes(wl):
-    # about 10-30 s of CPU work on the default workload: half of the weight rows, 1024 activation rows
-    return max(128, wl.rows // 2), min(1024, max(1, wl.m))
+    # about 10-30 s of CPU work on the default workload: all weight rows, up to 8192 activation rows
+    return wl.rows, min(8192, max(1, wl.m))
 
 
 def run_reference(args):
@@ -346,9 +349,10 @@ def run_gpu(args):
             "peak_source": peaks["source"] + " (sustained cuBLAS bf16)",
             "algorithmic_flops_per_launch": flops,
             # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the two-operand GEMM kernel
-            # (615.2 MB + 252.9 MB, ncu capture of this workload; see profiles/step_kernels_c4_ffn.md);
+            # (627.9 MB + 252.9 MB, ncu capture of this workload; see profiles/step_kernels_c4_ffn.md);
             # not taken for other workloads or for the fused path
-            "traffic": 868.1e6 if (ws_bytes and wl.name == "c4_ffn" and m == wl.m) else None,
+            "traffic": 880.8e6 if (ws_bytes and wl.name == "c4_ffn" and m == wl.m) else None,
+            # the whole mwu_project call (eight launches) against the 8 bytes per weight the method needs
             "projection": {"bound": "hbm", "achieved": abytes["projection"] / (proj_ms * 1e-3) / 1e9,
                            "peak": peaks["hbm_gbs"], "unit": "GB/s",
                            "frac": abytes["projection"] / (proj_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]},

@@ -395,6 +395,13 @@ __device__ void sample_select(const u64 (&key)[SAMP_PER], const bool (&valid)[SA
     __syncthreads();
 }
 
+// block of the i-th of ns evenly spaced samples: i * mb / ns without a division (ns is either
+// NSAMP, a power of two, or mb itself); i < 2^12 and mb < 2^31, so the product fits 64 bits
+__device__ __forceinline__ long long sample_block(int i, long long mb, int ns) {
+    static_assert((NSAMP & (NSAMP - 1)) == 0, "NSAMP is a power of two");
+    return ns == NSAMP ? (long long)(((u64)i * (u64)mb) / (u64)NSAMP) : (long long)i;
+}
+
 template <int B>
 __global__ void __launch_bounds__(SAMP_THREADS) sample_kernel(Params p, long long k_unify, long long k_prune) {
     const long long mb = p.n_blocks;
@@ -408,7 +415,7 @@ __global__ void __launch_bounds__(SAMP_THREADS) sample_kernel(Params p, long lon
         ku[t] = ~0ull;
         valid[t] = i < ns;
         if (i < ns) {
-            const long long j = (long long)(((u64)i * (u64)mb) / (u64)ns);     // i < 2^12, mb < 2^31
+            const long long j = sample_block(i, mb, ns);
             double S, Lu, Kp;
             block_keys_at<B>(p.W, p.U, j, p.use_l1, &S, &Lu, &Kp);
             kp[t] = key_bits(Kp);
@@ -463,8 +470,16 @@ __device__ void scan_hist(const unsigned *hist, int nb, u64 r, unsigned *bin_out
     __shared__ u64 s_part[32];
     const int PER = nb / FIN_THREADS;
     u64 sum = 0;
+    unsigned mine8[8];                                       // this thread's bins when there are eight of them
+    if (PER == 8) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) mine8[i] = ld_vol(&hist[threadIdx.x * 8 + i]);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) sum += mine8[i];
+    } else {
 #pragma unroll 8
-    for (int i = 0; i < PER; ++i) sum += ld_vol(&hist[threadIdx.x * PER + i]);
+        for (int i = 0; i < PER; ++i) sum += ld_vol(&hist[threadIdx.x * PER + i]);
+    }
     // inclusive scan of the per-thread sums: shuffles inside a warp, then over the 32 warp totals
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
     u64 incl = sum;
@@ -487,6 +502,20 @@ __device__ void scan_hist(const unsigned *hist, int nb, u64 r, unsigned *bin_out
     if (wid) incl += s_part[wid - 1];
     const u64 run = incl - sum;
     if (threadIdx.x == FIN_THREADS - 1 && incl < r) *err = 1;
+    if (PER == 8) {
+        // the thread whose range holds the r-th element finds the bin among its eight counts
+        if (run < r && r <= incl) {
+            u64 before = run;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const u64 c = mine8[i];
+                if (before < r && r <= before + c) { *bin_out = threadIdx.x * 8 + i; *r_in_bin = r - before; *cnt_out = c; }
+                before += c;
+            }
+        }
+        __syncthreads();
+        return;
+    }
     __shared__ int s_owner;
     __shared__ u64 s_run;
     if (threadIdx.x == 0) s_owner = -1;
