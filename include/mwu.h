@@ -114,6 +114,32 @@ int mwu_project(const mwu_proj_desc *desc, const float *W, const float *U_dual, 
                 void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 /*
+ * mwu_admm_step -- the Q-step and the dual step of one ADMM iteration in one sweep
+ * (Algorithm 1: Q = Unify(W + U), then U <- U + W - Q; the dual update is the last of the three
+ * ADMM steps of Section 3.3, and ||W - Q + U||_F^2 is the quadratic term of the augmented
+ * Lagrangian given there, without its factor rho/2).
+ *
+ * With v = W, or fp32(W + U_dual), and Q as mwu_project computes it:
+ *   U_next[l]    = fp32(v_l - Q_l)       one subtraction per entry: v_l for a pruned block,
+ *                                        +0 for a block that keeps its values
+ *   residual_sq  = sum over pruned blocks of sum v_l^2 + sum over unified blocks of L_u
+ *                = ||v - Q||_F^2 with the unified magnitudes unrounded, accumulated in fp64
+ *                  (the order of the additions is not fixed: expect the last bits to vary)
+ * rho * U_next is also the gradient of the quadratic term with respect to W, which the caller's
+ * optimiser needs for the next W-step.
+ *
+ *   U_next        out  fp32 [rows*cols]; may be NULL.  Must not overlap W or U_dual (they are read
+ *                      again after U_next has been written): MWU_ERR_INVALID_ARG
+ *   residual_sq   out  device fp64 [1], 8-byte aligned; may be NULL; zeroed by the call
+ *   At least one of the two must be given.  All other arguments, outputs, workspace and errors as
+ *   mwu_project (without the per-block loss outputs).
+ */
+int mwu_admm_step(const mwu_proj_desc *desc, const float *W, const float *U_dual, float *Q,
+                  float *U_next, double *residual_sq, float *u, uint32_t *pruned_bitmap,
+                  uint32_t *unified_bitmap, uint32_t *sign_bits, uint32_t *dev_status,
+                  void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
  * mwu_project_static -- mwu_project without a caller-supplied workspace.  (The paper has no
  * counterpart: this is a packaging variant of the same projection, with the same outputs.)
  *

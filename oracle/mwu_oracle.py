@@ -155,6 +155,26 @@ def project(W: np.ndarray, b: int, k_unify: int, k_prune: int,
                       sign=sign.reshape(N, K), stats=stats, V=V)
 
 
+@dataclasses.dataclass
+class DualUpdate:
+    U_next: np.ndarray     # fp32 [N][K]
+    residual_sq: float     # ||V - Q||_F^2 with unrounded unified magnitudes, fp64
+
+
+def dual_update(p: Projection, b: int) -> DualUpdate:
+    """Dual step of ADMM (Algorithm 1, last assignment of the loop; third ADMM step of Section
+    3.3): U_{k+1} = U_k + W_{k+1} - Q_{k+1}.  With V = fp32(W_{k+1} + U_k), the tensor that was
+    projected, this is V - Q: one fp32 subtraction per entry.  residual_sq is the quadratic term
+    ||W - Q + U||_F^2 of the augmented Lagrangian of Section 3.3 (without rho/2) after the Q-step,
+    summed per block from the fp64 block statistics: sum v^2 for a pruned block, the unification
+    loss for a unified block, nothing for a block that keeps its values."""
+    U_next = (p.V - p.Q).astype(np.float32)                 # fp32 - fp32, rounded once
+    Vb = p.V.reshape(-1, b).astype(np.float64)
+    sumsq = tree_sum(Vb * Vb)
+    residual = float(np.sum(sumsq[p.pruned]) + np.sum(p.stats.L_u[p.unified]))
+    return DualUpdate(U_next=U_next, residual_sq=residual)
+
+
 def bitmap_words(mask: np.ndarray) -> np.ndarray:
     """bool[n] -> uint32[ceil(n/32)], bit (j % 32) of word (j // 32)."""
     n = mask.shape[0]

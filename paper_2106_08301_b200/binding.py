@@ -16,11 +16,13 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libmwu.so")
 
 EXPORTS = ["mwu_status_string", "mwu_count_from_permille", "mwu_project_workspace_bytes",
-           "mwu_project", "mwu_project_static", "mwu_packed_bytes", "mwu_pack", "mwu_gemm", "mwu_decode", "mwu_gemm_workspace_bytes", "mwu_gemm_ws",
+           "mwu_project", "mwu_admm_step", "mwu_project_static", "mwu_packed_bytes", "mwu_pack", "mwu_gemm", "mwu_decode", "mwu_gemm_workspace_bytes", "mwu_gemm_ws",
            "mwu_conv_implicit"]
 MWU_STATIC_MAX_BLOCKS = 1048576
 
 MWU_OK = 0
+(MWU_ERR_INVALID_ARG, MWU_ERR_SHAPE, MWU_ERR_ALIGNMENT, MWU_ERR_WORKSPACE, MWU_ERR_UNSUPPORTED_DEVICE,
+ MWU_ERR_CUDA) = 1, 2, 3, 4, 5, 6
 MWU_DEV_NONFINITE, MWU_DEV_TIMEOUT, MWU_DEV_BOUNDS, MWU_DEV_SELECT = 1, 2, 4, 8
 MWU_PRUNE_KEY_L2SQ, MWU_PRUNE_KEY_L1 = 0, 1
 MWU_ALGO_AUTO, MWU_ALGO_ONE_PASS, MWU_ALGO_MULTI_PASS = 0, 1, 2
@@ -58,6 +60,8 @@ def lib() -> ctypes.CDLL:
         L.mwu_project_workspace_bytes.argtypes = [dp]
         L.mwu_project.restype = ctypes.c_int
         L.mwu_project.argtypes = [dp] + [vp] * 11 + [sz, vp]
+        L.mwu_admm_step.restype = ctypes.c_int
+        L.mwu_admm_step.argtypes = [dp] + [vp] * 11 + [sz, vp]
         L.mwu_project_static.restype = ctypes.c_int
         L.mwu_project_static.argtypes = [dp] + [vp] * 10 + [vp]
         L.mwu_packed_bytes.restype = sz
@@ -117,6 +121,19 @@ def mwu_project(desc, W, U_dual, Q, u, pruned_bitmap, unified_bitmap, sign_bits,
                            _stream(stream))
     if check and rc != MWU_OK:
         raise MwuError(rc, "mwu_project")
+    return rc
+
+
+def mwu_admm_step(desc, W, U_dual, Q, U_next, residual_sq, u, pruned_bitmap, unified_bitmap, sign_bits,
+                  dev_status, workspace, stream=None, check=True) -> int:
+    """Projection plus dual update U_next = V - Q and residual_sq = ||V - Q||_F^2 in one call."""
+    rc = lib().mwu_admm_step(ctypes.byref(desc), _ptr(W), _ptr(U_dual), _ptr(Q), _ptr(U_next),
+                             _ptr(residual_sq), _ptr(u), _ptr(pruned_bitmap), _ptr(unified_bitmap),
+                             _ptr(sign_bits), _ptr(dev_status), _ptr(workspace),
+                             workspace.numel() * workspace.element_size() if workspace is not None else 0,
+                             _stream(stream))
+    if check and rc != MWU_OK:
+        raise MwuError(rc, "mwu_admm_step")
     return rc
 
 
@@ -210,6 +227,11 @@ class ProjectionBuffers:
         return mwu_project(self.desc, W, U_dual, self.Q, self.u, self.pruned_bitmap,
                            self.unified_bitmap, self.sign_bits, self.loss_u, self.loss_p,
                            self.dev_status, self.workspace, stream)
+
+    def admm_step(self, W, U_dual, U_next, residual_sq, stream=None):
+        return mwu_admm_step(self.desc, W, U_dual, self.Q, U_next, residual_sq, self.u,
+                             self.pruned_bitmap, self.unified_bitmap, self.sign_bits,
+                             self.dev_status, self.workspace, stream)
 
     def pack(self, W, U_dual=None, packed=None, stream=None):
         if packed is None:

@@ -103,6 +103,8 @@ struct Params {
     uint2 *list;                // [list_cap] candidate list: (block index, bin codes)
     unsigned list_cap;
     int gated;                  // multi-pass kernels return at once unless work->failed is set
+    float *U_next;              // dual update V - Q (mwu_admm_step), else null
+    double *resid;              // ||V - Q||_F^2 accumulator (mwu_admm_step), else null
     u64 *cand_key;              // [CAP]
     unsigned *cand_idx;         // [CAP]
     unsigned *bins;             // [n_blocks]
@@ -163,6 +165,33 @@ __device__ __forceinline__ void block_keys(const float *v, int use_l1, double *S
 #pragma unroll
         for (int l = 0; l < B / 2; ++l) h[l] = __fma_rn(a[2 * l], a[2 * l], __dmul_rn(a[2 * l + 1], a[2 * l + 1]));
         *Kp_out = tree_sum<B / 2>(h);
+    }
+}
+
+// sum v^2 of a block with the same pairing as the prune key of block_keys
+template <int B>
+__device__ __forceinline__ double block_sumsq(const float *v) {
+    double h[B / 2];
+#pragma unroll
+    for (int l = 0; l < B / 2; ++l) {
+        const double a0 = (double)v[2 * l], a1 = (double)v[2 * l + 1];
+        h[l] = __fma_rn(a0, a0, __dmul_rn(a1, a1));
+    }
+    return tree_sum<B / 2>(h);
+}
+
+// sum over the CTA of one double per thread, added to *dst by one thread
+__device__ __forceinline__ void block_add_double(double x, double *dst) {
+    __shared__ double s_part[32];
+    for (int m = 16; m > 0; m >>= 1) x += __shfl_xor_sync(0xffffffffu, x, m);
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    if (lane == 0) s_part[wid] = x;
+    __syncthreads();
+    if (wid == 0) {
+        const int nw = (blockDim.x + 31) >> 5;
+        double t = lane < nw ? s_part[lane] : 0.0;
+        for (int m = 16; m > 0; m >>= 1) t += __shfl_xor_sync(0xffffffffu, t, m);
+        if (lane == 0 && t != 0.0) atomicAdd(dst, t);
     }
 }
 
@@ -634,6 +663,7 @@ template <int B>
 __global__ void __launch_bounds__(256) stats_kernel(Params p, double *loss_u, double *loss_p, float *u_out,
                                                     unsigned *sign_bits) {
     if (p.gated && p.work->failed == 0u) return;     // the one-pass result stands
+    if (p.gated && p.resid && blockIdx.x == 0 && threadIdx.x == 0) *p.resid = 0.0;   // emit_kernel sums afresh
     constexpr int NBT = 16 / B;                         // blocks per thread and step
     const Sel *sp = &p.work->sel[0];
     const Sel *su = &p.work->sel[1];
@@ -1076,6 +1106,7 @@ __global__ void __launch_bounds__(256, 3) emit_kernel(Params p, float *Q, float 
     const long long n_bm_words = (p.n_blocks + 31) / 32;
     __shared__ float4 s_stage[8][128];                       // one warp step of Q per warp
     float4 *ws = s_stage[threadIdx.x >> 5];
+    double resid_acc = 0.0;
 
     for (long long unit = (long long)blockIdx.x * blockDim.x + threadIdx.x; unit < n_iter;
          unit += (long long)gridDim.x * blockDim.x) {
@@ -1113,7 +1144,7 @@ __global__ void __launch_bounds__(256, 3) emit_kernel(Params p, float *Q, float 
             cls_u |= (un ? 1u : 0u) << e;
         }
         // q of the unified blocks and the sign plane come from stats_kernel; W is read again
-        // only where a block keeps its own values
+        // only where a block keeps its own values (everywhere for the dual update: it needs v)
         float uo[NBT];
 #pragma unroll
         for (int e = 0; e < NBT; ++e) uo[e] = 0.f;
@@ -1123,9 +1154,10 @@ __global__ void __launch_bounds__(256, 3) emit_kernel(Params p, float *Q, float 
                 if ((cls_u >> e) & 1u) uo[e] = u_out[j0 + e];
         }
         if (unit < n_units) {
-            if (Q) {
+            if (Q || p.U_next || p.resid) {
                 float v[16];
-                const bool need_v = ((~cls_p & ~cls_u) & valid & ALL) != 0u;
+                const bool admm = p.U_next != nullptr || p.resid != nullptr;
+                const bool need_v = admm || ((~cls_p & ~cls_u) & valid & ALL) != 0u;
                 if (need_v) load16(p.W, p.U, f, n, v);
                 else {
 #pragma unroll
@@ -1143,6 +1175,32 @@ __global__ void __launch_bounds__(256, 3) emit_kernel(Params p, float *Q, float 
                         q[e * B + l] = pr ? 0.f : (un ? (neg ? -uo[e] : uo[e]) : v[e * B + l]);
                     }
                 }
+                if (admm) {
+                    // dual update V - Q and ||V - Q||^2 (loss of the block's class)
+#pragma unroll
+                    for (int e = 0; e < NBT; ++e) {
+                        const bool pr = (cls_p >> e) & 1u, un = (cls_u >> e) & 1u;
+                        if (p.resid && (pr || un)) {
+                            double S, Lu, Kp;
+                            block_keys<B>(v + e * B, 0, &S, &Lu, &Kp);
+                            resid_acc += pr ? Kp : Lu;
+                        }
+                    }
+                    if (p.U_next) {
+                        if (f + 16 <= n) {
+                            float4 *dst = reinterpret_cast<float4 *>(p.U_next + f);
+#pragma unroll
+                            for (int c = 0; c < 4; ++c)
+                                dst[c] = make_float4(__fsub_rn(v[4 * c], q[4 * c]), __fsub_rn(v[4 * c + 1], q[4 * c + 1]),
+                                                     __fsub_rn(v[4 * c + 2], q[4 * c + 2]), __fsub_rn(v[4 * c + 3], q[4 * c + 3]));
+                        } else {
+#pragma unroll
+                            for (int l = 0; l < 16; ++l)
+                                if (f + l < n) p.U_next[f + l] = __fsub_rn(v[l], q[l]);
+                        }
+                    }
+                }
+                if (Q) {
                 if (!warp_full) {
                     if (f + 16 <= n) {
                         float4 *dst = reinterpret_cast<float4 *>(Q + f);
@@ -1159,6 +1217,7 @@ __global__ void __launch_bounds__(256, 3) emit_kernel(Params p, float *Q, float 
 #pragma unroll
                     for (int c = 0; c < 4; ++c)
                         ws[lane * 4 + (c ^ ((lane >> 1) & 3))] = make_float4(q[4 * c], q[4 * c + 1], q[4 * c + 2], q[4 * c + 3]);
+                }
                 }
             }
             if (j0 + NBT <= p.n_blocks) {
@@ -1206,6 +1265,7 @@ __global__ void __launch_bounds__(256, 3) emit_kernel(Params p, float *Q, float 
             }
         }
     }
+    if (p.resid) block_add_double(resid_acc, p.resid);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -1216,7 +1276,9 @@ __device__ __forceinline__ void one_pass_fail(const Params &p) { atomicExch(&p.w
 // pass_kernel: keys, provisional classes and every output in one sweep over W (+U).
 // A block is a candidate when its final class is still open: its prune key lies inside the prune
 // window, or it certainly survives pruning and its L_u lies inside the unify window.
-template <int B>
+// ADMM: also the dual update V - Q and ||V - Q||_F^2 (mwu_admm_step); a separate instantiation so
+// that the plain projection keeps its register count.
+template <int B, bool ADMM>
 __global__ void __launch_bounds__(256) pass_kernel(Params p, float *Q, double *loss_u, double *loss_p,
                                                    float *u_out, unsigned *pruned_bitmap,
                                                    unsigned *unified_bitmap, unsigned *sign_bits) {
@@ -1237,6 +1299,7 @@ __global__ void __launch_bounds__(256) pass_kernel(Params p, float *Q, double *l
     const unsigned lt_mask = (1u << lane) - 1u;
     unsigned fill = 0;                                   // warp-uniform
     unsigned under_p = 0, over_p = 0, under_u = 0, over_u = 0, nonfinite = 0;
+    double resid_acc = 0.0;
     // fewer than 2^31 blocks of at least two values: units (16 values) and blocks count in 32 bits
     const long long n = p.n_floats;
     const unsigned n_units = (unsigned)((n + 15) / 16);
@@ -1310,6 +1373,11 @@ __global__ void __launch_bounds__(256) pass_kernel(Params p, float *Q, double *l
                 cls_u |= (un ? 1u : 0u) << e;
                 cand |= (open ? 1u : 0u) << e;
                 if (un) uo[e] = qf;
+                if (ADMM && p.resid) {
+                    // squared distance of the block to its image: the loss of its (provisional) class
+                    if (un) resid_acc += Lu;
+                    else if (pr) resid_acc += p.use_l1 ? block_sumsq<B>(v + e * B) : Kp;
+                }
             }
         }
         if (live) {
@@ -1327,7 +1395,7 @@ __global__ void __launch_bounds__(256) pass_kernel(Params p, float *Q, double *l
                 for (int e = 0; e < NBT; ++e)
                     if (j0 + e < n_blocks) u_out[j0 + e] = uo[e];
             }
-            if (Q) {
+            if (Q || (ADMM && p.U_next)) {
                 // q = v (kept), +-u (unified: magnitude u, sign from the sign plane bits), or +0
                 float q[16];
 #pragma unroll
@@ -1343,7 +1411,23 @@ __global__ void __launch_bounds__(256) pass_kernel(Params p, float *Q, double *l
                     }
                 }
                 const long long f = (long long)unit * 16;
-                if (!warp_full) {
+                if (ADMM && p.U_next) {
+                    // dual update: one fp32 subtraction per entry (v for a pruned block, +0 for a kept one)
+                    if (f + 16 <= n) {
+                        float4 *dst = reinterpret_cast<float4 *>(p.U_next + f);
+#pragma unroll
+                        for (int c = 0; c < 4; ++c)
+                            dst[c] = make_float4(__fsub_rn(v[4 * c], q[4 * c]), __fsub_rn(v[4 * c + 1], q[4 * c + 1]),
+                                                 __fsub_rn(v[4 * c + 2], q[4 * c + 2]), __fsub_rn(v[4 * c + 3], q[4 * c + 3]));
+                    } else {
+#pragma unroll
+                        for (int l = 0; l < 16; ++l)
+                            if (f + l < n) p.U_next[f + l] = __fsub_rn(v[l], q[l]);
+                    }
+                }
+                if (!Q) {
+                    // only the dual update was wanted
+                } else if (!warp_full) {
                     if (f + 16 <= n) {
                         float4 *dst = reinterpret_cast<float4 *>(Q + f);
                         dst[0] = make_float4(q[0], q[1], q[2], q[3]);
@@ -1442,6 +1526,7 @@ __global__ void __launch_bounds__(256) pass_kernel(Params p, float *Q, double *l
         if (s_tot[2]) atomicAdd(&hist_u[0], s_tot[2]);
         if (s_tot[3]) atomicAdd(&hist_u[top], s_tot[3]);
     }
+    if (ADMM && p.resid) block_add_double(resid_acc, p.resid);
 }
 
 // Sort the n candidates (global cand_key / cand_idx) and write the threshold element, the r-th
@@ -1575,12 +1660,12 @@ __global__ void __launch_bounds__(FIN_THREADS) list_select_kernel(Params p) {
 // Final class of block j against what pass_kernel wrote (read back from the bitmaps); the
 // block's outputs are rewritten where they differ.
 template <int B>
-__device__ __forceinline__ void apply_class(const Params &p, float *Q, float *u_out, unsigned *pruned_bitmap,
-                                            unsigned *unified_bitmap, unsigned idx, bool pr, bool un) {
+__device__ __forceinline__ double apply_class(const Params &p, float *Q, float *u_out, unsigned *pruned_bitmap,
+                                              unsigned *unified_bitmap, unsigned idx, bool pr, bool un) {
     const unsigned bit = 1u << (idx & 31u);
     unsigned *wp = pruned_bitmap + (idx >> 5), *wu = unified_bitmap + (idx >> 5);
     const bool pr0 = (ld_vol(wp) & bit) != 0u, un0 = (ld_vol(wu) & bit) != 0u;
-    if (pr == pr0 && un == un0) return;
+    if (pr == pr0 && un == un0) return 0.0;
     if (pr != pr0) { if (pr) atomicOr(wp, bit); else atomicAnd(wp, ~bit); }
     if (un != un0) { if (un) atomicOr(wu, bit); else atomicAnd(wu, ~bit); }
     const long long j = (long long)idx;
@@ -1590,10 +1675,16 @@ __device__ __forceinline__ void apply_class(const Params &p, float *Q, float *u_
     block_keys<B>(v, p.use_l1, &S, &Lu, &Kp);
     const float qf = __double2float_rn(__dmul_rn(S, 1.0 / (double)B));
     u_out[j] = un ? qf : 0.f;
-    if (Q) {
 #pragma unroll
-        for (int l = 0; l < B; ++l) Q[j * B + l] = pr ? 0.f : (un ? (v[l] < 0.f ? -qf : qf) : v[l]);
+    for (int l = 0; l < B; ++l) {
+        const float q = pr ? 0.f : (un ? (v[l] < 0.f ? -qf : qf) : v[l]);
+        if (Q) Q[j * B + l] = q;
+        if (p.U_next) p.U_next[j * B + l] = __fsub_rn(v[l], q);
     }
+    // change of ||V - Q||^2: the loss of the new class minus that of the provisional one
+    if (!p.resid) return 0.0;
+    const double sq = p.use_l1 ? block_sumsq<B>(v) : Kp;
+    return (pr ? sq : (un ? Lu : 0.0)) - (pr0 ? sq : (un0 ? Lu : 0.0));
 }
 
 // list_finish_kernel: every listed block outside the unify threshold bin gets its final class at
@@ -1615,6 +1706,7 @@ __global__ void __launch_bounds__(FIN_THREADS) list_finish_kernel(Params p, floa
     const u128 lo = from_halves(su->lo_hi, su->lo_lo);
     const u128 hi = from_halves(su->hi_hi, su->hi_lo);
     const unsigned n_list = min(p.work->list_count, p.list_cap);
+    double resid_delta = 0.0;
     for (unsigned i = blockIdx.x * blockDim.x + threadIdx.x; i < n_list; i += gridDim.x * blockDim.x) {
         const uint2 e = __ldg(&p.list[i]);
         const unsigned bu = e.y >> 16;
@@ -1635,8 +1727,9 @@ __global__ void __launch_bounds__(FIN_THREADS) list_finish_kernel(Params p, floa
                 } else un = bu < Bu;
             }
         }
-        apply_class<B>(p, Q, u_out, pruned_bitmap, unified_bitmap, e.x, pr, un);
+        resid_delta += apply_class<B>(p, Q, u_out, pruned_bitmap, unified_bitmap, e.x, pr, un);
     }
+    if (p.resid) block_add_double(resid_delta, p.resid);
     if (mode_u != 0u) return;
     if (!last_block_done(&p.work->fticket[1])) return;
 
@@ -1647,8 +1740,10 @@ __global__ void __launch_bounds__(FIN_THREADS) list_finish_kernel(Params p, floa
         return;
     }
     const unsigned r = (unsigned)r_u;
+    double tail_delta = 0.0;
     for (unsigned i = threadIdx.x; i < m; i += blockDim.x)
-        apply_class<B>(p, Q, u_out, pruned_bitmap, unified_bitmap, c_idx[i], false, i < r);
+        tail_delta += apply_class<B>(p, Q, u_out, pruned_bitmap, unified_bitmap, c_idx[i], false, i < r);
+    if (p.resid) block_add_double(tail_delta, p.resid);
 }
 
 }  // namespace proj
@@ -1694,7 +1789,8 @@ static cudaError_t launch_project(const mwu::proj::Params &p, const mwu_proj_des
     const bool need_u = ksel_u > 0 && ksel_u < mb - desc->k_prune;
 
     if (one_pass) {
-        pass_kernel<B><<<grid_stream, 256, 0, st>>>(p, Q, loss_u, loss_p, u, pb, ub, sb);
+        if (p.U_next || p.resid) pass_kernel<B, true><<<grid_stream, 256, 0, st>>>(p, Q, loss_u, loss_p, u, pb, ub, sb);
+        else pass_kernel<B, false><<<grid_stream, 256, 0, st>>>(p, Q, loss_u, loss_p, u, pb, ub, sb);
         if (!need_p && !need_u) return cudaGetLastError();       // no threshold: every class is final
         // the list holds a few per cent of the blocks
         const long long lb = (mb / 8 + FIN_THREADS - 1) / FIN_THREADS;      // a thread per expected entry
@@ -1718,15 +1814,17 @@ static cudaError_t launch_project(const mwu::proj::Params &p, const mwu_proj_des
     return cudaGetLastError();
 }
 
-extern "C" int mwu_project(const mwu_proj_desc *desc, const float *W, const float *U_dual, float *Q,
-                           float *u, uint32_t *pruned_bitmap, uint32_t *unified_bitmap,
-                           uint32_t *sign_bits, double *loss_u, double *loss_p, uint32_t *dev_status,
-                           void *workspace, size_t workspace_bytes, void *cuda_stream) {
+// mwu_project and mwu_admm_step: the latter also wants U_next and / or residual_sq
+static int project_impl(const mwu_proj_desc *desc, const float *W, const float *U_dual, float *Q,
+                        float *U_next, double *residual_sq, float *u, uint32_t *pruned_bitmap,
+                        uint32_t *unified_bitmap, uint32_t *sign_bits, double *loss_u, double *loss_p,
+                        uint32_t *dev_status, void *workspace, size_t workspace_bytes, void *cuda_stream) {
     using namespace mwu;
     int rc = validate_desc(desc, false);
     if (rc != MWU_OK) return rc;
     if (!W || !u || !pruned_bitmap || !unified_bitmap || !sign_bits || !dev_status || !workspace)
         return MWU_ERR_INVALID_ARG;
+    if (!aligned_to(U_next, 16) || !aligned_to(residual_sq, 8)) return MWU_ERR_ALIGNMENT;
     if (!aligned_to(W, 16) || !aligned_to(U_dual, 16) || !aligned_to(Q, 16) || !aligned_to(u, 16) ||
         !aligned_to(pruned_bitmap, 16) || !aligned_to(unified_bitmap, 16) ||
         !aligned_to(sign_bits, 16) || !aligned_to(loss_u, 16) || !aligned_to(loss_p, 16) ||
@@ -1758,9 +1856,12 @@ extern "C" int mwu_project(const mwu_proj_desc *desc, const float *W, const floa
     p.list_cap = (unsigned)list_capacity((size_t)p.n_blocks);
     p.gated = one_pass ? 1 : 0;
     p.dev_status = dev_status;
+    p.U_next = U_next;
+    p.resid = residual_sq;
 
     if (cudaMemsetAsync(ws, 0, ws_off_hist() + 5 * (size_t)p.nb * sizeof(unsigned), st) != cudaSuccess)
         return MWU_ERR_CUDA;
+    if (residual_sq && cudaMemsetAsync(residual_sq, 0, sizeof(double), st) != cudaSuccess) return MWU_ERR_CUDA;
     cudaError_t e;
     switch (desc->block) {
         case 2: e = launch_project<2>(p, desc, Q, u, pruned_bitmap, unified_bitmap, sign_bits, loss_u, loss_p, sm_count, one_pass, st); break;
@@ -1769,4 +1870,30 @@ extern "C" int mwu_project(const mwu_proj_desc *desc, const float *W, const floa
         default: e = launch_project<16>(p, desc, Q, u, pruned_bitmap, unified_bitmap, sign_bits, loss_u, loss_p, sm_count, one_pass, st); break;
     }
     return e == cudaSuccess ? MWU_OK : MWU_ERR_CUDA;
+}
+
+extern "C" int mwu_project(const mwu_proj_desc *desc, const float *W, const float *U_dual, float *Q,
+                           float *u, uint32_t *pruned_bitmap, uint32_t *unified_bitmap,
+                           uint32_t *sign_bits, double *loss_u, double *loss_p, uint32_t *dev_status,
+                           void *workspace, size_t workspace_bytes, void *cuda_stream) {
+    return project_impl(desc, W, U_dual, Q, nullptr, nullptr, u, pruned_bitmap, unified_bitmap, sign_bits,
+                        loss_u, loss_p, dev_status, workspace, workspace_bytes, cuda_stream);
+}
+
+extern "C" int mwu_admm_step(const mwu_proj_desc *desc, const float *W, const float *U_dual, float *Q,
+                             float *U_next, double *residual_sq, float *u, uint32_t *pruned_bitmap,
+                             uint32_t *unified_bitmap, uint32_t *sign_bits, uint32_t *dev_status,
+                             void *workspace, size_t workspace_bytes, void *cuda_stream) {
+    if (!desc || !W) return MWU_ERR_INVALID_ARG;
+    if (!U_next && !residual_sq) return MWU_ERR_INVALID_ARG;       // nothing beyond mwu_project was asked for
+    if (U_next) {
+        // the kernels read W and U_dual again after U_next has been written: no overlap allowed
+        const size_t bytes = (size_t)desc->rows * (size_t)desc->cols * sizeof(float);
+        const char *o = (const char *)U_next;
+        const char *ins[2] = {(const char *)W, (const char *)U_dual};
+        for (int i = 0; i < 2; ++i)
+            if (ins[i] && o < ins[i] + bytes && ins[i] < o + bytes) return MWU_ERR_INVALID_ARG;
+    }
+    return project_impl(desc, W, U_dual, Q, U_next, residual_sq, u, pruned_bitmap, unified_bitmap, sign_bits,
+                        nullptr, nullptr, dev_status, workspace, workspace_bytes, cuda_stream);
 }

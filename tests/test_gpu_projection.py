@@ -199,3 +199,13 @@ def test_projection_one_pass_with_dual_and_l1():
     Mb = 512 * 1024 // 4
     check_against_oracle(W, 4, Mb * 6 // 10, Mb * 3 // 10, U=U, algos=(B.MWU_ALGO_AUTO,))
     check_against_oracle(W, 4, Mb * 6 // 10, Mb * 3 // 10, prune_key=1, algos=(B.MWU_ALGO_AUTO,))
+
+
+def test_projection_many_blocks_wide_histogram():
+    """More than 8 Mi blocks: both pipelines switch to the 65536-bin window histogram (64 bins per
+    thread in the threshold search) and the candidate list holds several hundred thousand entries."""
+    rows, cols, b = 2050, 8192, 2
+    W = inputs.normal_weights(rows, cols, 0.02, 2050)
+    Mb = rows * cols // b
+    assert Mb > 8 * 1024 * 1024
+    check_against_oracle(W, b, O.count_from_permille(Mb, 350), O.count_from_permille(Mb, 250))
