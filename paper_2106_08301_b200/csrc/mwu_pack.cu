@@ -26,6 +26,7 @@ struct Params {
     long long rows, cols;
     int b;
     PackedLayout L;
+    unsigned long long gap[5][2];   // byte ranges between the sections (alignment padding), zeroed by scan_kernel
 };
 
 // class masks of row r of a record; padding rows are all-pruned
@@ -166,6 +167,9 @@ __global__ void __launch_bounds__(1024) scan_kernel(Params p) {
             atomicOr(p.dev_status, (unsigned)MWU_DEV_BOUNDS);
         recs[n_rec] = make_uint4((unsigned)tu, (unsigned)td, (unsigned)tp, 0u);
     }
+    // the padding between the sections must read as zero (each gap is shorter than the alignment)
+    for (int g = 0; g < 5; ++g)
+        for (unsigned long long a = p.gap[g][0] + threadIdx.x; a < p.gap[g][1]; a += blockDim.x) p.packed[a] = 0;
     if (threadIdx.x < 32) {
         unsigned long long *h = reinterpret_cast<unsigned long long *>(p.packed);
         unsigned long long v = 0;
@@ -370,8 +374,8 @@ extern "C" int mwu_pack(const mwu_proj_desc *desc, const float *W, const float *
     p.dev_status = dev_status;
     p.rows = desc->rows; p.cols = desc->cols; p.b = desc->block;
     cudaStream_t st = (cudaStream_t)cuda_stream;
-    // header, and the gaps between sections, must read as zero
-    if (cudaMemsetAsync(packed, 0, kHeaderBytes, st) != cudaSuccess) return MWU_ERR_CUDA;
+    // header and the gaps between sections must read as zero: scan_kernel writes all 32 header
+    // words and clears the gaps
     const size_t n_rec = (size_t)p.L.n_tiles * p.L.n_stages;
     const size_t gaps[5][2] = {
         {p.L.off_rec + 16 * (n_rec + 1), p.L.off_ulist},
@@ -379,10 +383,7 @@ extern "C" int mwu_pack(const mwu_proj_desc *desc, const float *W, const float *
         {p.L.off_dpos + 2 * (size_t)p.L.n_dense, p.L.off_dpay},
         {p.L.off_dpay + 2 * (size_t)desc->block * p.L.n_dense, p.L.off_ppos},
         {p.L.off_ppos + 2 * (size_t)p.L.n_plist, p.L.total}};
-    for (int g = 0; g < 5; ++g)
-        if (gaps[g][1] > gaps[g][0])
-            if (cudaMemsetAsync((char *)packed + gaps[g][0], 0, gaps[g][1] - gaps[g][0], st) != cudaSuccess)
-                return MWU_ERR_CUDA;
+    for (int g = 0; g < 5; ++g) { p.gap[g][0] = gaps[g][0]; p.gap[g][1] = gaps[g][1] > gaps[g][0] ? gaps[g][1] : gaps[g][0]; }
     pack::count_kernel<<<(unsigned)n_rec, 128, 0, st>>>(p);
     pack::scan_kernel<<<1, 1024, 0, st>>>(p);
     switch (desc->block) {
