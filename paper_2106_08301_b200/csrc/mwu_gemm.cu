@@ -32,7 +32,8 @@ bool pair_eligible(const Params &p);
 cudaError_t launch_pair(int bw, const CUtensorMap &tmap, const Params &p, int sm_count, cudaStream_t st);
 // decode-once path, defined in mwu_gemm3.cu
 cudaError_t launch_decode(int bw, const Params &p, __nv_bfloat16 *Wd, long long ldw, cudaStream_t st);
-cudaError_t launch_dense(const CUtensorMap &tmap_x, const CUtensorMap &tmap_w, const Params &p, int sm_count,
+cudaError_t launch_dense(const CUtensorMap &tmap_x, const CUtensorMap &tmap_w, const CUtensorMap &tmap_y,
+                         const Params &p, int sm_count,
                          cudaStream_t st);
 
 // ------------------------------------------------------------------------------------------
@@ -630,9 +631,17 @@ extern "C" int mwu_gemm_ws(const mwu_proj_desc *desc, const void *packed, const 
         if (!encode_bf16_2d(encode, &tmap_x, X, desc->cols, M, ldx, BMH) ||
             !encode_bf16_2d(encode, &tmap_w, workspace, desc->cols, n_pad, desc->cols, kTileRows))
             return MWU_ERR_CUDA;
+        // bf16 output leaves through TMA tile stores of 64 columns x 32 rows; fp32 output through
+        // plain stores (the map is then a copy of the activation map, never used)
+        CUtensorMap tmap_y = tmap_x;
+        p.y_tma = 0;
+        if (y_dtype == 0) {
+            if (!encode_bf16_2d(encode, &tmap_y, Y, desc->rows, M, ldy, 32)) return MWU_ERR_CUDA;
+            p.y_tma = 1;
+        }
         if (launch_decode(desc->block, p, (__nv_bfloat16 *)workspace, desc->cols, st) != cudaSuccess)
             return MWU_ERR_CUDA;
-        return launch_dense(tmap_x, tmap_w, p, sm_count, st) == cudaSuccess ? MWU_OK : MWU_ERR_CUDA;
+        return launch_dense(tmap_x, tmap_w, tmap_y, p, sm_count, st) == cudaSuccess ? MWU_OK : MWU_ERR_CUDA;
     }
 
     // tiles of 256 activation rows unless the problem has no second half to fill

@@ -11,7 +11,9 @@
 // tcgen05.mma.cta_group::2; each CTA loads its own 128 activation rows and its own 128 weight
 // rows of a stage by TMA (no multicast), six stages deep.  The accumulators (128 lanes x 256
 // fp32 columns per CTA) are double-buffered in tensor memory, so the epilogue of a tile runs
-// under the main loop of the next one.
+// under the main loop of the next one.  bf16 output leaves through TMA: a warp converts 32 rows x
+// 64 columns, lays them out with the 128-byte swizzle in its 4 KB of shared memory and one lane
+// issues a tile store (whole 128-byte lines, clipped at the edges of Y by the tensor map).
 // Roles per CTA (10 warps): warp 0 TMA producer (both CTAs' loads report their bytes straight to
 // the leader's barrier, cp.async.bulk.tensor with .cta_group::2); warp 1 allocates tensor memory
 // and, in the leader CTA (cluster rank 0), issues the MMAs; warps 2-9 epilogue (two per 32-lane
@@ -91,6 +93,7 @@ constexpr int D_A_BYTES = AH_BYTES;                  // this CTA's 128 activatio
 constexpr int D_B_BYTES = REC_BYTES;                 // this CTA's 128 weight rows
 constexpr int D_STAGE_BYTES = D_A_BYTES + D_B_BYTES;
 constexpr int D_BAND = 8;                            // activation row tiles per band of the tile order
+constexpr int D_EPI_BYTES = 4096;                    // per epilogue warp: 32 rows x 64 bf16 columns
 
 struct DenseSmem {
     unsigned long long full[D_STAGES], empty[D_STAGES], tfull[2], tempty[2], drain;
@@ -102,14 +105,14 @@ struct DenseSmem {
 
 __global__ void __launch_bounds__(D_THREADS, 1)
 mwu_dense_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
-                      const Params p) {
+                      const __grid_constant__ CUtensorMap tmap_y, const Params p) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char *base = reinterpret_cast<unsigned char *>(
         (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     unsigned char *sA = base;
     unsigned char *sB = base + D_STAGES * D_A_BYTES;
-    unsigned char *stage_buf = sB + D_STAGES * D_B_BYTES;   // epilogue: 2 KB per warp
-    DenseSmem *sm = reinterpret_cast<DenseSmem *>(stage_buf + D_EPI_WARPS * 2048);
+    unsigned char *stage_buf = sB + D_STAGES * D_B_BYTES;   // epilogue: 4 KB per warp, 1024-byte aligned
+    DenseSmem *sm = reinterpret_cast<DenseSmem *>(stage_buf + D_EPI_WARPS * D_EPI_BYTES);
     const int n_stages = (int)p.n_stages;
     volatile int *abort = &sm->abort;
 
@@ -261,7 +264,7 @@ mwu_dense_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
         // ---------------- epilogue: this CTA's 128 rows x 256 columns ----------------
         const int quarter = warp & 3;                       // TMEM lanes this warp may read
         const int chalf = (warp - 2) >> 2;                  // which 128 columns
-        unsigned char *stg = stage_buf + (warp - 2) * 2048;
+        unsigned char *stg = stage_buf + (warp - 2) * D_EPI_BYTES;
         bool ok = true;
         for (long long k = 0; ok && tile_of(k, mt_, nt_); ++k) {
             const long long mt = mt_, nt = nt_;
@@ -276,6 +279,47 @@ mwu_dense_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
             const long long m = mt * 256 + rank * 128 + quarter * 32 + lane;
             const unsigned trow = tmem_base + ((unsigned)(quarter * 32) << 16) + buf * 256u + (unsigned)(chalf * 128);
             const long long ncol0 = nt * 256 + chalf * 128;
+            if (p.y_tma) {
+                const long long mrow0 = m - lane;
+                for (int c0 = 0; c0 < 128; c0 += 64) {
+                    if (ncol0 + c0 >= p.N || mrow0 >= p.M) break;
+                    unsigned v0[32], v1[32];
+                    if (any) {
+                        tmem_ld32_issue(trow + (unsigned)c0, v0);
+                        tmem_ld32_issue(trow + (unsigned)(c0 + 32), v1);
+                        tmem_ld_wait(v0);
+                        tmem_ld_wait(v1);
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) { v0[j] = 0u; v1[j] = 0u; }
+                    }
+                    // the previous store of this warp has read the staging buffer
+                    if (lane == 0) bulk_wait_read();
+                    __syncwarp();
+                    // row `lane`: eight 16-byte pieces, piece j at position j ^ (lane % 8) (128-byte swizzle)
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        const unsigned *src = (j < 4) ? (v0 + 8 * j) : (v1 + 8 * (j - 4));
+                        uint4 o;
+                        __nv_bfloat162 h2;
+                        h2 = __floats2bfloat162_rn(__uint_as_float(src[0]), __uint_as_float(src[1]));
+                        o.x = *reinterpret_cast<unsigned *>(&h2);
+                        h2 = __floats2bfloat162_rn(__uint_as_float(src[2]), __uint_as_float(src[3]));
+                        o.y = *reinterpret_cast<unsigned *>(&h2);
+                        h2 = __floats2bfloat162_rn(__uint_as_float(src[4]), __uint_as_float(src[5]));
+                        o.z = *reinterpret_cast<unsigned *>(&h2);
+                        h2 = __floats2bfloat162_rn(__uint_as_float(src[6]), __uint_as_float(src[7]));
+                        o.w = *reinterpret_cast<unsigned *>(&h2);
+                        *reinterpret_cast<uint4 *>(stg + lane * 128 + ((j ^ (lane & 7)) << 4)) = o;
+                    }
+                    fence_proxy_async();
+                    __syncwarp();
+                    if (lane == 0) {
+                        tma_store_2d(&tmap_y, smem_u32(stg), (int)(ncol0 + c0), (int)mrow0);
+                        bulk_commit();
+                    }
+                }
+            } else {
             for (int c0 = 0; c0 < 128; c0 += 32) {
                 if (ncol0 + c0 >= p.N) break;
                 unsigned v[32];
@@ -288,6 +332,7 @@ mwu_dense_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
                 if (p.y_fp32 || ncol0 + c0 + 32 > p.N) store_row_chunk<32>(p, m, ncol0 + c0, v);
                 else store_chunk_staged(p, m - lane, lane, ncol0 + c0, v, stg);
             }
+            }
             tc_fence_before();
             __syncwarp();
             if (lane == 0) {
@@ -295,6 +340,7 @@ mwu_dense_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
                 else mbar_arrive_cluster(smem_u32(&sm->tempty[buf]), 0);
             }
         }
+        if (lane == 0) bulk_wait_all();                     // this warp's tile stores are done
     }
 
     // teardown: nobody leaves while the other CTA may still read this one's memory or barriers
@@ -309,11 +355,11 @@ mwu_dense_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
 }
 
 static size_t dense_smem_bytes() {
-    return 1024 + (size_t)D_STAGES * D_STAGE_BYTES + (size_t)D_EPI_WARPS * 2048 + sizeof(DenseSmem);
+    return 1024 + (size_t)D_STAGES * D_STAGE_BYTES + (size_t)D_EPI_WARPS * D_EPI_BYTES + sizeof(DenseSmem);
 }
 
-cudaError_t launch_dense(const CUtensorMap &tmap_x, const CUtensorMap &tmap_w, const Params &p, int sm_count,
-                         cudaStream_t st) {
+cudaError_t launch_dense(const CUtensorMap &tmap_x, const CUtensorMap &tmap_w, const CUtensorMap &tmap_y,
+                         const Params &p, int sm_count, cudaStream_t st) {
     auto kern = mwu_dense_pair_kernel;
     const size_t smem = dense_smem_bytes();
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -333,7 +379,7 @@ cudaError_t launch_dense(const CUtensorMap &tmap_x, const CUtensorMap &tmap_w, c
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, kern, tmap_x, tmap_w, p);
+    return cudaLaunchKernelEx(&cfg, kern, tmap_x, tmap_w, tmap_y, p);
 }
 
 }  // namespace gemm

@@ -42,6 +42,7 @@ struct Params {
     int y_fp32;
     int resident;                       // pair kernel: a CTA pair keeps one weight tile (see mwu_gemm2.cu)
     int stage_epi;                      // single-CTA GEMM: 16 KB of shared memory is there for store_chunk_staged
+    int y_tma;                          // two-operand GEMM: bf16 output leaves through TMA stores (a tensor map of Y exists)
     unsigned *dev_status;
     // convolution only
     const __nv_bfloat16 *X;
@@ -181,6 +182,17 @@ __device__ __forceinline__ void tma_load_2d_pair(unsigned dst, const CUtensorMap
         "[%0], [%1, {%3, %4}], [%2];"
         ::"r"(dst), "l"(map), "r"(bar_cluster), "r"(x), "r"(y) : "memory");
 }
+// shared memory -> global tile store; the box is clipped at the tensor's bounds
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap *map, unsigned src, int x, int y) {
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+                 ::"l"(map), "r"(src), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// the issuing thread's earlier bulk stores have read their shared-memory source
+__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+// ... and have completed
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+
 __device__ __forceinline__ void tmem_alloc2(unsigned dst_smem, unsigned ncols) {
     asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
