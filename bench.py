@@ -378,9 +378,9 @@ def run_gpu(args):
             "peak_source": peaks["source"] + " (sustained cuBLAS bf16)",
             "algorithmic_flops_per_launch": flops,
             # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the two-operand GEMM kernel
-            # (627.9 MB + 252.9 MB, ncu capture of this workload; see profiles/step_kernels_c4_ffn.md);
+            # (610.1 MB + 250.0 MB, ncu capture of this workload; see profiles/step_kernels_c4_ffn.md);
             # not taken for other workloads or for the fused path
-            "traffic": 880.8e6 if (ws_bytes and wl.name == "c4_ffn" and m == wl.m) else None,
+            "traffic": 860.1e6 if (ws_bytes and wl.name == "c4_ffn" and m == wl.m) else None,
             # the whole mwu_project call (eight launches) against the 8 bytes per weight the method needs
             "projection": {"bound": "hbm", "achieved": abytes["projection"] / (proj_ms * 1e-3) / 1e9,
                            "peak": peaks["hbm_gbs"], "unit": "GB/s",
