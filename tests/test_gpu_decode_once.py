@@ -145,3 +145,27 @@ def test_gemm_ws_config4_shape_sampled_outputs():
     ref = O.gemm(X[rows].to(torch.float64).numpy(), O.decoded_weights(p, wl.block))
     fro, mx = errors(Y[rows].float().cpu().numpy(), ref)
     assert fro <= 2e-3 and mx <= 1e-2, (fro, mx)
+
+
+@pytest.mark.parametrize("b,pruned_permille", [(2, 900), (4, 0), (8, 500)])
+def test_gemm_ws_sweep_points_full_size_sampled_outputs(b, pruned_permille):
+    """Points of the 4096 x 4096 sweep at full size (M = 8192), among them the two ends: nothing
+    pruned, and 90 % pruned with every other block unified.  The class bitmaps and the packed
+    bytes are compared with the checker bit for bit, the GEMM on sampled rows."""
+    wl = inputs.sweep_workload(b, pruned_permille)
+    ku = B.mwu_count_from_permille(wl.n_blocks, wl.unified_permille)
+    kp = B.mwu_count_from_permille(wl.n_blocks, wl.pruned_permille)
+    desc, bufs, packed, p = project_and_pack(wl.weights(), wl.block, ku, kp)
+    assert np.array_equal(bufs.pruned_bitmap.cpu().numpy().view(np.uint32), O.bitmap_words(p.pruned))
+    assert np.array_equal(bufs.unified_bitmap.cpu().numpy().view(np.uint32), O.bitmap_words(p.unified))
+    assert np.array_equal(packed.cpu().numpy(), O.pack(p, wl.block))
+    X = wl.activations()
+    ws = torch.empty(B.mwu_gemm_workspace_bytes(desc, wl.m), dtype=torch.uint8, device="cuda")
+    Y = torch.empty((wl.m, wl.rows), dtype=torch.bfloat16, device="cuda")
+    B.mwu_gemm_ws(desc, packed, X.cuda(), wl.m, wl.cols, Y, wl.rows, 0, ws, bufs.dev_status)
+    torch.cuda.synchronize()
+    assert int(bufs.dev_status.item()) == 0
+    rows = [0, 31, 32, 255, 256, 4097, 8191]
+    ref = O.gemm(X[rows].to(torch.float64).numpy(), O.decoded_weights(p, wl.block))
+    fro, mx = errors(Y[rows].float().cpu().numpy(), ref)
+    assert fro <= 2e-3 and mx <= 1e-2, (fro, mx)
