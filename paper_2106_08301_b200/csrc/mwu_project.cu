@@ -505,6 +505,18 @@ __device__ void scan_hist(const unsigned *hist, int nb, u64 r, unsigned *bin_out
         for (int i = 0; i < 8; ++i) mine8[i] = ld_vol(&hist[threadIdx.x * 8 + i]);
 #pragma unroll
         for (int i = 0; i < 8; ++i) sum += mine8[i];
+    } else if (PER == 64) {
+        // A thread's 64 bins are 256 bytes: read by the thread itself, every load of a warp would
+        // touch 32 cache lines (the L1 tag stage then takes 65 000 cycles per CTA for 65536 bins).
+        // The warp sums them together instead: two coalesced loads and a shuffle tree per thread.
+        const int l = threadIdx.x & 31, w = threadIdx.x >> 5;
+#pragma unroll 4
+        for (int e = 0; e < 32; ++e) {
+            const int base = (w * 32 + e) * 64;
+            unsigned a = ld_vol(&hist[base + l]) + ld_vol(&hist[base + 32 + l]);
+            for (int m = 16; m > 0; m >>= 1) a += __shfl_xor_sync(0xffffffffu, a, m);
+            if (l == e) sum = a;
+        }
     } else {
 #pragma unroll 8
         for (int i = 0; i < PER; ++i) sum += ld_vol(&hist[threadIdx.x * PER + i]);
