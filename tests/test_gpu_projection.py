@@ -209,3 +209,43 @@ def test_projection_many_blocks_wide_histogram():
     Mb = rows * cols // b
     assert Mb > 8 * 1024 * 1024
     check_against_oracle(W, b, O.count_from_permille(Mb, 350), O.count_from_permille(Mb, 250))
+
+
+def test_projection_largest_sweep_size_properties():
+    """2^28 weights (the largest size of the projection sweep), where the CPU checker is out of
+    reach: properties that pin the result at any size.  Class counts are exact; pruned blocks are
+    zero, unified blocks carry +-u, other blocks are copied; and the selection is a valid one: no
+    pruned block has a larger prune key than a surviving one, no unified block a larger L_u than a
+    surviving one that kept its values (keys recomputed here with plain fp64 tensor operations)."""
+    rows = cols = 16384
+    b = 16
+    Mb = rows * cols // b
+    ku, kp = O.count_from_permille(Mb, 500), O.count_from_permille(Mb, 250)
+    W = inputs.normal_weights(rows, cols, 0.02, inputs.seed_for(5, 928))
+    desc, bufs, Wd, _ = run_project(W, b, ku, kp, want_loss=False)
+    del W
+    assert int(bufs.dev_status.item()) == 0
+
+    def unpack(words):
+        bits = (words.view(torch.int32).unsqueeze(1) >> torch.arange(32, device="cuda", dtype=torch.int32)) & 1
+        return bits.reshape(-1)[:Mb].bool()
+
+    pruned, unified = unpack(bufs.pruned_bitmap), unpack(bufs.unified_bitmap)
+    assert int(pruned.sum()) == kp and int(unified.sum()) == ku - kp and not bool((pruned & unified).any())
+    V = Wd.reshape(Mb, b)
+    Q = bufs.Q.reshape(Mb, b)
+    kept = ~(pruned | unified)
+    assert not bool(Q[pruned].any())
+    assert torch.equal(Q[kept].view(torch.int32), V[kept].view(torch.int32))
+    u = bufs.u
+    assert not bool(u[~unified].any())
+    assert torch.equal(Q[unified], torch.where(V[unified] < 0, -u[unified, None], u[unified, None]))
+    A = V.abs().double()
+    Lp = (A * A).sum(1)
+    q = A.mean(1, keepdim=True)
+    Lu = ((A - q) ** 2).sum(1)
+    del A
+    assert float(Lp[pruned].max()) <= float(Lp[~pruned].min()) * (1 + 1e-12)
+    assert float(Lu[unified].max()) <= float(Lu[kept].min()) * (1 + 1e-12)
+    # the unified value is the mean magnitude
+    assert torch.allclose(u[unified].double(), q[unified, 0], rtol=1e-6, atol=0)
