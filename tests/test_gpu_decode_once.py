@@ -169,3 +169,25 @@ def test_gemm_ws_sweep_points_full_size_sampled_outputs(b, pruned_permille):
     ref = O.gemm(X[rows].to(torch.float64).numpy(), O.decoded_weights(p, wl.block))
     fro, mx = errors(Y[rows].float().cpu().numpy(), ref)
     assert fro <= 2e-3 and mx <= 1e-2, (fro, mx)
+
+
+@pytest.mark.parametrize("N,K,M,b", [(504, 256, 40001, 8), (1024, 128, 50000, 16), (304, 384, 38000, 4),
+                                     (1104, 64, 20000, 2)])
+def test_gemm_ws_short_reduction_many_rows(N, K, M, b):
+    """Short reductions with many activation rows (the 1x1-convolution regime: a few k stages per
+    tile, hundreds of row tiles).  Ragged N, M and an odd number of 128-row weight tiles."""
+    W = inputs.normal_weights(N, K, 0.02, 7000 + N)
+    Mb = N * K // b
+    check_gemm_ws(W, b, Mb * 7 // 10, Mb * 4 // 10, M, seed=N)
+
+
+def test_gemm_ws_short_reduction_dead_stage():
+    """A 64-column stage that is pruned in every row is skipped (short reduction, many rows)."""
+    N, K, b, M = 512, 256, 16, 40000
+    W = inputs.normal_weights(N, K, 0.02, 7100)
+    W[:, 64:128] = 0.0
+    Mb = N * K // b
+    desc, bufs, packed, p, X, ref = check_gemm_ws(W, b, Mb // 2, Mb // 4, M, seed=3)
+    h = O.parse_header(O.pack(p, b))
+    rec = O.pack(p, b)[h["off_rec"]:h["off_rec"] + 16 * 16].view(np.uint32).reshape(-1, 4)
+    assert rec[1, 3] == 0                                    # stage 1 of the first row tile is dead
