@@ -361,11 +361,30 @@ def run_gpu(args):
         c1.record()
         torch.cuda.synchronize()
         cublas_ms = c0.elapsed_time(c1) / 10
+        # the fused ADMM step (projection + dual update + quadratic term) on the same weight with a
+        # dual tensor, timed beside the path: 16 bytes per weight are what it has to move
+        U_dual = torch.randn(W.shape, device="cuda", generator=torch.Generator("cuda").manual_seed(21060830)) * 0.004
+        U_next = torch.empty(W.numel(), dtype=torch.float32, device="cuda")
+        resid = torch.zeros(1, dtype=torch.float64, device="cuda")
+        for _ in range(3):
+            bufs.admm_step(W, U_dual, U_next, resid)
+        a0 = torch.cuda.Event(enable_timing=True)
+        a1 = torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        a0.record()
+        for _ in range(20):
+            bufs.admm_step(W, U_dual, U_next, resid)
+        a1.record()
+        torch.cuda.synchronize()
+        admm_ms = a0.elapsed_time(a1) / 20
+        del U_dual, U_next
         line["phases"] = {
             "project_ms": proj_ms, "pack_ms": pack_ms, "gemm_ms": gemm_ms,
             "projection_gbs_algorithmic": abytes["projection"] / (proj_ms * 1e-3) / 1e9,
             "gemm_effective_tflops": flops / (gemm_ms * 1e-3) / 1e12,
             "gemm_executed_dense_tflops": dense_flops / (gemm_ms * 1e-3) / 1e12,
+            "admm_step_ms": admm_ms,
+            "admm_step_gbs_algorithmic": 16.0 * W.numel() / (admm_ms * 1e-3) / 1e9,
             "cublas_dense_bf16_ms": cublas_ms,
             "cublas_dense_bf16_tflops": dense_flops / (cublas_ms * 1e-3) / 1e12,
         }
@@ -385,6 +404,10 @@ def run_gpu(args):
             "projection": {"bound": "hbm", "achieved": abytes["projection"] / (proj_ms * 1e-3) / 1e9,
                            "peak": peaks["hbm_gbs"], "unit": "GB/s",
                            "frac": abytes["projection"] / (proj_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]},
+            # mwu_admm_step: W, U in; Q, U_next out
+            "admm_step": {"bound": "hbm", "achieved": 16.0 * W.numel() / (admm_ms * 1e-3) / 1e9,
+                          "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                          "frac": 16.0 * W.numel() / (admm_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]},
         }
         line["clocks"] = sampler.summary()
         line["e2e"] = {"value": e2e_value, "unit": UNIT, "ms_per_step": e2e_ms, "steps": e2e_steps,
