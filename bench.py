@@ -291,7 +291,7 @@ def run_gpu(args):
     # memory and its Y back.  The copies run on their own streams with two sets of device buffers,
     # so step i's download and step i+1's upload overlap step i's kernels (the link is full duplex);
     # the kernels themselves stay in order on one stream and share the projection / packed buffers.
-    e2e_steps = max(2, min(args.steps, 10))
+    e2e_steps = max(2, min(args.steps, 30))
     Wb, Xb, Yb = [W, torch.empty_like(W)], [X, torch.empty_like(X)], [Y, torch.empty_like(Y)]
     Yh = [Y_host, torch.empty_like(Y_host).pin_memory()]
     s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
