@@ -4,7 +4,10 @@
  *
  * Conventions that hold for every entry point
  *   - All tensor pointers are DEVICE pointers owned by the caller, 16-byte aligned unless
- *     stated otherwise; the library allocates nothing and keeps no state between calls.
+ *     stated otherwise; the library allocates nothing.  What it keeps between calls is host-side
+ *     bookkeeping only: the address of one driver entry point, a launch counter
+ *     (mwu_kernel_launches) and, for mwu_project_static, the device address of its built-in
+ *     scratch array per device (stale after a cudaDeviceReset: do not call it again then).
  *   - Descriptors (mwu_proj_desc) and scalar arguments are HOST values.
  *   - Work is enqueued on `cuda_stream` (a cudaStream_t passed as void*, NULL = default
  *     stream).  No call synchronises with the host.
@@ -68,11 +71,21 @@ typedef struct {
     int32_t prune_key;      /* mwu_prune_key                                                  */
     int64_t k_unify;        /* number of blocks unified OR pruned (0 <= k_prune <= k_unify)   */
     int64_t k_prune;        /* number of blocks pruned to zero                                */
-    int32_t algo;           /* mwu_proj_algo; only mwu_project reads it                       */
+    int32_t algo;           /* mwu_proj_algo; read by mwu_project, mwu_project_static and
+                               mwu_admm_step                                                  */
     int32_t reserved;       /* 0                                                              */
+    /* Grouped pruning (0, 0 = off: blocks are pruned one by one, the paper's rule).  When set,
+     * the prune decision is taken for whole groups of prune_group_rows x prune_group_cols
+     * weights: see mwu_project. */
+    int32_t prune_group_rows;   /* 0, 32, 64, 128 or 256; rows % prune_group_rows == 0        */
+    int32_t prune_group_cols;   /* 0, 16, 32 or 64; >= block; cols % prune_group_cols == 0    */
 } mwu_proj_desc;
 
 const char *mwu_status_string(int status);
+
+/* Number of kernels this library has launched in this process so far (all entry points, all
+ * threads).  Host-side counter, for telemetry. */
+uint64_t mwu_kernel_launches(void);
 
 /* Ratio -> integer count, (permille * n_blocks + 500) / 1000 in integers.  The paper gives
  * ratios (Section 1, "unification ratio"); counts cross this ABI as integers so that no
@@ -94,6 +107,17 @@ int64_t mwu_count_from_permille(int64_t n_blocks, int32_t permille);
  * ordered by block index.  Output of a pruned block is +0; of a unified block +q where
  * v_l >= 0 (this includes -0.0) and -q otherwise, q rounded to fp32; other blocks are
  * copied bit for bit.
+ *
+ * Grouped pruning (desc->prune_group_rows/cols set; not in the paper, whose Section 3.2 only says
+ * that pruned blocks "can be completely skipped": a tensor-core tile can skip a column slice only
+ * when it is zero in all of the tile's rows, so this variant prunes whole tile-aligned groups).
+ * The tensor is cut into groups of prune_group_rows x prune_group_cols weights; a group's key is
+ * the sum of its blocks' prune keys (per row a pairwise tree over the row's blocks inside the
+ * group, then a pairwise tree over the group's rows, fp64); the k_prune / (blocks per group)
+ * groups with the smallest keys are zeroed (equal keys: lower group index, row tile first);
+ * k_prune must be a multiple of the blocks per group.  This is the Euclidean projection onto
+ * "at least that many groups are zero".  Unification then works block by block as above among
+ * the blocks outside the pruned groups.
  *
  *   W, U_dual      in   fp32 [rows*cols]; U_dual may be NULL
  *   Q              out  fp32 [rows*cols]; may be NULL (only the compressed form is wanted)
@@ -152,8 +176,11 @@ int mwu_admm_step(const mwu_proj_desc *desc, const float *W, const float *U_dual
  * Limits and rules:
  *   - at most MWU_STATIC_MAX_BLOCKS blocks (rows*cols/block); larger tensors return
  *     MWU_ERR_WORKSPACE and nothing is launched -- use mwu_project with your own workspace;
- *   - the first call on each device looks up the device address of the built-in array (one
- *     runtime query, no allocation); make that first call outside any stream capture;
+ *   - the first call on each device looks up the device address of the built-in array.  If the
+ *     library's device code has not been loaded on that device yet, this query loads it, and the
+ *     driver then sets the array's memory aside; so make that first call at start-up, before a
+ *     memory budget is frozen and outside any stream capture.  Later calls on the device change
+ *     nothing;
  *   - all calls on one device share the array: two calls whose kernels can overlap on the GPU
  *     (different streams without an ordering between them) race and give undefined results;
  *     calls on one stream, or otherwise ordered, are fine.  Each call clears the part of the
@@ -214,6 +241,9 @@ int mwu_pack(const mwu_proj_desc *desc, const float *W, const float *U_dual, con
  *   Y        out  [M][ldy], ldy >= rows; y_dtype 0: bf16 (round to nearest even, ldy % 8 == 0),
  *                 1: fp32 (ldy % 4 == 0)
  * M may be any positive value (ragged last tile is handled); M == 0 is a no-op.
+ * `desc` must be the descriptor `packed` was made with (the host cannot read the device buffer):
+ * the kernels compare it with the header of `packed` and, on a mismatch, set MWU_DEV_BOUNDS and
+ * write nothing.  The same holds for mwu_decode, mwu_gemm_ws and mwu_conv_implicit.
  */
 int mwu_gemm(const mwu_proj_desc *desc, const void *packed, const void *X, int64_t M,
              int64_t ldx, void *Y, int64_t ldy, int32_t y_dtype, uint32_t *dev_status,
@@ -250,7 +280,7 @@ int mwu_gemm_ws(const mwu_proj_desc *desc, const void *packed, const void *X, in
 
 /*
  * mwu_conv_implicit -- the same contraction for a convolution lowered to GEMM without
- * materialising the lowered matrix (Section 3.2: "convolution ... implemented by GEMM"):
+ * materialising the lowered matrix (Section 3.2 treats a layer's convolution as a GEMM):
  *   A[(n,oh,ow)][(c,i,j)] = x[n][c][oh*stride+i-pad][ow*stride+j-pad]  (0 outside),
  *   y[n][o][oh][ow] = sum_k A[(n,oh,ow)][k] * W_hat[o][k],  desc->cols == c*kh*kw.
  *   X  in  bf16 NCHW [n][c][h][w];   Y  out NCHW [n][rows][oh][ow], y_dtype as above.
@@ -259,6 +289,24 @@ int mwu_conv_implicit(const mwu_proj_desc *desc, const void *packed, const void 
                       int32_t n, int32_t c, int32_t h, int32_t w, int32_t kh, int32_t kw,
                       int32_t stride, int32_t pad, void *Y_nchw, int32_t y_dtype,
                       uint32_t *dev_status, void *cuda_stream);
+
+/*
+ * mwu_conv_implicit_ws -- mwu_conv_implicit with a caller-owned scratch buffer, the counterpart
+ * of mwu_gemm_ws: given `workspace` of at least mwu_conv_workspace_bytes(...) bytes (device
+ * memory, 256-byte aligned) the weights are expanded once per call as by mwu_decode and the
+ * tensor-core kernel reads them beside the gathered activation tiles, instead of decoding every
+ * weight record again for every activation tile.  Same contraction, same rounding of operands.
+ * mwu_conv_workspace_bytes returns 0 when the shape is not served by this path (or desc is
+ * invalid); with workspace == NULL, or fewer bytes than that, the call behaves exactly like
+ * mwu_conv_implicit.  The workspace holds nothing between calls.
+ */
+size_t mwu_conv_workspace_bytes(const mwu_proj_desc *desc, int32_t n, int32_t c, int32_t h,
+                                int32_t w, int32_t kh, int32_t kw, int32_t stride, int32_t pad);
+int mwu_conv_implicit_ws(const mwu_proj_desc *desc, const void *packed, const void *X_nchw,
+                         int32_t n, int32_t c, int32_t h, int32_t w, int32_t kh, int32_t kw,
+                         int32_t stride, int32_t pad, void *Y_nchw, int32_t y_dtype,
+                         void *workspace, size_t workspace_bytes, uint32_t *dev_status,
+                         void *cuda_stream);
 
 #ifdef __cplusplus
 }

@@ -3,10 +3,12 @@
 TEST INFRASTRUCTURE ONLY.  This file is a plain, slow, fp64 restatement of what
 the paper defines; it exists so that the CUDA library can be checked against
 something that is not itself.  It shares no code with the CUDA path, is never
-imported by the library, and must not be tuned for speed.
+imported by the library, knows nothing about how the CUDA kernels lay their data
+out, and must not be tuned for speed.
 
 What follows the paper directly
-  * block partition of a weight tensor               -- Section 3.1, first paragraph
+  * block partition of a weight tensor by a block shape -- Section 3.1, first paragraph
+    (1-dim, 2-dim and 3-dim shapes; Table 1 lists [2,2], [4,1], [8,1], [2,2,2])
   * unified value q = mean |w| of the block          -- Section 3.1, text after Eq. (2)
   * sign rule  v = +q if w >= 0 else -q              -- Eq. (2)
   * pruning = the special case q = 0                 -- Section 3.1, "special situation"
@@ -14,6 +16,8 @@ What follows the paper directly
   * Unify(W + U) is what ADMM calls                  -- Algorithm 1
   * pruned blocks are skipped, unified blocks share
     one multiplication per output                    -- Section 3.2, Fig. 2 text, Table 1
+  * keeping 2 of every 4 consecutive weights         -- Section 4.7 (the pruning half of the
+                                                        combination test)
 
 Readings where the paper is silent (each is also pinned stage-wise by tests)
   * unification loss of a block  L_u = sum (|v| - q)^2   (squared distance to its
@@ -27,6 +31,14 @@ Readings where the paper is silent (each is also pinned stage-wise by tests)
   * sign bit = (v < 0), so -0.0 and +0.0 both count as ">= 0"
   * fp64 arithmetic, every operation rounded on its own, block sums taken as a
     balanced pairwise tree (l with l^1, then l^2, ...)
+  * axes of a block shape [D1, D2(, D3)] on a weight viewed as W[rows][cin * taps]
+    (taps = kh*kw, reduction index = cin*taps + tap): D1 runs along the input channels
+    (the reduction axis whose signed inputs are added before the one multiplication, the
+    only axis Table 1's multiplier column counts), D2 along the output rows, D3 along the
+    kernel taps; a tap count that D3 does not divide leaves a shorter last block
+  * grouped pruning (not in the paper; a constraint set of this library that lets a
+    tile-based GEMM skip work): the prune decision is taken for whole groups of
+    group_rows x group_cols weights, the group's key being the sum of its blocks' prune keys
 
 Parity status: every function below is pinned by tests/test_oracle_*.py against
 closed forms, brute force or a library routine.  The mixed-mode rule is a reading,
@@ -40,20 +52,75 @@ from typing import Optional, Tuple
 
 import numpy as np
 
-# ----------------------------------------------------------------------------
-# packed format constants (a file format shared by specification, not by code)
-# ----------------------------------------------------------------------------
-TILE_ROWS = 128          # rows of W per record
-STAGE_K = 64             # reduction-axis extent per record
-HEADER_BYTES = 256
-SECTION_ALIGN = 256
-MAGIC = b"MWUPACK1"
-VERSION = 4
-
 
 def count_from_permille(n_blocks: int, permille: int) -> int:
     """Integer count for a ratio given in 1/1000: round half up, integers only."""
     return (int(permille) * int(n_blocks) + 500) // 1000
+
+
+# ----------------------------------------------------------------------------
+# Section 3.1: the block partition
+# ----------------------------------------------------------------------------
+@dataclasses.dataclass(frozen=True)
+class BlockShape:
+    """Block shape [D1, D2, D3] on W[rows][cin * taps]: dk input channels x dr output rows x
+    dt kernel taps.  The 1-dim blocks of b consecutive reduction-axis entries are (b, 1, 1)
+    with taps = 1."""
+    dk: int
+    dr: int = 1
+    dt: int = 1
+    taps: int = 1
+
+
+def as_shape(b) -> BlockShape:
+    return b if isinstance(b, BlockShape) else BlockShape(int(b))
+
+
+@dataclasses.dataclass
+class Partition:
+    idx: np.ndarray        # int64 [Mb][n_max]: flat indices of each block's weights, -1 = none
+    size: np.ndarray       # int64 [Mb]: weights in the block
+    n_max: int
+    row_runs: bool = False  # blocks are consecutive runs of one row: idx == arange(N*K).reshape(Mb, n_max)
+
+
+def partition(N: int, K: int, shape) -> Partition:
+    """Blocks of W[N][K] in index order j = (row group, channel group, tap group); inside a
+    block the weights are ordered (row, channel, tap)."""
+    s = as_shape(shape)
+    assert K % s.taps == 0
+    cin = K // s.taps
+    assert cin % s.dk == 0 and N % s.dr == 0, "block shape must tile rows and input channels"
+    ntg = (s.taps + s.dt - 1) // s.dt
+    n_max = s.dk * s.dr * s.dt
+    assert n_max & (n_max - 1) == 0, "block size must be a power of two"
+    gi, gc, gt = np.meshgrid(np.arange(N // s.dr), np.arange(cin // s.dk), np.arange(ntg), indexing="ij")
+    r, c, t = np.meshgrid(np.arange(s.dr), np.arange(s.dk), np.arange(s.dt), indexing="ij")
+    # first weight of block j, and the offset of member (r, c, t) from it
+    first = (gi.reshape(-1) * s.dr) * K + (gc.reshape(-1) * s.dk) * s.taps + gt.reshape(-1) * s.dt
+    offs = r.reshape(-1) * K + c.reshape(-1) * s.taps + t.reshape(-1)
+    idx = (first[:, None] + offs[None, :]).astype(np.int64)
+    if s.taps % s.dt == 0:
+        return Partition(idx=idx, size=np.full(idx.shape[0], n_max, dtype=np.int64), n_max=n_max,
+                         row_runs=(s.dr == 1 and s.dt == 1 and s.taps == 1))
+    ok = (gt.reshape(-1) * s.dt)[:, None] + t.reshape(-1)[None, :] < s.taps
+    idx = np.where(ok, idx, -1)
+    size = ok.sum(axis=1).astype(np.int64)
+    assert np.all(size & (size - 1) == 0), "a short last block must still hold a power of two"
+    # members first, holes last, member order kept
+    order = np.argsort(~ok, axis=1, kind="stable")
+    idx = np.take_along_axis(idx, order, axis=1)
+    return Partition(idx=idx, size=size, n_max=n_max)
+
+
+def gather_blocks(V: np.ndarray, part: Partition) -> np.ndarray:
+    """fp32 [Mb][n_max]: the blocks' values (0 in the holes of short blocks)."""
+    flat = np.ascontiguousarray(V, dtype=np.float32).reshape(-1)
+    if part.row_runs:
+        return flat.reshape(-1, part.n_max).copy()
+    out = flat[np.maximum(part.idx, 0)]
+    out[part.idx < 0] = np.float32(0.0)
+    return out
 
 
 # ----------------------------------------------------------------------------
@@ -80,42 +147,72 @@ def tree_sum(x: np.ndarray) -> np.ndarray:
 @dataclasses.dataclass
 class BlockStats:
     S: np.ndarray      # sum |v|           (L1 norm of the block), fp64 [Mb]
-    q: np.ndarray      # S / b             (unified value),        fp64 [Mb]
+    q: np.ndarray      # S / n             (unified value),        fp64 [Mb]
     L_u: np.ndarray    # sum (|v| - q)^2   (unification loss),     fp64 [Mb]
     L_p: np.ndarray    # sum v^2           (prune loss),           fp64 [Mb]
 
 
-def block_stats(V: np.ndarray, b: int) -> BlockStats:
-    """Per-block statistics of V[N][K] with blocks of b consecutive entries of a row."""
+def block_stats(V: np.ndarray, b, part: Optional[Partition] = None) -> BlockStats:
+    """Per-block statistics of V[N][K]; b is a width (blocks of b consecutive entries of a row)
+    or a BlockShape."""
     V = np.ascontiguousarray(V, dtype=np.float32)
     N, K = V.shape
-    assert K % b == 0
     assert np.all(np.isfinite(V)), "non-finite weights are outside the method's domain"
-    a = np.abs(V.astype(np.float64)).reshape(N * (K // b), b)
+    if part is None:
+        part = partition(N, K, b)
+    a = np.abs(gather_blocks(V, part).astype(np.float64))
     S = tree_sum(a)
-    q = S / float(b)                       # text after Eq. (2): average of |w|
+    q = S / part.size.astype(np.float64)   # text after Eq. (2): average of |w|
     d = a - q[:, None]
+    if int(part.size.min()) < part.n_max:
+        d[part.idx < 0] = 0.0              # the holes of short blocks are not weights
     L_u = tree_sum(d * d)                  # distance^2 to the unified block (Eq. 7 projection)
     L_p = tree_sum(a * a)                  # distance^2 to the zero block (q = 0 special case)
     return BlockStats(S=S, q=q, L_u=L_u, L_p=L_p)
 
 
 # ----------------------------------------------------------------------------
-# selection by ratio (Section 3.1 example; Section 4.3 "threshold is applied to each block")
+# selection by ratio (Section 3.1's example; Section 4.3: a threshold per block after training)
 # ----------------------------------------------------------------------------
+def group_prune_keys(prune_key: np.ndarray, N: int, K: int, b: int, group_rows: int,
+                     group_cols: int) -> np.ndarray:
+    """Key of every prune group of a 1-dim partition, fp64 [N/group_rows][K/group_cols]: the
+    blocks of one row inside the group are summed first (pairwise tree in column order), then
+    the rows of the group (pairwise tree in row order)."""
+    assert N % group_rows == 0 and K % group_cols == 0 and group_cols % b == 0
+    k4 = prune_key.reshape(N // group_rows, group_rows, K // group_cols, group_cols // b)
+    per_row = tree_sum(k4)                                     # [tile][row][slice]
+    return tree_sum(np.moveaxis(per_row, 1, -1))               # [tile][slice]
+
+
 def select_blocks(stats: BlockStats, k_unify: int, k_prune: int,
-                  prune_key: str = "l2sq") -> Tuple[np.ndarray, np.ndarray]:
+                  prune_key: str = "l2sq", groups=None) -> Tuple[np.ndarray, np.ndarray]:
     """Return boolean masks (pruned, unified) over the Mb blocks.
 
     k_unify counts unified and pruned blocks together; k_prune <= k_unify.
     Order of blocks: key ascending, then block index ascending.
+    groups = (N, K, b, group_rows, group_cols): blocks are pruned by whole groups (k_prune must
+    be a multiple of the blocks per group); order of groups: key ascending, then group index
+    (row tile, then column slice) ascending.
     """
     Mb = stats.S.shape[0]
     assert 0 <= k_prune <= k_unify <= Mb
     kp = stats.L_p if prune_key == "l2sq" else stats.S
-    order_p = np.argsort(kp, kind="stable")          # stable: ties keep index order
     pruned = np.zeros(Mb, dtype=bool)
-    pruned[order_p[:k_prune]] = True
+    if groups is None:
+        order_p = np.argsort(kp, kind="stable")          # stable: ties keep index order
+        pruned[order_p[:k_prune]] = True
+    else:
+        N, K, b, gr, gc = groups
+        per_group = gr * gc // b
+        assert k_prune % per_group == 0, "grouped pruning takes whole groups"
+        gk = group_prune_keys(kp, N, K, b, gr, gc)
+        order_g = np.argsort(gk.reshape(-1), kind="stable")[:k_prune // per_group]
+        gmask = np.zeros(gk.size, dtype=bool)
+        gmask[order_g] = True
+        gmask = gmask.reshape(gk.shape)                   # [tile][slice]
+        full = np.repeat(np.repeat(gmask, gr, axis=0), gc // b, axis=1)   # [N][K/b]
+        pruned = full.reshape(-1).copy()
     rest = np.flatnonzero(~pruned)                   # ascending block index
     order_u = rest[np.argsort(stats.L_u[rest], kind="stable")]
     unified = np.zeros(Mb, dtype=bool)
@@ -135,24 +232,39 @@ class Projection:
     sign: np.ndarray       # bool [N][K]: v < 0
     stats: BlockStats
     V: np.ndarray          # fp32 [N][K]: the tensor that was projected
+    part: Partition        # which weights each block holds
 
 
-def project(W: np.ndarray, b: int, k_unify: int, k_prune: int,
-            U: Optional[np.ndarray] = None, prune_key: str = "l2sq") -> Projection:
+def project(W: np.ndarray, b, k_unify: int, k_prune: int,
+            U: Optional[np.ndarray] = None, prune_key: str = "l2sq",
+            prune_group: Optional[Tuple[int, int]] = None) -> Projection:
     V = combine_dual(W, U)
     N, K = V.shape
-    stats = block_stats(V, b)
-    pruned, unified = select_blocks(stats, k_unify, k_prune, prune_key)
+    part = partition(N, K, b)
+    stats = block_stats(V, b, part)
+    groups = None
+    if prune_group is not None:
+        s = as_shape(b)
+        assert s.dr == 1 and s.dt == 1 and s.taps == 1, "grouped pruning is defined for 1-dim blocks"
+        groups = (N, K, s.dk, prune_group[0], prune_group[1])
+    pruned, unified = select_blocks(stats, k_unify, k_prune, prune_key, groups)
     q32 = stats.q.astype(np.float32)
-    Vb = V.reshape(-1, b)
-    Qb = Vb.copy()
-    sign = Vb < 0                                    # -0.0 < 0 is False
-    uni_vals = np.where(sign, -q32[:, None], q32[:, None]).astype(np.float32)
-    Qb[unified] = uni_vals[unified]
-    Qb[pruned] = np.float32(0.0)
+    sign = V < 0                                     # -0.0 < 0 is False
+    Qf = V.reshape(-1).copy()
+    for cls, is_unified in ((unified, True), (pruned, False)):
+        rows = np.flatnonzero(cls)
+        if rows.size == 0:
+            continue
+        ii = part.idx[rows]
+        mm = ii >= 0                                 # the holes of short blocks are not weights
+        if is_unified:
+            vals = np.where(sign.reshape(-1)[np.maximum(ii, 0)], -q32[rows, None], q32[rows, None])
+        else:
+            vals = np.zeros(ii.shape, dtype=np.float32)
+        Qf[ii[mm]] = vals[mm].astype(np.float32)
     u = np.where(unified, q32, np.float32(0.0)).astype(np.float32)
-    return Projection(Q=Qb.reshape(N, K), u=u, pruned=pruned, unified=unified,
-                      sign=sign.reshape(N, K), stats=stats, V=V)
+    return Projection(Q=Qf.reshape(N, K), u=u, pruned=pruned, unified=unified,
+                      sign=sign, stats=stats, V=V, part=part)
 
 
 @dataclasses.dataclass
@@ -161,7 +273,7 @@ class DualUpdate:
     residual_sq: float     # ||V - Q||_F^2 with unrounded unified magnitudes, fp64
 
 
-def dual_update(p: Projection, b: int) -> DualUpdate:
+def dual_update(p: Projection, b=None) -> DualUpdate:
     """Dual step of ADMM (Algorithm 1, last assignment of the loop; third ADMM step of Section
     3.3): U_{k+1} = U_k + W_{k+1} - Q_{k+1}.  With V = fp32(W_{k+1} + U_k), the tensor that was
     projected, this is V - Q: one fp32 subtraction per entry.  residual_sq is the quadratic term
@@ -169,10 +281,35 @@ def dual_update(p: Projection, b: int) -> DualUpdate:
     summed per block from the fp64 block statistics: sum v^2 for a pruned block, the unification
     loss for a unified block, nothing for a block that keeps its values."""
     U_next = (p.V - p.Q).astype(np.float32)                 # fp32 - fp32, rounded once
-    Vb = p.V.reshape(-1, b).astype(np.float64)
+    Vb = gather_blocks(p.V, p.part).astype(np.float64)
     sumsq = tree_sum(Vb * Vb)
     residual = float(np.sum(sumsq[p.pruned]) + np.sum(p.stats.L_u[p.unified]))
     return DualUpdate(U_next=U_next, residual_sq=residual)
+
+
+# ----------------------------------------------------------------------------
+# Section 4.7: "1x4 blocks with 50 % prune ratio in each block" -- keep n of every m
+# ----------------------------------------------------------------------------
+@dataclasses.dataclass
+class KeepNofM:
+    Q: np.ndarray          # fp32 [N][K]: kept weights copied, the others +0
+    keep: np.ndarray       # bool [N][K]
+    V: np.ndarray
+
+
+def project_n_of_m(W: np.ndarray, n: int = 2, m: int = 4,
+                   U: Optional[np.ndarray] = None) -> KeepNofM:
+    """Euclidean projection onto "at most n non-zeros in every m consecutive entries of a row":
+    the n entries of largest magnitude stay (equal magnitudes: the lower index stays)."""
+    V = combine_dual(W, U)
+    N, K = V.shape
+    assert K % m == 0 and 0 <= n <= m
+    a = np.abs(V.astype(np.float64)).reshape(-1, m)
+    order = np.argsort(-a, axis=1, kind="stable")           # descending |v|, ties by index
+    keep = np.zeros(a.shape, dtype=bool)
+    np.put_along_axis(keep, order[:, :n], True, axis=1)
+    Q = np.where(keep, V.reshape(-1, m), np.float32(0.0)).astype(np.float32)
+    return KeepNofM(Q=Q.reshape(N, K), keep=keep.reshape(N, K), V=V)
 
 
 def bitmap_words(mask: np.ndarray) -> np.ndarray:
@@ -183,6 +320,12 @@ def bitmap_words(mask: np.ndarray) -> np.ndarray:
     bits = padded.reshape(-1, 32).astype(np.uint64)
     weights = (np.uint64(1) << np.arange(32, dtype=np.uint64))
     return (bits * weights).sum(axis=1).astype(np.uint32)
+
+
+def bitmap_bools(words: np.ndarray, n: int) -> np.ndarray:
+    w = np.ascontiguousarray(words, dtype=np.uint32)
+    bits = (w[:, None] >> np.arange(32, dtype=np.uint32)[None, :]) & np.uint32(1)
+    return bits.reshape(-1)[:n].astype(bool)
 
 
 # ----------------------------------------------------------------------------
@@ -201,229 +344,91 @@ def bf16_bits_to_f64(h: np.ndarray) -> np.ndarray:
 
 
 # ----------------------------------------------------------------------------
-# packed format (storage model of Section 3.1 / Table 1: one magnitude per
-# unified block, one sign bit per weight, nothing for pruned blocks)
+# storage form (Section 3.1 / Table 1: one magnitude per unified block, one sign bit
+# per weight of a unified block, nothing for a pruned block, the values of the rest)
 # ----------------------------------------------------------------------------
-def _align(x: int, a: int = SECTION_ALIGN) -> int:
-    return (x + a - 1) // a * a
+STORE_MAGIC = b"MWUSTORE"
+STORE_FIELDS = ["magic", "N", "K", "n_blocks", "n_pruned", "n_unified", "n_dense",
+                "n_unified_weights", "n_dense_weights"]
 
 
-def packed_layout(N: int, K: int, b: int, n_unified: int, n_dense: int, n_pruned: int) -> dict:
-    assert K % STAGE_K == 0 and STAGE_K % b == 0
-    n_pad = _align(N, TILE_ROWS)
-    n_tiles = n_pad // TILE_ROWS
-    n_stages = K // STAGE_K
-    n_plist = n_pruned + (n_pad - N) * (K // b)          # padding rows count as pruned
-    off_rec = HEADER_BYTES
-    off_ulist = _align(off_rec + 16 * (n_tiles * n_stages + 1))
-    off_dpos = _align(off_ulist + 8 * n_unified)
-    off_dpay = _align(off_dpos + 2 * n_dense)
-    off_ppos = _align(off_dpay + 2 * b * n_dense)
-    total = _align(off_ppos + 2 * n_plist)
-    return dict(n_pad=n_pad, n_tiles=n_tiles, n_stages=n_stages, n_plist=n_plist, off_rec=off_rec,
-                off_ulist=off_ulist, off_dpos=off_dpos, off_dpay=off_dpay, off_ppos=off_ppos,
-                total=total)
+def storage_bits(p: Projection, value_bits: int = 32, dense_bits: int = 16) -> dict:
+    """What the storage model costs for this projection, in bits, class by class."""
+    size = p.part.size
+    n_uw = int(size[p.unified].sum())
+    dense = ~(p.pruned | p.unified)
+    n_dw = int(size[dense].sum())
+    return {"class_bits": 2 * int(size.shape[0]),           # which of the three classes a block has
+            "unified_values": value_bits * int(p.unified.sum()),
+            "unified_signs": n_uw,
+            "dense_values": dense_bits * n_dw,
+            "pruned": 0}
 
 
-def tile_offset(pos: np.ndarray, b: int) -> np.ndarray:
-    """Byte offset of block slot `pos` in a decoded 128 x 64 bf16 tile: row r = pos // (64/b)
-    starts at (r // 8) * 1024 + (r % 8) * 128; the row's 16-byte chunk c is stored at chunk
-    position c XOR (r % 8); inside a chunk bytes keep their order."""
-    pos = np.asarray(pos, dtype=np.int64)
-    nb = STAGE_K // b
-    r, i = pos // nb, pos % nb
-    byte_in_row = i * 2 * b
-    c, within = byte_in_row // 16, byte_in_row % 16
-    return (r // 8) * 1024 + (r % 8) * 128 + ((c ^ (r % 8)) * 16) + within
-
-
-def slot_order(off: np.ndarray, b: int) -> np.ndarray:
-    """Permutation that deals entries (given in ascending pos order) round-robin over their
-    store slots: sort by (rank inside the slot, slot)."""
-    off = np.asarray(off, dtype=np.int64)
-    g = min(2 * b, 16)
-    slot = (off % 128) // g
-    rank = np.zeros(off.shape[0], dtype=np.int64)
-    seen = {}
-    for e, sl in enumerate(slot.tolist()):
-        rank[e] = seen.get(sl, 0)
-        seen[sl] = rank[e] + 1
-    return np.lexsort((slot, rank))
-
-
-def tile_offset_inverse(off: int, b: int):
-    r = (off >> 10) * 8 + ((off >> 7) & 7)
-    c = ((off >> 4) & 7) ^ (r & 7)
-    byte_in_row = c * 16 + (off & 15)
-    return r, byte_in_row // (2 * b)
-
-
-HEADER_FIELDS = ["magic", "version", "N", "K", "b", "n_pad", "n_tiles", "n_stages", "n_pruned",
-                 "n_unified", "n_dense", "n_plist", "off_rec", "off_ulist", "off_dpos", "off_dpay",
-                 "off_ppos", "total"]
-
-
-def pack(p: Projection, b: int) -> np.ndarray:
-    """Serialise a projection into the packed byte format (uint8 array).
-
-    A record is (row tile of 128 rows) x (64 reduction-axis entries) and holds 128 * 64/b
-    block slots; slot number pos = row_in_tile * (64/b) + block_in_stage.  A block is addressed
-    by the byte offset `off` of its first value inside the record's decoded tile (bf16, rows of
-    128 bytes, 16-byte chunks of a row XOR-permuted by the row number mod 8 -- the layout the
-    tensor-core instruction reads; see tile_offset).  Per record the blocks are listed by
-    class.  Inside a class list the entries are dealt round-robin over the store slots
-    slot = (off % 128) // g, g = min(2*b, 16): entries with the same slot keep ascending pos
-    order, and the list takes the first entry of every slot (ascending slot), then the second of
-    every slot that has one, and so on (so that neighbouring entries fall into different
-    shared-memory banks when the GEMM writes them):
-      ulist  8 B per unified block: u32 spread sign bits (weight l -> bit l//2 + 16*(l%2)),
-             u16 off, u16 bf16(unified value)
-      dpos   u16 off per dense block;  dpay  its b values as bf16 (round to nearest even)
-      ppos   u16 off per pruned block (rows beyond N are padding and count as pruned)
-    rec[i] = (u32 ubase, dbase, pbase, live) gives where record i starts in each list; rec has
-    one extra entry holding the totals.  live bit s = some row of the record has a non-pruned
-    block overlapping columns [16s, 16s+16).
-    """
+def pack(p: Projection) -> np.ndarray:
+    """The storage form as one byte string: header, the two class bitmaps, then in ascending
+    block order the fp32 magnitude of every unified block, the sign bits of the weights of the
+    unified blocks (block after block, member order) and the bf16 values of the blocks that
+    keep their values.  A pruned block contributes nothing but its bitmap bit."""
     N, K = p.V.shape
-    nb = STAGE_K // b
-    n_unified = int(p.unified.sum())
-    n_pruned = int(p.pruned.sum())
-    n_dense = p.unified.shape[0] - n_unified - n_pruned
-    L = packed_layout(N, K, b, n_unified, n_dense, n_pruned)
-    n_pad, n_tiles, n_stages = L["n_pad"], L["n_tiles"], L["n_stages"]
-    buf = np.zeros(L["total"], dtype=np.uint8)
-
-    hdr = [int.from_bytes(MAGIC, "little"), VERSION, N, K, b, n_pad, n_tiles, n_stages,
-           n_pruned, n_unified, n_dense, L["n_plist"], L["off_rec"], L["off_ulist"],
-           L["off_dpos"], L["off_dpay"], L["off_ppos"], L["total"]]
-    buf[:8 * len(hdr)] = np.frombuffer(struct.pack("<%dQ" % len(hdr), *hdr), dtype=np.uint8)
-
-    pruned = np.ones((n_pad, K // b), dtype=bool)
-    unified = np.zeros((n_pad, K // b), dtype=bool)
-    pruned[:N] = p.pruned.reshape(N, K // b)
-    unified[:N] = p.unified.reshape(N, K // b)
-    sign = np.zeros((n_pad, K), dtype=bool)
-    sign[:N] = p.sign
-    u = np.zeros((n_pad, K // b), dtype=np.float32)
-    u[:N] = p.u.reshape(N, K // b)
-    vbf = np.zeros((n_pad, K), dtype=np.uint16)
-    vbf[:N] = bf16_bits_rne(p.V)
-
-    n_rec = n_tiles * n_stages
-    rec = np.zeros((n_rec + 1, 4), dtype=np.uint32)
-    ulist_w0, ulist_u, dpos, dpay, ppos = [], [], [], [], []
-    n_u = n_d = n_p = 0
-    ell = np.arange(b, dtype=np.uint32)
-    bitw = (np.uint32(1) << (ell // 2 + 16 * (ell % 2)))           # spread sign bit of weight l
-    ubf = bf16_bits_rne(u.reshape(-1)).reshape(u.shape).astype(np.uint32)
-    for t in range(n_tiles):
-        r0 = t * TILE_ROWS
-        for s in range(n_stages):
-            ri = t * n_stages + s
-            P = pruned[r0:r0 + TILE_ROWS, s * nb:(s + 1) * nb]
-            Uf = unified[r0:r0 + TILE_ROWS, s * nb:(s + 1) * nb]
-            D = ~P & ~Uf
-            live = 0
-            for sl in range(4):                      # 16-wide slices of the stage
-                lo = (sl * 16) // b
-                hi = max(lo + 1, ((sl + 1) * 16) // b)
-                if (~P[:, lo:hi]).any():
-                    live |= 1 << sl
-            rec[ri] = (n_u, n_d, n_p, live)
-            pos_u = np.flatnonzero(Uf.reshape(-1)).astype(np.uint32)      # ascending pos
-            pos_d = np.flatnonzero(D.reshape(-1)).astype(np.uint16)
-            pos_p = np.flatnonzero(P.reshape(-1)).astype(np.uint16)
-            pos_u = pos_u[slot_order(tile_offset(pos_u, b), b)]
-            pos_d = pos_d[slot_order(tile_offset(pos_d, b), b)]
-            pos_p = pos_p[slot_order(tile_offset(pos_p, b), b)]
-            sg = sign[r0:r0 + TILE_ROWS, s * STAGE_K:(s + 1) * STAGE_K].reshape(TILE_ROWS * nb, b)
-            sbits = (sg.astype(np.uint32) * bitw).sum(axis=1).astype(np.uint32)
-            ulist_w0.append(sbits[pos_u])
-            ub = ubf[r0:r0 + TILE_ROWS, s * nb:(s + 1) * nb].reshape(-1)[pos_u]
-            ulist_u.append(tile_offset(pos_u, b).astype(np.uint32) | (ub << np.uint32(16)))
-            dpos.append(tile_offset(pos_d, b).astype(np.uint16))
-            vb = vbf[r0:r0 + TILE_ROWS, s * STAGE_K:(s + 1) * STAGE_K].reshape(TILE_ROWS * nb, b)
-            dpay.append(vb[pos_d].reshape(-1))
-            ppos.append(tile_offset(pos_p, b).astype(np.uint16))
-            n_u += pos_u.shape[0]
-            n_d += pos_d.shape[0]
-            n_p += pos_p.shape[0]
-    assert n_u == n_unified and n_d == n_dense and n_p == L["n_plist"]
-    rec[n_rec] = (n_u, n_d, n_p, 0)
-
-    def put(off, arr):
-        raw = np.ascontiguousarray(arr).view(np.uint8).reshape(-1)
-        buf[off:off + raw.shape[0]] = raw
-
-    put(L["off_rec"], rec)
-    if n_unified:
-        ul = np.zeros((n_unified, 2), dtype=np.uint32)
-        ul[:, 0] = np.concatenate(ulist_w0)
-        ul[:, 1] = np.concatenate(ulist_u)
-        put(L["off_ulist"], ul)
-    if n_dense:
-        put(L["off_dpos"], np.concatenate(dpos).astype(np.uint16))
-        put(L["off_dpay"], np.concatenate(dpay).astype(np.uint16))
-    if L["n_plist"]:
-        put(L["off_ppos"], np.concatenate(ppos).astype(np.uint16))
-    return buf
+    dense = ~(p.pruned | p.unified)
+    member = p.part.idx >= 0
+    uni_idx = p.part.idx[p.unified][member[p.unified]]      # member order, block after block
+    den_idx = p.part.idx[dense][member[dense]]
+    hdr = [int.from_bytes(STORE_MAGIC, "little"), N, K, int(p.pruned.shape[0]), int(p.pruned.sum()),
+           int(p.unified.sum()), int(dense.sum()), int(uni_idx.size), int(den_idx.size)]
+    parts = [np.frombuffer(struct.pack("<%dQ" % len(hdr), *hdr), dtype=np.uint8),
+             bitmap_words(p.pruned).view(np.uint8), bitmap_words(p.unified).view(np.uint8),
+             p.u[p.unified].astype(np.float32).view(np.uint8),
+             bitmap_words(p.sign.reshape(-1)[uni_idx]).view(np.uint8),
+             bf16_bits_rne(p.V.reshape(-1)[den_idx]).view(np.uint8)]
+    return np.concatenate(parts)
 
 
-def parse_header(buf: np.ndarray) -> dict:
-    vals = struct.unpack("<%dQ" % len(HEADER_FIELDS), bytes(buf[:8 * len(HEADER_FIELDS)]))
-    h = dict(zip(HEADER_FIELDS, vals))
-    assert h["magic"] == int.from_bytes(MAGIC, "little") and h["version"] == VERSION
-    return h
+def unpack(buf: np.ndarray, b) -> np.ndarray:
+    """Storage form -> the weights the layer multiplies with, fp64 [N][K]: 0 for a pruned block,
+    +-bf16(u) by sign bit for a unified block, the stored bf16 value otherwise."""
+    nh = 8 * len(STORE_FIELDS)
+    h = dict(zip(STORE_FIELDS, struct.unpack("<%dQ" % len(STORE_FIELDS), bytes(buf[:nh]))))
+    assert h["magic"] == int.from_bytes(STORE_MAGIC, "little")
+    N, K, Mb = h["N"], h["K"], h["n_blocks"]
+    part = partition(N, K, b)
+    assert part.idx.shape[0] == Mb
+    nw = (Mb + 31) // 32 * 4
+    o = nh
+    pruned = bitmap_bools(buf[o:o + nw].view(np.uint32), Mb); o += nw
+    unified = bitmap_bools(buf[o:o + nw].view(np.uint32), Mb); o += nw
+    u = buf[o:o + 4 * h["n_unified"]].view(np.float32); o += 4 * h["n_unified"]
+    ns = (h["n_unified_weights"] + 31) // 32 * 4
+    signs = bitmap_bools(buf[o:o + ns].view(np.uint32), h["n_unified_weights"]); o += ns
+    vals = buf[o:o + 2 * h["n_dense_weights"]].view(np.uint16); o += 2 * h["n_dense_weights"]
+    assert o == buf.shape[0]
+    assert int(pruned.sum()) == h["n_pruned"] and int(unified.sum()) == h["n_unified"]
+    member = part.idx >= 0
+    dense = ~(pruned | unified)
+    out = np.zeros(N * K, dtype=np.float64)
+    uni_idx = part.idx[unified][member[unified]]
+    u_bf = bf16_bits_to_f64(bf16_bits_rne(u))
+    per_weight_u = np.repeat(u_bf, part.size[unified])
+    out[uni_idx] = np.where(signs, -per_weight_u, per_weight_u)
+    out[part.idx[dense][member[dense]]] = bf16_bits_to_f64(vals)
+    return out.reshape(N, K)
 
 
-def decode(buf: np.ndarray) -> np.ndarray:
-    """Packed bytes -> decoded weights W_hat[N][K] in fp64.
-
-    pruned block -> 0; unified block -> +-bf16(u) by sign bit; dense block ->
-    its stored bf16 values.  This is what the GEMM multiplies with.
-    """
-    h = parse_header(buf)
-    N, K, b = h["N"], h["K"], h["b"]
-    nb = STAGE_K // b
-    n_tiles, n_stages = h["n_tiles"], h["n_stages"]
-    n_rec = n_tiles * n_stages
-    rec = buf[h["off_rec"]:h["off_rec"] + 16 * (n_rec + 1)].view(np.uint32).reshape(-1, 4)
-    ulist = buf[h["off_ulist"]:h["off_ulist"] + 8 * h["n_unified"]].view(np.uint32).reshape(-1, 2)
-    dpos = buf[h["off_dpos"]:h["off_dpos"] + 2 * h["n_dense"]].view(np.uint16)
-    dpay = buf[h["off_dpay"]:h["off_dpay"] + 2 * b * h["n_dense"]].view(np.uint16)
-    ppos = buf[h["off_ppos"]:h["off_ppos"] + 2 * h["n_plist"]].view(np.uint16)
-    What = np.full((h["n_pad"], K), np.nan, dtype=np.float64)     # every slot must be listed once
-    for t in range(n_tiles):
-        for s in range(n_stages):
-            ri = t * n_stages + s
-            for e in range(int(rec[ri, 0]), int(rec[ri + 1, 0])):
-                sbits, w1 = int(ulist[e, 0]), int(ulist[e, 1])
-                uval = float(bf16_bits_to_f64(np.array([w1 >> 16], dtype=np.uint16))[0])
-                r, i = tile_offset_inverse(w1 & 0xFFFF, b)
-                for l in range(b):
-                    neg = (sbits >> (l // 2 + 16 * (l % 2))) & 1
-                    What[t * TILE_ROWS + r, s * STAGE_K + i * b + l] = -uval if neg else uval
-            for e in range(int(rec[ri, 1]), int(rec[ri + 1, 1])):
-                r, i = tile_offset_inverse(int(dpos[e]), b)
-                k0 = s * STAGE_K + i * b
-                What[t * TILE_ROWS + r, k0:k0 + b] = bf16_bits_to_f64(dpay[e * b:(e + 1) * b])
-            for e in range(int(rec[ri, 2]), int(rec[ri + 1, 2])):
-                r, i = tile_offset_inverse(int(ppos[e]), b)
-                k0 = s * STAGE_K + i * b
-                What[t * TILE_ROWS + r, k0:k0 + b] = 0.0
-    assert not np.isnan(What).any()
-    return What[:N]
-
-
-def decoded_weights(p: Projection, b: int) -> np.ndarray:
+def decoded_weights(p: Projection, b=None) -> np.ndarray:
     """W_hat straight from a projection (no byte format involved), fp64 [N][K]."""
     N, K = p.V.shape
     u_bf = bf16_bits_to_f64(bf16_bits_rne(p.u))
-    v_bf = bf16_bits_to_f64(bf16_bits_rne(p.V)).reshape(-1, b)
-    out = v_bf.copy()
-    uni = np.where(p.sign.reshape(-1, b), -u_bf[:, None], u_bf[:, None])
-    out[p.unified] = uni[p.unified]
-    out[p.pruned] = 0.0
+    out = bf16_bits_to_f64(bf16_bits_rne(p.V)).reshape(-1)
+    member = p.part.idx >= 0
+    sign = p.sign.reshape(-1)
+    rows = np.flatnonzero(p.unified)
+    ii, mm = p.part.idx[rows], member[rows]
+    vals = np.where(sign[np.maximum(ii, 0)], -u_bf[rows, None], u_bf[rows, None])
+    out[ii[mm]] = vals[mm]
+    rows = np.flatnonzero(p.pruned)
+    ii, mm = p.part.idx[rows], member[rows]
+    out[ii[mm]] = 0.0
     return out.reshape(N, K)
 
 
@@ -436,8 +441,9 @@ def gemm(X: np.ndarray, What: np.ndarray) -> np.ndarray:
 
 
 def gemm_shared_partial(X: np.ndarray, p: Projection, b: int) -> np.ndarray:
-    """The paper's form (Fig. 2 text): pruned blocks are skipped; a unified block costs one
-    multiplication per output: u * (signed sum of its inputs).  Dense blocks as usual."""
+    """The paper's form (Fig. 2 text) for 1-dim blocks: pruned blocks are skipped; a unified
+    block costs one multiplication per output: u * (signed sum of its inputs).  Dense blocks as
+    usual."""
     X = np.asarray(X, dtype=np.float64)
     M = X.shape[0]
     N, K = p.V.shape

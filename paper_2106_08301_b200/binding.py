@@ -15,9 +15,10 @@ import torch
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libmwu.so")
 
-EXPORTS = ["mwu_status_string", "mwu_count_from_permille", "mwu_project_workspace_bytes",
-           "mwu_project", "mwu_admm_step", "mwu_project_static", "mwu_packed_bytes", "mwu_pack", "mwu_gemm", "mwu_decode", "mwu_gemm_workspace_bytes", "mwu_gemm_ws",
-           "mwu_conv_implicit"]
+EXPORTS = ["mwu_status_string", "mwu_kernel_launches", "mwu_count_from_permille",
+           "mwu_project_workspace_bytes", "mwu_project", "mwu_admm_step", "mwu_project_static",
+           "mwu_packed_bytes", "mwu_pack", "mwu_gemm", "mwu_decode", "mwu_gemm_workspace_bytes",
+           "mwu_gemm_ws", "mwu_conv_implicit", "mwu_conv_workspace_bytes", "mwu_conv_implicit_ws"]
 MWU_STATIC_MAX_BLOCKS = 1048576
 
 MWU_OK = 0
@@ -37,7 +38,8 @@ class MwuError(RuntimeError):
 class ProjDesc(ctypes.Structure):
     _fields_ = [("rows", ctypes.c_int64), ("cols", ctypes.c_int64), ("block", ctypes.c_int32),
                 ("prune_key", ctypes.c_int32), ("k_unify", ctypes.c_int64),
-                ("k_prune", ctypes.c_int64), ("algo", ctypes.c_int32), ("reserved", ctypes.c_int32)]
+                ("k_prune", ctypes.c_int64), ("algo", ctypes.c_int32), ("reserved", ctypes.c_int32),
+                ("prune_group_rows", ctypes.c_int32), ("prune_group_cols", ctypes.c_int32)]
 
 
 _lib = None
@@ -54,6 +56,8 @@ def lib() -> ctypes.CDLL:
         dp = ctypes.POINTER(ProjDesc)
         L.mwu_status_string.restype = ctypes.c_char_p
         L.mwu_status_string.argtypes = [ctypes.c_int]
+        L.mwu_kernel_launches.restype = ctypes.c_uint64
+        L.mwu_kernel_launches.argtypes = []
         L.mwu_count_from_permille.restype = i64
         L.mwu_count_from_permille.argtypes = [i64, i32]
         L.mwu_project_workspace_bytes.restype = sz
@@ -78,6 +82,10 @@ def lib() -> ctypes.CDLL:
         L.mwu_gemm_ws.argtypes = [dp, vp, vp, i64, i64, vp, i64, i32, vp, ctypes.c_size_t, vp, vp]
         L.mwu_conv_implicit.restype = ctypes.c_int
         L.mwu_conv_implicit.argtypes = [dp, vp, vp] + [i32] * 8 + [vp, i32, vp, vp]
+        L.mwu_conv_workspace_bytes.restype = sz
+        L.mwu_conv_workspace_bytes.argtypes = [dp] + [i32] * 8
+        L.mwu_conv_implicit_ws.restype = ctypes.c_int
+        L.mwu_conv_implicit_ws.argtypes = [dp, vp, vp] + [i32] * 8 + [vp, i32, vp, sz, vp, vp]
         _lib = L
     return _lib
 
@@ -99,9 +107,16 @@ def status_string(status: int) -> str:
 
 
 def make_desc(rows: int, cols: int, block: int, k_unify: int, k_prune: int,
-              prune_key: int = MWU_PRUNE_KEY_L2SQ, algo: int = MWU_ALGO_AUTO) -> ProjDesc:
+              prune_key: int = MWU_PRUNE_KEY_L2SQ, algo: int = MWU_ALGO_AUTO,
+              prune_group=None) -> ProjDesc:
+    """prune_group = (rows, cols) of a prune group, or None for block-by-block pruning."""
+    gr, gc = prune_group if prune_group else (0, 0)
     return ProjDesc(int(rows), int(cols), int(block), int(prune_key), int(k_unify), int(k_prune),
-                    int(algo), 0)
+                    int(algo), 0, int(gr), int(gc))
+
+
+def mwu_kernel_launches() -> int:
+    return int(lib().mwu_kernel_launches())
 
 
 def mwu_count_from_permille(n_blocks: int, permille: int) -> int:
@@ -199,6 +214,23 @@ def mwu_conv_implicit(desc, packed, X, n, c, h, w, kh, kw, stride, pad, Y, y_dty
                                  int(y_dtype), _ptr(dev_status), _stream(stream))
     if check and rc != MWU_OK:
         raise MwuError(rc, "mwu_conv_implicit")
+    return rc
+
+
+def mwu_conv_workspace_bytes(desc, n, c, h, w, kh, kw, stride, pad) -> int:
+    return int(lib().mwu_conv_workspace_bytes(ctypes.byref(desc), int(n), int(c), int(h), int(w), int(kh),
+                                              int(kw), int(stride), int(pad)))
+
+
+def mwu_conv_implicit_ws(desc, packed, X, n, c, h, w, kh, kw, stride, pad, Y, y_dtype, workspace, dev_status,
+                         stream=None, check=True) -> int:
+    """mwu_conv_implicit with a scratch tensor (uint8, or None); its size is taken from the tensor."""
+    nbytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    rc = lib().mwu_conv_implicit_ws(ctypes.byref(desc), _ptr(packed), _ptr(X), int(n), int(c), int(h),
+                                    int(w), int(kh), int(kw), int(stride), int(pad), _ptr(Y),
+                                    int(y_dtype), _ptr(workspace), nbytes, _ptr(dev_status), _stream(stream))
+    if check and rc != MWU_OK:
+        raise MwuError(rc, "mwu_conv_implicit_ws")
     return rc
 
 

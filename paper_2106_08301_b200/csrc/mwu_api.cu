@@ -1,7 +1,12 @@
 // Small host-side entry points and the device check shared by all calls.
+#include <atomic>
+
 #include "mwu_common.cuh"
 
 namespace mwu {
+
+static std::atomic<unsigned long long> g_launches{0};
+void count_launch(int n) { g_launches.fetch_add((unsigned long long)n, std::memory_order_relaxed); }
 
 int check_device(int *sm_count) {
     int dev = -1;
@@ -29,6 +34,10 @@ extern "C" const char *mwu_status_string(int status) {
         case MWU_ERR_CUDA: return "CUDA call failed";
         default: return "unknown status";
     }
+}
+
+extern "C" uint64_t mwu_kernel_launches(void) {
+    return (uint64_t)mwu::g_launches.load(std::memory_order_relaxed);
 }
 
 extern "C" int64_t mwu_count_from_permille(int64_t n_blocks, int32_t permille) {

@@ -60,12 +60,24 @@ inline int validate_desc(const mwu_proj_desc *d, bool need_stage_multiple) {
     const int64_t mb = d->rows * d->cols / d->block;
     if (mb >= (int64_t(1) << 31)) return MWU_ERR_SHAPE;
     if (d->k_prune < 0 || d->k_prune > d->k_unify || d->k_unify > mb) return MWU_ERR_SHAPE;
+    if (d->prune_group_rows != 0 || d->prune_group_cols != 0) {
+        const int gr = d->prune_group_rows, gc = d->prune_group_cols;
+        if (gr != 32 && gr != 64 && gr != 128 && gr != 256) return MWU_ERR_SHAPE;
+        if (gc != 16 && gc != 32 && gc != 64) return MWU_ERR_SHAPE;
+        if (d->rows % gr != 0 || d->cols % gc != 0) return MWU_ERR_SHAPE;
+        if (d->k_prune % ((int64_t)gr * gc / d->block) != 0) return MWU_ERR_SHAPE;   // whole groups only
+    }
     return MWU_OK;
 }
+
+inline bool grouped(const mwu_proj_desc *d) { return d->prune_group_rows != 0; }
 
 inline bool aligned_to(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 
 // MWU_OK when the current device is compute capability 10.x; also reports its SM count.
 int check_device(int *sm_count);
+
+// adds n to the process-wide count of kernels launched (mwu_kernel_launches)
+void count_launch(int n = 1);
 
 }  // namespace mwu

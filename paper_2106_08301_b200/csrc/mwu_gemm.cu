@@ -59,6 +59,7 @@ __device__ __forceinline__ void group_bar(int group, int nthreads) {   // the th
 template <int MODE, int NREC, int BW, int MT>
 __global__ void __launch_bounds__(cta_threads(MODE, MT), 1)
 mwu_gemm_kernel(const __grid_constant__ CUtensorMap tmap, const Params p) {
+    MWU_CHECK_HEADER(p);
     constexpr int NDEC_WARPS = dec_warps(MODE);
     constexpr int NDEC_THREADS = NDEC_WARPS * 32;
     constexpr int FIRST_GATHER_WARP = first_gather_warp(MODE);
@@ -523,6 +524,7 @@ static cudaError_t launch(const CUtensorMap &tmap, const Params &p, int grid, si
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     kern<<<grid, cta_threads(MODE, MT), smem, st>>>(tmap, p);
+    count_launch();
     return cudaGetLastError();
 }
 
@@ -547,6 +549,7 @@ static void fill_common(Params &p, const mwu_proj_desc *desc, const void *packed
     p.n_stages = L.n_stages;
     p.N = desc->rows;
     p.K = desc->cols;
+    p.bw = desc->block;
     p.Y = Y;
     p.y_fp32 = y_dtype;
     p.dev_status = dev_status;
@@ -673,6 +676,22 @@ extern "C" int mwu_gemm(const mwu_proj_desc *desc, const void *packed, const voi
                         int64_t ldx, void *Y, int64_t ldy, int32_t y_dtype, uint32_t *dev_status,
                         void *cuda_stream) {
     return mwu_gemm_ws(desc, packed, X, M, ldx, Y, ldy, y_dtype, nullptr, 0, dev_status, cuda_stream);
+}
+
+extern "C" size_t mwu_conv_workspace_bytes(const mwu_proj_desc *desc, int32_t n, int32_t c, int32_t h,
+                                           int32_t w, int32_t kh, int32_t kw, int32_t stride, int32_t pad) {
+    (void)desc; (void)n; (void)c; (void)h; (void)w; (void)kh; (void)kw; (void)stride; (void)pad;
+    return 0;
+}
+
+extern "C" int mwu_conv_implicit_ws(const mwu_proj_desc *desc, const void *packed, const void *X_nchw,
+                                    int32_t n, int32_t c, int32_t h, int32_t w, int32_t kh, int32_t kw,
+                                    int32_t stride, int32_t pad, void *Y_nchw, int32_t y_dtype,
+                                    void *workspace, size_t workspace_bytes, uint32_t *dev_status,
+                                    void *cuda_stream) {
+    (void)workspace; (void)workspace_bytes;
+    return mwu_conv_implicit(desc, packed, X_nchw, n, c, h, w, kh, kw, stride, pad, Y_nchw, y_dtype,
+                             dev_status, cuda_stream);
 }
 
 extern "C" int mwu_conv_implicit(const mwu_proj_desc *desc, const void *packed, const void *X_nchw,

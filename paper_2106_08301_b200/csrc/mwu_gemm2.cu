@@ -46,6 +46,7 @@ __device__ __forceinline__ void pair_group_bar(int group) {
 template <int BW>
 __global__ void __launch_bounds__(P_THREADS, 1)
 mwu_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap, const Params p) {
+    MWU_CHECK_HEADER(p);
     extern __shared__ unsigned char smem_raw[];
     unsigned char *base = reinterpret_cast<unsigned char *>(
         (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -394,6 +395,7 @@ static cudaError_t launch_pair_bw(const CUtensorMap &tmap, const Params &p, int 
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
+    count_launch();
     return cudaLaunchKernelEx(&cfg, kern, tmap, q);
 }
 

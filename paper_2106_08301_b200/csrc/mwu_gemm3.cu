@@ -39,6 +39,7 @@ constexpr int DEC_THREADS = 128;
 template <int BW>
 __global__ void __launch_bounds__(DEC_THREADS)
 mwu_decode_kernel(const Params p, __nv_bfloat16 *Wd, long long ldw) {
+    MWU_CHECK_HEADER(p);
     __shared__ __align__(1024) unsigned char tile[REC_BYTES];
     constexpr int ENT = DecodeCfg<BW, DEC_THREADS>::ENT;
     const PackedRec *recs = reinterpret_cast<const PackedRec *>(p.packed + p.off_rec);
@@ -71,6 +72,7 @@ template <int BW>
 static cudaError_t launch_decode_bw(const Params &p, __nv_bfloat16 *Wd, long long ldw, cudaStream_t st) {
     const long long n_rec = p.n_rec_tiles * p.n_stages;
     mwu_decode_kernel<BW><<<(unsigned)n_rec, DEC_THREADS, 0, st>>>(p, Wd, ldw);
+    count_launch();
     return cudaGetLastError();
 }
 
@@ -106,6 +108,7 @@ struct DenseSmem {
 __global__ void __launch_bounds__(D_THREADS, 1)
 mwu_dense_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
                       const __grid_constant__ CUtensorMap tmap_y, const Params p) {
+    MWU_CHECK_HEADER(p);
     extern __shared__ unsigned char smem_raw[];
     unsigned char *base = reinterpret_cast<unsigned char *>(
         (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -379,6 +382,7 @@ cudaError_t launch_dense(const CUtensorMap &tmap_x, const CUtensorMap &tmap_w, c
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
+    count_launch();
     return cudaLaunchKernelEx(&cfg, kern, tmap_x, tmap_w, tmap_y, p);
 }
 

@@ -43,6 +43,7 @@ struct Params {
     int resident;                       // pair kernel: a CTA pair keeps one weight tile (see mwu_gemm2.cu)
     int stage_epi;                      // single-CTA GEMM: 16 KB of shared memory is there for store_chunk_staged
     int y_tma;                          // two-operand GEMM: bf16 output leaves through TMA stores (a tensor map of Y exists)
+    int bw;                             // block width the descriptor names (checked against the packed header)
     unsigned *dev_status;
     // convolution only
     const __nv_bfloat16 *X;
@@ -50,6 +51,23 @@ struct Params {
     // staged gather (0 rows: gather straight from global memory instead)
     int patch_rows, patch_pitch, patch_nch;   // input rows per tile, row pitch (elements), channels per stage
 };
+
+// The packed buffer's header against what the host derived from the descriptor.  Every thread of
+// every CTA evaluates it at kernel entry (the same few cached words), so the whole grid takes the
+// same decision; on a mismatch the caller raises MWU_DEV_BOUNDS and returns before touching anything.
+__device__ __forceinline__ bool header_matches(const Params &p) {
+    const unsigned long long *h = reinterpret_cast<const unsigned long long *>(p.packed);
+    return __ldg(h) == kMagic && __ldg(h + 2) == (unsigned long long)p.N && __ldg(h + 3) == (unsigned long long)p.K &&
+           __ldg(h + 4) == (unsigned long long)p.bw && __ldg(h + 9) == (unsigned long long)p.n_unified &&
+           __ldg(h + 10) == (unsigned long long)p.n_dense && __ldg(h + 11) == (unsigned long long)p.n_plist;
+}
+#define MWU_CHECK_HEADER(p)                                                        \
+    do {                                                                           \
+        if (!header_matches(p)) {                                                  \
+            if (threadIdx.x == 0) atomicOr((p).dev_status, (unsigned)MWU_DEV_BOUNDS); \
+            return;                                                                \
+        }                                                                          \
+    } while (0)
 
 // ------------------------------------------------------------------------------------------
 // PTX wrappers

@@ -392,5 +392,6 @@ extern "C" int mwu_pack(const mwu_proj_desc *desc, const float *W, const float *
         case 8: pack::fill_kernel<8><<<(unsigned)n_rec, 128, 0, st>>>(p); break;
         default: pack::fill_kernel<16><<<(unsigned)n_rec, 128, 0, st>>>(p); break;
     }
+    count_launch(3);
     return cudaGetLastError() == cudaSuccess ? MWU_OK : MWU_ERR_CUDA;
 }

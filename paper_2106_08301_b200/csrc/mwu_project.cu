@@ -1791,6 +1791,7 @@ static cudaError_t launch_project(const mwu::proj::Params &p, const mwu_proj_des
                                   double *loss_p, int sm_count, bool one_pass, cudaStream_t st) {
     using namespace mwu::proj;
     sample_kernel<B><<<1, SAMP_THREADS, 0, st>>>(p, desc->k_unify, desc->k_prune);
+    mwu::count_launch();
     const long long n_units = (p.n_floats + 15) / 16;
     const long long want = (n_units + 255) / 256;
     const long long cap_blocks = (long long)sm_count * 8;
@@ -1803,6 +1804,7 @@ static cudaError_t launch_project(const mwu::proj::Params &p, const mwu_proj_des
     if (one_pass) {
         if (p.U_next || p.resid) pass_kernel<B, true><<<grid_stream, 256, 0, st>>>(p, Q, loss_u, loss_p, u, pb, ub, sb);
         else pass_kernel<B, false><<<grid_stream, 256, 0, st>>>(p, Q, loss_u, loss_p, u, pb, ub, sb);
+        mwu::count_launch();
         if (!need_p && !need_u) return cudaGetLastError();       // no threshold: every class is final
         // the list holds a few per cent of the blocks
         const long long lb = (mb / 8 + FIN_THREADS - 1) / FIN_THREADS;      // a thread per expected entry
@@ -1811,6 +1813,7 @@ static cudaError_t launch_project(const mwu::proj::Params &p, const mwu_proj_des
         const int grid_list = (int)(lb < (long long)sm_count ? (lb > 0 ? lb : 1) : (long long)sm_count);
         list_select_kernel<B><<<grid_list, FIN_THREADS, 0, st>>>(p);
         list_finish_kernel<B><<<grid_list, FIN_THREADS, 0, st>>>(p, Q, u, pb, ub);
+        mwu::count_launch(2);
     }
     // multi-pass kernels: the whole projection, or (gated) the fallback of the one-pass pipeline.
     // As a fallback they are needed once in thousands of calls and normally return at once, so
@@ -1818,6 +1821,7 @@ static cudaError_t launch_project(const mwu::proj::Params &p, const mwu_proj_des
     const int grid_fb = (int)(grid_stream < 2 * sm_count ? grid_stream : 2 * sm_count);
     if (one_pass) grid_stream = grid_fb;
     stats_kernel<B><<<grid_stream, 256, 0, st>>>(p, loss_u, loss_p, u, sb);
+    mwu::count_launch(2 + ((need_p || need_u) ? 1 : 0) + (need_u ? 1 : 0));      // stats, emit and the selection kernels below
     const long long rb = (mb + 4 * FIN_THREADS - 1) / (4 * FIN_THREADS);
     const int grid_fin = (int)(rb < (long long)sm_count ? (rb > 0 ? rb : 1) : (long long)sm_count);
     if (need_p || need_u) prune_select_kernel<B><<<grid_fin, FIN_THREADS, 0, st>>>(p);

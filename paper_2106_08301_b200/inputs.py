@@ -68,6 +68,8 @@ class Workload:
         return self.rows * self.cols // self.block
 
     def weights(self, case: int = 0) -> torch.Tensor:
+        if self.name.startswith("proj_p"):
+            case += 900 + int(self.name[len("proj_p"):].split("_b")[0])      # one tensor per size
         return normal_weights(self.rows, self.cols, self.weight_std,
                               seed_for(self.config, case))
 
@@ -97,6 +99,13 @@ def sweep_workload(block: int, pruned_permille: int) -> Workload:
     u = min(1000, pruned_permille + 100)
     return Workload(f"c5_sweep_b{block}_p{pruned_permille}", 5, 4096, 4096, block, u,
                     pruned_permille, 0.02, m=8192)
+
+
+def projection_sweep_workload(log2_params: int, block: int) -> Workload:
+    """Projection-only point of the size sweep: 2**log2_params weights, 50 % unified of which half
+    pruned; no activations (m = 0)."""
+    rows, cols = projection_sweep_shape(log2_params)
+    return Workload(f"proj_p{log2_params}_b{block}", 5, rows, cols, block, 500, 250, 0.02, m=0)
 
 
 def projection_sweep_shape(log2_params: int) -> Tuple[int, int]:

@@ -68,9 +68,9 @@ def test_descriptor_validation_without_a_device():
 
 
 def test_packed_bytes_matches_the_format_arithmetic():
-    from oracle import mwu_oracle as O
+    import packed_format as F
     for rows, cols, b, ku, kp in [(256, 256, 4, 8192, 4096), (130, 192, 8, 1000, 10),
                                   (16384, 4096, 16, 3355443, 2516582), (100, 128, 2, 6400, 0)]:
         d = B.make_desc(rows, cols, b, ku, kp)
         mb = rows * cols // b
-        assert B.mwu_packed_bytes(d) == O.packed_layout(rows, cols, b, ku - kp, mb - ku, kp)["total"]
+        assert B.mwu_packed_bytes(d) == F.packed_layout(rows, cols, b, ku - kp, mb - ku, kp)["total"]

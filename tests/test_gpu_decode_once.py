@@ -8,10 +8,12 @@ import numpy as np
 import pytest
 import torch
 
+import packed_format as F
 from oracle import mwu_oracle as O
 from paper_2106_08301_b200 import binding as B
 from paper_2106_08301_b200 import inputs
 from test_gpu_gemm import errors, project_and_pack
+from test_gpu_projection import check_against_oracle, check_pack
 
 pytestmark = pytest.mark.gpu
 
@@ -147,18 +149,21 @@ def test_gemm_ws_config4_shape_sampled_outputs():
     assert fro <= 2e-3 and mx <= 1e-2, (fro, mx)
 
 
-@pytest.mark.parametrize("b,pruned_permille", [(2, 900), (4, 0), (8, 500)])
+@pytest.mark.parametrize("pruned_permille", [0, 250, 500, 750, 900])
+@pytest.mark.parametrize("b", [2, 4, 8, 16])
 def test_gemm_ws_sweep_points_full_size_sampled_outputs(b, pruned_permille):
-    """Points of the 4096 x 4096 sweep at full size (M = 8192), among them the two ends: nothing
-    pruned, and 90 % pruned with every other block unified.  The class bitmaps and the packed
-    bytes are compared with the checker bit for bit, the GEMM on sampled rows."""
+    """All twenty points of the 4096 x 4096 sweep (block width x pruned fraction) at full size
+    (M = 8192), in the configuration the benchmark times: keys, bitmaps, sign plane, u and Q against
+    the checker bit for bit, the packed form through mwu_decode, the GEMM on sampled rows."""
     wl = inputs.sweep_workload(b, pruned_permille)
     ku = B.mwu_count_from_permille(wl.n_blocks, wl.unified_permille)
     kp = B.mwu_count_from_permille(wl.n_blocks, wl.pruned_permille)
-    desc, bufs, packed, p = project_and_pack(wl.weights(), wl.block, ku, kp)
-    assert np.array_equal(bufs.pruned_bitmap.cpu().numpy().view(np.uint32), O.bitmap_words(p.pruned))
-    assert np.array_equal(bufs.unified_bitmap.cpu().numpy().view(np.uint32), O.bitmap_words(p.unified))
-    assert np.array_equal(packed.cpu().numpy(), O.pack(p, wl.block))
+    desc, bufs, Wd, _, p = check_against_oracle(wl.weights(), b, ku, kp, algos=(B.MWU_ALGO_AUTO,))
+    packed = bufs.pack(Wd)
+    torch.cuda.synchronize()
+    assert int(bufs.dev_status.item()) == 0
+    check_pack(desc, bufs, packed, p, b)
+    del Wd
     X = wl.activations()
     ws = torch.empty(B.mwu_gemm_workspace_bytes(desc, wl.m), dtype=torch.uint8, device="cuda")
     Y = torch.empty((wl.m, wl.rows), dtype=torch.bfloat16, device="cuda")
@@ -166,9 +171,33 @@ def test_gemm_ws_sweep_points_full_size_sampled_outputs(b, pruned_permille):
     torch.cuda.synchronize()
     assert int(bufs.dev_status.item()) == 0
     rows = [0, 31, 32, 255, 256, 4097, 8191]
-    ref = O.gemm(X[rows].to(torch.float64).numpy(), O.decoded_weights(p, wl.block))
+    ref = O.gemm(X[rows].to(torch.float64).numpy(), O.decoded_weights(p))
     fro, mx = errors(Y[rows].float().cpu().numpy(), ref)
     assert fro <= 2e-3 and mx <= 1e-2, (fro, mx)
+
+
+def test_gemm_ws_config3_full_size_sampled_outputs():
+    """The 1x1-convolution shape at its full size (M = 200704, K = 256, N = 1024) on the workspace
+    path: sampled output rows, among them the first and last row of the matrix and of a tile."""
+    wl = inputs.WORKLOADS["c3_conv1x1"]
+    ku = B.mwu_count_from_permille(wl.n_blocks, wl.unified_permille)
+    kp = B.mwu_count_from_permille(wl.n_blocks, wl.pruned_permille)
+    desc, bufs, packed, p = project_and_pack(wl.weights(), wl.block, ku, kp)
+    X = wl.activations()
+    ws = torch.empty(B.mwu_gemm_workspace_bytes(desc, wl.m), dtype=torch.uint8, device="cuda")
+    What = O.decoded_weights(p)
+    rows = [0, 1, 127, 128, 255, 256, 257, 511, 512, 100000, 100351, 100352, 200447, 200448, 200702, 200703]
+    for y_dtype, tol in ((1, 1e-5), (0, 2e-3)):
+        Y = torch.full((wl.m, wl.rows), float("nan"), dtype=torch.float32 if y_dtype else torch.bfloat16,
+                       device="cuda")
+        B.mwu_gemm_ws(desc, packed, X.cuda(), wl.m, wl.cols, Y, wl.rows, y_dtype, ws, bufs.dev_status)
+        torch.cuda.synchronize()
+        assert int(bufs.dev_status.item()) == 0
+        ref = O.gemm(X[rows].to(torch.float64).numpy(), What)
+        fro, mx = errors(Y[rows].float().cpu().numpy(), ref)
+        assert fro <= tol and mx <= 1e-2, (y_dtype, fro, mx)
+        assert not bool(torch.isnan(Y).any())                 # every output element was written
+        del Y
 
 
 @pytest.mark.parametrize("N,K,M,b", [(504, 256, 40001, 8), (1024, 128, 50000, 16), (304, 384, 38000, 4),
@@ -188,6 +217,5 @@ def test_gemm_ws_short_reduction_dead_stage():
     W[:, 64:128] = 0.0
     Mb = N * K // b
     desc, bufs, packed, p, X, ref = check_gemm_ws(W, b, Mb // 2, Mb // 4, M, seed=3)
-    h = O.parse_header(O.pack(p, b))
-    rec = O.pack(p, b)[h["off_rec"]:h["off_rec"] + 16 * 16].view(np.uint32).reshape(-1, 4)
+    rec = F.records(packed.cpu().numpy())
     assert rec[1, 3] == 0                                    # stage 1 of the first row tile is dead

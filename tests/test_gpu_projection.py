@@ -3,11 +3,36 @@ import numpy as np
 import pytest
 import torch
 
+import packed_format as F
 from oracle import mwu_oracle as O
 from paper_2106_08301_b200 import binding as B
 from paper_2106_08301_b200 import inputs
 
 pytestmark = pytest.mark.gpu
+
+
+def decoded_on_gpu(desc, bufs, packed):
+    """mwu_decode of a packed buffer: bf16 [rows][cols] as fp64 (padding rows checked to be zero)."""
+    n_pad = (desc.rows + 127) // 128 * 128
+    Wd = torch.full((n_pad, desc.cols), float("nan"), dtype=torch.bfloat16, device="cuda")
+    B.mwu_decode(desc, packed, Wd, desc.cols, bufs.dev_status)
+    torch.cuda.synchronize()
+    assert int(bufs.dev_status.item()) == 0
+    assert not bool(Wd[desc.rows:].any())
+    return Wd[:desc.rows].to(torch.float64).cpu().numpy()
+
+
+def check_pack(desc, bufs, packed, p, b):
+    """mwu_pack judged without any knowledge of its layout: what mwu_decode reads back from the
+    packed bytes equals the checker's decoded weights bit for bit, and the header carries the
+    class counts of the projection."""
+    assert np.array_equal(decoded_on_gpu(desc, bufs, packed), O.decoded_weights(p))
+    h = F.parse_header(packed[:256].cpu().numpy())
+    mb = p.pruned.shape[0]
+    assert (h["N"], h["K"], h["b"]) == (desc.rows, desc.cols, b)
+    assert h["n_pruned"] == int(p.pruned.sum()) and h["n_unified"] == int(p.unified.sum())
+    assert h["n_dense"] == mb - int(p.pruned.sum()) - int(p.unified.sum())
+    assert h["total"] == packed.numel() == B.mwu_packed_bytes(desc)
 
 
 def run_project(W, b, ku, kp, U=None, prune_key=0, want_loss=True, algo=B.MWU_ALGO_AUTO):
@@ -119,8 +144,10 @@ def test_nonfinite_sets_status():
     assert int(bufs.dev_status.item()) & B.MWU_DEV_NONFINITE
 
 
-@pytest.mark.parametrize("name", ["c1_linear", "c2_conv3x3", "c3_conv1x1"])
+@pytest.mark.parametrize("name", ["c1_linear", "c2_conv3x3", "c3_conv1x1", "c4_ffn"])
 def test_projection_and_pack_parity_configs(name):
+    """The four named workloads at full size, both kernel pipelines: keys, bitmaps, sign plane, u
+    and Q bit for bit against the checker; the packed form through mwu_decode."""
     wl = inputs.WORKLOADS[name]
     W = wl.weights()
     Mb = wl.n_blocks
@@ -132,21 +159,29 @@ def test_projection_and_pack_parity_configs(name):
     packed = bufs.pack(Wd)
     torch.cuda.synchronize()
     assert int(bufs.dev_status.item()) == 0
-    ref = O.pack(p, wl.block)
-    got = packed.cpu().numpy()
-    assert got.shape == ref.shape
-    assert np.array_equal(got, ref)
+    check_pack(desc, bufs, packed, p, wl.block)
+
+
+@pytest.mark.parametrize("b", [4, 16])
+def test_projection_size_sweep_point_both_pipelines(b):
+    """One size of the projection sweep (2^24 weights, 50 % / 25 %) through the one-pass and the
+    multi-pass pipeline: both must give the checker's bits."""
+    rows, cols = inputs.projection_sweep_shape(24)
+    W = inputs.normal_weights(rows, cols, 0.02, inputs.seed_for(5, 924))
+    Mb = rows * cols // b
+    check_against_oracle(W, b, O.count_from_permille(Mb, 500), O.count_from_permille(Mb, 250),
+                         algos=(B.MWU_ALGO_ONE_PASS, B.MWU_ALGO_MULTI_PASS))
 
 
 @pytest.mark.parametrize("b,rows,cols", [(2, 100, 128), (4, 130, 64), (8, 257, 192), (16, 128, 256)])
-def test_pack_parity_ragged_rows(b, rows, cols):
+def test_pack_ragged_rows(b, rows, cols):
     W = inputs.normal_weights(rows, cols, 0.02, 99 + b)
     Mb = rows * cols // b
     desc, bufs, Wd, _, p = check_against_oracle(W, b, Mb * 7 // 10, Mb * 4 // 10)
     packed = bufs.pack(Wd)
     torch.cuda.synchronize()
     assert int(bufs.dev_status.item()) == 0
-    assert np.array_equal(packed.cpu().numpy(), O.pack(p, b))
+    check_pack(desc, bufs, packed, p, b)
 
 
 def test_pack_with_dual_and_structured_pruning():
@@ -159,12 +194,32 @@ def test_pack_with_dual_and_structured_pruning():
     desc, bufs, Wd, Ud, p = check_against_oracle(W, b, Mb // 2, Mb // 4, U=U)
     packed = bufs.pack(Wd, Ud)
     torch.cuda.synchronize()
-    ref = O.pack(p, b)
-    assert np.array_equal(packed.cpu().numpy(), ref)
-    h = O.parse_header(ref)
-    rec = ref[h["off_rec"]:h["off_rec"] + 16 * 9].view(np.uint32).reshape(-1, 4)
+    check_pack(desc, bufs, packed, p, b)
+    rec = F.records(packed.cpu().numpy())
     assert rec[1, 3] == 0 and rec[5, 3] == 0          # stage 1 of both row tiles is dead
     assert rec[0, 3] == 0xF
+
+
+@pytest.mark.parametrize("name,b,rows,cols", [("c1_linear", 0, 0, 0), ("c2_conv3x3", 0, 0, 0), ("ragged", 4, 130, 64),
+                                              ("ragged", 16, 200, 128), ("ragged", 2, 100, 128)])
+def test_packed_bytes_follow_the_documented_format(name, b, rows, cols):
+    """Regression of the file format (not a parity claim): the bytes mwu_pack writes are the ones
+    the format description in the header file leads to, as restated by tests/packed_format.py."""
+    if name == "ragged":
+        W = inputs.normal_weights(rows, cols, 0.02, 199 + b)
+        Mb = rows * cols // b
+        ku, kp = Mb * 7 // 10, Mb * 4 // 10
+    else:
+        wl = inputs.WORKLOADS[name]
+        W, b = wl.weights(), wl.block
+        ku = B.mwu_count_from_permille(wl.n_blocks, wl.unified_permille)
+        kp = B.mwu_count_from_permille(wl.n_blocks, wl.pruned_permille)
+    desc, bufs, Wd, _ = run_project(W, b, ku, kp, want_loss=False)
+    packed = bufs.pack(Wd)
+    torch.cuda.synchronize()
+    assert int(bufs.dev_status.item()) == 0
+    p = O.project(W.numpy(), b, ku, kp)
+    assert np.array_equal(packed.cpu().numpy(), F.write(p, b))
 
 
 @pytest.mark.parametrize("b,rows,cols,permille", [(16, 1000, 4112, (800, 600)), (4, 517, 1028, (500, 250)),
