@@ -308,6 +308,49 @@ int mwu_conv_implicit_ws(const mwu_proj_desc *desc, const void *packed, const vo
                          void *workspace, size_t workspace_bytes, uint32_t *dev_status,
                          void *cuda_stream);
 
+/*
+ * mwu_keep_n_of_m -- the in-block pruning of Section 4.7 (the pruning half of the paper's
+ * combination test: 1x4 blocks with half of every block pruned, the pattern sparse tensor cores
+ * accept).  Of every m = 4 consecutive entries of a row of v = W, or fp32(W + U_dual), the n with
+ * the largest magnitude are kept (equal magnitudes: the lower index) and the others become +0:
+ * the Euclidean projection (Eq. 7) onto "at most n non-zeros in every group of m".
+ *
+ *   W, U_dual   in   fp32 [rows*cols], cols % 4 == 0; U_dual may be NULL
+ *   Q           out  fp32 [rows*cols]; may be NULL
+ *   keep_bits   out  uint32 [ceil(rows*cols/32)], bit (f%32) of word (f/32) set when weight f is kept
+ *   Wd          out  bf16 [rows][ldw], ldw >= cols, ldw % 8 == 0; may be NULL: Q rounded to bf16, the
+ *                    weight matrix mwu_gemm_dense multiplies with
+ * Only m == 4 is built (n = 0..4): MWU_ERR_SHAPE otherwise.  A non-finite input sets
+ * MWU_DEV_NONFINITE.
+ */
+int mwu_keep_n_of_m(int64_t rows, int64_t cols, int32_t n, int32_t m, const float *W,
+                    const float *U_dual, float *Q, uint32_t *keep_bits, void *Wd, int64_t ldw,
+                    uint32_t *dev_status, void *cuda_stream);
+
+/*
+ * mwu_gemm_dense -- Y = X . Wd^T for a plain bf16 weight matrix Wd[rows][ldw] (Section 3.2's layer
+ * forward for weights that carry no block classes, e.g. the output of mwu_keep_n_of_m or of
+ * mwu_decode): the two-operand tensor-core kernel behind mwu_gemm_ws, bf16 x bf16 accumulated in
+ * fp32.  X, Y, M, ldx, ldy, y_dtype as mwu_gemm; ldw >= cols, ldw % 8 == 0.  The kept / dropped
+ * pattern of mwu_keep_n_of_m saves storage only: every product is executed.
+ */
+int mwu_gemm_dense(int64_t rows, int64_t cols, const void *Wd, int64_t ldw, const void *X, int64_t M,
+                   int64_t ldx, void *Y, int64_t ldy, int32_t y_dtype, uint32_t *dev_status,
+                   void *cuda_stream);
+
+/*
+ * mwu_debug_conv_wait -- testing aid for the bounded waits inside the kernels (the paper has no
+ * counterpart).  Every wait of a kernel on one of its own barriers has a limit, after which the
+ * kernel sets MWU_DEV_TIMEOUT in *dev_status, lets the copies it has in flight land, releases its
+ * tensor memory and returns, leaving the context usable.  This call makes that path observable on
+ * the tensor-core kernel of mwu_conv_implicit_ws: `limit_cycles` replaces the limit (about two
+ * seconds by default; <= 0 restores it) and `withhold_stage` names the running number of one
+ * pipeline stage whose loads the producer leaves out in every CTA, so that the consumer's wait for
+ * it must run out (-1: none).  Process-wide host setting, read when mwu_conv_implicit_ws is called;
+ * not meant for production code.
+ */
+void mwu_debug_conv_wait(int64_t limit_cycles, int64_t withhold_stage);
+
 #ifdef __cplusplus
 }
 #endif

@@ -18,7 +18,8 @@ LIB_PATH = os.path.join(_HERE, "libmwu.so")
 EXPORTS = ["mwu_status_string", "mwu_kernel_launches", "mwu_count_from_permille",
            "mwu_project_workspace_bytes", "mwu_project", "mwu_admm_step", "mwu_project_static",
            "mwu_packed_bytes", "mwu_pack", "mwu_gemm", "mwu_decode", "mwu_gemm_workspace_bytes",
-           "mwu_gemm_ws", "mwu_conv_implicit", "mwu_conv_workspace_bytes", "mwu_conv_implicit_ws"]
+           "mwu_gemm_ws", "mwu_conv_implicit", "mwu_conv_workspace_bytes", "mwu_conv_implicit_ws",
+           "mwu_debug_conv_wait", "mwu_keep_n_of_m", "mwu_gemm_dense"]
 MWU_STATIC_MAX_BLOCKS = 1048576
 
 MWU_OK = 0
@@ -86,6 +87,12 @@ def lib() -> ctypes.CDLL:
         L.mwu_conv_workspace_bytes.argtypes = [dp] + [i32] * 8
         L.mwu_conv_implicit_ws.restype = ctypes.c_int
         L.mwu_conv_implicit_ws.argtypes = [dp, vp, vp] + [i32] * 8 + [vp, i32, vp, sz, vp, vp]
+        L.mwu_keep_n_of_m.restype = ctypes.c_int
+        L.mwu_keep_n_of_m.argtypes = [i64, i64, i32, i32, vp, vp, vp, vp, vp, i64, vp, vp]
+        L.mwu_gemm_dense.restype = ctypes.c_int
+        L.mwu_gemm_dense.argtypes = [i64, i64, vp, i64, vp, i64, i64, vp, i64, i32, vp, vp]
+        L.mwu_debug_conv_wait.restype = None
+        L.mwu_debug_conv_wait.argtypes = [i64, i64]
         _lib = L
     return _lib
 
@@ -215,6 +222,26 @@ def mwu_conv_implicit(desc, packed, X, n, c, h, w, kh, kw, stride, pad, Y, y_dty
     if check and rc != MWU_OK:
         raise MwuError(rc, "mwu_conv_implicit")
     return rc
+
+
+def mwu_keep_n_of_m(rows, cols, n, m, W, U_dual, Q, keep_bits, Wd, ldw, dev_status, stream=None, check=True) -> int:
+    rc = lib().mwu_keep_n_of_m(int(rows), int(cols), int(n), int(m), _ptr(W), _ptr(U_dual), _ptr(Q),
+                               _ptr(keep_bits), _ptr(Wd), int(ldw), _ptr(dev_status), _stream(stream))
+    if check and rc != MWU_OK:
+        raise MwuError(rc, "mwu_keep_n_of_m")
+    return rc
+
+
+def mwu_gemm_dense(rows, cols, Wd, ldw, X, M, ldx, Y, ldy, y_dtype, dev_status, stream=None, check=True) -> int:
+    rc = lib().mwu_gemm_dense(int(rows), int(cols), _ptr(Wd), int(ldw), _ptr(X), int(M), int(ldx), _ptr(Y),
+                              int(ldy), int(y_dtype), _ptr(dev_status), _stream(stream))
+    if check and rc != MWU_OK:
+        raise MwuError(rc, "mwu_gemm_dense")
+    return rc
+
+
+def mwu_debug_conv_wait(limit_cycles: int, withhold_stage: int) -> None:
+    lib().mwu_debug_conv_wait(int(limit_cycles), int(withhold_stage))
 
 
 def mwu_conv_workspace_bytes(desc, n, c, h, w, kh, kw, stride, pad) -> int:

@@ -494,12 +494,7 @@ mwu_gemm_kernel(const __grid_constant__ CUtensorMap tmap, const Params p) {
 // ------------------------------------------------------------------------------------------
 // host
 // ------------------------------------------------------------------------------------------
-typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
-                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *,
-                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
-                                  CUtensorMapFloatOOBfill);
-
-static EncodeTiledFn get_encode_fn() {
+EncodeTiledFn get_encode_fn() {
     static EncodeTiledFn fn = nullptr;
     if (!fn) {
         void *ptr = nullptr;
@@ -676,22 +671,6 @@ extern "C" int mwu_gemm(const mwu_proj_desc *desc, const void *packed, const voi
                         int64_t ldx, void *Y, int64_t ldy, int32_t y_dtype, uint32_t *dev_status,
                         void *cuda_stream) {
     return mwu_gemm_ws(desc, packed, X, M, ldx, Y, ldy, y_dtype, nullptr, 0, dev_status, cuda_stream);
-}
-
-extern "C" size_t mwu_conv_workspace_bytes(const mwu_proj_desc *desc, int32_t n, int32_t c, int32_t h,
-                                           int32_t w, int32_t kh, int32_t kw, int32_t stride, int32_t pad) {
-    (void)desc; (void)n; (void)c; (void)h; (void)w; (void)kh; (void)kw; (void)stride; (void)pad;
-    return 0;
-}
-
-extern "C" int mwu_conv_implicit_ws(const mwu_proj_desc *desc, const void *packed, const void *X_nchw,
-                                    int32_t n, int32_t c, int32_t h, int32_t w, int32_t kh, int32_t kw,
-                                    int32_t stride, int32_t pad, void *Y_nchw, int32_t y_dtype,
-                                    void *workspace, size_t workspace_bytes, uint32_t *dev_status,
-                                    void *cuda_stream) {
-    (void)workspace; (void)workspace_bytes;
-    return mwu_conv_implicit(desc, packed, X_nchw, n, c, h, w, kh, kw, stride, pad, Y_nchw, y_dtype,
-                             dev_status, cuda_stream);
 }
 
 extern "C" int mwu_conv_implicit(const mwu_proj_desc *desc, const void *packed, const void *X_nchw,

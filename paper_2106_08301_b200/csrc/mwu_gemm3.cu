@@ -108,7 +108,7 @@ struct DenseSmem {
 __global__ void __launch_bounds__(D_THREADS, 1)
 mwu_dense_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
                       const __grid_constant__ CUtensorMap tmap_y, const Params p) {
-    MWU_CHECK_HEADER(p);
+    if (!p.all_live) MWU_CHECK_HEADER(p);
     extern __shared__ unsigned char smem_raw[];
     unsigned char *base = reinterpret_cast<unsigned char *>(
         (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -162,6 +162,7 @@ mwu_dense_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
 
     // live mask of stage ks for tile column nt: OR over its (one or two) 128-row records
     auto live_of = [&](long long nt, int ks) -> unsigned {
+        if (p.all_live) return 0xFu;
         unsigned l = __ldg(&recs[(nt * 2) * n_stages + ks].live);
         if (nt * 2 + 1 < p.n_rec_tiles) l |= __ldg(&recs[(nt * 2 + 1) * n_stages + ks].live);
         return l;

@@ -30,6 +30,12 @@ __host__ __device__ constexpr int cta_threads(int mode, int mt) {
 constexpr int MAX_STAGES_K = 256;       // cols <= 16384
 constexpr long long WAIT_LIMIT_CYCLES = 4000000000ll;   // about two seconds
 
+// cuTensorMapEncodeTiled, looked up through the runtime (no link against the driver library)
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
 struct Params {
     const unsigned char *packed;
     size_t off_rec, off_ulist, off_dpos, off_dpay, off_ppos;
@@ -44,6 +50,7 @@ struct Params {
     int stage_epi;                      // single-CTA GEMM: 16 KB of shared memory is there for store_chunk_staged
     int y_tma;                          // two-operand GEMM: bf16 output leaves through TMA stores (a tensor map of Y exists)
     int bw;                             // block width the descriptor names (checked against the packed header)
+    int all_live;                       // two-operand GEMM on a plain dense matrix: no packed record table to consult
     unsigned *dev_status;
     // convolution only
     const __nv_bfloat16 *X;

@@ -82,11 +82,14 @@ struct Work {
     unsigned cand_count[2];
     unsigned ticket[4];         // [1]: prune_select, [3]: collect<1>
     // one-pass pipeline
-    unsigned fcand_count[2];    // threshold-bin candidates of list_select / list_collect
+    unsigned fcand_count[2];    // threshold-bin candidates of the two halves of resolve_kernel
     unsigned fticket[2];
     unsigned list_count;        // entries appended to the candidate list
-    unsigned failed;            // != 0: the one-pass result is void, the multi-pass kernels run
+    unsigned failed;            // != 0: the one-pass result is void, the multi-pass kernel runs
     u64 That[2];                // provisional thresholds (key bit patterns)
+    unsigned release;           // resolve_kernel: the prune threshold and the unify bin are published
+    unsigned bar;               // multipass_kernel: arrivals at its grid barriers (only ever grows)
+    unsigned pad1[2];
 };
 
 struct Params {
@@ -102,7 +105,14 @@ struct Params {
     unsigned *fhist;            // [2][nb]: prune, unify (one-pass kernels)
     uint2 *list;                // [list_cap] candidate list: (block index, bin codes)
     unsigned list_cap;
-    int gated;                  // multi-pass kernels return at once unless work->failed is set
+    int gated;                  // the multi-pass kernel returns at once unless work->failed is set
+    int run_sample;             // the multi-pass kernel also chooses the windows (no sample_kernel before it)
+    // grouped pruning: the prune class of a block is the bit of its group (nullptr: pruning by key)
+    const unsigned *gprune;     // [ceil(n_groups / 32)]
+    unsigned group_rows, group_cols;     // extent of a prune group in rows and columns of W
+    unsigned blocks_per_row;    // cols / b
+    unsigned groups_per_row;    // cols / group_cols
+    long long k_unify, k_prune;
     float *U_next;              // dual update V - Q (mwu_admm_step), else null
     double *resid;              // ||V - Q||_F^2 accumulator (mwu_admm_step), else null
     u64 *cand_key;              // [CAP]
@@ -124,6 +134,48 @@ template <typename T>
 __device__ __forceinline__ T ld_vol(const T *p) { return *reinterpret_cast<const volatile T *>(p); }
 
 __device__ __forceinline__ u64 key_bits(double x) { return (u64)__double_as_longlong(x); }
+
+// Fresh copy of the selection state in shared memory, made by the whole CTA.  Inside a kernel that
+// spans several phases (grid barriers between them) plain loads of words another CTA has written
+// may be served from a stale L1 line, so every phase reads its own copy, taken with volatile loads.
+__device__ __forceinline__ void load_work(const Work *g, Work *s) {
+    __syncthreads();
+    const volatile unsigned *src = reinterpret_cast<const volatile unsigned *>(g);
+    unsigned *dst = reinterpret_cast<unsigned *>(s);
+    for (unsigned i = threadIdx.x; i < sizeof(Work) / 4; i += blockDim.x) dst[i] = src[i];
+    __syncthreads();
+}
+
+// grouped pruning: is block j inside a pruned group?
+__device__ __forceinline__ bool group_pruned(const Params &p, unsigned j) {
+    const unsigned row = j / p.blocks_per_row, kb = j - row * p.blocks_per_row;
+    const unsigned g = (row / p.group_rows) * p.groups_per_row + (kb * (unsigned)p.b) / p.group_cols;
+    return (__ldg(p.gprune + (g >> 5)) >> (g & 31u)) & 1u;
+}
+
+// Barrier over all CTAs of a cooperative launch (all resident at once).  `counter` only grows:
+// the k-th barrier of a kernel is passed when it reaches k * gridDim.x.  The wait is bounded: when
+// it runs out the caller raises MWU_DEV_TIMEOUT and leaves.
+constexpr long long GRID_WAIT_CYCLES = 4000000000ll;          // about two seconds
+__device__ __forceinline__ bool grid_sync(unsigned *counter, unsigned k) {
+    __shared__ int s_grid_ok;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        __threadfence();
+        atomicAdd(counter, 1u);
+        const unsigned target = k * gridDim.x;
+        int ok = 1;
+        const long long t0 = clock64();
+        unsigned spins = 0;
+        while (ld_vol(counter) < target) {
+            if ((++spins & 63u) == 0u && clock64() - t0 > GRID_WAIT_CYCLES) { ok = 0; break; }
+        }
+        __threadfence();
+        s_grid_ok = ok;
+    }
+    __syncthreads();
+    return s_grid_ok != 0;
+}
 
 // ---------------------------------------------------------------------------------------------
 // fp64 statistics of one block held in registers (fixed pairwise tree, every op rounded alone)
@@ -431,40 +483,59 @@ __device__ __forceinline__ long long sample_block(int i, long long mb, int ns) {
     return ns == NSAMP ? (long long)(((u64)i * (u64)mb) / (u64)NSAMP) : (long long)i;
 }
 
+// Run by one whole CTA of SAMP_THREADS threads: windows and provisional thresholds of the two
+// selections, written into p.work.
 template <int B>
-__global__ void __launch_bounds__(SAMP_THREADS) sample_kernel(Params p, long long k_unify, long long k_prune) {
+__device__ void sample_body(const Params &p) {
+    const long long k_unify = p.k_unify, k_prune = p.k_prune;
     const long long mb = p.n_blocks;
+    const bool by_group = p.gprune != nullptr;
     const int ns = (int)(mb < (long long)NSAMP ? mb : (long long)NSAMP);
     u64 kp[SAMP_PER], ku[SAMP_PER];
-    bool valid[SAMP_PER];
+    bool valid[SAMP_PER], in_group[SAMP_PER];
 #pragma unroll
     for (int t = 0; t < SAMP_PER; ++t) {
         const int i = threadIdx.x * SAMP_PER + t;
         kp[t] = ~0ull;
         ku[t] = ~0ull;
         valid[t] = i < ns;
+        in_group[t] = false;
         if (i < ns) {
             const long long j = sample_block(i, mb, ns);
             double S, Lu, Kp;
             block_keys_at<B>(p.W, p.U, j, p.use_l1, &S, &Lu, &Kp);
             kp[t] = key_bits(Kp);
             ku[t] = key_bits(Lu);
+            if (by_group) in_group[t] = group_pruned(p, (unsigned)j);
         }
     }
     Sel *sp = &p.work->sel[0];
     Sel *su = &p.work->sel[1];
     const long long ksel_u = k_unify - k_prune;
-    u64 lo, hi, That;
-    sample_select(kp, valid, (float)((double)k_prune / (double)mb), &lo, &hi, &That);
-    if (threadIdx.x == 0) {
-        set_window(sp, lo, hi, p.nb);
-        sp->mode = (k_prune == 0) ? 1u : (k_prune == mb ? 2u : 0u);
-        sp->k = (u64)k_prune;
-        p.work->That[0] = That;
-    }
-    // the sample blocks that survive the (estimated) prune threshold
+    u64 lo, hi, That = 0;
+    if (threadIdx.x == 0 && p.resid) *p.resid = 0.0;  // the kernels that follow add to it
+    if (by_group) {
+        // the prune classes are known (bit of the block's group): nothing to estimate
+        if (threadIdx.x == 0) {
+            set_window(sp, 0, 0, p.nb);
+            sp->mode = 3u;
+            sp->k = (u64)k_prune;
+            p.work->That[0] = 0;
+        }
 #pragma unroll
-    for (int t = 0; t < SAMP_PER; ++t) valid[t] = valid[t] && (k_prune == 0 || kp[t] > That);
+        for (int t = 0; t < SAMP_PER; ++t) valid[t] = valid[t] && !in_group[t];
+    } else {
+        sample_select(kp, valid, (float)((double)k_prune / (double)mb), &lo, &hi, &That);
+        if (threadIdx.x == 0) {
+            set_window(sp, lo, hi, p.nb);
+            sp->mode = (k_prune == 0) ? 1u : (k_prune == mb ? 2u : 0u);
+            sp->k = (u64)k_prune;
+            p.work->That[0] = That;
+        }
+        // the sample blocks that survive the (estimated) prune threshold
+#pragma unroll
+        for (int t = 0; t < SAMP_PER; ++t) valid[t] = valid[t] && (k_prune == 0 || kp[t] > That);
+    }
     const long long elig = mb - k_prune;
     sample_select(ku, valid, elig > 0 ? (float)((double)ksel_u / (double)elig) : 0.f, &lo, &hi, &That);
     if (threadIdx.x == 0) {
@@ -473,6 +544,23 @@ __global__ void __launch_bounds__(SAMP_THREADS) sample_kernel(Params p, long lon
         su->k = (u64)ksel_u;
         p.work->That[1] = That;
     }
+}
+
+// First kernel of the one-pass pipeline.  CTA 0 clears the selection state and chooses the windows;
+// the other CTAs clear the histograms (n_zero 32-bit words starting at zero_base).
+template <int B>
+__global__ void __launch_bounds__(SAMP_THREADS) sample_kernel(Params p, unsigned *zero_base, unsigned n_zero) {
+    if (blockIdx.x > 0) {
+        const unsigned per = (n_zero / 4 + gridDim.x - 2) / (gridDim.x - 1);          // uint4 pieces per CTA
+        uint4 *z = reinterpret_cast<uint4 *>(zero_base);
+        const unsigned lo = (blockIdx.x - 1) * per, hi = min(lo + per, n_zero / 4);
+        for (unsigned i = lo + threadIdx.x; i < hi; i += blockDim.x) z[i] = make_uint4(0, 0, 0, 0);
+        return;
+    }
+    unsigned *w = reinterpret_cast<unsigned *>(p.work);
+    for (unsigned i = threadIdx.x; i < sizeof(Work) / 4; i += blockDim.x) w[i] = 0u;
+    __syncthreads();
+    sample_body<B>(p);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -595,25 +683,26 @@ struct BinSel {
 };
 
 // level 0: which bin holds the k-th element; writes the bin and its composite range
-__device__ void select_bin(const Params &p, Sel *s, const unsigned *hist, BinSel *out, bool publish) {
+// sr: the CTA's copy of the selection (count and window); s: the global one, written when `publish`
+__device__ void select_bin(const Params &p, const Sel *sr, Sel *s, const unsigned *hist, BinSel *out, bool publish) {
     __shared__ unsigned s_bin, s_err;
     __shared__ u64 s_r, s_cnt;
     if (threadIdx.x == 0) { s_err = 0; s_bin = 0; s_r = 0; s_cnt = 0; }
     __syncthreads();
-    scan_hist(hist, p.nb, s->k, &s_bin, &s_r, &s_cnt, &s_err);
+    scan_hist(hist, p.nb, sr->k, &s_bin, &s_r, &s_cnt, &s_err);
     if (threadIdx.x == 0) {
         if (s_err) atomicOr(p.dev_status, (unsigned)MWU_DEV_SELECT);
         const unsigned B = s_bin;
         u64 klo, khi;
-        if (B == 0) { klo = 0; khi = s->lo0; }
-        else if (B == (unsigned)p.nb - 1u) { klo = s->hi0; khi = ~0ull >> 1; }     // keys are < 2^63
+        if (B == 0) { klo = 0; khi = sr->lo0; }
+        else if (B == (unsigned)p.nb - 1u) { klo = sr->hi0; khi = ~0ull >> 1; }     // keys are < 2^63
         else {
-            klo = s->lo0 + ((u64)(B - 1) << s->shift0);
-            khi = s->lo0 + ((u64)B << s->shift0);
-            if (khi > s->hi0) khi = s->hi0;
+            klo = sr->lo0 + ((u64)(B - 1) << sr->shift0);
+            khi = sr->lo0 + ((u64)B << sr->shift0);
+            if (khi > sr->hi0) khi = sr->hi0;
         }
         const u128 lo = make_c(klo, 0), hi = make_c(khi, 0);
-        if (publish) {                                   // for the kernels that follow
+        if (publish) {                                   // for the phases that follow
             s->B = B;
             s->r = s_r;
             s->cnt = s_cnt;
@@ -662,6 +751,7 @@ __device__ __forceinline__ bool selected(const Params &p, const SelView &s, long
                                          int which) {
     if (s.mode == 1u) return false;
     if (s.mode == 2u) return true;
+    if (s.mode == 3u) return group_pruned(p, (unsigned)j);      // grouped pruning: the group's bit
     if (bin < s.B) return true;
     if (bin > s.B) return false;
     const u64 key = exact_key<B>(p, j, which);
@@ -672,13 +762,12 @@ __device__ __forceinline__ bool selected(const Params &p, const SelView &s, long
 // stats_kernel
 // ---------------------------------------------------------------------------------------------
 template <int B>
-__global__ void __launch_bounds__(256) stats_kernel(Params p, double *loss_u, double *loss_p, float *u_out,
-                                                    unsigned *sign_bits) {
-    if (p.gated && p.work->failed == 0u) return;     // the one-pass result stands
-    if (p.gated && p.resid && blockIdx.x == 0 && threadIdx.x == 0) *p.resid = 0.0;   // emit_kernel sums afresh
+__device__ void stats_body(const Params &p, const Work &w, double *loss_u, double *loss_p, float *u_out,
+                           unsigned *sign_bits) {
+    if (p.gated && p.resid && blockIdx.x == 0 && threadIdx.x == 0) *p.resid = 0.0;   // emit_body sums afresh
     constexpr int NBT = 16 / B;                         // blocks per thread and step
-    const Sel *sp = &p.work->sel[0];
-    const Sel *su = &p.work->sel[1];
+    const Sel *sp = &w.sel[0];
+    const Sel *su = &w.sel[1];
     const u64 plo = sp->lo0, phi = sp->hi0, ulo = su->lo0, uhi = su->hi0;
     const unsigned psh = sp->shift0, ush = su->shift0;
     const unsigned nb = (unsigned)p.nb;
@@ -772,11 +861,11 @@ __global__ void __launch_bounds__(256) stats_kernel(Params p, double *loss_u, do
 // four consecutive bin codes starting at j4 (j4 % 4 == 0); codes beyond n read as 0
 __device__ __forceinline__ void load_codes4(const unsigned *bins, long long j4, long long n, unsigned (&c)[4]) {
     if (j4 + 4 <= n) {
-        const uint4 v = __ldg(reinterpret_cast<const uint4 *>(bins + j4));
+        const uint4 v = __ldcg(reinterpret_cast<const uint4 *>(bins + j4));
         c[0] = v.x; c[1] = v.y; c[2] = v.z; c[3] = v.w;
     } else {
 #pragma unroll
-        for (int e = 0; e < 4; ++e) c[e] = (j4 + e < n) ? __ldg(bins + j4 + e) : 0u;
+        for (int e = 0; e < 4; ++e) c[e] = (j4 + e < n) ? __ldcg(bins + j4 + e) : 0u;
     }
 }
 
@@ -801,24 +890,23 @@ __device__ void sort_candidates(u64 *key, unsigned *idx, int n_pow2) {
     }
 }
 
+// Exact threshold element of selection KIND.  w: this phase's copy of the selection state;
+// c_key / c_idx: CAP entries of shared memory each.
 template <int KIND, int B>
-__global__ void __launch_bounds__(FIN_THREADS) collect_kernel(Params p) {
-    if (p.gated && p.work->failed == 0u) return;     // the one-pass result stands
+__device__ void collect_body(const Params &p, const Work &w, u64 *c_key, unsigned *c_idx) {
     Sel *s = &p.work->sel[KIND];
-    if (s->mode != 0u) return;
-    __shared__ u64 c_key[CAP];
-    __shared__ unsigned c_idx[CAP];
+    const Sel *sw = &w.sel[KIND];
+    if (sw->mode != 0u) return;                       // the same in every CTA
     __shared__ unsigned s_bin, s_err, s_n;
     __shared__ u64 s_r, s_cnt;
-    // the selection state comes from the previous kernel: plain loads
-    const SelView pv = view_of(&p.work->sel[0]);
-    const unsigned Bsel = s->B;
-    const bool too_many = s->cnt > (u64)CAP;
+    const SelView pv = view_of(&w.sel[0]);
+    const unsigned Bsel = sw->B;
+    const bool too_many = sw->cnt > (u64)CAP;
     const long long stride = (long long)gridDim.x * blockDim.x;
 
     if (!too_many) {
-        const u128 lo = from_halves(s->lo_hi, s->lo_lo);
-        const u128 hi = from_halves(s->hi_hi, s->hi_lo);
+        const u128 lo = from_halves(sw->lo_hi, sw->lo_lo);
+        const u128 hi = from_halves(sw->hi_hi, sw->hi_lo);
         for (long long j0 = ((long long)blockIdx.x * blockDim.x + threadIdx.x) * 4; j0 < p.n_blocks;
              j0 += stride * 4 * PASS_LOADS) {
             unsigned codes[PASS_LOADS][4];
@@ -936,21 +1024,18 @@ __global__ void __launch_bounds__(FIN_THREADS) collect_kernel(Params p) {
 // candidates.  The last CTA sorts the candidates, which fixes the threshold element, counts the
 // L_u bins of the candidates that survive, and locates the unify threshold bin.
 template <int B>
-__global__ void __launch_bounds__(FIN_THREADS) prune_select_kernel(Params p) {
-    if (p.gated && p.work->failed == 0u) return;     // the one-pass result stands
+__device__ void prune_select_body(const Params &p, const Work &w, u64 *c_key, unsigned *c_idx) {
     Sel *sp = &p.work->sel[0];
     Sel *su = &p.work->sel[1];
-    const unsigned mode_p = sp->mode, mode_u = su->mode;
-    if (mode_p != 0u && mode_u != 0u) return;
-    __shared__ u64 c_key[CAP];
-    __shared__ unsigned c_idx[CAP];
+    const unsigned mode_p = w.sel[0].mode, mode_u = w.sel[1].mode;
+    if (mode_p != 0u && mode_u != 0u) return;         // the same in every CTA
     __shared__ unsigned s_bin, s_err, s_n;
     __shared__ u64 s_r, s_cnt;
     __shared__ BinSel s_sel;
     unsigned *hist_u = p.hist + p.nb;
     if (threadIdx.x == 0) { s_sel.B = 0; s_sel.r = 0; s_sel.cnt = 0; s_sel.lo_hi = s_sel.lo_lo = s_sel.hi_hi = s_sel.hi_lo = 0; }
     __syncthreads();
-    if (mode_p == 0u) select_bin(p, sp, p.hist, &s_sel, true);
+    if (mode_p == 0u) select_bin(p, &w.sel[0], sp, p.hist, &s_sel, true);
     const unsigned Bp = s_sel.B;
     const bool too_many = mode_p == 0u && s_sel.cnt > (u64)CAP;
     const u128 lo0 = from_halves(s_sel.lo_hi, s_sel.lo_lo);
@@ -984,6 +1069,8 @@ __global__ void __launch_bounds__(FIN_THREADS) prune_select_kernel(Params p) {
                             }
                             continue;
                         }
+                    } else if (mode_p == 3u) {
+                        if (group_pruned(p, (unsigned)j)) continue;
                     }
                     if (mode_u != 0u) continue;
                     if (bu == 0) ++under;
@@ -1097,27 +1184,25 @@ __global__ void __launch_bounds__(FIN_THREADS) prune_select_kernel(Params p) {
         __threadfence();
         __syncthreads();
     }
-    if (mode_u == 0u) select_bin(p, su, hist_u, &s_sel, true);
+    if (mode_u == 0u) select_bin(p, &w.sel[1], su, hist_u, &s_sel, true);
 }
 
 // ---------------------------------------------------------------------------------------------
-// emit_kernel
+// emit_body
 // ---------------------------------------------------------------------------------------------
+// s_stage: 128 float4 of shared memory per warp of the CTA
 template <int B>
-__global__ void __launch_bounds__(256, 3) emit_kernel(Params p, float *Q, float *u_out,
-                                                   unsigned *pruned_bitmap, unsigned *unified_bitmap,
-                                                   unsigned *sign_bits) {
-    if (p.gated && p.work->failed == 0u) return;     // the one-pass result stands
+__device__ void emit_body(const Params &p, const Work &w, float *Q, float *u_out, unsigned *pruned_bitmap,
+                          unsigned *unified_bitmap, unsigned *sign_bits, float4 *s_stage) {
     constexpr int NBT = 16 / B;
-    const SelView vp = view_of(&p.work->sel[0]);
-    const SelView vu = view_of(&p.work->sel[1]);
+    const SelView vp = view_of(&w.sel[0]);
+    const SelView vu = view_of(&w.sel[1]);
     const long long n = p.n_floats;
     const int lane = threadIdx.x & 31;
     const long long n_units = (n + 15) / 16;
     const long long n_iter = (n_units + 31) / 32 * 32;      // whole warps take part in every step
     const long long n_bm_words = (p.n_blocks + 31) / 32;
-    __shared__ float4 s_stage[8][128];                       // one warp step of Q per warp
-    float4 *ws = s_stage[threadIdx.x >> 5];
+    float4 *ws = s_stage + (threadIdx.x >> 5) * 128;         // one warp step of Q per warp
     double resid_acc = 0.0;
 
     for (long long unit = (long long)blockIdx.x * blockDim.x + threadIdx.x; unit < n_iter;
@@ -1127,18 +1212,18 @@ __global__ void __launch_bounds__(256, 3) emit_kernel(Params p, float *Q, float 
         unsigned code[NBT];
         const long long j0 = unit * NBT;
         if (j0 + NBT <= p.n_blocks) {
-            if (NBT == 1) code[0] = __ldg(p.bins + j0);
-            else if (NBT == 2) { const uint2 c = __ldg(reinterpret_cast<const uint2 *>(p.bins + j0)); code[0] = c.x; code[1 % NBT] = c.y; }
+            if (NBT == 1) code[0] = __ldcg(p.bins + j0);
+            else if (NBT == 2) { const uint2 c = __ldcg(reinterpret_cast<const uint2 *>(p.bins + j0)); code[0] = c.x; code[1 % NBT] = c.y; }
             else {
 #pragma unroll
                 for (int e = 0; e < NBT; e += 4) {
-                    const uint4 c = __ldg(reinterpret_cast<const uint4 *>(p.bins + j0 + e));
+                    const uint4 c = __ldcg(reinterpret_cast<const uint4 *>(p.bins + j0 + e));
                     code[e % NBT] = c.x; code[(e + 1) % NBT] = c.y; code[(e + 2) % NBT] = c.z; code[(e + 3) % NBT] = c.w;
                 }
             }
         } else {
 #pragma unroll
-            for (int e = 0; e < NBT; ++e) code[e] = (j0 + e < p.n_blocks) ? __ldg(p.bins + j0 + e) : 0u;
+            for (int e = 0; e < NBT; ++e) code[e] = (j0 + e < p.n_blocks) ? __ldcg(p.bins + j0 + e) : 0u;
         }
         unsigned cls_p = 0, cls_u = 0;                       // bit e: block e of this thread
         constexpr unsigned ALL = (1u << NBT) - 1u;
@@ -1348,6 +1433,8 @@ __global__ void __launch_bounds__(256) pass_kernel(Params p, float *Q, double *l
         unsigned code[NBT];
         float uo[NBT];
         const unsigned j0 = unit * NBT;
+        // grouped pruning: a unit's 16 values lie in one group (groups are at least 16 columns wide)
+        const bool grp = mode_p == 3u && j0 < n_blocks && group_pruned(p, j0);
 #pragma unroll
         for (int e = 0; e < NBT; ++e) {
             double S, Lu, Kp;
@@ -1371,6 +1458,9 @@ __global__ void __launch_bounds__(256) pass_kernel(Params p, float *Q, double *l
                     if (bp == 0u) ++under_p;
                     else if (bp == top) ++over_p;
                     else { atomicAdd(&hist_p[bp], 1u); open = true; }
+                } else if (mode_p == 3u) {
+                    pr = grp;                              // grouped pruning: the class is the group's bit
+                    survives = !grp;
                 } else {
                     pr = mode_p == 2u;
                     survives = mode_p == 1u;
@@ -1586,89 +1676,6 @@ __device__ bool pick_threshold(const Params &p, Sel *s, u64 r, unsigned n, u64 *
     return ok;
 }
 
-// list_select_kernel: exact prune threshold; the L_u histogram gains the listed blocks that
-// survive pruning; the unify threshold bin.
-template <int B>
-__global__ void __launch_bounds__(FIN_THREADS) list_select_kernel(Params p) {
-    if (p.work->failed != 0u) return;
-    Sel *sp = &p.work->sel[0];
-    Sel *su = &p.work->sel[1];
-    const unsigned mode_p = sp->mode, mode_u = su->mode;
-    if (mode_p != 0u && mode_u != 0u) return;
-    __shared__ u64 c_key[CAP];
-    __shared__ unsigned c_idx[CAP];
-    __shared__ BinSel s_sel;
-    const unsigned nb = (unsigned)p.nb, top = nb - 1u;
-    unsigned *hist_u = p.fhist + p.nb;
-    const u64 ulo = su->lo0, uhi = su->hi0;
-    const unsigned ush = su->shift0;
-    if (threadIdx.x == 0) { s_sel.B = 0; s_sel.r = 0; s_sel.cnt = 0; s_sel.lo_hi = s_sel.lo_lo = s_sel.hi_hi = s_sel.hi_lo = 0; }
-    __syncthreads();
-    if (mode_p == 0u) select_bin(p, sp, p.fhist, &s_sel, blockIdx.x == 0);   // every CTA computes the same values
-    const unsigned Bp = s_sel.B;
-    const u64 r_p = s_sel.r;
-    // the threshold bin must be a real bin of the window and small enough to sort
-    const bool hit_p = mode_p != 0u || (Bp >= 1u && Bp <= nb - 2u && s_sel.cnt <= (u64)CAP);
-    unsigned under = 0, over = 0;
-    if (mode_p == 0u && hit_p) {
-        const u128 lo0 = from_halves(s_sel.lo_hi, s_sel.lo_lo);
-        const u128 hi0 = from_halves(s_sel.hi_hi, s_sel.hi_lo);
-        const unsigned n_list = min(p.work->list_count, p.list_cap);
-        for (unsigned i = blockIdx.x * blockDim.x + threadIdx.x; i < n_list; i += gridDim.x * blockDim.x) {
-            const uint2 e = __ldg(&p.list[i]);
-            const unsigned bp = e.y & 0xffffu, bu = e.y >> 16;
-            if (bp == 0u || bp == top) continue;          // not in the prune window: counted by pass_kernel
-            if (bp < Bp) continue;                        // pruned
-            if (bp == Bp) {                               // decided by the last CTA
-                const u64 key = exact_key<B>(p, (long long)e.x, 0);
-                const u128 c = make_c(key, (u64)e.x);
-                if (c >= lo0 && c < hi0) {
-                    const unsigned slot = atomicAdd(&p.work->fcand_count[0], 1u);
-                    if (slot < (unsigned)CAP) { p.cand_key[slot] = key; p.cand_idx[slot] = e.x; }
-                }
-                continue;
-            }
-            if (mode_u != 0u) continue;
-            if (bu == 0u) ++under;
-            else if (bu == top) ++over;
-            else atomicAdd(&hist_u[bu], 1u);
-        }
-    }
-    for (int m = 16; m > 0; m >>= 1) {
-        under += __shfl_xor_sync(0xffffffffu, under, m);
-        over += __shfl_xor_sync(0xffffffffu, over, m);
-    }
-    if ((threadIdx.x & 31) == 0) {
-        if (under) atomicAdd(&hist_u[0], under);
-        if (over) atomicAdd(&hist_u[top], over);
-    }
-    if (!last_block_done(&p.work->fticket[0])) return;
-
-    // ---- last CTA only ----
-    if (mode_p == 0u) {
-        bool ok = hit_p;
-        const unsigned m = ld_vol(&p.work->fcand_count[0]);
-        if (ok) ok = pick_threshold(p, sp, r_p, m, c_key, c_idx);
-        if (!ok) {
-            if (threadIdx.x == 0) one_pass_fail(p);
-            return;
-        }
-        // the blocks of the threshold bin that survive join the L_u histogram
-        if (mode_u == 0u) {
-            for (unsigned i = (unsigned)r_p + threadIdx.x; i < m; i += blockDim.x) {
-                const u64 ku = exact_key<B>(p, (long long)c_idx[i], 1);
-                atomicAdd(&hist_u[bin_of(ku, ulo, uhi, ush, nb)], 1u);
-            }
-        }
-        __threadfence();
-        __syncthreads();
-    }
-    if (mode_u == 0u) {
-        select_bin(p, su, hist_u, &s_sel, true);
-        if (threadIdx.x == 0 && !(s_sel.B >= 1u && s_sel.B <= nb - 2u && s_sel.cnt <= (u64)CAP)) one_pass_fail(p);
-    }
-}
-
 // Final class of block j against what pass_kernel wrote (read back from the bitmaps); the
 // block's outputs are rewritten where they differ.
 template <int B>
@@ -1699,25 +1706,133 @@ __device__ __forceinline__ double apply_class(const Params &p, float *Q, float *
     return (pr ? sq : (un ? Lu : 0.0)) - (pr0 ? sq : (un0 ? Lu : 0.0));
 }
 
-// list_finish_kernel: every listed block outside the unify threshold bin gets its final class at
-// once; the blocks inside it are sorted by the last CTA, which fixes the threshold element and
-// their classes.
+// resolve_kernel (cooperative launch: all CTAs resident): the exact thresholds of the one-pass
+// pipeline and the final classes of the listed blocks, in one launch.
+//   first half   exact prune threshold bin from the window histogram; the listed blocks of that bin
+//                become candidates, the listed survivors complete the L_u histogram.  The CTA that
+//                finishes last ranks the candidates (exact threshold element), adds the surviving
+//                ones to the L_u histogram, locates the unify threshold bin and releases the others,
+//                which wait for it (bounded).
+//   second half  every listed block outside the unify threshold bin gets its final class at once
+//                (outputs rewritten where it differs from the provisional one); the blocks inside
+//                it are ranked by the CTA that finishes last, which fixes the threshold element and
+//                their classes.
+// A threshold outside its window, a threshold bin or tie group too large to rank, or a full list
+// gives the one-pass result up (work->failed): the multi-pass kernel behind redoes the projection.
 template <int B>
-__global__ void __launch_bounds__(FIN_THREADS) list_finish_kernel(Params p, float *Q, float *u_out,
-                                                                  unsigned *pruned_bitmap,
-                                                                  unsigned *unified_bitmap) {
-    // everything read here was written by earlier kernels: plain loads
-    if (p.work->failed != 0u) return;
-    Sel *su = &p.work->sel[1];
+__global__ void __launch_bounds__(FIN_THREADS) resolve_kernel(Params p, float *Q, float *u_out,
+                                                              unsigned *pruned_bitmap, unsigned *unified_bitmap) {
+    __shared__ Work w;                                 // selection state as the earlier kernels left it
     __shared__ u64 c_key[CAP];
     __shared__ unsigned c_idx[CAP];
-    const SelView vp = view_of(&p.work->sel[0]);
-    const unsigned mode_u = su->mode;
-    const unsigned Bu = su->B;
-    const u64 r_u = su->r;
-    const u128 lo = from_halves(su->lo_hi, su->lo_lo);
-    const u128 hi = from_halves(su->hi_hi, su->hi_lo);
-    const unsigned n_list = min(p.work->list_count, p.list_cap);
+    __shared__ BinSel s_sel;
+    __shared__ int s_go;
+    load_work(p.work, &w);
+    if (w.failed != 0u) return;                        // list overflow in pass_kernel: the same in every CTA
+    Sel *sp = &p.work->sel[0];
+    Sel *su = &p.work->sel[1];
+    const unsigned mode_p = w.sel[0].mode, mode_u = w.sel[1].mode;
+    if (mode_p != 0u && mode_u != 0u) return;
+    const unsigned nb = (unsigned)p.nb, top = nb - 1u;
+    unsigned *hist_u = p.fhist + p.nb;
+    const u64 ulo = w.sel[1].lo0, uhi = w.sel[1].hi0;
+    const unsigned ush = w.sel[1].shift0;
+    const unsigned n_list = min(w.list_count, p.list_cap);
+    if (threadIdx.x == 0) { s_sel.B = 0; s_sel.r = 0; s_sel.cnt = 0; s_sel.lo_hi = s_sel.lo_lo = s_sel.hi_hi = s_sel.hi_lo = 0; }
+    __syncthreads();
+
+    // ---------------- first half: the prune threshold ----------------
+    if (mode_p == 0u) select_bin(p, &w.sel[0], sp, p.fhist, &s_sel, blockIdx.x == 0);   // every CTA computes the same values
+    const unsigned Bp = s_sel.B;
+    const u64 r_p = s_sel.r;
+    // the threshold bin must be a real bin of the window and small enough to rank
+    const bool hit_p = mode_p != 0u || (Bp >= 1u && Bp <= nb - 2u && s_sel.cnt <= (u64)CAP);
+    if (!hit_p) {                                      // the same in every CTA
+        if (blockIdx.x == 0 && threadIdx.x == 0) one_pass_fail(p);
+        return;
+    }
+    if (mode_p == 0u) {
+        unsigned under = 0, over = 0;
+        const u128 lo0 = from_halves(s_sel.lo_hi, s_sel.lo_lo);
+        const u128 hi0 = from_halves(s_sel.hi_hi, s_sel.hi_lo);
+        for (unsigned i = blockIdx.x * blockDim.x + threadIdx.x; i < n_list; i += gridDim.x * blockDim.x) {
+            const uint2 e = __ldg(&p.list[i]);
+            const unsigned bp = e.y & 0xffffu, bu = e.y >> 16;
+            if (bp == 0u || bp == top) continue;          // not in the prune window: counted by pass_kernel
+            if (bp < Bp) continue;                        // pruned
+            if (bp == Bp) {                               // decided by the last CTA
+                const u64 key = exact_key<B>(p, (long long)e.x, 0);
+                const u128 c = make_c(key, (u64)e.x);
+                if (c >= lo0 && c < hi0) {
+                    const unsigned slot = atomicAdd(&p.work->fcand_count[0], 1u);
+                    if (slot < (unsigned)CAP) { p.cand_key[slot] = key; p.cand_idx[slot] = e.x; }
+                }
+                continue;
+            }
+            if (mode_u != 0u) continue;
+            if (bu == 0u) ++under;
+            else if (bu == top) ++over;
+            else atomicAdd(&hist_u[bu], 1u);
+        }
+        for (int m = 16; m > 0; m >>= 1) {
+            under += __shfl_xor_sync(0xffffffffu, under, m);
+            over += __shfl_xor_sync(0xffffffffu, over, m);
+        }
+        if ((threadIdx.x & 31) == 0) {
+            if (under) atomicAdd(&hist_u[0], under);
+            if (over) atomicAdd(&hist_u[top], over);
+        }
+    }
+    if (last_block_done(&p.work->fticket[0])) {
+        // ---- the CTA that finished last: exact prune threshold, unify threshold bin ----
+        bool ok = true;
+        if (mode_p == 0u) {
+            const unsigned m = ld_vol(&p.work->fcand_count[0]);
+            ok = pick_threshold(p, sp, r_p, m, c_key, c_idx);
+            // the blocks of the threshold bin that survive join the L_u histogram
+            if (ok && mode_u == 0u) {
+                for (unsigned i = (unsigned)r_p + threadIdx.x; i < m; i += blockDim.x) {
+                    const u64 ku = exact_key<B>(p, (long long)c_idx[i], 1);
+                    atomicAdd(&hist_u[bin_of(ku, ulo, uhi, ush, nb)], 1u);
+                }
+            }
+            __threadfence();
+            __syncthreads();
+        }
+        if (ok && mode_u == 0u) {
+            select_bin(p, &w.sel[1], su, hist_u, &s_sel, true);
+            if (!(s_sel.B >= 1u && s_sel.B <= nb - 2u && s_sel.cnt <= (u64)CAP)) ok = false;
+        }
+        if (threadIdx.x == 0) {
+            if (!ok) one_pass_fail(p);
+            __threadfence();
+            atomicExch(&p.work->release, 1u);
+        }
+    } else {
+        // the others wait for the thresholds (all CTAs are resident, the wait is bounded)
+        if (threadIdx.x == 0) {
+            int go = 1;
+            const long long t0 = clock64();
+            unsigned spins = 0;
+            while (ld_vol(&p.work->release) == 0u) {
+                if ((++spins & 63u) == 0u && clock64() - t0 > GRID_WAIT_CYCLES) { go = 0; break; }
+            }
+            __threadfence();
+            if (!go) { atomicOr(p.dev_status, (unsigned)MWU_DEV_TIMEOUT); one_pass_fail(p); }
+            s_go = go;
+        }
+        __syncthreads();
+        if (!s_go) return;
+    }
+    load_work(p.work, &w);                             // thresholds as the last CTA published them
+    if (w.failed != 0u) return;
+
+    // ---------------- second half: final classes of the listed blocks ----------------
+    const SelView vp = view_of(&w.sel[0]);
+    const unsigned Bu = w.sel[1].B;
+    const u64 r_u = w.sel[1].r;
+    const u128 lo = from_halves(w.sel[1].lo_hi, w.sel[1].lo_lo);
+    const u128 hi = from_halves(w.sel[1].hi_hi, w.sel[1].hi_lo);
     double resid_delta = 0.0;
     for (unsigned i = blockIdx.x * blockDim.x + threadIdx.x; i < n_list; i += gridDim.x * blockDim.x) {
         const uint2 e = __ldg(&p.list[i]);
@@ -1732,7 +1847,7 @@ __global__ void __launch_bounds__(FIN_THREADS) list_finish_kernel(Params p, floa
                     const u128 c = make_c(key, (u64)e.x);
                     if (c >= lo && c < hi) {
                         const unsigned slot = atomicAdd(&p.work->fcand_count[1], 1u);
-                        if (slot < (unsigned)CAP) { p.cand_key[slot] = key; p.cand_idx[slot] = e.x; }
+                        if (slot < (unsigned)CAP) { p.cand_key[CAP + slot] = key; p.cand_idx[CAP + slot] = e.x; }
                         continue;
                     }
                     un = c < lo;
@@ -1747,7 +1862,10 @@ __global__ void __launch_bounds__(FIN_THREADS) list_finish_kernel(Params p, floa
 
     // ---- last CTA only ----
     const unsigned m = ld_vol(&p.work->fcand_count[1]);
-    if (!pick_threshold(p, su, r_u, m, c_key, c_idx)) {
+    Params pc = p;                                     // the second half's candidates sit behind the first half's
+    pc.cand_key = p.cand_key + CAP;
+    pc.cand_idx = p.cand_idx + CAP;
+    if (!pick_threshold(pc, su, r_u, m, c_key, c_idx)) {
         if (threadIdx.x == 0) one_pass_fail(p);
         return;
     }
@@ -1758,6 +1876,173 @@ __global__ void __launch_bounds__(FIN_THREADS) list_finish_kernel(Params p, floa
     if (p.resid) block_add_double(tail_delta, p.resid);
 }
 
+// ---------------------------------------------------------------------------------------------
+// grouped pruning: keys of the prune groups, and the groups to zero
+// ---------------------------------------------------------------------------------------------
+// One CTA takes 256 rows x 64 columns of W (+U).  A half warp reads 64 consecutive values of one row;
+// every lane squares (or takes the magnitude of) its four values and the sums climb the pairwise tree
+// over the group's columns with shuffles (the pairing of the block keys continued across blocks);
+// the rows of a group are then summed as a pairwise tree in shared memory.  Everything is fp64 with
+// one rounding per operation, in a fixed order: the keys do not depend on the launch shape.
+__global__ void __launch_bounds__(256) group_stats_kernel(Params p, double *gkey, long long rows, long long cols) {
+    __shared__ double s_row[256][4];
+    const unsigned gc = p.group_cols, gr = p.group_rows;
+    const unsigned nsl = 64u / gc;                      // group slices per CTA tile: 4, 2 or 1
+    const unsigned lanes_per_slice = gc / 4u;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const long long row0 = (long long)blockIdx.y * 256, col0 = (long long)blockIdx.x * 64;
+    const long long col = col0 + (lane & 15) * 4;
+#pragma unroll 4
+    for (int it = 0; it < 16; ++it) {
+        const int r = warp * 32 + it * 2 + (lane >> 4);
+        const long long row = row0 + r;
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (row < rows && col < cols) {
+            v = __ldg(reinterpret_cast<const float4 *>(p.W + row * cols + col));
+            if (p.U) {
+                const float4 d = __ldg(reinterpret_cast<const float4 *>(p.U + row * cols + col));
+                v.x = __fadd_rn(v.x, d.x); v.y = __fadd_rn(v.y, d.y); v.z = __fadd_rn(v.z, d.z); v.w = __fadd_rn(v.w, d.w);
+            }
+        }
+        const double a0 = (double)fabsf(v.x), a1 = (double)fabsf(v.y), a2 = (double)fabsf(v.z), a3 = (double)fabsf(v.w);
+        double t;
+        if (p.use_l1) t = __dadd_rn(__dadd_rn(a0, a1), __dadd_rn(a2, a3));
+        else t = __dadd_rn(__fma_rn(a0, a0, __dmul_rn(a1, a1)), __fma_rn(a2, a2, __dmul_rn(a3, a3)));   // squares are exact
+        for (unsigned m = 1; m < lanes_per_slice; m <<= 1) t = __dadd_rn(t, __shfl_xor_sync(0xffffffffu, t, m));
+        if (((unsigned)lane & (lanes_per_slice - 1u)) == 0u) s_row[r][((unsigned)lane & 15u) / lanes_per_slice] = t;
+    }
+    __syncthreads();
+    // rows of a group: r with r ^ 1, then r ^ 2, ...
+    for (unsigned sdist = 1; sdist < gr; sdist <<= 1) {
+        for (unsigned i = threadIdx.x; i < 256u * nsl; i += blockDim.x) {
+            const unsigned r = i / nsl, sl = i % nsl;
+            if ((r & (2u * sdist - 1u)) == 0u) s_row[r][sl] = __dadd_rn(s_row[r][sl], s_row[r + sdist][sl]);
+        }
+        __syncthreads();
+    }
+    const long long gpr = cols / gc;                    // groups per row tile
+    for (unsigned i = threadIdx.x; i < (256u / gr) * nsl; i += blockDim.x) {
+        const unsigned g = i / nsl, sl = i % nsl;
+        const long long row = row0 + (long long)g * gr, c = col0 + (long long)sl * gc;
+        if (row < rows && c < cols) gkey[(row / gr) * gpr + c / gc] = s_row[g * gr][sl];
+    }
+}
+
+// One CTA: the kg groups with the smallest (key, index) get their bit in gprune.  Radix selection on
+// the keys' bit patterns (eight passes of eight bits) gives the threshold key and how many groups
+// holding exactly that key are taken; those are the ones with the lowest indices.
+__global__ void __launch_bounds__(FIN_THREADS) group_select_kernel(const double *gkey, unsigned n_groups, unsigned kg,
+                                                                   unsigned *gprune) {
+    __shared__ unsigned s_hist[256];
+    __shared__ u64 s_prefix;
+    __shared__ unsigned s_r;
+    __shared__ unsigned s_warp[32];
+    const u64 *keys = reinterpret_cast<const u64 *>(gkey);
+    const unsigned n_words = (n_groups + 31u) / 32u;
+    if (kg == 0u || kg >= n_groups) {
+        for (unsigned i = threadIdx.x; i < n_words; i += blockDim.x) {
+            unsigned wv = kg == 0u ? 0u : 0xffffffffu;
+            if (kg != 0u && i == n_words - 1u && (n_groups & 31u)) wv = (1u << (n_groups & 31u)) - 1u;
+            gprune[i] = wv;
+        }
+        return;
+    }
+    if (threadIdx.x == 0) { s_prefix = 0; s_r = kg; }
+    u64 mask = 0;
+    for (int shift = 56; shift >= 0; shift -= 8) {
+        for (unsigned i = threadIdx.x; i < 256u; i += blockDim.x) s_hist[i] = 0;
+        __syncthreads();
+        const u64 prefix = s_prefix;
+        for (unsigned i = threadIdx.x; i < n_groups; i += blockDim.x) {
+            const u64 k = __ldg(keys + i);
+            if ((k & mask) == prefix) atomicAdd(&s_hist[(unsigned)(k >> shift) & 255u], 1u);
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            unsigned r = s_r, d = 0;
+            while (d < 255u && s_hist[d] < r) { r -= s_hist[d]; ++d; }
+            s_r = r;
+            s_prefix = prefix | ((u64)d << shift);
+        }
+        mask |= (u64)255 << shift;
+        __syncthreads();
+    }
+    const u64 T = s_prefix;
+    const unsigned r_ties = s_r;                        // groups with key == T that are taken (>= 1)
+    // every thread owns a run of whole bitmap words; ties are numbered in index order
+    const unsigned words_per = (n_words + blockDim.x - 1u) / blockDim.x;
+    const unsigned w0 = threadIdx.x * words_per, w1 = min(w0 + words_per, n_words);
+    unsigned ties = 0;
+    for (unsigned wi = w0; wi < w1; ++wi)
+        for (unsigned bit = 0; bit < 32u; ++bit) {
+            const unsigned i = wi * 32u + bit;
+            if (i < n_groups && __ldg(keys + i) == T) ++ties;
+        }
+    const unsigned incl = block_scan_incl(ties, s_warp);
+    unsigned ordinal = incl - ties;                     // ties before this thread's run
+    for (unsigned wi = w0; wi < w1; ++wi) {
+        unsigned wv = 0;
+        for (unsigned bit = 0; bit < 32u; ++bit) {
+            const unsigned i = wi * 32u + bit;
+            if (i >= n_groups) break;
+            const u64 k = __ldg(keys + i);
+            bool take = k < T;
+            if (k == T) { take = ordinal < r_ties; ++ordinal; }
+            wv |= (take ? 1u : 0u) << bit;
+        }
+        gprune[wi] = wv;
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// multipass_kernel (cooperative launch): the whole multi-pass projection in one launch, its phases
+// separated by grid barriers -- [windows from a sample] -> statistics -> prune threshold -> unify
+// threshold -> emit.  It is the projection of small tensors (launch latency decides there), and the
+// fallback of the one-pass pipeline, behind which it is always enqueued and returns at once unless
+// work->failed is set.
+// ---------------------------------------------------------------------------------------------
+constexpr int MP_SMEM_BYTES = (FIN_THREADS / 32) * 128 * 16;     // emit staging: 2 KB per warp
+static_assert(MP_SMEM_BYTES >= CAP * 12, "the candidate sort buffers share the staging memory");
+
+template <int B>
+__global__ void __launch_bounds__(FIN_THREADS) multipass_kernel(Params p, float *Q, double *loss_u, double *loss_p,
+                                                                float *u_out, unsigned *pruned_bitmap,
+                                                                unsigned *unified_bitmap, unsigned *sign_bits) {
+    extern __shared__ __align__(16) unsigned char mp_smem[];
+    __shared__ Work w;
+    u64 *c_key = reinterpret_cast<u64 *>(mp_smem);
+    unsigned *c_idx = reinterpret_cast<unsigned *>(mp_smem + CAP * sizeof(u64));
+    if (p.gated) {
+        load_work(p.work, &w);
+        if (w.failed == 0u) return;                    // the one-pass result stands (the same in every CTA)
+    }
+    unsigned k = 0;                                    // grid barriers passed so far
+    bool ok = true;
+    if (p.run_sample) {
+        if (blockIdx.x == 0) sample_body<B>(p);
+        ok = grid_sync(&p.work->bar, ++k);
+    }
+    if (ok) {
+        load_work(p.work, &w);
+        stats_body<B>(p, w, loss_u, loss_p, u_out, sign_bits);
+        ok = grid_sync(&p.work->bar, ++k);
+    }
+    if (ok) {
+        prune_select_body<B>(p, w, c_key, c_idx);
+        ok = grid_sync(&p.work->bar, ++k);
+    }
+    if (ok) {
+        load_work(p.work, &w);
+        collect_body<1, B>(p, w, c_key, c_idx);
+        ok = grid_sync(&p.work->bar, ++k);
+    }
+    if (ok) {
+        load_work(p.work, &w);
+        emit_body<B>(p, w, Q, u_out, pruned_bitmap, unified_bitmap, sign_bits, reinterpret_cast<float4 *>(mp_smem));
+    }
+    if (!ok && threadIdx.x == 0) atomicOr(p.dev_status, (unsigned)MWU_DEV_TIMEOUT);
+}
+
 }  // namespace proj
 
 // ---------------------------------------------------------------------------------------------
@@ -1765,11 +2050,17 @@ __global__ void __launch_bounds__(FIN_THREADS) list_finish_kernel(Params p, floa
 // ---------------------------------------------------------------------------------------------
 static size_t ws_off_hist() { return align_up(sizeof(proj::Work)); }
 static size_t ws_off_cand_key() { return align_up(ws_off_hist() + 5 * proj::NB_MAX * sizeof(unsigned)); }
-static size_t ws_off_cand_idx() { return align_up(ws_off_cand_key() + proj::CAP * sizeof(proj::u64)); }
-static size_t ws_off_bins() { return align_up(ws_off_cand_idx() + proj::CAP * sizeof(unsigned)); }
+// two sets of candidates: the two halves of resolve_kernel each keep their own
+static size_t ws_off_cand_idx() { return align_up(ws_off_cand_key() + 2 * proj::CAP * sizeof(proj::u64)); }
+static size_t ws_off_bins() { return align_up(ws_off_cand_idx() + 2 * proj::CAP * sizeof(unsigned)); }
 static size_t ws_off_list(size_t mb) { return align_up(ws_off_bins() + (mb + 8) * sizeof(unsigned)); }
 // candidate list of the one-pass pipeline: a quarter of the blocks (the windows hold a few per cent)
 static size_t list_capacity(size_t mb) { return mb / 4 + 4096; }
+static size_t ws_off_gkey(size_t mb) { return align_up(ws_off_list(mb) + list_capacity(mb) * sizeof(uint2)); }
+static size_t n_groups_of(const mwu_proj_desc *d) {
+    return grouped(d) ? (size_t)(d->rows / d->prune_group_rows) * (size_t)(d->cols / d->prune_group_cols) : 0;
+}
+static size_t ws_off_gprune(const mwu_proj_desc *d, size_t mb) { return align_up(ws_off_gkey(mb) + n_groups_of(d) * sizeof(double)); }
 
 static bool use_one_pass(const mwu_proj_desc *desc) {
     if (desc->algo == MWU_ALGO_ONE_PASS) return true;
@@ -1782,51 +2073,78 @@ static bool use_one_pass(const mwu_proj_desc *desc) {
 extern "C" size_t mwu_project_workspace_bytes(const mwu_proj_desc *desc) {
     if (mwu::validate_desc(desc, false) != MWU_OK) return 0;
     const size_t mb = (size_t)(desc->rows * desc->cols / desc->block);
-    return mwu::align_up(mwu::ws_off_list(mb) + mwu::list_capacity(mb) * sizeof(uint2));
+    return mwu::align_up(mwu::ws_off_gprune(desc, mb) + (mwu::n_groups_of(desc) + 31) / 32 * 4 + 16);
+}
+
+// Cooperative launch (every CTA resident at once, which the grid barriers of the kernel rely on):
+// the grid is cut to what the device can hold of this kernel.
+template <typename... Args>
+static cudaError_t launch_cooperative(void (*kern)(Args...), int grid, int threads, size_t smem, int sm_count,
+                                      cudaStream_t st, Args... args) {
+    int per_sm = 0;
+    cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, threads, smem);
+    if (e != cudaSuccess) return e;
+    if (per_sm < 1) return cudaErrorCooperativeLaunchTooLarge;
+    const long long cap = (long long)per_sm * sm_count;
+    if (grid > cap) grid = (int)cap;
+    void *argv[] = {(void *)&args...};
+    mwu::count_launch();
+    return cudaLaunchCooperativeKernel((const void *)kern, dim3((unsigned)grid), dim3((unsigned)threads), argv, smem, st);
 }
 
 template <int B>
 static cudaError_t launch_project(const mwu::proj::Params &p, const mwu_proj_desc *desc, float *Q,
                                   float *u, unsigned *pb, unsigned *ub, unsigned *sb, double *loss_u,
-                                  double *loss_p, int sm_count, bool one_pass, cudaStream_t st) {
+                                  double *loss_p, int sm_count, bool one_pass, double *gkey, unsigned *gprune,
+                                  cudaStream_t st) {
     using namespace mwu::proj;
-    sample_kernel<B><<<1, SAMP_THREADS, 0, st>>>(p, desc->k_unify, desc->k_prune);
-    mwu::count_launch();
+    cudaError_t e;
+    if (p.gprune) {
+        // grouped pruning: the groups' keys, then the groups to zero (a bit per group)
+        const dim3 grid((unsigned)((desc->cols + 63) / 64), (unsigned)((desc->rows + 255) / 256));
+        group_stats_kernel<<<grid, 256, 0, st>>>(p, gkey, desc->rows, desc->cols);
+        const unsigned n_groups = (unsigned)mwu::n_groups_of(desc);
+        const unsigned per_group = (unsigned)(desc->prune_group_rows * desc->prune_group_cols / desc->block);
+        group_select_kernel<<<1, FIN_THREADS, 0, st>>>(gkey, n_groups, (unsigned)(desc->k_prune / per_group), gprune);
+        mwu::count_launch(2);
+    }
     const long long n_units = (p.n_floats + 15) / 16;
     const long long want = (n_units + 255) / 256;
     const long long cap_blocks = (long long)sm_count * 8;
-    int grid_stream = (int)(want < cap_blocks ? (want > 0 ? want : 1) : cap_blocks);
+    const int grid_stream = (int)(want < cap_blocks ? (want > 0 ? want : 1) : cap_blocks);
     const long long mb = p.n_blocks;
-    const bool need_p = desc->k_prune > 0 && desc->k_prune < mb;
+    const bool need_p = !p.gprune && desc->k_prune > 0 && desc->k_prune < mb;
     const long long ksel_u = desc->k_unify - desc->k_prune;
     const bool need_u = ksel_u > 0 && ksel_u < mb - desc->k_prune;
+    const long long want_mp = (n_units + FIN_THREADS - 1) / FIN_THREADS;
+    const int grid_mp = (int)(want_mp < (long long)sm_count ? (want_mp > 0 ? want_mp : 1) : (long long)sm_count);
+    static bool smem_set = false;                       // per instantiation: the attribute sticks to the function
+    if (!smem_set) {
+        e = cudaFuncSetAttribute(multipass_kernel<B>, cudaFuncAttributeMaxDynamicSharedMemorySize, MP_SMEM_BYTES);
+        if (e != cudaSuccess) return e;
+        smem_set = true;
+    }
 
     if (one_pass) {
+        // CTA 0 clears the selection state and samples; further CTAs clear the five histograms
+        const unsigned n_zero = 5u * (unsigned)p.nb;
+        const int zero_ctas = p.nb == NB_SMALL ? 1 : 8;
+        sample_kernel<B><<<1 + zero_ctas, SAMP_THREADS, 0, st>>>(p, p.hist, n_zero);
         if (p.U_next || p.resid) pass_kernel<B, true><<<grid_stream, 256, 0, st>>>(p, Q, loss_u, loss_p, u, pb, ub, sb);
         else pass_kernel<B, false><<<grid_stream, 256, 0, st>>>(p, Q, loss_u, loss_p, u, pb, ub, sb);
-        mwu::count_launch();
-        if (!need_p && !need_u) return cudaGetLastError();       // no threshold: every class is final
-        // the list holds a few per cent of the blocks
-        const long long lb = (mb / 8 + FIN_THREADS - 1) / FIN_THREADS;      // a thread per expected entry
-        // one CTA per SM at most: 1024 threads of 64 registers fill an SM's register file, a second
-        // CTA would only start when the first has ended
-        const int grid_list = (int)(lb < (long long)sm_count ? (lb > 0 ? lb : 1) : (long long)sm_count);
-        list_select_kernel<B><<<grid_list, FIN_THREADS, 0, st>>>(p);
-        list_finish_kernel<B><<<grid_list, FIN_THREADS, 0, st>>>(p, Q, u, pb, ub);
         mwu::count_launch(2);
+        if (!need_p && !need_u) return cudaGetLastError();       // no threshold: every class is final
+        // the list holds a few per cent of the blocks: a thread per expected entry, one CTA per SM at most
+        const long long lb = (mb / 8 + FIN_THREADS - 1) / FIN_THREADS;
+        const int grid_list = (int)(lb < (long long)sm_count ? (lb > 0 ? lb : 1) : (long long)sm_count);
+        e = launch_cooperative(resolve_kernel<B>, grid_list, FIN_THREADS, 0, sm_count, st, p, Q, u, pb, ub);
+        if (e != cudaSuccess) return e;
+        // behind it the multi-pass kernel, which returns at once unless the one-pass result was given up
+        // (once in thousands of calls)
     }
-    // multi-pass kernels: the whole projection, or (gated) the fallback of the one-pass pipeline.
-    // As a fallback they are needed once in thousands of calls and normally return at once, so
-    // they get one small wave of CTAs (every loop is grid-strided).
-    const int grid_fb = (int)(grid_stream < 2 * sm_count ? grid_stream : 2 * sm_count);
-    if (one_pass) grid_stream = grid_fb;
-    stats_kernel<B><<<grid_stream, 256, 0, st>>>(p, loss_u, loss_p, u, sb);
-    mwu::count_launch(2 + ((need_p || need_u) ? 1 : 0) + (need_u ? 1 : 0));      // stats, emit and the selection kernels below
-    const long long rb = (mb + 4 * FIN_THREADS - 1) / (4 * FIN_THREADS);
-    const int grid_fin = (int)(rb < (long long)sm_count ? (rb > 0 ? rb : 1) : (long long)sm_count);
-    if (need_p || need_u) prune_select_kernel<B><<<grid_fin, FIN_THREADS, 0, st>>>(p);
-    if (need_u) collect_kernel<1, B><<<grid_fin, FIN_THREADS, 0, st>>>(p);
-    emit_kernel<B><<<grid_stream, 256, 0, st>>>(p, Q, u, pb, ub, sb);
+    e = launch_cooperative(multipass_kernel<B>, grid_mp, FIN_THREADS, (size_t)MP_SMEM_BYTES, sm_count, st, p, Q, loss_u,
+                           loss_p, u, pb, ub, sb);
+    if (e != cudaSuccess) return e;
     return cudaGetLastError();
 }
 
@@ -1871,19 +2189,37 @@ static int project_impl(const mwu_proj_desc *desc, const float *W, const float *
     p.list = (uint2 *)(ws + ws_off_list((size_t)p.n_blocks));
     p.list_cap = (unsigned)list_capacity((size_t)p.n_blocks);
     p.gated = one_pass ? 1 : 0;
+    p.run_sample = one_pass ? 0 : 1;
     p.dev_status = dev_status;
     p.U_next = U_next;
     p.resid = residual_sq;
+    p.k_unify = desc->k_unify;
+    p.k_prune = desc->k_prune;
+    p.blocks_per_row = (unsigned)(desc->cols / desc->block);
+    double *gkey = nullptr;
+    unsigned *gprune = nullptr;
+    p.gprune = nullptr;
+    p.group_rows = p.group_cols = p.groups_per_row = 1;
+    if (grouped(desc)) {
+        gkey = (double *)(ws + ws_off_gkey((size_t)p.n_blocks));
+        gprune = (unsigned *)(ws + ws_off_gprune(desc, (size_t)p.n_blocks));
+        p.gprune = gprune;
+        p.group_rows = (unsigned)desc->prune_group_rows;
+        p.group_cols = (unsigned)desc->prune_group_cols;
+        p.groups_per_row = (unsigned)(desc->cols / desc->prune_group_cols);
+    }
 
-    if (cudaMemsetAsync(ws, 0, ws_off_hist() + 5 * (size_t)p.nb * sizeof(unsigned), st) != cudaSuccess)
+    // The one-pass pipeline clears its selection state and histograms in its first kernel; the
+    // multi-pass kernel, launched alone, needs them (and its barrier counter) cleared beforehand.
+    if (!one_pass &&
+        cudaMemsetAsync(ws, 0, ws_off_hist() + 5 * (size_t)p.nb * sizeof(unsigned), st) != cudaSuccess)
         return MWU_ERR_CUDA;
-    if (residual_sq && cudaMemsetAsync(residual_sq, 0, sizeof(double), st) != cudaSuccess) return MWU_ERR_CUDA;
     cudaError_t e;
     switch (desc->block) {
-        case 2: e = launch_project<2>(p, desc, Q, u, pruned_bitmap, unified_bitmap, sign_bits, loss_u, loss_p, sm_count, one_pass, st); break;
-        case 4: e = launch_project<4>(p, desc, Q, u, pruned_bitmap, unified_bitmap, sign_bits, loss_u, loss_p, sm_count, one_pass, st); break;
-        case 8: e = launch_project<8>(p, desc, Q, u, pruned_bitmap, unified_bitmap, sign_bits, loss_u, loss_p, sm_count, one_pass, st); break;
-        default: e = launch_project<16>(p, desc, Q, u, pruned_bitmap, unified_bitmap, sign_bits, loss_u, loss_p, sm_count, one_pass, st); break;
+        case 2: e = launch_project<2>(p, desc, Q, u, pruned_bitmap, unified_bitmap, sign_bits, loss_u, loss_p, sm_count, one_pass, gkey, gprune, st); break;
+        case 4: e = launch_project<4>(p, desc, Q, u, pruned_bitmap, unified_bitmap, sign_bits, loss_u, loss_p, sm_count, one_pass, gkey, gprune, st); break;
+        case 8: e = launch_project<8>(p, desc, Q, u, pruned_bitmap, unified_bitmap, sign_bits, loss_u, loss_p, sm_count, one_pass, gkey, gprune, st); break;
+        default: e = launch_project<16>(p, desc, Q, u, pruned_bitmap, unified_bitmap, sign_bits, loss_u, loss_p, sm_count, one_pass, gkey, gprune, st); break;
     }
     return e == cudaSuccess ? MWU_OK : MWU_ERR_CUDA;
 }

@@ -116,7 +116,7 @@ def test_gemm_output_leading_dimension():
     W = inputs.normal_weights(256, 128, 0.02, 65)
     desc, bufs, packed, p = project_and_pack(W, 8, 2000, 1000)
     X = inputs.normal_activations_bf16((100, 128), 3)
-    ref = O.gemm(X.to(torch.float64).numpy(), O.decoded_weights(p, 8))
+    ref = O.gemm(X.to(torch.float64).numpy(), O.decoded_weights(p))
     Y = run_gemm(desc, bufs, packed, X, 1, ldy=264)
     assert errors(Y, ref)[0] <= 1e-5
 
@@ -142,21 +142,33 @@ def test_gemm_config3_shape_reduced_rows():
                B.mwu_count_from_permille(Mb, wl.pruned_permille), 1000)
 
 
-def conv_case(W, b, ku, kp, x, kh, kw, stride, pad):
+def conv_case(W, b, ku, kp, x, kh, kw, stride, pad, expect_ws=None):
+    """Both entry points: mwu_conv_implicit (decode fused into the kernel) and mwu_conv_implicit_ws
+    (weights expanded once into a workspace; falls back to the first for shapes it does not serve)."""
     desc, bufs, packed, p = project_and_pack(W, b, ku, kp)
     n, c, h, w = x.shape
     oh = (h + 2 * pad - kh) // stride + 1
     ow = (w + 2 * pad - kw) // stride + 1
-    ref = O.conv2d_direct(x.to(torch.float64).numpy(), O.decoded_weights(p, b), kh, kw, stride, pad)
+    ref = O.conv2d_direct(x.to(torch.float64).numpy(), O.decoded_weights(p), kh, kw, stride, pad)
     xd = x.cuda().contiguous()
-    for y_dtype, tol in [(1, 1e-5), (0, 2e-3)]:
-        Y = torch.full((n, W.shape[0], oh, ow), float("nan"),
-                       dtype=torch.float32 if y_dtype else torch.bfloat16, device="cuda")
-        B.mwu_conv_implicit(desc, packed, xd, n, c, h, w, kh, kw, stride, pad, Y, y_dtype, bufs.dev_status)
-        torch.cuda.synchronize()
-        assert int(bufs.dev_status.item()) == 0
-        fro, mx = errors(Y.float().cpu().numpy(), ref)
-        assert fro <= tol and mx <= 1e-2, (y_dtype, fro, mx)
+    ws_bytes = B.mwu_conv_workspace_bytes(desc, n, c, h, w, kh, kw, stride, pad)
+    if expect_ws is not None:
+        assert (ws_bytes > 0) == expect_ws
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda") if ws_bytes else None
+    for use_ws in (False, True):
+        for y_dtype, tol in [(1, 1e-5), (0, 2e-3)]:
+            Y = torch.full((n, W.shape[0], oh, ow), float("nan"),
+                           dtype=torch.float32 if y_dtype else torch.bfloat16, device="cuda")
+            if use_ws:
+                B.mwu_conv_implicit_ws(desc, packed, xd, n, c, h, w, kh, kw, stride, pad, Y, y_dtype, ws,
+                                       bufs.dev_status)
+            else:
+                B.mwu_conv_implicit(desc, packed, xd, n, c, h, w, kh, kw, stride, pad, Y, y_dtype, bufs.dev_status)
+            torch.cuda.synchronize()
+            assert int(bufs.dev_status.item()) == 0
+            fro, mx = errors(Y.float().cpu().numpy(), ref)
+            assert fro <= tol and mx <= 1e-2, (use_ws, y_dtype, fro, mx)
+    return desc, bufs, packed, p, xd, ref
 
 
 def test_conv_small_cases():
@@ -172,6 +184,57 @@ def test_conv_small_cases():
     # 1x1 convolution equals a GEMM over channels
     W = inputs.normal_weights(128, 64, 0.05, 73)
     conv_case(W, 8, 300, 100, x, 1, 1, 1, 0)
+
+
+@pytest.mark.parametrize("filters,cin,h,w,k,pad,b", [(128, 64, 13, 12, 3, 1, 4),     # second tile of an image has 3 of 10 rows
+                                                     (256, 128, 28, 28, 3, 1, 16),   # two filter tiles, two channel chunks, 4-row tiles
+                                                     (200, 64, 9, 11, 5, 2, 8),      # 5x5 taps, filters ragged inside a tile
+                                                     (128, 64, 10, 10, 3, 0, 2),     # no padding: 8x8 output
+                                                     (128, 192, 6, 40, 1, 0, 8)])    # 1x1, three channel chunks, 3-row tiles
+def test_conv_workspace_path_shapes(filters, cin, h, w, k, pad, b):
+    W = inputs.normal_weights(filters, cin * k * k, 0.05, 740 + filters + cin + k)
+    x = inputs.normal_activations_bf16((3, cin, h, w), 741 + h)
+    Mb = W.numel() // b
+    conv_case(W, b, Mb * 6 // 10, Mb * 3 // 10, x, k, k, 1, pad, expect_ws=True)
+
+
+def test_conv_workspace_path_declines_other_shapes():
+    x = inputs.normal_activations_bf16((2, 64, 9, 7), 71)
+    W = inputs.normal_weights(128, 576, 0.05, 72)
+    d = B.make_desc(128, 576, 16, 1000, 500)
+    assert B.mwu_conv_workspace_bytes(d, 2, 64, 9, 7, 3, 3, 2, 0) == 0          # stride 2
+    assert B.mwu_conv_workspace_bytes(d, 2, 64, 9, 200, 3, 3, 1, 1) == 0        # 200 output pixels per row
+    assert B.mwu_conv_workspace_bytes(d, 2, 64, 9, 7, 3, 3, 1, 1) > 0
+    d2 = B.make_desc(128, 288, 16, 500, 200)                                     # 32 channels
+    assert B.mwu_conv_workspace_bytes(d2, 2, 32, 9, 7, 3, 3, 1, 1) == 0
+
+
+def test_bounded_wait_runs_out_and_the_context_stays_usable():
+    """Every wait of a kernel on its own barriers has a limit.  Here the producer of the convolution
+    kernel leaves one stage's loads out (a barrier that nothing completes) and the limit is cut to
+    about a millisecond: the kernel must come back by itself with MWU_DEV_TIMEOUT set, and the next
+    call on the same stream must give the right result."""
+    W = inputs.normal_weights(128, 576, 0.05, 760)
+    x = inputs.normal_activations_bf16((4, 64, 8, 8), 761)
+    Mb = W.numel() // 4
+    desc, bufs, packed, p = project_and_pack(W, 4, Mb // 2, Mb // 4)
+    ref = O.conv2d_direct(x.to(torch.float64).numpy(), O.decoded_weights(p), 3, 3, 1, 1)
+    xd = x.cuda()
+    ws = torch.empty(B.mwu_conv_workspace_bytes(desc, 4, 64, 8, 8, 3, 3, 1, 1), dtype=torch.uint8, device="cuda")
+    assert ws.numel() > 0
+    Y = torch.zeros((4, 128, 8, 8), dtype=torch.float32, device="cuda")
+    B.mwu_debug_conv_wait(2_000_000, 3)                  # ~1 ms; the fourth stage of every CTA never arrives
+    try:
+        B.mwu_conv_implicit_ws(desc, packed, xd, 4, 64, 8, 8, 3, 3, 1, 1, Y, 1, ws, bufs.dev_status)
+        torch.cuda.synchronize()
+    finally:
+        B.mwu_debug_conv_wait(0, -1)
+    assert int(bufs.dev_status.item()) & B.MWU_DEV_TIMEOUT
+    bufs.dev_status.zero_()
+    B.mwu_conv_implicit_ws(desc, packed, xd, 4, 64, 8, 8, 3, 3, 1, 1, Y, 1, ws, bufs.dev_status)
+    torch.cuda.synchronize()
+    assert int(bufs.dev_status.item()) == 0
+    assert errors(Y.cpu().numpy(), ref)[0] <= 1e-5
 
 
 def test_conv_config2():
