@@ -67,18 +67,28 @@ typedef enum {
 
 typedef struct {
     int64_t rows, cols;     /* W[rows][cols], row-major, cols % block == 0                    */
-    int32_t block;          /* micro-block width along cols: 2, 4, 8 or 16                    */
+    int32_t block;          /* micro-block width along cols: 2, 4, 8 or 16 (D1 of a 2- or
+                               3-dim block shape, see block_rows / block_taps below)          */
     int32_t prune_key;      /* mwu_prune_key                                                  */
     int64_t k_unify;        /* number of blocks unified OR pruned (0 <= k_prune <= k_unify)   */
     int64_t k_prune;        /* number of blocks pruned to zero                                */
     int32_t algo;           /* mwu_proj_algo; read by mwu_project, mwu_project_static and
                                mwu_admm_step                                                  */
-    int32_t reserved;       /* 0                                                              */
+    int32_t block_rows;     /* D2: rows a block spans; 0 or 1 = blocks lie in one row, 2 or 4 */
     /* Grouped pruning (0, 0 = off: blocks are pruned one by one, the paper's rule).  When set,
      * the prune decision is taken for whole groups of prune_group_rows x prune_group_cols
      * weights: see mwu_project. */
     int32_t prune_group_rows;   /* 0, 32, 64, 128 or 256; rows % prune_group_rows == 0        */
     int32_t prune_group_cols;   /* 0, 16, 32 or 64; >= block; cols % prune_group_cols == 0    */
+    /* 2- and 3-dim block shapes [D1, D2, D3] of Section 3.1 / Table 1 ([2,2], [2,2,2]) on a weight
+     * viewed as W[rows][cin * taps] (taps = kh*kw, column = channel * taps + tap): a block spans
+     * `block` input channels x block_rows rows x block_taps kernel taps.  Blocks are numbered
+     * (row group, channel group, tap group), their weights ordered (row, channel, tap) for the
+     * pairwise sums.  When block_taps does not divide taps the last tap group is shorter and its
+     * blocks hold fewer weights (their unified value is the mean over the weights they hold).
+     * block * block_rows * block_taps <= 16.  All zero (or one): the 1-dim blocks described above. */
+    int32_t block_taps;     /* D3: kernel taps a block spans; 0 or 1, or 2                      */
+    int32_t taps;           /* kh*kw of the weight (cols = cin * taps); 0 or 1 for a linear layer */
 } mwu_proj_desc;
 
 const char *mwu_status_string(int status);
@@ -337,6 +347,22 @@ int mwu_keep_n_of_m(int64_t rows, int64_t cols, int32_t n, int32_t m, const floa
 int mwu_gemm_dense(int64_t rows, int64_t cols, const void *Wd, int64_t ldw, const void *X, int64_t M,
                    int64_t ldx, void *Y, int64_t ldy, int32_t y_dtype, uint32_t *dev_status,
                    void *cuda_stream);
+
+/*
+ * mwu_conv_dense -- the convolution of mwu_conv_implicit for a plain bf16 weight matrix
+ * Wd[rows][ldw] whose first c*kh*kw columns are in [c][kh][kw] order (the counterpart of
+ * mwu_gemm_dense; it serves the block shapes that have no packed form: project with Q, round Q to
+ * bf16, multiply).  Shapes: stride 1, c % 64 == 0, at most 128 output pixels per row;
+ * mwu_conv_dense_workspace_bytes returns 0 for any other shape and the call then returns
+ * MWU_ERR_SHAPE.  `workspace`: device memory of that many bytes, 256-byte aligned, holding nothing
+ * between calls.
+ */
+size_t mwu_conv_dense_workspace_bytes(int64_t rows, int32_t n, int32_t c, int32_t h, int32_t w,
+                                      int32_t kh, int32_t kw, int32_t stride, int32_t pad);
+int mwu_conv_dense(int64_t rows, const void *Wd, int64_t ldw, const void *X_nchw, int32_t n, int32_t c,
+                   int32_t h, int32_t w, int32_t kh, int32_t kw, int32_t stride, int32_t pad,
+                   void *Y_nchw, int32_t y_dtype, void *workspace, size_t workspace_bytes,
+                   uint32_t *dev_status, void *cuda_stream);
 
 /*
  * mwu_debug_conv_wait -- testing aid for the bounded waits inside the kernels (the paper has no

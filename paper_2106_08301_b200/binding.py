@@ -19,7 +19,8 @@ EXPORTS = ["mwu_status_string", "mwu_kernel_launches", "mwu_count_from_permille"
            "mwu_project_workspace_bytes", "mwu_project", "mwu_admm_step", "mwu_project_static",
            "mwu_packed_bytes", "mwu_pack", "mwu_gemm", "mwu_decode", "mwu_gemm_workspace_bytes",
            "mwu_gemm_ws", "mwu_conv_implicit", "mwu_conv_workspace_bytes", "mwu_conv_implicit_ws",
-           "mwu_debug_conv_wait", "mwu_keep_n_of_m", "mwu_gemm_dense"]
+           "mwu_debug_conv_wait", "mwu_keep_n_of_m", "mwu_gemm_dense", "mwu_conv_dense_workspace_bytes",
+           "mwu_conv_dense"]
 MWU_STATIC_MAX_BLOCKS = 1048576
 
 MWU_OK = 0
@@ -39,8 +40,15 @@ class MwuError(RuntimeError):
 class ProjDesc(ctypes.Structure):
     _fields_ = [("rows", ctypes.c_int64), ("cols", ctypes.c_int64), ("block", ctypes.c_int32),
                 ("prune_key", ctypes.c_int32), ("k_unify", ctypes.c_int64),
-                ("k_prune", ctypes.c_int64), ("algo", ctypes.c_int32), ("reserved", ctypes.c_int32),
-                ("prune_group_rows", ctypes.c_int32), ("prune_group_cols", ctypes.c_int32)]
+                ("k_prune", ctypes.c_int64), ("algo", ctypes.c_int32), ("block_rows", ctypes.c_int32),
+                ("prune_group_rows", ctypes.c_int32), ("prune_group_cols", ctypes.c_int32),
+                ("block_taps", ctypes.c_int32), ("taps", ctypes.c_int32)]
+
+    @property
+    def n_blocks(self) -> int:
+        """Blocks of the partition this descriptor names (1-, 2- or 3-dim shape)."""
+        dr, dt, taps = max(self.block_rows, 1), max(self.block_taps, 1), max(self.taps, 1)
+        return (self.rows // dr) * ((self.cols // taps) // self.block) * ((taps + dt - 1) // dt)
 
 
 _lib = None
@@ -91,6 +99,10 @@ def lib() -> ctypes.CDLL:
         L.mwu_keep_n_of_m.argtypes = [i64, i64, i32, i32, vp, vp, vp, vp, vp, i64, vp, vp]
         L.mwu_gemm_dense.restype = ctypes.c_int
         L.mwu_gemm_dense.argtypes = [i64, i64, vp, i64, vp, i64, i64, vp, i64, i32, vp, vp]
+        L.mwu_conv_dense_workspace_bytes.restype = sz
+        L.mwu_conv_dense_workspace_bytes.argtypes = [i64] + [i32] * 8
+        L.mwu_conv_dense.restype = ctypes.c_int
+        L.mwu_conv_dense.argtypes = [i64, vp, i64, vp] + [i32] * 8 + [vp, i32, vp, sz, vp, vp]
         L.mwu_debug_conv_wait.restype = None
         L.mwu_debug_conv_wait.argtypes = [i64, i64]
         _lib = L
@@ -115,11 +127,12 @@ def status_string(status: int) -> str:
 
 def make_desc(rows: int, cols: int, block: int, k_unify: int, k_prune: int,
               prune_key: int = MWU_PRUNE_KEY_L2SQ, algo: int = MWU_ALGO_AUTO,
-              prune_group=None) -> ProjDesc:
-    """prune_group = (rows, cols) of a prune group, or None for block-by-block pruning."""
+              prune_group=None, block_rows: int = 0, block_taps: int = 0, taps: int = 0) -> ProjDesc:
+    """prune_group = (rows, cols) of a prune group, or None for block-by-block pruning.
+    block_rows / block_taps / taps: 2- and 3-dim block shapes (block = channels of a block)."""
     gr, gc = prune_group if prune_group else (0, 0)
     return ProjDesc(int(rows), int(cols), int(block), int(prune_key), int(k_unify), int(k_prune),
-                    int(algo), 0, int(gr), int(gc))
+                    int(algo), int(block_rows), int(gr), int(gc), int(block_taps), int(taps))
 
 
 def mwu_kernel_launches() -> int:
@@ -240,6 +253,22 @@ def mwu_gemm_dense(rows, cols, Wd, ldw, X, M, ldx, Y, ldy, y_dtype, dev_status, 
     return rc
 
 
+def mwu_conv_dense_workspace_bytes(rows, n, c, h, w, kh, kw, stride, pad) -> int:
+    return int(lib().mwu_conv_dense_workspace_bytes(int(rows), int(n), int(c), int(h), int(w), int(kh), int(kw),
+                                                    int(stride), int(pad)))
+
+
+def mwu_conv_dense(rows, Wd, ldw, X, n, c, h, w, kh, kw, stride, pad, Y, y_dtype, workspace, dev_status,
+                   stream=None, check=True) -> int:
+    nbytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    rc = lib().mwu_conv_dense(int(rows), _ptr(Wd), int(ldw), _ptr(X), int(n), int(c), int(h), int(w), int(kh),
+                              int(kw), int(stride), int(pad), _ptr(Y), int(y_dtype), _ptr(workspace), nbytes,
+                              _ptr(dev_status), _stream(stream))
+    if check and rc != MWU_OK:
+        raise MwuError(rc, "mwu_conv_dense")
+    return rc
+
+
 def mwu_debug_conv_wait(limit_cycles: int, withhold_stage: int) -> None:
     lib().mwu_debug_conv_wait(int(limit_cycles), int(withhold_stage))
 
@@ -268,7 +297,7 @@ class ProjectionBuffers:
     """Device buffers for one mwu_project call on a [rows, cols] weight."""
 
     def __init__(self, desc: ProjDesc, device="cuda", want_q=True, want_loss=False):
-        mb = desc.rows * desc.cols // desc.block
+        mb = desc.n_blocks
         n = desc.rows * desc.cols
         self.desc = desc
         self.Q = torch.empty(n, dtype=torch.float32, device=device) if want_q else None

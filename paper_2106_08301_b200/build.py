@@ -15,7 +15,7 @@ INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 LIB = os.path.join(HERE, "libmwu.so")
 OBJ_DIR = os.path.join(HERE, "_build")
 SOURCES = ["mwu_api.cu", "mwu_project.cu", "mwu_pack.cu", "mwu_gemm.cu", "mwu_gemm2.cu", "mwu_gemm3.cu",
-           "mwu_conv.cu", "mwu_nm.cu", "mwu_noalloc.cu"]
+           "mwu_conv.cu", "mwu_nm.cu", "mwu_shapes.cu", "mwu_noalloc.cu"]
 ARCH = ["-gencode", "arch=compute_100a,code=sm_100a"]
 
 

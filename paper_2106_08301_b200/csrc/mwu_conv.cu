@@ -131,13 +131,25 @@ __global__ void __launch_bounds__(128) mwu_decode_taps_kernel(const Params p, un
     }
 }
 
+// a plain dense weight matrix [rows][ldw] in [c][tap] column order -> [n_pad][c * taps] tap-major
+// (rows beyond `rows` are written as zeros)
+__global__ void __launch_bounds__(256) permute_taps_kernel(const unsigned short *Wd, long long ldw, long long rows,
+                                                           long long n_pad, int taps, int C, unsigned short *out) {
+    const long long K = (long long)taps * C, total = n_pad * K;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
+        const long long row = i / K, kk = i - row * K;
+        const int tap = (int)(kk / C), c = (int)(kk - (long long)tap * C);
+        out[i] = row < rows ? Wd[row * ldw + (long long)c * taps + tap] : (unsigned short)0;
+    }
+}
+
 // ------------------------------------------------------------------------------------------
 // the tensor-core kernel
 // ------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(C_THREADS, 1)
 mwu_conv_taps_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
                      const ConvParams p) {
-    MWU_CHECK_HEADER(p.g);
+    if (!p.g.all_live) MWU_CHECK_HEADER(p.g);
     extern __shared__ unsigned char smem_raw[];
     unsigned char *base = reinterpret_cast<unsigned char *>(
         (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -297,9 +309,10 @@ mwu_conv_taps_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_co
     }
 
     // teardown
-    if (*abort && threadIdx.x == 0) atomicOr(p.g.dev_status, (unsigned)MWU_DEV_TIMEOUT);
     tc_fence_before();
     __syncthreads();
+    // after the barrier: a role that finished its own work early must still see a flag raised later
+    if (*abort && threadIdx.x == 0) atomicOr(p.g.dev_status, (unsigned)MWU_DEV_TIMEOUT);
     if (warp == 1) {
         tc_fence_after();
         tmem_dealloc(tmem_base, 256);
@@ -347,6 +360,78 @@ extern "C" size_t mwu_conv_workspace_bytes(const mwu_proj_desc *desc, int32_t n,
     return gemm::x_bytes_aligned(n, c, h, w) + (size_t)L.n_pad * (size_t)desc->cols * 2;
 }
 
+namespace mwu {
+namespace gemm {
+
+// shape of the convolution alone (no descriptor): stride 1, channels in chunks of 64, at most 128
+// output pixels per row
+static bool taps_geometry(int n, int c, int h, int w, int kh, int kw, int stride, int pad, int *OH, int *OW, int *R) {
+    if (n <= 0 || c <= 0 || h <= 0 || w <= 0 || kh <= 0 || kw <= 0 || stride != 1 || pad < 0) return false;
+    if (c % BK != 0 || h + 2 * pad < kh || w + 2 * pad < kw || pad > 32767) return false;
+    const int oh = h + 2 * pad - kh + 1, ow = w + 2 * pad - kw + 1;
+    if (ow > 128 || w > 65535 || h > 65535) return false;
+    int r = 128 / ow;
+    if (r > oh) r = oh;
+    if (r > 256) r = 256;
+    *OH = oh; *OW = ow; *R = r;
+    return true;
+}
+
+// image copy, tensor maps and the tensor-core kernel; the tap-major weights must already be in `wd`
+// (or be produced by `make_weights`, which is enqueued between the image copy and the main kernel)
+template <typename F>
+static int run_taps(ConvParams &p, const void *X_nchw, int n, int c, int h, int w, int kh, int kw, int pad,
+                    unsigned short *xt, unsigned short *wd, long long n_pad, int sm_count, cudaStream_t st,
+                    F make_weights) {
+    EncodeTiledFn encode = get_encode_fn();
+    if (!encode) return MWU_ERR_CUDA;
+    int OH, OW, R;
+    if (!taps_geometry(n, c, h, w, kh, kw, 1, pad, &OH, &OW, &R)) return MWU_ERR_SHAPE;
+    const long long K = (long long)c * kh * kw;
+    p.C = c; p.H = h; p.W = w; p.KH = kh; p.KW = kw; p.pad = pad; p.OH = OH; p.OW = OW; p.NIMG = n;
+    p.R = R;
+    p.tiles_per_img = (OH + R - 1) / R;
+    p.n_ntiles = (int)(n_pad / kTileRows);
+    p.a_bytes = (unsigned)(R * OW * 128);
+    p.wait_limit = g_wait_limit;
+    p.withhold = g_withhold;
+    // tensor maps: the pixel-major image as [n][h][w][c] (innermost first: c, w, h, n), and the weights
+    CUtensorMap tmap_x, tmap_w;
+    {
+        const cuuint64_t gdim[4] = {(cuuint64_t)c, (cuuint64_t)w, (cuuint64_t)h, (cuuint64_t)n};
+        const cuuint64_t gstr[3] = {(cuuint64_t)c * 2, (cuuint64_t)w * c * 2, (cuuint64_t)h * w * c * 2};
+        const cuuint32_t box[4] = {(cuuint32_t)BK, (cuuint32_t)OW, (cuuint32_t)R, 1};
+        const cuuint32_t estr[4] = {1, 1, 1, 1};
+        if (encode(&tmap_x, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, xt, gdim, gstr, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                   CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return MWU_ERR_CUDA;
+        const cuuint64_t wdim[2] = {(cuuint64_t)K, (cuuint64_t)n_pad};
+        const cuuint64_t wstr[1] = {(cuuint64_t)K * 2};
+        const cuuint32_t wbox[2] = {(cuuint32_t)BK, (cuuint32_t)kTileRows};
+        const cuuint32_t west[2] = {1, 1};
+        if (encode(&tmap_w, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, wd, wdim, wstr, wbox, west, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                   CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return MWU_ERR_CUDA;
+    }
+    const int HW = h * w;
+    nchw_to_nhwc_kernel<<<dim3((unsigned)((HW + 31) / 32), (unsigned)((c + 31) / 32), (unsigned)n), 256, 0, st>>>(
+        (const unsigned short *)X_nchw, xt, c, HW);
+    make_weights();
+    const size_t smem = conv_smem_bytes();
+    if (cudaFuncSetAttribute(mwu_conv_taps_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+        return MWU_ERR_CUDA;
+    const long long tiles = (long long)n * p.tiles_per_img * p.n_ntiles;
+    const int grid = (int)(tiles < sm_count ? tiles : sm_count);
+    mwu_conv_taps_kernel<<<grid, C_THREADS, smem, st>>>(tmap_x, tmap_w, p);
+    count_launch(3);
+    return cudaGetLastError() == cudaSuccess ? MWU_OK : MWU_ERR_CUDA;
+}
+
+}  // namespace gemm
+}  // namespace mwu
+
 extern "C" int mwu_conv_implicit_ws(const mwu_proj_desc *desc, const void *packed, const void *X_nchw,
                                     int32_t n, int32_t c, int32_t h, int32_t w, int32_t kh, int32_t kw,
                                     int32_t stride, int32_t pad, void *Y_nchw, int32_t y_dtype,
@@ -366,13 +451,9 @@ extern "C" int mwu_conv_implicit_ws(const mwu_proj_desc *desc, const void *packe
     int sm_count = 0;
     int rc = check_device(&sm_count);
     if (rc != MWU_OK) return rc;
-    EncodeTiledFn encode = get_encode_fn();
-    if (!encode) return MWU_ERR_CUDA;
     cudaStream_t st = (cudaStream_t)cuda_stream;
 
     ConvParams p = {};
-    int OH, OW, R;
-    taps_path(desc, n, c, h, w, kh, kw, stride, pad, &OH, &OW, &R);
     const PackedLayout L = packed_layout(desc);
     p.g.packed = (const unsigned char *)packed;
     p.g.off_rec = L.off_rec; p.g.off_ulist = L.off_ulist; p.g.off_dpos = L.off_dpos;
@@ -386,53 +467,63 @@ extern "C" int mwu_conv_implicit_ws(const mwu_proj_desc *desc, const void *packe
     p.g.Y = Y_nchw;
     p.g.y_fp32 = y_dtype;
     p.g.dev_status = dev_status;
-    p.C = c; p.H = h; p.W = w; p.KH = kh; p.KW = kw; p.pad = pad; p.OH = OH; p.OW = OW; p.NIMG = n;
-    p.R = R;
-    p.tiles_per_img = (OH + R - 1) / R;
-    p.n_ntiles = (int)L.n_tiles;
-    p.a_bytes = (unsigned)(R * OW * 128);
-    p.wait_limit = g_wait_limit;
-    p.withhold = g_withhold;
-
     unsigned short *xt = (unsigned short *)workspace;
     unsigned short *wd = (unsigned short *)((char *)workspace + x_bytes_aligned(n, c, h, w));
-    // tensor maps: the pixel-major image as [n][h][w][c] (innermost first: c, w, h, n), and the weights
-    CUtensorMap tmap_x, tmap_w;
-    {
-        const cuuint64_t gdim[4] = {(cuuint64_t)c, (cuuint64_t)w, (cuuint64_t)h, (cuuint64_t)n};
-        const cuuint64_t gstr[3] = {(cuuint64_t)c * 2, (cuuint64_t)w * c * 2, (cuuint64_t)h * w * c * 2};
-        const cuuint32_t box[4] = {(cuuint32_t)BK, (cuuint32_t)OW, (cuuint32_t)R, 1};
-        const cuuint32_t estr[4] = {1, 1, 1, 1};
-        if (encode(&tmap_x, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, xt, gdim, gstr, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                   CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-            return MWU_ERR_CUDA;
-        const cuuint64_t wdim[2] = {(cuuint64_t)desc->cols, (cuuint64_t)L.n_pad};
-        const cuuint64_t wstr[1] = {(cuuint64_t)desc->cols * 2};
-        const cuuint32_t wbox[2] = {(cuuint32_t)BK, (cuuint32_t)kTileRows};
-        const cuuint32_t west[2] = {1, 1};
-        if (encode(&tmap_w, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, wd, wdim, wstr, wbox, west, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                   CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-            return MWU_ERR_CUDA;
-    }
-    const int HW = h * w;
-    nchw_to_nhwc_kernel<<<dim3((unsigned)((HW + 31) / 32), (unsigned)((c + 31) / 32), (unsigned)n), 256, 0, st>>>(
-        (const unsigned short *)X_nchw, xt, c, HW);
     const unsigned n_rec = (unsigned)(L.n_tiles * L.n_stages);
+    const int taps = kh * kw, bw = desc->block;
+    const Params g = p.g;
+    return run_taps(p, X_nchw, n, c, h, w, kh, kw, pad, xt, wd, L.n_pad, sm_count, st, [&]() {
+        switch (bw) {
+            case 2: mwu_decode_taps_kernel<2><<<n_rec, 128, 0, st>>>(g, wd, taps, c); break;
+            case 4: mwu_decode_taps_kernel<4><<<n_rec, 128, 0, st>>>(g, wd, taps, c); break;
+            case 8: mwu_decode_taps_kernel<8><<<n_rec, 128, 0, st>>>(g, wd, taps, c); break;
+            default: mwu_decode_taps_kernel<16><<<n_rec, 128, 0, st>>>(g, wd, taps, c); break;
+        }
+    });
+}
+
+extern "C" size_t mwu_conv_dense_workspace_bytes(int64_t rows, int32_t n, int32_t c, int32_t h, int32_t w,
+                                                 int32_t kh, int32_t kw, int32_t stride, int32_t pad) {
+    using namespace mwu;
+    int OH, OW, R;
+    if (rows <= 0 || !gemm::taps_geometry(n, c, h, w, kh, kw, stride, pad, &OH, &OW, &R)) return 0;
+    const int64_t n_pad = (rows + kTileRows - 1) / kTileRows * kTileRows;
+    return gemm::x_bytes_aligned(n, c, h, w) + (size_t)n_pad * (size_t)c * kh * kw * 2;
+}
+
+extern "C" int mwu_conv_dense(int64_t rows, const void *Wd, int64_t ldw, const void *X_nchw, int32_t n, int32_t c,
+                              int32_t h, int32_t w, int32_t kh, int32_t kw, int32_t stride, int32_t pad,
+                              void *Y_nchw, int32_t y_dtype, void *workspace, size_t workspace_bytes,
+                              uint32_t *dev_status, void *cuda_stream) {
+    using namespace mwu;
+    using namespace mwu::gemm;
+    if (!Wd || !X_nchw || !Y_nchw || !dev_status || !workspace) return MWU_ERR_INVALID_ARG;
+    if (y_dtype != 0 && y_dtype != 1) return MWU_ERR_INVALID_ARG;
+    const size_t need = mwu_conv_dense_workspace_bytes(rows, n, c, h, w, kh, kw, stride, pad);
+    if (need == 0 || ldw < (int64_t)c * kh * kw) return MWU_ERR_SHAPE;
+    if (workspace_bytes < need) return MWU_ERR_WORKSPACE;
+    if (!aligned_to(Wd, 2) || !aligned_to(X_nchw, 16) || !aligned_to(Y_nchw, 16) || !aligned_to(dev_status, 4) ||
+        !aligned_to(workspace, 256))
+        return MWU_ERR_ALIGNMENT;
+    int sm_count = 0;
+    const int rc = check_device(&sm_count);
+    if (rc != MWU_OK) return rc;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    ConvParams p = {};
+    p.g.all_live = 1;                                   // plain weights: no packed header to compare with
+    p.g.N = rows;
+    p.g.K = (long long)c * kh * kw;
+    p.g.Y = Y_nchw;
+    p.g.y_fp32 = y_dtype;
+    p.g.dev_status = dev_status;
+    const long long n_pad = (rows + kTileRows - 1) / kTileRows * kTileRows;
+    unsigned short *xt = (unsigned short *)workspace;
+    unsigned short *wd = (unsigned short *)((char *)workspace + x_bytes_aligned(n, c, h, w));
     const int taps = kh * kw;
-    switch (desc->block) {
-        case 2: mwu_decode_taps_kernel<2><<<n_rec, 128, 0, st>>>(p.g, wd, taps, c); break;
-        case 4: mwu_decode_taps_kernel<4><<<n_rec, 128, 0, st>>>(p.g, wd, taps, c); break;
-        case 8: mwu_decode_taps_kernel<8><<<n_rec, 128, 0, st>>>(p.g, wd, taps, c); break;
-        default: mwu_decode_taps_kernel<16><<<n_rec, 128, 0, st>>>(p.g, wd, taps, c); break;
-    }
-    const size_t smem = conv_smem_bytes();
-    if (cudaFuncSetAttribute(mwu_conv_taps_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-        return MWU_ERR_CUDA;
-    const long long tiles = (long long)n * p.tiles_per_img * p.n_ntiles;
-    const int grid = (int)(tiles < sm_count ? tiles : sm_count);
-    mwu_conv_taps_kernel<<<grid, C_THREADS, smem, st>>>(tmap_x, tmap_w, p);
-    count_launch(3);
-    return cudaGetLastError() == cudaSuccess ? MWU_OK : MWU_ERR_CUDA;
+    return run_taps(p, X_nchw, n, c, h, w, kh, kw, pad, xt, wd, n_pad, sm_count, st, [&]() {
+        const long long total = n_pad * p.g.K;
+        const long long want = (total + 255) / 256, cap = (long long)sm_count * 16;
+        permute_taps_kernel<<<(unsigned)(want < cap ? want : cap), 256, 0, st>>>((const unsigned short *)Wd, ldw, rows,
+                                                                                  n_pad, taps, c, wd);
+    });
 }

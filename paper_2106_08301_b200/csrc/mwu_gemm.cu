@@ -482,9 +482,10 @@ mwu_gemm_kernel(const __grid_constant__ CUtensorMap tmap, const Params p) {
     }
 
     // teardown
-    if (*abort && threadIdx.x == 0) atomicOr(p.dev_status, (unsigned)MWU_DEV_TIMEOUT);
     tc_fence_before();
     __syncthreads();
+    // after the barrier: a role that finished its own work early must still see a flag raised later
+    if (*abort && threadIdx.x == 0) atomicOr(p.dev_status, (unsigned)MWU_DEV_TIMEOUT);
     if (warp == 1) {
         tc_fence_after();
         tmem_dealloc(tmem_base, 512);

@@ -348,9 +348,10 @@ mwu_dense_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
     }
 
     // teardown: nobody leaves while the other CTA may still read this one's memory or barriers
-    if (*abort && threadIdx.x == 0) atomicOr(p.dev_status, (unsigned)MWU_DEV_TIMEOUT);
     tc_fence_before();
     __syncthreads();
+    // after the barrier: a role that finished its own work early must still see a flag raised later
+    if (*abort && threadIdx.x == 0) atomicOr(p.dev_status, (unsigned)MWU_DEV_TIMEOUT);
     cluster_sync_all();
     if (warp == 1) {
         tc_fence_after();

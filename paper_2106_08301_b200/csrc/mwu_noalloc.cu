@@ -49,7 +49,7 @@ extern "C" int mwu_project_static(const mwu_proj_desc *desc, const float *W, con
                                   double *loss_p, uint32_t *dev_status, void *cuda_stream) {
     const int rc = mwu::validate_desc(desc, false);
     if (rc != MWU_OK) return rc;
-    const int64_t n_blocks = desc->rows * desc->cols / desc->block;
+    const int64_t n_blocks = mwu::shape_of(desc).mb;
     const size_t need = mwu_project_workspace_bytes(desc);
     if (n_blocks > (int64_t)MWU_STATIC_MAX_BLOCKS || need == 0 || need > kScratchBytes)
         return MWU_ERR_WORKSPACE;            // tensor too large for the built-in scratch

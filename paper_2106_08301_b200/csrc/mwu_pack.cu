@@ -346,7 +346,9 @@ __global__ void __launch_bounds__(128) fill_kernel(Params p) {
 
 extern "C" size_t mwu_packed_bytes(const mwu_proj_desc *desc) {
     if (mwu::validate_desc(desc, true) != MWU_OK) return 0;
-    return mwu::packed_layout(desc).total;
+    // a 2-dim block shape is packed through per-row arrays, which mwu_pack builds behind the packed bytes
+    const size_t extra = mwu::shape_of(desc).shaped ? mwu::shapes::lowering_bytes(desc) : 0;
+    return mwu::packed_layout(desc).total + extra;
 }
 
 extern "C" int mwu_pack(const mwu_proj_desc *desc, const float *W, const float *U_dual, const float *u,
@@ -364,10 +366,17 @@ extern "C" int mwu_pack(const mwu_proj_desc *desc, const float *W, const float *
         return MWU_ERR_ALIGNMENT;
     pack::Params p;
     p.L = packed_layout(desc);
-    if (packed_bytes < p.L.total) return MWU_ERR_WORKSPACE;
+    if (packed_bytes < mwu_packed_bytes(desc)) return MWU_ERR_WORKSPACE;
     if (p.L.n_tiles * p.L.n_stages >= (int64_t(1) << 31)) return MWU_ERR_SHAPE;
-    rc = check_device(nullptr);
+    int sm_count = 0;
+    rc = check_device(&sm_count);
     if (rc != MWU_OK) return rc;
+    if (shape_of(desc).shaped) {
+        // every run of `block` entries of a row becomes a 1-dim block with its block's class and magnitude
+        rc = shapes::lower(desc, u, pruned_bitmap, unified_bitmap, (char *)packed + p.L.total, &u, &pruned_bitmap,
+                           &unified_bitmap, sm_count, (cudaStream_t)cuda_stream);
+        if (rc != MWU_OK) return rc;
+    }
     p.W = W; p.U = U_dual; p.u = u;
     p.pruned_bitmap = pruned_bitmap; p.unified_bitmap = unified_bitmap; p.sign_bits = sign_bits;
     p.packed = (unsigned char *)packed;

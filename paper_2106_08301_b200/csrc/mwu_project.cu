@@ -1372,7 +1372,10 @@ __device__ __forceinline__ void one_pass_fail(const Params &p) { atomicExch(&p.w
 
 // pass_kernel: keys, provisional classes and every output in one sweep over W (+U).
 // A block is a candidate when its final class is still open: its prune key lies inside the prune
-// window, or it certainly survives pruning and its L_u lies inside the unify window.
+// window, or it certainly survives pruning and its L_u lies inside the unify window.  Candidates
+// are staged per warp with their two keys; when 32 have gathered, the whole warp turns them into
+// bin codes, window-histogram counts and list entries (every lane busy), so the sweep itself only
+// compares keys with the window edges.
 // ADMM: also the dual update V - Q and ||V - Q||_F^2 (mwu_admm_step); a separate instantiation so
 // that the plain projection keeps its register count.
 template <int B, bool ADMM>
@@ -1389,10 +1392,13 @@ __global__ void __launch_bounds__(256) pass_kernel(Params p, float *Q, double *l
     const unsigned nb = (unsigned)p.nb, top = nb - 1u;
     unsigned *hist_p = p.fhist, *hist_u = p.fhist + p.nb;
     __shared__ float4 s_q[8][128];                       // one warp step of Q per warp
-    __shared__ uint2 s_cand[8][STAGE_ENTRIES];           // list entries waiting for a full 32-entry flush
+    // candidates waiting for a full 32-entry flush: block index and both keys
+    __shared__ unsigned s_cidx[8][STAGE_ENTRIES];
+    __shared__ u64 s_ckp[8][STAGE_ENTRIES], s_cku[8][STAGE_ENTRIES];
     const int lane = threadIdx.x & 31;
     float4 *wq = s_q[threadIdx.x >> 5];
-    uint2 *wc = s_cand[threadIdx.x >> 5];
+    unsigned *cidx = s_cidx[threadIdx.x >> 5];
+    u64 *ckp = s_ckp[threadIdx.x >> 5], *cku = s_cku[threadIdx.x >> 5];
     const unsigned lt_mask = (1u << lane) - 1u;
     unsigned fill = 0;                                   // warp-uniform
     unsigned under_p = 0, over_p = 0, under_u = 0, over_u = 0, nonfinite = 0;
@@ -1404,6 +1410,25 @@ __global__ void __launch_bounds__(256) pass_kernel(Params p, float *Q, double *l
     const unsigned n_blocks = (unsigned)p.n_blocks;
     const unsigned n_bm_words = (n_blocks + 31u) / 32u;
     const unsigned ustride = gridDim.x * blockDim.x;
+
+    // staged candidates [from, from + cnt) -> bin codes, window histograms, list entries (whole warp)
+    auto flush = [&](unsigned from, unsigned cnt) {
+        unsigned base = 0;
+        if (lane == 0) base = atomicAdd(&p.work->list_count, cnt);
+        base = __shfl_sync(0xffffffffu, base, 0);
+        if (base + cnt > p.list_cap) {
+            if (lane == 0) one_pass_fail(p);
+            return;
+        }
+        if ((unsigned)lane < cnt) {
+            const u64 kp = ckp[from + lane], ku = cku[from + lane];
+            const unsigned bp = bin_of(kp, plo, phi, psh, nb), bu = bin_of(ku, ulo, uhi, ush, nb);
+            if (mode_p == 0u && bp != 0u && bp != top) atomicAdd(&hist_p[bp], 1u);       // open because of the prune window
+            else if (mode_u == 0u && bu != 0u && bu != top) atomicAdd(&hist_u[bu], 1u);  // a survivor inside the unify window
+            p.list[base + lane] = make_uint2(cidx[from + lane], bp | (bu << 16));
+        }
+    };
+
     unsigned unit = blockIdx.x * blockDim.x + threadIdx.x;
     float nxt[16];
 #pragma unroll
@@ -1421,20 +1446,31 @@ __global__ void __launch_bounds__(256) pass_kernel(Params p, float *Q, double *l
         }
         const bool live = unit < n_units;
         const bool warp_full = (long long)(unit - lane + 32u) * 16 <= n;      // all 512 floats of this warp step exist
-        unsigned sb = 0;
+        const unsigned j0 = unit * NBT;
+        // Sign plane: bit l = (v[l] < 0).  Without a zero among the warp's values that is the IEEE sign
+        // bit, gathered with one funnel shift per value; a zero (it may be -0.0) takes the compare.
+        float vmin = fabsf(v[0]);
 #pragma unroll
-        for (int l = 0; l < 16; ++l) sb |= (v[l] < 0.f ? 1u : 0u) << l;
+        for (int l = 1; l < 16; ++l) vmin = fminf(vmin, fabsf(v[l]));
+        const bool has_zero = __any_sync(0xffffffffu, vmin == 0.f);
+        unsigned sb = 0;
+        if (!has_zero) {
+#pragma unroll
+            for (int l = 15; l >= 0; --l) sb = __funnelshift_l(__float_as_uint(v[l]), sb, 1);
+        } else {
+#pragma unroll
+            for (int l = 0; l < 16; ++l) sb |= (v[l] < 0.f ? 1u : 0u) << l;
+        }
         if (live) {
             unsigned short *halves = reinterpret_cast<unsigned short *>(sign_bits);
             halves[unit] = (unsigned short)sb;
             if (unit == n_units - 1 && (n_units & 1)) halves[unit + 1] = 0;
         }
-        unsigned cls_p = 0, cls_u = 0, cand = 0;             // bit e: block e of this thread
-        unsigned code[NBT];
-        float uo[NBT];
-        const unsigned j0 = unit * NBT;
         // grouped pruning: a unit's 16 values lie in one group (groups are at least 16 columns wide)
         const bool grp = mode_p == 3u && j0 < n_blocks && group_pruned(p, j0);
+        unsigned cls_p = 0, cls_u = 0, cand = 0;             // bit e: block e of this thread
+        u64 kpb[NBT], kub[NBT];
+        float uo[NBT];
 #pragma unroll
         for (int e = 0; e < NBT; ++e) {
             double S, Lu, Kp;
@@ -1442,10 +1478,8 @@ __global__ void __launch_bounds__(256) pass_kernel(Params p, float *Q, double *l
             const float qf = __double2float_rn(__dmul_rn(S, 1.0 / (double)B));
             // S = sum |v| is Inf or NaN exactly when some value of the block is
             nonfinite |= ((unsigned)__double2hiint(S) >= 0x7ff00000u) ? 1u : 0u;
-            const u64 kpb = key_bits(Kp), kub = key_bits(Lu);
-            const unsigned bp = bin_of(kpb, plo, phi, psh, nb);
-            const unsigned bu = bin_of(kub, ulo, uhi, ush, nb);
-            code[e] = bp | (bu << 16);
+            kpb[e] = key_bits(Kp);
+            kub[e] = key_bits(Lu);
             uo[e] = 0.f;
             const unsigned j = j0 + e;
             if (j < n_blocks) {
@@ -1453,11 +1487,12 @@ __global__ void __launch_bounds__(256) pass_kernel(Params p, float *Q, double *l
                 if (loss_p) loss_p[j] = Kp;
                 bool pr, survives, open = false;
                 if (mode_p == 0u) {
-                    pr = kpb <= Tp;
-                    survives = bp == top;
-                    if (bp == 0u) ++under_p;
-                    else if (bp == top) ++over_p;
-                    else { atomicAdd(&hist_p[bp], 1u); open = true; }
+                    const bool below = kpb[e] < plo, above = kpb[e] >= phi;
+                    pr = kpb[e] <= Tp;
+                    survives = above;
+                    under_p += below ? 1u : 0u;
+                    over_p += above ? 1u : 0u;
+                    open = !(below || above);
                 } else if (mode_p == 3u) {
                     pr = grp;                              // grouped pruning: the class is the group's bit
                     survives = !grp;
@@ -1465,11 +1500,12 @@ __global__ void __launch_bounds__(256) pass_kernel(Params p, float *Q, double *l
                     pr = mode_p == 2u;
                     survives = mode_p == 1u;
                 }
-                const bool un = !pr && (mode_u == 2u || (mode_u == 0u && kub <= Tu));
+                const bool un = !pr && (mode_u == 2u || (mode_u == 0u && kub[e] <= Tu));
                 if (survives && mode_u == 0u) {
-                    if (bu == 0u) ++under_u;
-                    else if (bu == top) ++over_u;
-                    else { atomicAdd(&hist_u[bu], 1u); open = true; }
+                    const bool below = kub[e] < ulo, above = kub[e] >= uhi;
+                    under_u += below ? 1u : 0u;
+                    over_u += above ? 1u : 0u;
+                    open = open || !(below || above);
                 }
                 cls_p |= (pr ? 1u : 0u) << e;
                 cls_u |= (un ? 1u : 0u) << e;
@@ -1498,18 +1534,25 @@ __global__ void __launch_bounds__(256) pass_kernel(Params p, float *Q, double *l
                     if (j0 + e < n_blocks) u_out[j0 + e] = uo[e];
             }
             if (Q || (ADMM && p.U_next)) {
-                // q = v (kept), +-u (unified: magnitude u, sign from the sign plane bits), or +0
+                // q = v (kept), +-u (unified: magnitude u, sign of v), or +0
                 float q[16];
 #pragma unroll
                 for (int e = 0; e < NBT; ++e) {
                     const bool pr = (cls_p >> e) & 1u, un = (cls_u >> e) & 1u;
-                    const unsigned keep = (pr || un) ? 0u : 0xffffffffu;
                     const unsigned mag = un ? __float_as_uint(uo[e]) : 0u;
-                    const unsigned sgn = un ? 0x80000000u : 0u;
+                    if (!has_zero) {
+                        // no zero in the warp: the sign of v is its IEEE sign bit
+                        const unsigned m1 = pr ? 0u : (un ? 0x80000000u : 0xffffffffu);
 #pragma unroll
-                    for (int l = 0; l < B; ++l) {
-                        const int k = e * B + l;
-                        q[k] = __uint_as_float((__float_as_uint(v[k]) & keep) | mag | ((sb << (31 - k)) & sgn));
+                        for (int l = 0; l < B; ++l) q[e * B + l] = __uint_as_float((__float_as_uint(v[e * B + l]) & m1) | mag);
+                    } else {
+                        const unsigned keep = (pr || un) ? 0u : 0xffffffffu;
+                        const unsigned sgn = un ? 0x80000000u : 0u;
+#pragma unroll
+                        for (int l = 0; l < B; ++l) {
+                            const int k = e * B + l;
+                            q[k] = __uint_as_float((__float_as_uint(v[k]) & keep) | mag | ((sb << (31 - k)) & sgn));
+                        }
                     }
                 }
                 const long long f = (long long)unit * 16;
@@ -1576,34 +1619,30 @@ __global__ void __launch_bounds__(256) pass_kernel(Params p, float *Q, double *l
                 }
             }
         }
-        // candidate list: entries gather in the warp's staging buffer and leave 32 at a time
+        // candidates gather in the warp's staging buffer and leave 32 at a time
+        if (__any_sync(0xffffffffu, cand != 0u)) {
 #pragma unroll
-        for (int e = 0; e < NBT; ++e) {
-            const bool c = (cand >> e) & 1u;
-            const unsigned bal = __ballot_sync(0xffffffffu, c);
-            if (bal == 0u) continue;
-            if (c) wc[fill + __popc(bal & lt_mask)] = make_uint2(j0 + e, code[e]);
-            fill += __popc(bal);
-            __syncwarp();
-            if (fill >= 32u) {
-                unsigned base = 0;
-                if (lane == 0) base = atomicAdd(&p.work->list_count, 32u);
-                base = __shfl_sync(0xffffffffu, base, 0);
-                fill -= 32u;
-                if (base + 32u <= p.list_cap) p.list[base + lane] = wc[fill + lane];
-                else if (lane == 0) one_pass_fail(p);
+            for (int e = 0; e < NBT; ++e) {
+                const bool c = (cand >> e) & 1u;
+                const unsigned bal = __ballot_sync(0xffffffffu, c);
+                if (bal == 0u) continue;
+                if (c) {
+                    const unsigned pos = fill + __popc(bal & lt_mask);
+                    cidx[pos] = j0 + e;
+                    ckp[pos] = kpb[e];
+                    cku[pos] = kub[e];
+                }
+                fill += __popc(bal);
                 __syncwarp();
+                if (fill >= 32u) {
+                    fill -= 32u;
+                    flush(fill, 32u);
+                    __syncwarp();
+                }
             }
         }
     }
-    if (fill > 0u) {
-        unsigned base = 0;
-        if (lane == 0) base = atomicAdd(&p.work->list_count, fill);
-        base = __shfl_sync(0xffffffffu, base, 0);
-        if (base + fill <= p.list_cap) {
-            if ((unsigned)lane < fill) p.list[base + lane] = wc[lane];
-        } else if (lane == 0) one_pass_fail(p);
-    }
+    if (fill > 0u) flush(0u, fill);
     // block-level totals of the catch-all bins
     __shared__ unsigned s_tot[4];
     if (threadIdx.x < 4) s_tot[threadIdx.x] = 0;
@@ -2072,6 +2111,7 @@ static bool use_one_pass(const mwu_proj_desc *desc) {
 
 extern "C" size_t mwu_project_workspace_bytes(const mwu_proj_desc *desc) {
     if (mwu::validate_desc(desc, false) != MWU_OK) return 0;
+    if (mwu::shape_of(desc).shaped) return mwu::shapes::workspace_bytes(desc);
     const size_t mb = (size_t)(desc->rows * desc->cols / desc->block);
     return mwu::align_up(mwu::ws_off_gprune(desc, mb) + (mwu::n_groups_of(desc) + 31) / 32 * 4 + 16);
 }
@@ -2171,6 +2211,9 @@ static int project_impl(const mwu_proj_desc *desc, const float *W, const float *
 
     cudaStream_t st = (cudaStream_t)cuda_stream;
     char *ws = (char *)workspace;
+    if (shape_of(desc).shaped)                          // 2- and 3-dim blocks: the block-by-block path
+        return shapes::project(desc, W, U_dual, Q, U_next, residual_sq, u, pruned_bitmap, unified_bitmap, sign_bits,
+                               loss_u, loss_p, dev_status, workspace, sm_count, st);
     const bool one_pass = use_one_pass(desc);
     proj::Params p;
     p.W = W;
