@@ -116,7 +116,9 @@ struct Params {
     float *U_next;              // dual update V - Q (mwu_admm_step), else null
     double *resid;              // ||V - Q||_F^2 accumulator (mwu_admm_step), else null
     u64 *cand_key;              // [CAP]
-    unsigned *cand_idx;         // [CAP]
+    unsigned *cand_idx;         // [2 * CAP]
+    unsigned *cand_aux;         // [2 * CAP] what resolve_kernel wants to know about a candidate besides its key
+    u64 *samp_kp, *samp_ku;     // [NSAMP] each: keys of the sample blocks (one-pass pipeline)
     unsigned *bins;             // [n_blocks]
     unsigned *dev_status;
 };
@@ -277,7 +279,26 @@ __device__ __forceinline__ void load_block(const float *W, const float *U, long 
     }
 }
 
-// exact keys of block j, read from global memory (sampling and threshold-bin blocks)
+// Approximate keys of block j in fp32, for the sample only: the sample steers the windows (any
+// window gives the same result), so its keys need no more than a few good digits, and sample_kernel,
+// a single CTA, has one SM's fp64 units.
+template <int B>
+__device__ __forceinline__ void block_keys_sample(const float *W, const float *U, long long j, int use_l1, u64 *kp,
+                                                  u64 *ku) {
+    float v[B];
+    load_block<B>(W, U, j, v);
+    float S = 0.f, sq = 0.f;
+#pragma unroll
+    for (int l = 0; l < B; ++l) { S += fabsf(v[l]); sq = fmaf(v[l], v[l], sq); }
+    const float q = S * (1.f / (float)B);
+    float lu = 0.f;
+#pragma unroll
+    for (int l = 0; l < B; ++l) { const float d = fabsf(v[l]) - q; lu = fmaf(d, d, lu); }
+    *kp = key_bits((double)(use_l1 ? S : sq));
+    *ku = key_bits((double)lu);
+}
+
+// exact keys of block j, read from global memory (threshold-bin blocks)
 template <int B>
 __device__ __forceinline__ void block_keys_at(const float *W, const float *U, long long j, int use_l1,
                                               double *S, double *Lu, double *Kp) {
@@ -483,10 +504,35 @@ __device__ __forceinline__ long long sample_block(int i, long long mb, int ns) {
     return ns == NSAMP ? (long long)(((u64)i * (u64)mb) / (u64)NSAMP) : (long long)i;
 }
 
-// Run by one whole CTA of SAMP_THREADS threads: windows and provisional thresholds of the two
-// selections, written into p.work.
+// sample_keys_kernel: approximate keys of the NSAMP evenly spaced sample blocks, one block per
+// thread, spread over many SMs (4096 scattered 64-byte reads issued by a single SM take about
+// 9 us; over 32 SMs they take one memory round trip).  The same launch clears the histograms.
 template <int B>
-__device__ void sample_body(const Params &p) {
+__global__ void __launch_bounds__(128) sample_keys_kernel(Params p, unsigned *zero_base, unsigned n_zero) {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    const long long mb = p.n_blocks;
+    const int ns = (int)(mb < (long long)NSAMP ? mb : (long long)NSAMP);
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < NSAMP) {
+        u64 kp = ~0ull, ku = ~0ull;
+        unsigned in_group = 0;
+        if (i < ns) {
+            const long long j = sample_block(i, mb, ns);
+            block_keys_sample<B>(p.W, p.U, j, p.use_l1, &kp, &ku);
+            if (p.gprune) in_group = group_pruned(p, (unsigned)j) ? 1u : 0u;
+        }
+        p.samp_kp[i] = kp;
+        p.samp_ku[i] = ku | ((u64)in_group << 63);       // keys are non-negative doubles: bit 63 is free
+    }
+    uint4 *z = reinterpret_cast<uint4 *>(zero_base);
+    for (unsigned q = blockIdx.x * blockDim.x + threadIdx.x; q < n_zero / 4; q += gridDim.x * blockDim.x)
+        z[q] = make_uint4(0, 0, 0, 0);
+}
+
+// Run by one whole CTA of SAMP_THREADS threads: windows and provisional thresholds of the two
+// selections, written into p.work.  from_keys: the sample keys were computed by sample_keys_kernel.
+template <int B>
+__device__ void sample_body(const Params &p, bool from_keys = false) {
     const long long k_unify = p.k_unify, k_prune = p.k_prune;
     const long long mb = p.n_blocks;
     const bool by_group = p.gprune != nullptr;
@@ -500,12 +546,14 @@ __device__ void sample_body(const Params &p) {
         ku[t] = ~0ull;
         valid[t] = i < ns;
         in_group[t] = false;
-        if (i < ns) {
+        if (i < ns && from_keys) {
+            kp[t] = p.samp_kp[i];
+            const u64 x = p.samp_ku[i];
+            ku[t] = x & (~0ull >> 1);
+            in_group[t] = (x >> 63) != 0ull;
+        } else if (i < ns) {
             const long long j = sample_block(i, mb, ns);
-            double S, Lu, Kp;
-            block_keys_at<B>(p.W, p.U, j, p.use_l1, &S, &Lu, &Kp);
-            kp[t] = key_bits(Kp);
-            ku[t] = key_bits(Lu);
+            block_keys_sample<B>(p.W, p.U, j, p.use_l1, &kp[t], &ku[t]);
             if (by_group) in_group[t] = group_pruned(p, (unsigned)j);
         }
     }
@@ -546,21 +594,17 @@ __device__ void sample_body(const Params &p) {
     }
 }
 
-// First kernel of the one-pass pipeline.  CTA 0 clears the selection state and chooses the windows;
-// the other CTAs clear the histograms (n_zero 32-bit words starting at zero_base).
+// Second kernel of the one-pass pipeline (one CTA): clears the selection state and chooses the
+// windows from the sample keys.  Launched with programmatic stream serialization behind
+// sample_keys_kernel, and itself lets pass_kernel's CTAs start early.
 template <int B>
-__global__ void __launch_bounds__(SAMP_THREADS) sample_kernel(Params p, unsigned *zero_base, unsigned n_zero) {
-    if (blockIdx.x > 0) {
-        const unsigned per = (n_zero / 4 + gridDim.x - 2) / (gridDim.x - 1);          // uint4 pieces per CTA
-        uint4 *z = reinterpret_cast<uint4 *>(zero_base);
-        const unsigned lo = (blockIdx.x - 1) * per, hi = min(lo + per, n_zero / 4);
-        for (unsigned i = lo + threadIdx.x; i < hi; i += blockDim.x) z[i] = make_uint4(0, 0, 0, 0);
-        return;
-    }
+__global__ void __launch_bounds__(SAMP_THREADS) sample_kernel(Params p) {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     unsigned *w = reinterpret_cast<unsigned *>(p.work);
     for (unsigned i = threadIdx.x; i < sizeof(Work) / 4; i += blockDim.x) w[i] = 0u;
+    asm volatile("griddepcontrol.wait;" ::: "memory");     // the sample keys are complete and visible
     __syncthreads();
-    sample_body<B>(p);
+    sample_body<B>(p, true);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -582,15 +626,27 @@ __device__ __forceinline__ bool last_block_done(unsigned *ticket) {
 }
 
 // find the bin holding the r-th element; hist has nb entries
+// `extra` (shared memory, n_extra bin numbers, may be null): one more element in each of these bins,
+// counted on top of what the histogram holds (the CTA's own corrections, not yet in global memory).
 __device__ void scan_hist(const unsigned *hist, int nb, u64 r, unsigned *bin_out, u64 *r_in_bin, u64 *cnt_out,
-                          unsigned *err) {
+                          unsigned *err, const unsigned *extra = nullptr, unsigned n_extra = 0) {
     __shared__ u64 s_part[32];
     const int PER = nb / FIN_THREADS;
     u64 sum = 0;
     unsigned mine8[8];                                       // this thread's bins when there are eight of them
     if (PER == 8) {
+        // two 16-byte loads that bypass L1 (the histogram may have been updated by other CTAs of this kernel)
+        const uint4 h0 = __ldcg(reinterpret_cast<const uint4 *>(hist) + threadIdx.x * 2);
+        const uint4 h1 = __ldcg(reinterpret_cast<const uint4 *>(hist) + threadIdx.x * 2 + 1);
+        mine8[0] = h0.x; mine8[1] = h0.y; mine8[2] = h0.z; mine8[3] = h0.w;
+        mine8[4] = h1.x; mine8[5] = h1.y; mine8[6] = h1.z; mine8[7] = h1.w;
+        for (unsigned x = 0; x < n_extra; ++x) {
+            const unsigned bx = extra[x];
+            if ((bx >> 3) == threadIdx.x) {
 #pragma unroll
-        for (int i = 0; i < 8; ++i) mine8[i] = ld_vol(&hist[threadIdx.x * 8 + i]);
+                for (int i = 0; i < 8; ++i) mine8[i] += ((bx & 7u) == (unsigned)i) ? 1u : 0u;
+            }
+        }
 #pragma unroll
         for (int i = 0; i < 8; ++i) sum += mine8[i];
     } else if (PER == 64) {
@@ -605,9 +661,11 @@ __device__ void scan_hist(const unsigned *hist, int nb, u64 r, unsigned *bin_out
             for (int m = 16; m > 0; m >>= 1) a += __shfl_xor_sync(0xffffffffu, a, m);
             if (l == e) sum = a;
         }
+        for (unsigned x = 0; x < n_extra; ++x) sum += ((extra[x] >> 6) == threadIdx.x) ? 1u : 0u;
     } else {
 #pragma unroll 8
         for (int i = 0; i < PER; ++i) sum += ld_vol(&hist[threadIdx.x * PER + i]);
+        for (unsigned x = 0; x < n_extra; ++x) sum += (extra[x] / (unsigned)PER == threadIdx.x) ? 1u : 0u;
     }
     // inclusive scan of the per-thread sums: shuffles inside a warp, then over the 32 warp totals
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
@@ -654,8 +712,12 @@ __device__ void scan_hist(const unsigned *hist, int nb, u64 r, unsigned *bin_out
     // warp 0 scans the owner's PER (<= 64) bins together
     if (wid == 0 && s_owner >= 0) {
         const int base = s_owner * PER;
-        const u64 c0 = lane < PER ? (u64)ld_vol(&hist[base + lane]) : 0ull;
-        const u64 c1 = lane + 32 < PER ? (u64)ld_vol(&hist[base + lane + 32]) : 0ull;
+        u64 c0 = lane < PER ? (u64)ld_vol(&hist[base + lane]) : 0ull;
+        u64 c1 = lane + 32 < PER ? (u64)ld_vol(&hist[base + lane + 32]) : 0ull;
+        for (unsigned x = 0; x < n_extra; ++x) {
+            c0 += (extra[x] == (unsigned)(base + lane)) ? 1u : 0u;
+            c1 += (extra[x] == (unsigned)(base + lane + 32)) ? 1u : 0u;
+        }
         u64 i0 = c0;                                   // inclusive scan over bins 0..31, then 32..63
         for (int m = 1; m < 32; m <<= 1) {
             const u64 y = __shfl_up_sync(0xffffffffu, i0, m);
@@ -684,12 +746,13 @@ struct BinSel {
 
 // level 0: which bin holds the k-th element; writes the bin and its composite range
 // sr: the CTA's copy of the selection (count and window); s: the global one, written when `publish`
-__device__ void select_bin(const Params &p, const Sel *sr, Sel *s, const unsigned *hist, BinSel *out, bool publish) {
+__device__ void select_bin(const Params &p, const Sel *sr, Sel *s, const unsigned *hist, BinSel *out, bool publish,
+                           const unsigned *extra = nullptr, unsigned n_extra = 0) {
     __shared__ unsigned s_bin, s_err;
     __shared__ u64 s_r, s_cnt;
     if (threadIdx.x == 0) { s_err = 0; s_bin = 0; s_r = 0; s_cnt = 0; }
     __syncthreads();
-    scan_hist(hist, p.nb, sr->k, &s_bin, &s_r, &s_cnt, &s_err);
+    scan_hist(hist, p.nb, sr->k, &s_bin, &s_r, &s_cnt, &s_err, extra, n_extra);
     if (threadIdx.x == 0) {
         if (s_err) atomicOr(p.dev_status, (unsigned)MWU_DEV_SELECT);
         const unsigned B = s_bin;
@@ -1383,6 +1446,17 @@ __global__ void __launch_bounds__(256) pass_kernel(Params p, float *Q, double *l
                                                    float *u_out, unsigned *pruned_bitmap,
                                                    unsigned *unified_bitmap, unsigned *sign_bits) {
     constexpr int NBT = 16 / B;
+    // Launched with programmatic stream serialization: the CTAs may start while sample_kernel still
+    // runs.  The first 64 bytes of W do not depend on it and are requested at once; everything
+    // sample_kernel writes (windows, cleared histograms) is read only behind the wait.
+    const long long n = p.n_floats;
+    const unsigned n_units = (unsigned)((n + 15) / 16);
+    unsigned unit = blockIdx.x * blockDim.x + threadIdx.x;
+    float nxt[16];
+#pragma unroll
+    for (int l = 0; l < 16; ++l) nxt[l] = 0.f;
+    if (unit < n_units) load16(p.W, p.U, (long long)unit * 16, n, nxt);
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const Sel *sp = &p.work->sel[0];
     const Sel *su = &p.work->sel[1];
     const u64 plo = sp->lo0, phi = sp->hi0, ulo = su->lo0, uhi = su->hi0;
@@ -1404,8 +1478,6 @@ __global__ void __launch_bounds__(256) pass_kernel(Params p, float *Q, double *l
     unsigned under_p = 0, over_p = 0, under_u = 0, over_u = 0, nonfinite = 0;
     double resid_acc = 0.0;
     // fewer than 2^31 blocks of at least two values: units (16 values) and blocks count in 32 bits
-    const long long n = p.n_floats;
-    const unsigned n_units = (unsigned)((n + 15) / 16);
     const unsigned n_iter = (n_units + 31u) / 32u * 32u;  // whole warps take part in every step
     const unsigned n_blocks = (unsigned)p.n_blocks;
     const unsigned n_bm_words = (n_blocks + 31u) / 32u;
@@ -1429,11 +1501,6 @@ __global__ void __launch_bounds__(256) pass_kernel(Params p, float *Q, double *l
         }
     };
 
-    unsigned unit = blockIdx.x * blockDim.x + threadIdx.x;
-    float nxt[16];
-#pragma unroll
-    for (int l = 0; l < 16; ++l) nxt[l] = 0.f;
-    if (unit < n_units) load16(p.W, p.U, (long long)unit * 16, n, nxt);
     for (; unit < n_iter; unit += ustride) {
         float v[16];
 #pragma unroll
@@ -1628,7 +1695,8 @@ __global__ void __launch_bounds__(256) pass_kernel(Params p, float *Q, double *l
                 if (bal == 0u) continue;
                 if (c) {
                     const unsigned pos = fill + __popc(bal & lt_mask);
-                    cidx[pos] = j0 + e;
+                    // block index with the provisional class in its top bits (fewer than 2^30 blocks)
+                    cidx[pos] = (j0 + e) | (((cls_p >> e) & 1u) << 31) | (((cls_u >> e) & 1u) << 30);
                     ckp[pos] = kpb[e];
                     cku[pos] = kub[e];
                 }
@@ -1670,60 +1738,16 @@ __global__ void __launch_bounds__(256) pass_kernel(Params p, float *Q, double *l
     if (ADMM && p.resid) block_add_double(resid_acc, p.resid);
 }
 
-// Sort the n candidates (global cand_key / cand_idx) and write the threshold element, the r-th
-// smallest (key, index), into the selection.  Run by one whole CTA; false when the counts do
-// not fit (the caller then gives the one-pass result up).
-__device__ bool pick_threshold(const Params &p, Sel *s, u64 r, unsigned n, u64 *c_key, unsigned *c_idx) {
-    const unsigned m = n < (unsigned)CAP ? n : (unsigned)CAP;
-    if (m <= blockDim.x) {
-        // the usual case, a few dozen candidates: every thread ranks its own by counting
-        u64 k = ~0ull;
-        unsigned ix = ~0u;
-        if (threadIdx.x < m) {
-            k = ld_vol(&p.cand_key[threadIdx.x]);
-            ix = ld_vol(&p.cand_idx[threadIdx.x]);
-            c_key[threadIdx.x] = k;
-            c_idx[threadIdx.x] = ix;
-        }
-        __syncthreads();
-        unsigned rank = 0;
-        if (threadIdx.x < m) {
-            for (unsigned t = 0; t < m; ++t) {
-                const u64 x = c_key[t];
-                const unsigned y = c_idx[t];
-                rank += (x < k || (x == k && y < ix)) ? 1u : 0u;
-            }
-        }
-        __syncthreads();
-        if (threadIdx.x < m) { c_key[rank] = k; c_idx[rank] = ix; }
-        __syncthreads();
-    } else {
-        for (int i = threadIdx.x; i < CAP; i += blockDim.x) {
-            c_key[i] = (i < (int)m) ? ld_vol(&p.cand_key[i]) : ~0ull;
-            c_idx[i] = (i < (int)m) ? ld_vol(&p.cand_idx[i]) : ~0u;
-        }
-        __syncthreads();
-        int np2 = 2;
-        while (np2 < (int)m) np2 <<= 1;
-        sort_candidates(c_key, c_idx, np2);
-    }
-    const bool ok = n <= (unsigned)CAP && r >= 1 && r <= (u64)m;
-    if (threadIdx.x == 0 && ok) {
-        s->T_key = c_key[r - 1];
-        s->T_idx = (u64)c_idx[r - 1];
-    }
-    return ok;
-}
+constexpr unsigned IDX_MASK = 0x3fffffffu;           // list entry: block index; bit 31 / 30: provisional pruned / unified
 
-// Final class of block j against what pass_kernel wrote (read back from the bitmaps); the
-// block's outputs are rewritten where they differ.
+// Block idx gets final class (pr, un) where pass_kernel had written (pr0, un0): bitmaps, u, Q (and
+// the dual update) are rewritten.  Returns the change of ||V - Q||^2.
 template <int B>
 __device__ __forceinline__ double apply_class(const Params &p, float *Q, float *u_out, unsigned *pruned_bitmap,
-                                              unsigned *unified_bitmap, unsigned idx, bool pr, bool un) {
+                                              unsigned *unified_bitmap, unsigned idx, bool pr, bool un, bool pr0,
+                                              bool un0) {
     const unsigned bit = 1u << (idx & 31u);
     unsigned *wp = pruned_bitmap + (idx >> 5), *wu = unified_bitmap + (idx >> 5);
-    const bool pr0 = (ld_vol(wp) & bit) != 0u, un0 = (ld_vol(wu) & bit) != 0u;
-    if (pr == pr0 && un == un0) return 0.0;
     if (pr != pr0) { if (pr) atomicOr(wp, bit); else atomicAnd(wp, ~bit); }
     if (un != un0) { if (un) atomicOr(wu, bit); else atomicAnd(wu, ~bit); }
     const long long j = (long long)idx;
@@ -1745,174 +1769,341 @@ __device__ __forceinline__ double apply_class(const Params &p, float *Q, float *
     return (pr ? sq : (un ? Lu : 0.0)) - (pr0 ? sq : (un0 ? Lu : 0.0));
 }
 
+constexpr int MP_SMEM_BYTES = (FIN_THREADS / 32) * 128 * 16;     // emit staging: 2 KB per warp
+constexpr int CHG_PER_THREAD = 3;                    // list entries a thread classifies before the changed ones are applied
+static_assert(MP_SMEM_BYTES >= CAP * 20 + CHG_PER_THREAD * FIN_THREADS * 8,
+              "candidate buffers, corrections and the compaction buffer share the staging memory");
+
+// The multi-pass projection as a sequence of phases separated by grid barriers (cooperative launch):
+// [windows from a sample] -> statistics -> prune threshold -> unify threshold -> emit.  k counts the
+// barriers of the running kernel that have been passed.
+template <int B>
+__device__ void multipass_phases(const Params &p, Work &w, unsigned &k, bool run_sample, unsigned char *smem, float *Q,
+                                 double *loss_u, double *loss_p, float *u_out, unsigned *pruned_bitmap,
+                                 unsigned *unified_bitmap, unsigned *sign_bits) {
+    u64 *c_key = reinterpret_cast<u64 *>(smem);
+    unsigned *c_idx = reinterpret_cast<unsigned *>(smem + CAP * sizeof(u64));
+    bool ok = true;
+    if (run_sample) {
+        if (blockIdx.x == 0) sample_body<B>(p);
+        ok = grid_sync(&p.work->bar, ++k);
+    }
+    if (ok) {
+        load_work(p.work, &w);
+        stats_body<B>(p, w, loss_u, loss_p, u_out, sign_bits);
+        ok = grid_sync(&p.work->bar, ++k);
+    }
+    if (ok) {
+        prune_select_body<B>(p, w, c_key, c_idx);
+        ok = grid_sync(&p.work->bar, ++k);
+    }
+    if (ok) {
+        load_work(p.work, &w);
+        collect_body<1, B>(p, w, c_key, c_idx);
+        ok = grid_sync(&p.work->bar, ++k);
+    }
+    if (ok) {
+        load_work(p.work, &w);
+        emit_body<B>(p, w, Q, u_out, pruned_bitmap, unified_bitmap, sign_bits, reinterpret_cast<float4 *>(smem));
+    }
+    if (!ok && threadIdx.x == 0) atomicOr(p.dev_status, (unsigned)MWU_DEV_TIMEOUT);
+}
+
+// rank the m candidates in shared memory (c_key, c_idx) by (key, index); m <= CAP
+// c_aux (when the candidates fit one per thread: the return value) receives g_aux in the same order
+__device__ bool rank_candidates(const Params &p, const u64 *g_key, const unsigned *g_idx, const unsigned *g_aux,
+                                unsigned m, u64 *c_key, unsigned *c_idx, unsigned *c_aux) {
+    if (m <= blockDim.x) {
+        // the usual case, a few dozen candidates: every thread ranks its own by counting
+        u64 k = ~0ull;
+        unsigned ix = ~0u, ax = 0u;
+        if (threadIdx.x < m) {
+            k = ld_vol(&g_key[threadIdx.x]);
+            ix = ld_vol(&g_idx[threadIdx.x]);
+            ax = ld_vol(&g_aux[threadIdx.x]);
+            c_key[threadIdx.x] = k;
+            c_idx[threadIdx.x] = ix;
+        }
+        __syncthreads();
+        unsigned rank = 0;
+        if (threadIdx.x < m) {
+            for (unsigned t = 0; t < m; ++t) {
+                const u64 x = c_key[t];
+                const unsigned y = c_idx[t];
+                rank += (x < k || (x == k && y < ix)) ? 1u : 0u;
+            }
+        }
+        __syncthreads();
+        if (threadIdx.x < m) { c_key[rank] = k; c_idx[rank] = ix; c_aux[rank] = ax; }
+        __syncthreads();
+        return true;
+    }
+    for (int i = threadIdx.x; i < CAP; i += blockDim.x) {
+        c_key[i] = (i < (int)m) ? ld_vol(&g_key[i]) : ~0ull;
+        c_idx[i] = (i < (int)m) ? ld_vol(&g_idx[i]) : ~0u;
+    }
+    __syncthreads();
+    int np2 = 2;
+    while (np2 < (int)m) np2 <<= 1;
+    sort_candidates(c_key, c_idx, np2);
+    return false;
+}
+
 // resolve_kernel (cooperative launch: all CTAs resident): the exact thresholds of the one-pass
 // pipeline and the final classes of the listed blocks, in one launch.
-//   first half   exact prune threshold bin from the window histogram; the listed blocks of that bin
-//                become candidates, the listed survivors complete the L_u histogram.  The CTA that
-//                finishes last ranks the candidates (exact threshold element), adds the surviving
-//                ones to the L_u histogram, locates the unify threshold bin and releases the others,
-//                which wait for it (bounded).
-//   second half  every listed block outside the unify threshold bin gets its final class at once
-//                (outputs rewritten where it differs from the provisional one); the blocks inside
-//                it are ranked by the CTA that finishes last, which fixes the threshold element and
-//                their classes.
-// A threshold outside its window, a threshold bin or tie group too large to rank, or a full list
-// gives the one-pass result up (work->failed): the multi-pass kernel behind redoes the projection.
+//   1  every CTA finds the prune threshold bin from the window histogram (the same values in
+//      all of them) and scans its slice of the list: blocks of that bin become candidates, listed
+//      survivors complete the L_u histogram.
+//      -- grid barrier --
+//   2  every CTA ranks the few dozen candidates itself (exact threshold element, no hand-over
+//      between CTAs), keeps the bins of the surviving candidates as corrections to the L_u
+//      histogram, and finds the unify threshold bin.
+//   3  every CTA gives the blocks of its list slice their final class: the class pass_kernel wrote
+//      travels in the entry, so nothing is read for the nine in ten whose class stands; the others
+//      are gathered 32 to a warp and rewritten.  Blocks of the unify threshold bin are ranked by
+//      the CTA that finishes last, which fixes the threshold element and their classes.
+//      -- grid barrier --
+//   4  if any step gave the one-pass result up (a threshold outside its window, a threshold bin or
+//      tie group too large to rank, a full list), the multi-pass phases redo the projection here.
 template <int B>
-__global__ void __launch_bounds__(FIN_THREADS) resolve_kernel(Params p, float *Q, float *u_out,
-                                                              unsigned *pruned_bitmap, unsigned *unified_bitmap) {
+__global__ void __launch_bounds__(FIN_THREADS) resolve_kernel(Params p, float *Q, double *loss_u, double *loss_p,
+                                                              float *u_out, unsigned *pruned_bitmap,
+                                                              unsigned *unified_bitmap, unsigned *sign_bits) {
+    extern __shared__ __align__(16) unsigned char mp_smem[];
     __shared__ Work w;                                 // selection state as the earlier kernels left it
-    __shared__ u64 c_key[CAP];
-    __shared__ unsigned c_idx[CAP];
     __shared__ BinSel s_sel;
-    __shared__ int s_go;
+    __shared__ unsigned s_n_extra, s_n_chg;
+    u64 *c_key = reinterpret_cast<u64 *>(mp_smem);
+    unsigned *c_idx = reinterpret_cast<unsigned *>(mp_smem + CAP * sizeof(u64));
+    unsigned *c_aux = reinterpret_cast<unsigned *>(mp_smem + CAP * 12);
+    unsigned *s_extra = reinterpret_cast<unsigned *>(mp_smem + CAP * 16);               // bins of surviving candidates
+    unsigned *s_chg = reinterpret_cast<unsigned *>(mp_smem + CAP * 20);                 // entries whose class changes
+    unsigned k = 0;                                    // grid barriers passed
     load_work(p.work, &w);
-    if (w.failed != 0u) return;                        // list overflow in pass_kernel: the same in every CTA
     Sel *sp = &p.work->sel[0];
     Sel *su = &p.work->sel[1];
     const unsigned mode_p = w.sel[0].mode, mode_u = w.sel[1].mode;
-    if (mode_p != 0u && mode_u != 0u) return;
     const unsigned nb = (unsigned)p.nb, top = nb - 1u;
     unsigned *hist_u = p.fhist + p.nb;
     const u64 ulo = w.sel[1].lo0, uhi = w.sel[1].hi0;
     const unsigned ush = w.sel[1].shift0;
     const unsigned n_list = min(w.list_count, p.list_cap);
-    if (threadIdx.x == 0) { s_sel.B = 0; s_sel.r = 0; s_sel.cnt = 0; s_sel.lo_hi = s_sel.lo_lo = s_sel.hi_hi = s_sel.hi_lo = 0; }
+    // every condition up to the second barrier is the same in all CTAs: they all take the same path
+    bool alive = w.failed == 0u && !(mode_p != 0u && mode_u != 0u);
+    if (threadIdx.x == 0) { s_sel.B = 0; s_sel.r = 0; s_sel.cnt = 0; s_sel.lo_hi = s_sel.lo_lo = s_sel.hi_hi = s_sel.hi_lo = 0; s_n_extra = 0; }
     __syncthreads();
 
-    // ---------------- first half: the prune threshold ----------------
-    if (mode_p == 0u) select_bin(p, &w.sel[0], sp, p.fhist, &s_sel, blockIdx.x == 0);   // every CTA computes the same values
-    const unsigned Bp = s_sel.B;
-    const u64 r_p = s_sel.r;
-    // the threshold bin must be a real bin of the window and small enough to rank
-    const bool hit_p = mode_p != 0u || (Bp >= 1u && Bp <= nb - 2u && s_sel.cnt <= (u64)CAP);
-    if (!hit_p) {                                      // the same in every CTA
-        if (blockIdx.x == 0 && threadIdx.x == 0) one_pass_fail(p);
-        return;
-    }
-    if (mode_p == 0u) {
-        unsigned under = 0, over = 0;
-        const u128 lo0 = from_halves(s_sel.lo_hi, s_sel.lo_lo);
-        const u128 hi0 = from_halves(s_sel.hi_hi, s_sel.hi_lo);
-        for (unsigned i = blockIdx.x * blockDim.x + threadIdx.x; i < n_list; i += gridDim.x * blockDim.x) {
-            const uint2 e = __ldg(&p.list[i]);
-            const unsigned bp = e.y & 0xffffu, bu = e.y >> 16;
-            if (bp == 0u || bp == top) continue;          // not in the prune window: counted by pass_kernel
-            if (bp < Bp) continue;                        // pruned
-            if (bp == Bp) {                               // decided by the last CTA
-                const u64 key = exact_key<B>(p, (long long)e.x, 0);
-                const u128 c = make_c(key, (u64)e.x);
-                if (c >= lo0 && c < hi0) {
-                    const unsigned slot = atomicAdd(&p.work->fcand_count[0], 1u);
-                    if (slot < (unsigned)CAP) { p.cand_key[slot] = key; p.cand_idx[slot] = e.x; }
+    SelView vp = view_of(&w.sel[0]);
+    if (alive && mode_p == 0u) {
+        // ---------------- 1: the prune threshold bin, its candidates, the survivors' L_u counts ----------------
+        select_bin(p, &w.sel[0], sp, p.fhist, &s_sel, blockIdx.x == 0);
+        const unsigned Bp = s_sel.B;
+        const u64 r_p = s_sel.r;
+        // the threshold bin must be a real bin of the window and small enough to rank
+        if (!(Bp >= 1u && Bp <= nb - 2u && s_sel.cnt <= (u64)CAP)) {
+            if (blockIdx.x == 0 && threadIdx.x == 0) one_pass_fail(p);
+            alive = false;
+        }
+        if (alive) {
+            unsigned under = 0, over = 0;
+            const u128 lo0 = from_halves(s_sel.lo_hi, s_sel.lo_lo);
+            const u128 hi0 = from_halves(s_sel.hi_hi, s_sel.hi_lo);
+            // a thread's entries are requested together (each iteration would otherwise wait for its own load)
+            const unsigned gstride = gridDim.x * blockDim.x;
+            for (unsigned i0 = blockIdx.x * blockDim.x + threadIdx.x; i0 < n_list; i0 += 4u * gstride) {
+              uint2 ent[4];
+#pragma unroll
+              for (int t4 = 0; t4 < 4; ++t4) {
+                  const unsigned i = i0 + (unsigned)t4 * gstride;
+                  ent[t4] = i < n_list ? __ldg(&p.list[i]) : make_uint2(0u, 0u);      // code 0: skipped below
+              }
+#pragma unroll
+              for (int t4 = 0; t4 < 4; ++t4) {
+                const uint2 e = ent[t4];
+                const unsigned idx = e.x & IDX_MASK;
+                const unsigned bp = e.y & 0xffffu, bu = e.y >> 16;
+                if (bp == 0u || bp == top) continue;          // not in the prune window: counted by pass_kernel
+                if (bp < Bp) continue;                        // pruned
+                if (bp == Bp) {                               // ranked after the barrier
+                    double S, Lu, Kp;
+                    block_keys_at<B>(p.W, p.U, (long long)idx, p.use_l1, &S, &Lu, &Kp);
+                    const u64 key = key_bits(Kp);
+                    const u128 c = make_c(key, (u64)idx);
+                    if (c >= lo0 && c < hi0) {
+                        const unsigned slot = atomicAdd(&p.work->fcand_count[0], 1u);
+                        if (slot < (unsigned)CAP) {
+                            p.cand_key[slot] = key;
+                            p.cand_idx[slot] = idx;
+                            p.cand_aux[slot] = bin_of(key_bits(Lu), ulo, uhi, ush, nb);   // where it counts if it survives
+                        }
+                    }
+                    continue;
                 }
-                continue;
+                if (mode_u != 0u) continue;
+                if (bu == 0u) ++under;
+                else if (bu == top) ++over;
+                else atomicAdd(&hist_u[bu], 1u);
+              }
             }
-            if (mode_u != 0u) continue;
-            if (bu == 0u) ++under;
-            else if (bu == top) ++over;
-            else atomicAdd(&hist_u[bu], 1u);
+            for (int m = 16; m > 0; m >>= 1) {
+                under += __shfl_xor_sync(0xffffffffu, under, m);
+                over += __shfl_xor_sync(0xffffffffu, over, m);
+            }
+            if ((threadIdx.x & 31) == 0) {
+                if (under) atomicAdd(&hist_u[0], under);
+                if (over) atomicAdd(&hist_u[top], over);
+            }
         }
-        for (int m = 16; m > 0; m >>= 1) {
-            under += __shfl_xor_sync(0xffffffffu, under, m);
-            over += __shfl_xor_sync(0xffffffffu, over, m);
+        if (!grid_sync(&p.work->bar, ++k)) {              // bounded; every CTA runs into the same limit
+            if (threadIdx.x == 0) atomicOr(p.dev_status, (unsigned)MWU_DEV_TIMEOUT);
+            return;
         }
-        if ((threadIdx.x & 31) == 0) {
-            if (under) atomicAdd(&hist_u[0], under);
-            if (over) atomicAdd(&hist_u[top], over);
-        }
-    }
-    if (last_block_done(&p.work->fticket[0])) {
-        // ---- the CTA that finished last: exact prune threshold, unify threshold bin ----
-        bool ok = true;
-        if (mode_p == 0u) {
+        if (alive) {
+            // ---------------- 2: exact prune threshold, corrections, unify threshold bin ----------------
             const unsigned m = ld_vol(&p.work->fcand_count[0]);
-            ok = pick_threshold(p, sp, r_p, m, c_key, c_idx);
-            // the blocks of the threshold bin that survive join the L_u histogram
-            if (ok && mode_u == 0u) {
-                for (unsigned i = (unsigned)r_p + threadIdx.x; i < m; i += blockDim.x) {
-                    const u64 ku = exact_key<B>(p, (long long)c_idx[i], 1);
-                    atomicAdd(&hist_u[bin_of(ku, ulo, uhi, ush, nb)], 1u);
+            if (m > (unsigned)CAP || r_p < 1 || r_p > (u64)m) {
+                if (blockIdx.x == 0 && threadIdx.x == 0) one_pass_fail(p);
+                alive = false;
+            } else {
+                const bool have_aux = rank_candidates(p, p.cand_key, p.cand_idx, p.cand_aux, m, c_key, c_idx, c_aux);
+                vp.B = Bp;
+                vp.T_key = c_key[r_p - 1];
+                vp.T_idx = (u64)c_idx[r_p - 1];
+                if (blockIdx.x == 0 && threadIdx.x == 0) { sp->T_key = vp.T_key; sp->T_idx = vp.T_idx; }
+                // the candidates that survive belong in the L_u histogram: kept here as corrections
+                if (mode_u == 0u) {
+                    for (unsigned i = (unsigned)r_p + threadIdx.x; i < m; i += blockDim.x) {
+                        const unsigned bu = have_aux ? c_aux[i] : bin_of(exact_key<B>(p, (long long)c_idx[i], 1), ulo, uhi, ush, nb);
+                        s_extra[atomicAdd(&s_n_extra, 1u)] = bu;
+                    }
+                }
+                __syncthreads();
+            }
+        }
+    }
+    unsigned Bu = 0;
+    u64 r_u = 0;
+    u128 lo = 0, hi = 0;
+    if (alive && mode_u == 0u) {
+        select_bin(p, &w.sel[1], su, hist_u, &s_sel, blockIdx.x == 0, s_extra, s_n_extra);
+        Bu = s_sel.B;
+        r_u = s_sel.r;
+        lo = from_halves(s_sel.lo_hi, s_sel.lo_lo);
+        hi = from_halves(s_sel.hi_hi, s_sel.hi_lo);
+        if (!(Bu >= 1u && Bu <= nb - 2u && s_sel.cnt <= (u64)CAP)) {
+            if (blockIdx.x == 0 && threadIdx.x == 0) one_pass_fail(p);
+            alive = false;
+        }
+    }
+    if (alive) {
+        // ---------------- 3: final classes of the listed blocks ----------------
+        double resid_delta = 0.0;
+        const unsigned per_round = CHG_PER_THREAD * gridDim.x * blockDim.x;
+        const unsigned rounds = (n_list + per_round - 1u) / per_round;
+        for (unsigned rd = 0; rd < rounds; ++rd) {
+            if (threadIdx.x == 0) s_n_chg = 0;
+            __syncthreads();
+            uint2 ent[CHG_PER_THREAD];
+            bool have[CHG_PER_THREAD];
+#pragma unroll
+            for (int t3 = 0; t3 < CHG_PER_THREAD; ++t3) {
+                const unsigned i = ((rd * CHG_PER_THREAD + t3) * gridDim.x + blockIdx.x) * blockDim.x + threadIdx.x;
+                have[t3] = i < n_list;
+                ent[t3] = have[t3] ? __ldg(&p.list[i]) : make_uint2(0u, 0u);
+            }
+#pragma unroll
+            for (int t3 = 0; t3 < CHG_PER_THREAD; ++t3) {
+                if (!have[t3]) continue;
+                const uint2 e = ent[t3];
+                const unsigned idx = e.x & IDX_MASK;
+                const bool pr0 = (e.x >> 31) & 1u, un0 = (e.x >> 30) & 1u;
+                const unsigned bu = e.y >> 16;
+                const bool pr = selected<B>(p, vp, (long long)idx, e.y & 0xffffu, 0);
+                bool un = false, held = false;
+                if (!pr) {
+                    if (mode_u == 2u) un = true;
+                    else if (mode_u == 0u) {
+                        if (bu == Bu) {                            // ranked by the last CTA
+                            const u64 key = exact_key<B>(p, (long long)idx, 1);
+                            const u128 c = make_c(key, (u64)idx);
+                            if (c >= lo && c < hi) {
+                                const unsigned slot = atomicAdd(&p.work->fcand_count[1], 1u);
+                                if (slot < (unsigned)CAP) {
+                                    p.cand_key[CAP + slot] = key;
+                                    p.cand_idx[CAP + slot] = idx;
+                                    p.cand_aux[CAP + slot] = (pr0 ? 2u : 0u) | (un0 ? 1u : 0u);   // the class pass_kernel wrote
+                                }
+                                held = true;
+                            }
+                            un = c < lo;
+                        } else un = bu < Bu;
+                    }
+                }
+                if (!held && (pr != pr0 || un != un0)) {
+                    // index with the final class in bits 31 / 30, the provisional class in a second word
+                    const unsigned slot = atomicAdd(&s_n_chg, 1u);
+                    s_chg[2 * slot] = idx | ((pr ? 1u : 0u) << 31) | ((un ? 1u : 0u) << 30);
+                    s_chg[2 * slot + 1] = (pr0 ? 2u : 0u) | (un0 ? 1u : 0u);
                 }
             }
-            __threadfence();
+            __syncthreads();
+            // the changed blocks of this round, one per thread (every lane of the leading warps busy)
+            const unsigned n_chg = s_n_chg;
+            for (unsigned c = threadIdx.x; c < n_chg; c += blockDim.x) {
+                const unsigned pe = s_chg[2 * c], old = s_chg[2 * c + 1];
+                resid_delta += apply_class<B>(p, Q, u_out, pruned_bitmap, unified_bitmap, pe & IDX_MASK, (pe >> 31) & 1u,
+                                              (pe >> 30) & 1u, (old >> 1) & 1u, old & 1u);
+            }
             __syncthreads();
         }
-        if (ok && mode_u == 0u) {
-            select_bin(p, &w.sel[1], su, hist_u, &s_sel, true);
-            if (!(s_sel.B >= 1u && s_sel.B <= nb - 2u && s_sel.cnt <= (u64)CAP)) ok = false;
-        }
-        if (threadIdx.x == 0) {
-            if (!ok) one_pass_fail(p);
-            __threadfence();
-            atomicExch(&p.work->release, 1u);
-        }
-    } else {
-        // the others wait for the thresholds (all CTAs are resident, the wait is bounded)
-        if (threadIdx.x == 0) {
-            int go = 1;
-            const long long t0 = clock64();
-            unsigned spins = 0;
-            while (ld_vol(&p.work->release) == 0u) {
-                if ((++spins & 63u) == 0u && clock64() - t0 > GRID_WAIT_CYCLES) { go = 0; break; }
-            }
-            __threadfence();
-            if (!go) { atomicOr(p.dev_status, (unsigned)MWU_DEV_TIMEOUT); one_pass_fail(p); }
-            s_go = go;
-        }
-        __syncthreads();
-        if (!s_go) return;
-    }
-    load_work(p.work, &w);                             // thresholds as the last CTA published them
-    if (w.failed != 0u) return;
-
-    // ---------------- second half: final classes of the listed blocks ----------------
-    const SelView vp = view_of(&w.sel[0]);
-    const unsigned Bu = w.sel[1].B;
-    const u64 r_u = w.sel[1].r;
-    const u128 lo = from_halves(w.sel[1].lo_hi, w.sel[1].lo_lo);
-    const u128 hi = from_halves(w.sel[1].hi_hi, w.sel[1].hi_lo);
-    double resid_delta = 0.0;
-    for (unsigned i = blockIdx.x * blockDim.x + threadIdx.x; i < n_list; i += gridDim.x * blockDim.x) {
-        const uint2 e = __ldg(&p.list[i]);
-        const unsigned bu = e.y >> 16;
-        const bool pr = selected<B>(p, vp, (long long)e.x, e.y & 0xffffu, 0);
-        bool un = false;
-        if (!pr) {
-            if (mode_u == 2u) un = true;
-            else if (mode_u == 0u) {
-                if (bu == Bu) {                            // decided by the last CTA
-                    const u64 key = exact_key<B>(p, (long long)e.x, 1);
-                    const u128 c = make_c(key, (u64)e.x);
-                    if (c >= lo && c < hi) {
-                        const unsigned slot = atomicAdd(&p.work->fcand_count[1], 1u);
-                        if (slot < (unsigned)CAP) { p.cand_key[CAP + slot] = key; p.cand_idx[CAP + slot] = e.x; }
-                        continue;
-                    }
-                    un = c < lo;
-                } else un = bu < Bu;
+        if (p.resid) block_add_double(resid_delta, p.resid);
+        if (mode_u == 0u && last_block_done(&p.work->fticket[1])) {
+            // ---- the CTA that finishes last: the blocks of the unify threshold bin ----
+            const unsigned m = ld_vol(&p.work->fcand_count[1]);
+            if (m > (unsigned)CAP || r_u < 1 || r_u > (u64)m) {
+                if (threadIdx.x == 0) one_pass_fail(p);
+            } else {
+                const bool have_aux = rank_candidates(p, p.cand_key + CAP, p.cand_idx + CAP, p.cand_aux + CAP, m, c_key,
+                                                      c_idx, c_aux);
+                if (threadIdx.x == 0) { su->T_key = c_key[r_u - 1]; su->T_idx = (u64)c_idx[r_u - 1]; }
+                const unsigned r = (unsigned)r_u;
+                double tail_delta = 0.0;
+                for (unsigned i = threadIdx.x; i < m; i += blockDim.x) {
+                    // the class pass_kernel wrote for this block: carried with the candidate, else read back
+                    const unsigned idx = c_idx[i], bit = 1u << (idx & 31u);
+                    const bool pr0 = have_aux ? ((c_aux[i] >> 1) & 1u) != 0u : (ld_vol(pruned_bitmap + (idx >> 5)) & bit) != 0u;
+                    const bool un0 = have_aux ? (c_aux[i] & 1u) != 0u : (ld_vol(unified_bitmap + (idx >> 5)) & bit) != 0u;
+                    const bool un = i < r;
+                    if (pr0 || un != un0)
+                        tail_delta += apply_class<B>(p, Q, u_out, pruned_bitmap, unified_bitmap, idx, false, un, pr0, un0);
+                }
+                if (p.resid) block_add_double(tail_delta, p.resid);
             }
         }
-        resid_delta += apply_class<B>(p, Q, u_out, pruned_bitmap, unified_bitmap, e.x, pr, un);
     }
-    if (p.resid) block_add_double(resid_delta, p.resid);
-    if (mode_u != 0u) return;
-    if (!last_block_done(&p.work->fticket[1])) return;
-
-    // ---- last CTA only ----
-    const unsigned m = ld_vol(&p.work->fcand_count[1]);
-    Params pc = p;                                     // the second half's candidates sit behind the first half's
-    pc.cand_key = p.cand_key + CAP;
-    pc.cand_idx = p.cand_idx + CAP;
-    if (!pick_threshold(pc, su, r_u, m, c_key, c_idx)) {
-        if (threadIdx.x == 0) one_pass_fail(p);
+    // ---------------- 4: the fallback, if the one-pass result was given up anywhere ----------------
+    if (!grid_sync(&p.work->bar, ++k)) {
+        if (threadIdx.x == 0) atomicOr(p.dev_status, (unsigned)MWU_DEV_TIMEOUT);
         return;
     }
-    const unsigned r = (unsigned)r_u;
-    double tail_delta = 0.0;
-    for (unsigned i = threadIdx.x; i < m; i += blockDim.x)
-        tail_delta += apply_class<B>(p, Q, u_out, pruned_bitmap, unified_bitmap, c_idx[i], false, i < r);
-    if (p.resid) block_add_double(tail_delta, p.resid);
+    load_work(p.work, &w);
+    if (w.failed == 0u) return;
+    multipass_phases<B>(p, w, k, false, mp_smem, Q, loss_u, loss_p, u_out, pruned_bitmap, unified_bitmap, sign_bits);
+}
+
+// ---------------------------------------------------------------------------------------------
+// multipass_kernel (cooperative launch): the whole multi-pass projection in one launch.  It is the
+// projection of small tensors (launch latency decides there) and of MWU_ALGO_MULTI_PASS.
+// ---------------------------------------------------------------------------------------------
+template <int B>
+__global__ void __launch_bounds__(FIN_THREADS) multipass_kernel(Params p, float *Q, double *loss_u, double *loss_p,
+                                                                float *u_out, unsigned *pruned_bitmap,
+                                                                unsigned *unified_bitmap, unsigned *sign_bits) {
+    extern __shared__ __align__(16) unsigned char mp_smem[];
+    __shared__ Work w;
+    unsigned k = 0;
+    multipass_phases<B>(p, w, k, p.run_sample != 0, mp_smem, Q, loss_u, loss_p, u_out, pruned_bitmap, unified_bitmap,
+                        sign_bits);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -2033,55 +2224,6 @@ __global__ void __launch_bounds__(FIN_THREADS) group_select_kernel(const double 
     }
 }
 
-// ---------------------------------------------------------------------------------------------
-// multipass_kernel (cooperative launch): the whole multi-pass projection in one launch, its phases
-// separated by grid barriers -- [windows from a sample] -> statistics -> prune threshold -> unify
-// threshold -> emit.  It is the projection of small tensors (launch latency decides there), and the
-// fallback of the one-pass pipeline, behind which it is always enqueued and returns at once unless
-// work->failed is set.
-// ---------------------------------------------------------------------------------------------
-constexpr int MP_SMEM_BYTES = (FIN_THREADS / 32) * 128 * 16;     // emit staging: 2 KB per warp
-static_assert(MP_SMEM_BYTES >= CAP * 12, "the candidate sort buffers share the staging memory");
-
-template <int B>
-__global__ void __launch_bounds__(FIN_THREADS) multipass_kernel(Params p, float *Q, double *loss_u, double *loss_p,
-                                                                float *u_out, unsigned *pruned_bitmap,
-                                                                unsigned *unified_bitmap, unsigned *sign_bits) {
-    extern __shared__ __align__(16) unsigned char mp_smem[];
-    __shared__ Work w;
-    u64 *c_key = reinterpret_cast<u64 *>(mp_smem);
-    unsigned *c_idx = reinterpret_cast<unsigned *>(mp_smem + CAP * sizeof(u64));
-    if (p.gated) {
-        load_work(p.work, &w);
-        if (w.failed == 0u) return;                    // the one-pass result stands (the same in every CTA)
-    }
-    unsigned k = 0;                                    // grid barriers passed so far
-    bool ok = true;
-    if (p.run_sample) {
-        if (blockIdx.x == 0) sample_body<B>(p);
-        ok = grid_sync(&p.work->bar, ++k);
-    }
-    if (ok) {
-        load_work(p.work, &w);
-        stats_body<B>(p, w, loss_u, loss_p, u_out, sign_bits);
-        ok = grid_sync(&p.work->bar, ++k);
-    }
-    if (ok) {
-        prune_select_body<B>(p, w, c_key, c_idx);
-        ok = grid_sync(&p.work->bar, ++k);
-    }
-    if (ok) {
-        load_work(p.work, &w);
-        collect_body<1, B>(p, w, c_key, c_idx);
-        ok = grid_sync(&p.work->bar, ++k);
-    }
-    if (ok) {
-        load_work(p.work, &w);
-        emit_body<B>(p, w, Q, u_out, pruned_bitmap, unified_bitmap, sign_bits, reinterpret_cast<float4 *>(mp_smem));
-    }
-    if (!ok && threadIdx.x == 0) atomicOr(p.dev_status, (unsigned)MWU_DEV_TIMEOUT);
-}
-
 }  // namespace proj
 
 // ---------------------------------------------------------------------------------------------
@@ -2091,7 +2233,9 @@ static size_t ws_off_hist() { return align_up(sizeof(proj::Work)); }
 static size_t ws_off_cand_key() { return align_up(ws_off_hist() + 5 * proj::NB_MAX * sizeof(unsigned)); }
 // two sets of candidates: the two halves of resolve_kernel each keep their own
 static size_t ws_off_cand_idx() { return align_up(ws_off_cand_key() + 2 * proj::CAP * sizeof(proj::u64)); }
-static size_t ws_off_bins() { return align_up(ws_off_cand_idx() + 2 * proj::CAP * sizeof(unsigned)); }
+static size_t ws_off_cand_aux() { return align_up(ws_off_cand_idx() + 2 * proj::CAP * sizeof(unsigned)); }
+static size_t ws_off_samp() { return align_up(ws_off_cand_aux() + 2 * proj::CAP * sizeof(unsigned)); }
+static size_t ws_off_bins() { return align_up(ws_off_samp() + 2 * proj::NSAMP * sizeof(proj::u64)); }
 static size_t ws_off_list(size_t mb) { return align_up(ws_off_bins() + (mb + 8) * sizeof(unsigned)); }
 // candidate list of the one-pass pipeline: a quarter of the blocks (the windows hold a few per cent)
 static size_t list_capacity(size_t mb) { return mb / 4 + 4096; }
@@ -2102,9 +2246,11 @@ static size_t n_groups_of(const mwu_proj_desc *d) {
 static size_t ws_off_gprune(const mwu_proj_desc *d, size_t mb) { return align_up(ws_off_gkey(mb) + n_groups_of(d) * sizeof(double)); }
 
 static bool use_one_pass(const mwu_proj_desc *desc) {
+    const long long mb = desc->rows * desc->cols / desc->block;
+    if (mb >= (1ll << 30)) return false;               // list entries keep two class bits above the block index
     if (desc->algo == MWU_ALGO_ONE_PASS) return true;
     if (desc->algo == MWU_ALGO_MULTI_PASS) return false;
-    return desc->rows * desc->cols / desc->block >= proj::ONE_PASS_MIN_BLOCKS;
+    return mb >= proj::ONE_PASS_MIN_BLOCKS;
 }
 
 }  // namespace mwu
@@ -2162,30 +2308,47 @@ static cudaError_t launch_project(const mwu::proj::Params &p, const mwu_proj_des
     if (!smem_set) {
         e = cudaFuncSetAttribute(multipass_kernel<B>, cudaFuncAttributeMaxDynamicSharedMemorySize, MP_SMEM_BYTES);
         if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(resolve_kernel<B>, cudaFuncAttributeMaxDynamicSharedMemorySize, MP_SMEM_BYTES);
+        if (e != cudaSuccess) return e;
         smem_set = true;
     }
 
     if (one_pass) {
-        // CTA 0 clears the selection state and samples; further CTAs clear the five histograms
+        // the sample keys (and the cleared histograms) from 32 SMs, then one CTA ranks the sample; the two
+        // kernels behind are launched with programmatic stream serialization, so their CTAs are in place
+        // (and the sweep's first loads in flight) when their predecessor ends
         const unsigned n_zero = 5u * (unsigned)p.nb;
-        const int zero_ctas = p.nb == NB_SMALL ? 1 : 8;
-        sample_kernel<B><<<1 + zero_ctas, SAMP_THREADS, 0, st>>>(p, p.hist, n_zero);
-        if (p.U_next || p.resid) pass_kernel<B, true><<<grid_stream, 256, 0, st>>>(p, Q, loss_u, loss_p, u, pb, ub, sb);
-        else pass_kernel<B, false><<<grid_stream, 256, 0, st>>>(p, Q, loss_u, loss_p, u, pb, ub, sb);
-        mwu::count_launch(2);
+        sample_keys_kernel<B><<<NSAMP / 128, 128, 0, st>>>(p, p.hist, n_zero);
+        {
+            cudaLaunchConfig_t cfg = {};
+            cfg.stream = st;
+            cudaLaunchAttribute attr[1];
+            attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+            attr[0].val.programmaticStreamSerializationAllowed = 1;
+            cfg.attrs = attr;
+            cfg.numAttrs = 1;
+            cfg.gridDim = dim3(1);
+            cfg.blockDim = dim3(SAMP_THREADS);
+            e = cudaLaunchKernelEx(&cfg, sample_kernel<B>, p);
+            if (e != cudaSuccess) return e;
+            cfg.gridDim = dim3((unsigned)grid_stream);
+            cfg.blockDim = dim3(256);
+            if (p.U_next || p.resid) e = cudaLaunchKernelEx(&cfg, pass_kernel<B, true>, p, Q, loss_u, loss_p, u, pb, ub, sb);
+            else e = cudaLaunchKernelEx(&cfg, pass_kernel<B, false>, p, Q, loss_u, loss_p, u, pb, ub, sb);
+            if (e != cudaSuccess) return e;
+        }
+        mwu::count_launch(3);
         if (!need_p && !need_u) return cudaGetLastError();       // no threshold: every class is final
-        // the list holds a few per cent of the blocks: a thread per expected entry, one CTA per SM at most
+        // the list holds a few per cent of the blocks: a thread per expected entry, one CTA per SM at most.
+        // Should the one-pass result be given up (once in thousands of calls), the same kernel redoes the
+        // projection with the multi-pass phases.
         const long long lb = (mb / 8 + FIN_THREADS - 1) / FIN_THREADS;
-        const int grid_list = (int)(lb < (long long)sm_count ? (lb > 0 ? lb : 1) : (long long)sm_count);
-        e = launch_cooperative(resolve_kernel<B>, grid_list, FIN_THREADS, 0, sm_count, st, p, Q, u, pb, ub);
-        if (e != cudaSuccess) return e;
-        // behind it the multi-pass kernel, which returns at once unless the one-pass result was given up
-        // (once in thousands of calls)
+        const int grid_list = (int)(lb < (long long)sm_count ? (lb > 16 ? lb : 16) : (long long)sm_count);
+        return launch_cooperative(resolve_kernel<B>, grid_list, FIN_THREADS, (size_t)MP_SMEM_BYTES, sm_count, st, p, Q,
+                                  loss_u, loss_p, u, pb, ub, sb);
     }
-    e = launch_cooperative(multipass_kernel<B>, grid_mp, FIN_THREADS, (size_t)MP_SMEM_BYTES, sm_count, st, p, Q, loss_u,
-                           loss_p, u, pb, ub, sb);
-    if (e != cudaSuccess) return e;
-    return cudaGetLastError();
+    return launch_cooperative(multipass_kernel<B>, grid_mp, FIN_THREADS, (size_t)MP_SMEM_BYTES, sm_count, st, p, Q, loss_u,
+                              loss_p, u, pb, ub, sb);
 }
 
 // mwu_project and mwu_admm_step: the latter also wants U_next and / or residual_sq
@@ -2228,6 +2391,9 @@ static int project_impl(const mwu_proj_desc *desc, const float *W, const float *
     p.fhist = p.hist + 3 * (size_t)p.nb;
     p.cand_key = (proj::u64 *)(ws + ws_off_cand_key());
     p.cand_idx = (unsigned *)(ws + ws_off_cand_idx());
+    p.cand_aux = (unsigned *)(ws + ws_off_cand_aux());
+    p.samp_kp = (proj::u64 *)(ws + ws_off_samp());
+    p.samp_ku = p.samp_kp + proj::NSAMP;
     p.bins = (unsigned *)(ws + ws_off_bins());
     p.list = (uint2 *)(ws + ws_off_list((size_t)p.n_blocks));
     p.list_cap = (unsigned)list_capacity((size_t)p.n_blocks);
