@@ -2,11 +2,12 @@
 //
 // The fused kernel behind mwu_conv_implicit decodes every weight record again for each activation
 // tile and assembles its im2col rows element by element.  With a workspace the work is split:
-//   nchw_to_nhwc_kernel     copies the input image into pixel-major order (channels innermost), so
-//                           that the 64 channels of a pixel are one 128-byte line;
-//   mwu_decode_taps_kernel  expands the packed weights once, as mwu_decode does, but orders the
-//                           reduction axis tap-major: column (i*kw + j) * cin + c instead of
-//                           c * kh*kw + i*kw + j (the same products, summed tap by tap);
+//   conv_prep_kernel        one launch, two jobs side by side: image tiles are copied into
+//                           pixel-major order (channels innermost, so that the 64 channels of a
+//                           pixel are one 128-byte line), and the packed weights are expanded once,
+//                           as mwu_decode does, but with the reduction axis tap-major: column
+//                           (i*kw + j) * cin + c instead of c * kh*kw + i*kw + j (the same products,
+//                           summed tap by tap);
 //   mwu_conv_taps_kernel    one CTA per tile of R output rows x OW pixels (R * OW <= 128) and 128
 //                           filters.  A k stage is one filter tap and 64 channels: its activation
 //                           operand is a box of the pixel-major image shifted by the tap's offset,
@@ -71,36 +72,53 @@ __device__ __forceinline__ void tma_load_4d(unsigned dst, const CUtensorMap *map
 }
 
 // ------------------------------------------------------------------------------------------
-// input image: [n][c][h*w] -> [n][h*w][c]
+// preparation, one launch: the input image [n][c][h*w] -> [n][h*w][c], and the weights
 // ------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256) nchw_to_nhwc_kernel(const unsigned short *x, unsigned short *xt, int C, int HW) {
-    __shared__ unsigned short tile[32][34];
-    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
-    const long long img = blockIdx.z;
-    const int hw0 = blockIdx.x * 32, c0 = blockIdx.y * 32;
+constexpr int PREP_THREADS = 512;
+
+// one CTA: a tile of 64 pixels x 64 channels of one image, read as pixel pairs, written as channel pairs
+__device__ __forceinline__ void nchw_to_nhwc_tile(const unsigned short *x, unsigned short *xt, int C, int HW,
+                                                  int tile, int tiles_hw, int tiles_c) {
+    __shared__ unsigned short s_t[64][66];
+    const int img = tile / (tiles_hw * tiles_c), rem = tile % (tiles_hw * tiles_c);
+    const int hw0 = (rem % tiles_hw) * 64, c0 = (rem / tiles_hw) * 64;
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;            // 32 x 16
+    const long long base = (long long)img * C * HW;
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-        const int c = c0 + ty + 8 * i, hw = hw0 + tx;
-        tile[ty + 8 * i][tx] = (c < C && hw < HW) ? x[(img * C + c) * HW + hw] : (unsigned short)0;
+        const int c = c0 + ty + 16 * i, hw = hw0 + 2 * tx;
+        unsigned short a = 0, b = 0;
+        if (c < C) {
+            if (hw + 1 < HW && (HW & 1) == 0) {
+                const unsigned v = *reinterpret_cast<const unsigned *>(x + base + (long long)c * HW + hw);
+                a = (unsigned short)v; b = (unsigned short)(v >> 16);
+            } else {
+                if (hw < HW) a = x[base + (long long)c * HW + hw];
+                if (hw + 1 < HW) b = x[base + (long long)c * HW + hw + 1];
+            }
+        }
+        s_t[ty + 16 * i][2 * tx] = a;
+        s_t[ty + 16 * i][2 * tx + 1] = b;
     }
     __syncthreads();
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-        const int hw = hw0 + ty + 8 * i, c = c0 + tx;
-        if (hw < HW && c < C) xt[(img * HW + hw) * C + c] = tile[tx][ty + 8 * i];
+        const int hw = hw0 + ty + 16 * i, c = c0 + 2 * tx;
+        if (hw < HW && c + 1 < C + 1) {
+            unsigned short *dst = xt + ((long long)img * HW + hw) * C + c;
+            const unsigned short a = s_t[2 * tx][ty + 16 * i], b = s_t[2 * tx + 1][ty + 16 * i];
+            if (c + 1 < C) *reinterpret_cast<unsigned *>(dst) = (unsigned)a | ((unsigned)b << 16);     // C is even
+            else if (c < C) dst[0] = a;
+        }
     }
 }
 
-// ------------------------------------------------------------------------------------------
-// packed records -> row-major bf16 with the reduction axis in tap-major order
-// ------------------------------------------------------------------------------------------
+// one CTA: a packed 128 x 64 record -> row-major bf16 with the reduction axis in tap-major order
 template <int BW>
-__global__ void __launch_bounds__(128) mwu_decode_taps_kernel(const Params p, unsigned short *Wd, int taps, int C) {
-    MWU_CHECK_HEADER(p);
+__device__ __forceinline__ void decode_taps_record(const Params &p, unsigned short *Wd, int taps, int C, long long rec) {
     __shared__ __align__(1024) unsigned char tile[REC_BYTES];
-    constexpr int ENT = DecodeCfg<BW, 128>::ENT;
+    constexpr int ENT = DecodeCfg<BW, PREP_THREADS>::ENT;
     const PackedRec *recs = reinterpret_cast<const PackedRec *>(p.packed + p.off_rec);
-    const long long rec = blockIdx.x;
     const long long rt = rec / p.n_stages, ks = rec % p.n_stages;
     const int tid = threadIdx.x;
     PackedRec r0, r1;
@@ -111,13 +129,13 @@ __global__ void __launch_bounds__(128) mwu_decode_taps_kernel(const Params p, un
         r1.ubase = b.x; r1.dbase = b.y; r1.pbase = b.z; r1.live = b.w;
     }
     unsigned m0[ENT], m1[ENT];
-    fetch_entries<BW, 128>(r0, r1, p, tid, m0, m1);
-    write_entries<BW, 128>(tile, r0, r1, p, tid, m0, m1);
+    fetch_entries<BW, PREP_THREADS>(r0, r1, p, tid, m0, m1);
+    write_entries<BW, PREP_THREADS>(tile, r0, r1, p, tid, m0, m1);
     asm volatile("cp.async.wait_all;" ::: "memory");
     __syncthreads();
 #pragma unroll
-    for (int i = 0; i < (REC_BYTES / 16) / 128; ++i) {
-        const int q = tid + i * 128;                        // 16-byte piece: row q / 8, piece q % 8
+    for (int i = 0; i < (REC_BYTES / 16) / PREP_THREADS; ++i) {
+        const int q = tid + i * PREP_THREADS;               // 16-byte piece: row q / 8, piece q % 8
         const int r = q >> 3, j = q & 7;
         const uint4 v = *reinterpret_cast<const uint4 *>(tile + r * 128 + ((j ^ (r & 7)) << 4));
         const unsigned wds[4] = {v.x, v.y, v.z, v.w};
@@ -129,6 +147,26 @@ __global__ void __launch_bounds__(128) mwu_decode_taps_kernel(const Params p, un
             row[(long long)tap * C + c] = (unsigned short)(wds[e >> 1] >> (16 * (e & 1)));
         }
     }
+}
+
+// CTAs [0, n_rec): weight records; the rest: image tiles.  The two jobs do not depend on each other,
+// so one launch runs them side by side.
+template <int BW>
+__global__ void __launch_bounds__(PREP_THREADS) conv_prep_kernel(const Params p, unsigned short *Wd, int taps, int C,
+                                                                 unsigned n_rec, const unsigned short *x,
+                                                                 unsigned short *xt, int HW, int tiles_hw, int tiles_c) {
+    if (blockIdx.x < n_rec) {
+        MWU_CHECK_HEADER(p);
+        decode_taps_record<BW>(p, Wd, taps, C, blockIdx.x);
+    } else {
+        nchw_to_nhwc_tile(x, xt, C, HW, (int)(blockIdx.x - n_rec), tiles_hw, tiles_c);
+    }
+}
+
+// the image alone (weights come from somewhere else)
+__global__ void __launch_bounds__(PREP_THREADS) nchw_to_nhwc_kernel(const unsigned short *x, unsigned short *xt, int C,
+                                                                    int HW, int tiles_hw, int tiles_c) {
+    nchw_to_nhwc_tile(x, xt, C, HW, (int)blockIdx.x, tiles_hw, tiles_c);
 }
 
 // a plain dense weight matrix [rows][ldw] in [c][tap] column order -> [n_pad][c * taps] tap-major
@@ -377,12 +415,12 @@ static bool taps_geometry(int n, int c, int h, int w, int kh, int kw, int stride
     return true;
 }
 
-// image copy, tensor maps and the tensor-core kernel; the tap-major weights must already be in `wd`
-// (or be produced by `make_weights`, which is enqueued between the image copy and the main kernel)
+// tensor maps, the preparation (`prepare` enqueues the image copy and whatever puts the tap-major
+// weights into `wd`) and the tensor-core kernel
 template <typename F>
 static int run_taps(ConvParams &p, const void *X_nchw, int n, int c, int h, int w, int kh, int kw, int pad,
                     unsigned short *xt, unsigned short *wd, long long n_pad, int sm_count, cudaStream_t st,
-                    F make_weights) {
+                    F prepare) {
     EncodeTiledFn encode = get_encode_fn();
     if (!encode) return MWU_ERR_CUDA;
     int OH, OW, R;
@@ -416,16 +454,15 @@ static int run_taps(ConvParams &p, const void *X_nchw, int n, int c, int h, int 
             return MWU_ERR_CUDA;
     }
     const int HW = h * w;
-    nchw_to_nhwc_kernel<<<dim3((unsigned)((HW + 31) / 32), (unsigned)((c + 31) / 32), (unsigned)n), 256, 0, st>>>(
-        (const unsigned short *)X_nchw, xt, c, HW);
-    make_weights();
+    const int tiles_hw = (HW + 63) / 64, tiles_c = (c + 63) / 64;
+    prepare((const unsigned short *)X_nchw, xt, HW, tiles_hw, tiles_c, (unsigned)(n * tiles_hw * tiles_c));
     const size_t smem = conv_smem_bytes();
     if (cudaFuncSetAttribute(mwu_conv_taps_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return MWU_ERR_CUDA;
     const long long tiles = (long long)n * p.tiles_per_img * p.n_ntiles;
     const int grid = (int)(tiles < sm_count ? tiles : sm_count);
     mwu_conv_taps_kernel<<<grid, C_THREADS, smem, st>>>(tmap_x, tmap_w, p);
-    count_launch(3);
+    count_launch();
     return cudaGetLastError() == cudaSuccess ? MWU_OK : MWU_ERR_CUDA;
 }
 
@@ -472,13 +509,16 @@ extern "C" int mwu_conv_implicit_ws(const mwu_proj_desc *desc, const void *packe
     const unsigned n_rec = (unsigned)(L.n_tiles * L.n_stages);
     const int taps = kh * kw, bw = desc->block;
     const Params g = p.g;
-    return run_taps(p, X_nchw, n, c, h, w, kh, kw, pad, xt, wd, L.n_pad, sm_count, st, [&]() {
+    return run_taps(p, X_nchw, n, c, h, w, kh, kw, pad, xt, wd, L.n_pad, sm_count, st,
+                    [&](const unsigned short *x, unsigned short *xo, int HW, int tiles_hw, int tiles_c, unsigned n_tiles) {
+        const unsigned grid = n_rec + n_tiles;
         switch (bw) {
-            case 2: mwu_decode_taps_kernel<2><<<n_rec, 128, 0, st>>>(g, wd, taps, c); break;
-            case 4: mwu_decode_taps_kernel<4><<<n_rec, 128, 0, st>>>(g, wd, taps, c); break;
-            case 8: mwu_decode_taps_kernel<8><<<n_rec, 128, 0, st>>>(g, wd, taps, c); break;
-            default: mwu_decode_taps_kernel<16><<<n_rec, 128, 0, st>>>(g, wd, taps, c); break;
+            case 2: conv_prep_kernel<2><<<grid, PREP_THREADS, 0, st>>>(g, wd, taps, c, n_rec, x, xo, HW, tiles_hw, tiles_c); break;
+            case 4: conv_prep_kernel<4><<<grid, PREP_THREADS, 0, st>>>(g, wd, taps, c, n_rec, x, xo, HW, tiles_hw, tiles_c); break;
+            case 8: conv_prep_kernel<8><<<grid, PREP_THREADS, 0, st>>>(g, wd, taps, c, n_rec, x, xo, HW, tiles_hw, tiles_c); break;
+            default: conv_prep_kernel<16><<<grid, PREP_THREADS, 0, st>>>(g, wd, taps, c, n_rec, x, xo, HW, tiles_hw, tiles_c); break;
         }
+        count_launch();
     });
 }
 
@@ -520,10 +560,14 @@ extern "C" int mwu_conv_dense(int64_t rows, const void *Wd, int64_t ldw, const v
     unsigned short *xt = (unsigned short *)workspace;
     unsigned short *wd = (unsigned short *)((char *)workspace + x_bytes_aligned(n, c, h, w));
     const int taps = kh * kw;
-    return run_taps(p, X_nchw, n, c, h, w, kh, kw, pad, xt, wd, n_pad, sm_count, st, [&]() {
-        const long long total = n_pad * p.g.K;
+    const long long K = p.g.K;
+    return run_taps(p, X_nchw, n, c, h, w, kh, kw, pad, xt, wd, n_pad, sm_count, st,
+                    [&](const unsigned short *x, unsigned short *xo, int HW, int tiles_hw, int tiles_c, unsigned n_tiles) {
+        nchw_to_nhwc_kernel<<<n_tiles, PREP_THREADS, 0, st>>>(x, xo, c, HW, tiles_hw, tiles_c);
+        const long long total = n_pad * K;
         const long long want = (total + 255) / 256, cap = (long long)sm_count * 16;
         permute_taps_kernel<<<(unsigned)(want < cap ? want : cap), 256, 0, st>>>((const unsigned short *)Wd, ldw, rows,
                                                                                   n_pad, taps, c, wd);
+        count_launch(2);
     });
 }

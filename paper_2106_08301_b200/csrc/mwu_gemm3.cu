@@ -97,12 +97,16 @@ constexpr int D_STAGE_BYTES = D_A_BYTES + D_B_BYTES;
 constexpr int D_BAND = 8;                            // activation row tiles per band of the tile order
 constexpr int D_EPI_BYTES = 4096;                    // per epilogue warp: 32 rows x 64 bf16 columns
 
+constexpr int D_LIVE_TAB = 4096;                     // live masks of all weight tiles, when they fit
+
 struct DenseSmem {
     unsigned long long full[D_STAGES], empty[D_STAGES], tfull[2], tempty[2], drain;
     unsigned tmem_base;
     int abort;
     unsigned char live_prod[MAX_STAGES_K];
     unsigned char live_mma[MAX_STAGES_K];
+    unsigned char live_tab[D_LIVE_TAB];                // [weight tile][stage], filled once at kernel start
+    unsigned char any_tab[D_LIVE_TAB / 4];             // [weight tile]: some stage of the tile is live
 };
 
 __global__ void __launch_bounds__(D_THREADS, 1)
@@ -154,12 +158,6 @@ mwu_dense_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) tmem_alloc2(smem_u32(&sm->tmem_base), 512);
-    tc_fence_before();
-    __syncthreads();
-    cluster_sync_all();                                 // both CTAs' barriers exist before any remote arrive
-    tc_fence_after();
-    const unsigned tmem_base = *reinterpret_cast<volatile unsigned *>(&sm->tmem_base);
-
     // live mask of stage ks for tile column nt: OR over its (one or two) 128-row records
     auto live_of = [&](long long nt, int ks) -> unsigned {
         if (p.all_live) return 0xFu;
@@ -167,10 +165,33 @@ mwu_dense_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
         if (nt * 2 + 1 < p.n_rec_tiles) l |= __ldg(&recs[(nt * 2 + 1) * n_stages + ks].live);
         return l;
     };
-    auto load_live = [&](unsigned char *table, long long nt) {
+    // The masks of every weight tile are read once, here, when they fit: read tile by tile they put a
+    // global-memory round trip in front of every tile of the producer and of the MMA issuer, which is
+    // a third of a tile's time when the reduction is only four stages long.
+    const bool tab_ok = n_tiles * n_stages <= D_LIVE_TAB && n_tiles <= D_LIVE_TAB / 4;
+    if (tab_ok) {
+        for (int i = threadIdx.x; i < (int)(n_tiles * n_stages); i += blockDim.x)
+            sm->live_tab[i] = (unsigned char)live_of(i / n_stages, i % n_stages);
+        __syncthreads();
+        for (int t = threadIdx.x; t < (int)n_tiles; t += blockDim.x) {
+            unsigned any = 0;
+            for (int ks = 0; ks < n_stages; ++ks) any |= sm->live_tab[t * n_stages + ks];
+            sm->any_tab[t] = (unsigned char)any;
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();                                 // both CTAs' barriers exist before any remote arrive
+    tc_fence_after();
+    const unsigned tmem_base = *reinterpret_cast<volatile unsigned *>(&sm->tmem_base);
+
+    // the masks of tile nt: a view into the table, or a fresh copy in the role's own buffer
+    auto load_live = [&](unsigned char *table, long long nt) -> const unsigned char * {
+        if (tab_ok) return &sm->live_tab[nt * n_stages];
         __syncwarp();
         for (int ks = lane; ks < n_stages; ks += 32) table[ks] = (unsigned char)live_of(nt, ks);
         __syncwarp();
+        return table;
     };
 
     if (warp == 0) {
@@ -183,9 +204,9 @@ mwu_dense_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
         bool ok = true;
         for (long long k = 0; ok && tile_of(k, mt_, nt_); ++k) {
             const long long mt = mt_, nt = nt_;
-            load_live(sm->live_prod, nt);
+            const unsigned char *lv = load_live(sm->live_prod, nt);
             for (int ks = 0; ks < n_stages; ++ks) {
-                if (!sm->live_prod[ks]) continue;
+                if (!lv[ks]) continue;
                 if (!mbar_wait_spin(smem_u32(&sm->empty[stage]), phase ^ 1u, abort)) ok = false;
                 if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
                 if (elect_one()) {
@@ -209,13 +230,13 @@ mwu_dense_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
         for (long long k = 0; ok && tile_of(k, mt_, nt_); ++k) {
             const long long nt = nt_;
             const unsigned buf = (unsigned)(k & 1), use_phase = (unsigned)((k >> 1) & 1);
-            load_live(sm->live_mma, nt);
+            const unsigned char *lv = load_live(sm->live_mma, nt);
             if (!mbar_wait(smem_u32(&sm->tempty[buf]), use_phase ^ 1u, abort)) ok = false;
             if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
             tc_fence_after();
             bool first = true;
             for (int ks = 0; ks < n_stages; ++ks) {
-                const unsigned live = sm->live_mma[ks];
+                const unsigned live = lv[ks];
                 if (!live) continue;
                 if (!ready) {
                     if (!mbar_wait_spin(smem_u32(&sm->full[stage]), phase, abort)) ok = false;
@@ -274,8 +295,11 @@ mwu_dense_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
             const long long mt = mt_, nt = nt_;
             const unsigned buf = (unsigned)(k & 1), use_phase = (unsigned)((k >> 1) & 1);
             unsigned any = 0;
-            for (int ks = lane; ks < n_stages; ks += 32) any |= live_of(nt, ks);
-            any = __reduce_or_sync(0xffffffffu, any);
+            if (tab_ok) any = sm->any_tab[nt];
+            else {
+                for (int ks = lane; ks < n_stages; ks += 32) any |= live_of(nt, ks);
+                any = __reduce_or_sync(0xffffffffu, any);
+            }
             if (!mbar_wait(smem_u32(&sm->tfull[buf]), use_phase, abort)) ok = false;
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
