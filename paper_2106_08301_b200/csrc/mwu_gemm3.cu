@@ -88,26 +88,33 @@ cudaError_t launch_decode(int bw, const Params &p, __nv_bfloat16 *Wd, long long 
 // ------------------------------------------------------------------------------------------
 // two-operand GEMM over the decoded weights
 // ------------------------------------------------------------------------------------------
-constexpr int D_STAGES = 6;
+constexpr int D_STAGES = 5;
 constexpr int D_EPI_WARPS = 8;
-constexpr int D_THREADS = 32 * (2 + D_EPI_WARPS);
+constexpr int D_MMA_WARP_B = 2 + D_EPI_WARPS;        // the second MMA issuer (the first is warp 1)
+constexpr int D_THREADS = 32 * (3 + D_EPI_WARPS);
 constexpr int D_A_BYTES = AH_BYTES;                  // this CTA's 128 activation rows
 constexpr int D_B_BYTES = REC_BYTES;                 // this CTA's 128 weight rows
 constexpr int D_STAGE_BYTES = D_A_BYTES + D_B_BYTES;
 constexpr int D_BAND = 8;                            // activation row tiles per band of the tile order
-constexpr int D_EPI_BYTES = 4096;                    // per epilogue warp: 32 rows x 64 bf16 columns
+constexpr int D_EPI_BUFS = 2;                        // staging buffers per epilogue warp
+constexpr int D_EPI_BYTES = 4096 * D_EPI_BUFS;       // each buffer: 32 rows x 64 bf16 columns
 
-constexpr int D_LIVE_TAB = 4096;                     // live masks of all weight tiles, when they fit
+constexpr int D_LIVE_TAB = 512;                      // live masks of all weight tiles, when they fit (short reductions)
 
 struct DenseSmem {
-    unsigned long long full[D_STAGES], empty[D_STAGES], tfull[2], tempty[2], drain;
+    unsigned long long full[D_STAGES], empty[D_STAGES], tfull[2], tempty[2], drain[2];
     unsigned tmem_base;
     int abort;
     unsigned char live_prod[MAX_STAGES_K];
     unsigned char live_mma[MAX_STAGES_K];
+    unsigned char live_mma_b[MAX_STAGES_K];              // the second MMA issuer's copy
+    unsigned ho_tiles, ho_ring;                        // hand-over between the two MMA issuers
     unsigned char live_tab[D_LIVE_TAB];                // [weight tile][stage], filled once at kernel start
-    unsigned char any_tab[D_LIVE_TAB / 4];             // [weight tile]: some stage of the tile is live
+    unsigned short cnt_tab[D_LIVE_TAB / 4];            // [weight tile]: how many of its stages are live
 };
+
+static_assert(1024 + D_STAGES * D_STAGE_BYTES + D_EPI_WARPS * D_EPI_BYTES + sizeof(DenseSmem) <= 232448,
+              "dense pair kernel: shared memory above the 227 KB a CTA may have");
 
 __global__ void __launch_bounds__(D_THREADS, 1)
 mwu_dense_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
@@ -126,21 +133,25 @@ mwu_dense_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const unsigned rank = cluster_rank();               // 0: leader (issues the MMAs), 1: peer
     const PackedRec *recs = reinterpret_cast<const PackedRec *>(p.packed + p.off_rec);
-    const long long m_tiles = (p.M + 255) / 256;
-    const long long n_tiles = (p.n_rec_tiles + 1) / 2;
-    const long long total_tiles = m_tiles * n_tiles;
-    const long long pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+    // 32-bit tile arithmetic (the host refuses a tile count of 2^31 or more): the MMA issuer computes
+    // the next tile's position between two tiles, while the tensor pipe runs dry
+    const unsigned m_tiles = (unsigned)((p.M + 255) / 256);
+    const unsigned n_tiles = (unsigned)((p.n_rec_tiles + 1) / 2);
+    const unsigned total_tiles = m_tiles * n_tiles;
+    const unsigned pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
     // k-th tile of this CTA pair.  Tiles are dealt round-robin in an order that walks bands of
     // D_BAND activation row tiles, weight tile by weight tile: the pairs running at one time then
     // share a few weight tiles and a band of activation rows, which stay in L2.
     long long mt_ = 0, nt_ = 0;
     auto tile_of = [&](long long k, long long &mt, long long &nt) -> bool {
-        const long long t = pair + k * n_pairs;
-        if (t >= total_tiles) return false;
-        const long long band = t / (D_BAND * n_tiles), r = t % (D_BAND * n_tiles);
-        const long long rows = (m_tiles - band * D_BAND) < D_BAND ? (m_tiles - band * D_BAND) : D_BAND;
-        nt = r / rows;
-        mt = band * D_BAND + r % rows;
+        const unsigned long long t64 = pair + (unsigned long long)k * n_pairs;
+        if (t64 >= total_tiles) return false;
+        const unsigned t = (unsigned)t64, per_band = D_BAND * n_tiles;
+        const unsigned band = t / per_band, r = t - band * per_band;
+        const unsigned left = m_tiles - band * D_BAND, rows = left < (unsigned)D_BAND ? left : (unsigned)D_BAND;
+        const unsigned q = r / rows;
+        nt = q;
+        mt = band * D_BAND + (r - q * rows);
         return true;
     };
 
@@ -153,8 +164,11 @@ mwu_dense_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
             mbar_init(smem_u32(&sm->tfull[b]), 1);
             mbar_init(smem_u32(&sm->tempty[b]), 2 * D_EPI_WARPS);
         }
-        mbar_init(smem_u32(&sm->drain), 1);
+        mbar_init(smem_u32(&sm->drain[0]), 1);
+        mbar_init(smem_u32(&sm->drain[1]), 1);
         sm->abort = 0;
+        sm->ho_tiles = 0;
+        sm->ho_ring = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) tmem_alloc2(smem_u32(&sm->tmem_base), 512);
@@ -168,15 +182,15 @@ mwu_dense_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
     // The masks of every weight tile are read once, here, when they fit: read tile by tile they put a
     // global-memory round trip in front of every tile of the producer and of the MMA issuer, which is
     // a third of a tile's time when the reduction is only four stages long.
-    const bool tab_ok = n_tiles * n_stages <= D_LIVE_TAB && n_tiles <= D_LIVE_TAB / 4;
+    const bool tab_ok = (long long)n_tiles * n_stages <= D_LIVE_TAB && n_tiles <= (unsigned)(D_LIVE_TAB / 4);
     if (tab_ok) {
-        for (int i = threadIdx.x; i < (int)(n_tiles * n_stages); i += blockDim.x)
+        for (int i = threadIdx.x; i < (int)n_tiles * n_stages; i += blockDim.x)
             sm->live_tab[i] = (unsigned char)live_of(i / n_stages, i % n_stages);
         __syncthreads();
         for (int t = threadIdx.x; t < (int)n_tiles; t += blockDim.x) {
-            unsigned any = 0;
-            for (int ks = 0; ks < n_stages; ++ks) any |= sm->live_tab[t * n_stages + ks];
-            sm->any_tab[t] = (unsigned char)any;
+            unsigned cnt = 0;
+            for (int ks = 0; ks < n_stages; ++ks) cnt += sm->live_tab[t * n_stages + ks] != 0;
+            sm->cnt_tab[t] = (unsigned short)cnt;
         }
     }
     tc_fence_before();
@@ -221,18 +235,40 @@ mwu_dense_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
                 if (++stage == D_STAGES) { stage = 0; phase ^= 1u; }
             }
         }
-    } else if (warp == 1 && rank == 0) {
-        // ---------------- MMA issuer (leader) ----------------
-        int stage = 0;
-        unsigned phase = 0;
-        bool ok = true, issued_any = false, ready = false;
+    } else if ((warp == 1 || warp == D_MMA_WARP_B) && rank == 0) {
+        // ---------------- MMA issuers (leader): warp 1 takes the even tiles, the other the odd ones ----------------
+        // A tcgen05.mma is accepted only shortly before the tensor pipe gets to it, so whatever the
+        // issuing thread does between two tiles (next tile's position, the accumulator hand-over, the
+        // first stage's barrier) leaves the pipe idle.  With two issuers each one does that work while
+        // the other one's MMAs run; each owns one accumulator buffer.  The issuer of tile k starts on
+        // its stages only once the issuer of tile k-1 has got past the barrier of its last stage (the
+        // hand-over word): a wait by parity is only meaningful within one phase of the barrier, and
+        // an issuer running a whole tile ahead could be two phases away from a slot's barrier.  The
+        // hand-over also carries the ring position, so nobody counts the other one's stages.
+        const unsigned mine = (warp == 1) ? 0u : 1u;
+        bool ok = true, issued_any = false;
         const unsigned idesc = make_idesc_pair(256);
+        volatile unsigned *ho_tiles = &sm->ho_tiles, *ho_ring = &sm->ho_ring;
         for (long long k = 0; ok && tile_of(k, mt_, nt_); ++k) {
+            if ((unsigned)(k & 1) != mine) continue;
             const long long nt = nt_;
-            const unsigned buf = (unsigned)(k & 1), use_phase = (unsigned)((k >> 1) & 1);
-            const unsigned char *lv = load_live(sm->live_mma, nt);
+            const unsigned buf = mine, use_phase = (unsigned)((k >> 1) & 1);
+            const unsigned char *lv = load_live(mine ? sm->live_mma_b : sm->live_mma, nt);
+            bool ready = false;
             if (!mbar_wait(smem_u32(&sm->tempty[buf]), use_phase ^ 1u, abort)) ok = false;
             if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
+            // the hand-over: tiles 0 .. k-1 have been issued
+            if (*ho_tiles != (unsigned)k) {
+                const long long t0 = clock64();
+                while (*ho_tiles != (unsigned)k) {
+                    if (*abort) { ok = false; break; }
+                    if (clock64() - t0 > WAIT_LIMIT_CYCLES) { *abort = 1; ok = false; break; }
+                }
+            }
+            if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
+            const unsigned ring = *ho_ring;                 // position in the ring of slots: 0 .. 2 * D_STAGES - 1
+            int stage = (int)(ring % D_STAGES);
+            unsigned phase = ring / D_STAGES;
             tc_fence_after();
             bool first = true;
             for (int ks = 0; ks < n_stages; ++ks) {
@@ -267,6 +303,11 @@ mwu_dense_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
                 if (++stage == D_STAGES) { stage = 0; phase ^= 1u; }
             }
             if (!ok) break;
+            if (lane == 0) {
+                *ho_ring = (unsigned)stage + phase * D_STAGES;
+                __threadfence_block();
+                *ho_tiles = (unsigned)(k + 1);
+            }
             if (elect_one()) {
                 if (!first) {
                     umma2_commit_both(smem_u32(&sm->tfull[buf]));
@@ -279,11 +320,11 @@ mwu_dense_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
         }
         // everything this thread issued must have retired before tensor memory is freed
         if (lane == 0 && issued_any) {
-            umma2_commit_local(smem_u32(&sm->drain));
-            mbar_wait(smem_u32(&sm->drain), 0, abort);
+            umma2_commit_local(smem_u32(&sm->drain[mine]));
+            mbar_wait(smem_u32(&sm->drain[mine]), 0, abort);
         }
         __syncwarp();
-    } else if (warp == 1) {
+    } else if (warp == 1 || warp == D_MMA_WARP_B) {
         // the peer's warp 1 only owns the tensor-memory allocation
     } else {
         // ---------------- epilogue: this CTA's 128 rows x 256 columns ----------------
@@ -295,7 +336,7 @@ mwu_dense_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
             const long long mt = mt_, nt = nt_;
             const unsigned buf = (unsigned)(k & 1), use_phase = (unsigned)((k >> 1) & 1);
             unsigned any = 0;
-            if (tab_ok) any = sm->any_tab[nt];
+            if (tab_ok) any = sm->cnt_tab[nt];
             else {
                 for (int ks = lane; ks < n_stages; ks += 32) any |= live_of(nt, ks);
                 any = __reduce_or_sync(0xffffffffu, any);
@@ -309,25 +350,40 @@ mwu_dense_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
             const long long ncol0 = nt * 256 + chalf * 128;
             if (p.y_tma) {
                 const long long mrow0 = m - lane;
-                for (int c0 = 0; c0 < 128; c0 += 64) {
-                    if (ncol0 + c0 >= p.N || mrow0 >= p.M) break;
-                    unsigned v0[32], v1[32];
-                    if (any) {
-                        tmem_ld32_issue(trow + (unsigned)c0, v0);
-                        tmem_ld32_issue(trow + (unsigned)(c0 + 32), v1);
-                        tmem_ld_wait(v0);
-                        tmem_ld_wait(v1);
-                    } else {
+                // All 128 columns go to registers first and the accumulator buffer is handed back at
+                // once: the hand-over to the leader's MMA issuers crosses to the other SM for one of
+                // the two CTAs, and that message queues behind this SM's outgoing store data, so the
+                // buffer should not also wait for the conversion and the stores.
+                unsigned v[4][32];
+                if (any) {
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) { v0[j] = 0u; v1[j] = 0u; }
-                    }
-                    // the previous store of this warp has read the staging buffer
-                    if (lane == 0) bulk_wait_read();
+                    for (int q = 0; q < 4; ++q) tmem_ld32_issue(trow + (unsigned)(32 * q), v[q]);
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) tmem_ld_wait(v[q]);
+                } else {
+#pragma unroll
+                    for (int q = 0; q < 4; ++q)
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) v[q][j] = 0u;
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) {
+                    if (rank == 0) mbar_arrive(smem_u32(&sm->tempty[buf]));
+                    else mbar_arrive_cluster(smem_u32(&sm->tempty[buf]), 0);
+                }
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const int c0 = 64 * h;
+                    if (ncol0 + c0 >= p.N || mrow0 >= p.M) break;
+                    unsigned char *sbuf = stg + (D_EPI_BUFS == 2 ? h * 4096 : 0);
+                    // the last store out of this buffer has read it
+                    if (lane == 0) { if (D_EPI_BUFS == 2) bulk_wait_read_1(); else bulk_wait_read(); }
                     __syncwarp();
                     // row `lane`: eight 16-byte pieces, piece j at position j ^ (lane % 8) (128-byte swizzle)
 #pragma unroll
                     for (int j = 0; j < 8; ++j) {
-                        const unsigned *src = (j < 4) ? (v0 + 8 * j) : (v1 + 8 * (j - 4));
+                        const unsigned *src = (j < 4) ? (v[2 * h] + 8 * j) : (v[2 * h + 1] + 8 * (j - 4));
                         uint4 o;
                         __nv_bfloat162 h2;
                         h2 = __floats2bfloat162_rn(__uint_as_float(src[0]), __uint_as_float(src[1]));
@@ -338,15 +394,16 @@ mwu_dense_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
                         o.z = *reinterpret_cast<unsigned *>(&h2);
                         h2 = __floats2bfloat162_rn(__uint_as_float(src[6]), __uint_as_float(src[7]));
                         o.w = *reinterpret_cast<unsigned *>(&h2);
-                        *reinterpret_cast<uint4 *>(stg + lane * 128 + ((j ^ (lane & 7)) << 4)) = o;
+                        *reinterpret_cast<uint4 *>(sbuf + lane * 128 + ((j ^ (lane & 7)) << 4)) = o;
                     }
                     fence_proxy_async();
                     __syncwarp();
                     if (lane == 0) {
-                        tma_store_2d(&tmap_y, smem_u32(stg), (int)(ncol0 + c0), (int)mrow0);
+                        tma_store_2d(&tmap_y, smem_u32(sbuf), (int)(ncol0 + c0), (int)mrow0);
                         bulk_commit();
                     }
                 }
+                continue;                                   // the buffer went back above
             } else {
             for (int c0 = 0; c0 < 128; c0 += 32) {
                 if (ncol0 + c0 >= p.N) break;
@@ -394,6 +451,7 @@ cudaError_t launch_dense(const CUtensorMap &tmap_x, const CUtensorMap &tmap_w, c
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     const long long tiles = ((p.M + 255) / 256) * ((p.n_rec_tiles + 1) / 2);
+    if (tiles >= (1ll << 31)) return cudaErrorInvalidValue;
     long long pairs = sm_count / 2;
     if (tiles < pairs) pairs = tiles;
     cudaLaunchConfig_t cfg = {};

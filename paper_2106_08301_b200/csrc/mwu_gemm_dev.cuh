@@ -112,24 +112,24 @@ __device__ __forceinline__ bool mbar_test(unsigned bar, unsigned parity) {
 }
 // bounded wait: false when aborted or out of time (then *abort is set)
 __device__ __forceinline__ bool mbar_wait(unsigned bar, unsigned parity, volatile int *abort) {
-    if (mbar_test(bar, parity)) return true;
+    // Polling, not a suspended try_wait: a waiter that went to sleep on a barrier which the OTHER CTA
+    // of the pair completes (a multicast commit, a remote arrive) was seen to wake a microsecond or
+    // two late, which serialised the pair's epilogue with the next tile's MMAs.
 #pragma unroll 1
-    for (int i = 0; i < 128; ++i)
-        if (mbar_try_wait(bar, parity)) return true;
+    for (int i = 0; i < 4096; ++i)
+        if (mbar_test(bar, parity)) return true;
     const long long t0 = clock64();
 #pragma unroll 1
     while (true) {
-        if (mbar_try_wait(bar, parity)) return true;
+#pragma unroll 1
+        for (int i = 0; i < 64; ++i)
+            if (mbar_test(bar, parity)) return true;
         if (*abort) return false;
         if (clock64() - t0 > WAIT_LIMIT_CYCLES) { *abort = 1; return false; }
     }
 }
-// the same for a single latency-critical thread: probe in a tight loop first (a suspended try_wait
-// wakes up a few hundred cycles late), then fall back to the bounded wait
+// kept as a name of its own where a single latency-critical thread waits
 __device__ __forceinline__ bool mbar_wait_spin(unsigned bar, unsigned parity, volatile int *abort) {
-#pragma unroll 1
-    for (int i = 0; i < 2048; ++i)
-        if (mbar_test(bar, parity)) return true;
     return mbar_wait(bar, parity, abort);
 }
 template <int BYTES>
@@ -215,6 +215,8 @@ __device__ __forceinline__ void tma_store_2d(const CUtensorMap *map, unsigned sr
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 // the issuing thread's earlier bulk stores have read their shared-memory source
 __device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+// ... all but the latest one have
+__device__ __forceinline__ void bulk_wait_read_1() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
 // ... and have completed
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 
