@@ -88,7 +88,7 @@ cudaError_t launch_decode(int bw, const Params &p, __nv_bfloat16 *Wd, long long 
 // ------------------------------------------------------------------------------------------
 // two-operand GEMM over the decoded weights
 // ------------------------------------------------------------------------------------------
-constexpr int D_STAGES = 5;
+constexpr int D_STAGES = 6;
 constexpr int D_EPI_WARPS = 8;
 constexpr int D_MMA_WARP_B = 2 + D_EPI_WARPS;        // the second MMA issuer (the first is warp 1)
 constexpr int D_THREADS = 32 * (3 + D_EPI_WARPS);
@@ -96,7 +96,7 @@ constexpr int D_A_BYTES = AH_BYTES;                  // this CTA's 128 activatio
 constexpr int D_B_BYTES = REC_BYTES;                 // this CTA's 128 weight rows
 constexpr int D_STAGE_BYTES = D_A_BYTES + D_B_BYTES;
 constexpr int D_BAND = 8;                            // activation row tiles per band of the tile order
-constexpr int D_EPI_BUFS = 2;                        // staging buffers per epilogue warp
+constexpr int D_EPI_BUFS = 1;                        // staging buffers per epilogue warp (2 with one slot fewer measured no faster)
 constexpr int D_EPI_BYTES = 4096 * D_EPI_BUFS;       // each buffer: 32 rows x 64 bf16 columns
 
 constexpr int D_LIVE_TAB = 512;                      // live masks of all weight tiles, when they fit (short reductions)

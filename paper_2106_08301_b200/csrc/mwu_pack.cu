@@ -2,13 +2,16 @@
 // magnitude per unified block, nothing but its position for a pruned block, one sign bit per
 // weight of a unified block, bf16 values for the rest), arranged per GEMM tile.
 //
-//   count_kernel  one CTA per record (128 rows x 64 columns): number of unified / dense / pruned
-//                 blocks and the record's live-slice mask.
-//   scan_kernel   one CTA: exclusive scan of the per-record counts over all records, header.
-//   fill_kernel   one CTA per record, one thread per row: class masks, then a scan over the rows
-//                 of the number of blocks per (class, store slot), which gives every block its
-//                 place in the round-robin order of its class list; a dense block's values are
-//                 read as whole 64-byte (or shorter) runs of W and written as one bf16 vector.
+//   count_kernel  one CTA per tile of 128 rows, a lane per record (128 rows x 64 columns) walking the
+//                 rows: number of unified / dense / pruned blocks and the record's live-slice mask.
+//   scan_kernel   one CTA: exclusive scan of the per-record counts over all records (1024 records
+//                 at a time, read and written as whole lines), header.
+//   fill_kernel   one CTA per record.  First one thread per row: class masks, then a scan over the
+//                 rows of the number of blocks per (class, store slot), which gives every block its
+//                 place in the round-robin order of its class list; the places go to shared memory.
+//                 Then the lists leave in list order, consecutive threads writing consecutive
+//                 entries; a dense block's values are read by the lanes that share its 64-byte run.
+// The three are chained with programmatic stream serialization.
 #include "mwu_common.cuh"
 
 namespace mwu {
@@ -56,11 +59,20 @@ __device__ __forceinline__ unsigned tile_offset(unsigned r, unsigned i, int b) {
     return (r >> 3) * 1024u + (r & 7u) * 128u + ((c ^ (r & 7u)) << 4) + within;
 }
 
-// sign bits of one block (bit l = weight l) -> bit l/2 + 16 * (l % 2)
+// sign bits of one block (bit l = weight l) -> bit l/2 + 16 * (l % 2): the even bits closed up in the
+// low half, the odd bits in the high half
+__device__ __forceinline__ unsigned close_up_even_bits(unsigned x) {
+    x &= 0x55555555u;
+    x = (x | (x >> 1)) & 0x33333333u;
+    x = (x | (x >> 2)) & 0x0f0f0f0fu;
+    x = (x | (x >> 4)) & 0x00ff00ffu;
+    x = (x | (x >> 8)) & 0x0000ffffu;
+    return x;
+}
 __device__ __forceinline__ unsigned spread_signs(unsigned sb, int b) {
-    unsigned out = 0;
-    for (int l = 0; l < b; ++l) out |= ((sb >> l) & 1u) << (l / 2 + 16 * (l & 1));
-    return out;
+    const unsigned m = (b >= 32) ? 0xffffffffu : ((1u << b) - 1u);
+    sb &= m;
+    return close_up_even_bits(sb) | (close_up_even_bits(sb >> 1) << 16);
 }
 
 __device__ __forceinline__ unsigned live_of(unsigned P, int b) {
@@ -76,96 +88,109 @@ __device__ __forceinline__ unsigned live_of(unsigned P, int b) {
     return live;
 }
 
-__global__ void __launch_bounds__(128) count_kernel(Params p) {
-    const int r = threadIdx.x;
-    const long long rec = blockIdx.x;
-    const long long tile = rec / p.L.n_stages, stage = rec % p.L.n_stages;
+constexpr int COUNT_WARPS = 16;                         // each takes 8 of the tile's 128 rows
+
+__global__ void __launch_bounds__(32 * COUNT_WARPS) count_kernel(Params p) {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const long long chunks = (p.L.n_stages + 31) / 32;      // 32 records of a tile at a time: lane = record (stage)
+    const long long tile = blockIdx.x / chunks;
+    const long long stage = (blockIdx.x % chunks) * 32 + lane;
     const int nb = kStageK / p.b;
-    unsigned P, U;
-    unsigned long long sgn;
-    row_masks(p, tile, stage, r, &P, &U, &sgn);
-    unsigned cu = __popc(U), cp = __popc(P);
-    unsigned live = live_of(P, p.b);
-    for (int m = 16; m > 0; m >>= 1) {
-        cu += __shfl_xor_sync(0xffffffffu, cu, m);
-        cp += __shfl_xor_sync(0xffffffffu, cp, m);
-        live |= __shfl_xor_sync(0xffffffffu, live, m);
+    const unsigned mask = (nb >= 32) ? 0xffffffffu : ((1u << nb) - 1u);
+    const long long bpr = p.cols / p.b;                     // blocks per row
+    constexpr int RPW = kTileRows / COUNT_WARPS;
+    __shared__ unsigned s_cu[COUNT_WARPS][32], s_cp[COUNT_WARPS][32], s_live[COUNT_WARPS][32];
+    unsigned cu = 0, cp = 0, live = 0;
+    if (stage < p.L.n_stages) {
+        unsigned P[RPW], U[RPW];
+#pragma unroll
+        for (int rr = 0; rr < RPW; ++rr) {                  // all of the warp's loads are in flight together
+            const long long n = tile * kTileRows + warp * RPW + rr;
+            P[rr] = 0xffffffffu;                            // padding rows are all-pruned
+            U[rr] = 0;
+            if (n < p.rows) {
+                const long long j0 = n * bpr + stage * nb;
+                P[rr] = __ldg(p.pruned_bitmap + (j0 >> 5)) >> (j0 & 31);
+                U[rr] = __ldg(p.unified_bitmap + (j0 >> 5)) >> (j0 & 31);
+            }
+        }
+#pragma unroll
+        for (int rr = 0; rr < RPW; ++rr) {
+            const unsigned Pm = P[rr] & mask;
+            cu += __popc(U[rr] & mask & ~Pm);
+            cp += __popc(Pm);
+            live |= live_of(Pm, p.b);
+        }
     }
-    __shared__ unsigned s_cu[4], s_cp[4], s_live[4];
-    if ((r & 31) == 0) { s_cu[r >> 5] = cu; s_cp[r >> 5] = cp; s_live[r >> 5] = live; }
+    s_cu[warp][lane] = cu; s_cp[warp][lane] = cp; s_live[warp][lane] = live;
     __syncthreads();
-    if (r == 0) {
-        const unsigned tu = s_cu[0] + s_cu[1] + s_cu[2] + s_cu[3];
-        const unsigned tp = s_cp[0] + s_cp[1] + s_cp[2] + s_cp[3];
-        PackedRec *recs = reinterpret_cast<PackedRec *>(p.packed + p.L.off_rec);
-        recs[rec].ubase = tu;                         // counts for now; scan_kernel makes bases
-        recs[rec].dbase = kTileRows * nb - tu - tp;
-        recs[rec].pbase = tp;
-        recs[rec].live = s_live[0] | s_live[1] | s_live[2] | s_live[3];
+    if (warp == 0 && stage < p.L.n_stages) {
+        unsigned tu = 0, tp = 0, tl = 0;
+#pragma unroll
+        for (int w = 0; w < COUNT_WARPS; ++w) { tu += s_cu[w][lane]; tp += s_cp[w][lane]; tl |= s_live[w][lane]; }
+        // counts for now (ubase, dbase, pbase, live); scan_kernel makes bases
+        uint4 *recs = reinterpret_cast<uint4 *>(p.packed + p.L.off_rec);
+        recs[tile * p.L.n_stages + stage] = make_uint4(tu, (unsigned)(kTileRows * nb) - tu - tp, tp, tl);
     }
 }
 
 __global__ void __launch_bounds__(1024) scan_kernel(Params p) {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const long long n_rec = p.L.n_tiles * p.L.n_stages;
     uint4 *recs = reinterpret_cast<uint4 *>(p.packed + p.L.off_rec);     // ubase, dbase, pbase, live
-    __shared__ unsigned long long s_u[64], s_d[64], s_p[64];
-    const long long per = (n_rec + 1023) / 1024;
-    const long long lo = threadIdx.x * per;
-    const long long hi = (lo + per < n_rec) ? lo + per : n_rec;
-    constexpr int KEEP = 8;                                 // records held in registers
-    uint4 held[KEEP];
-    unsigned long long su = 0, sd = 0, sp = 0;
-#pragma unroll
-    for (int k = 0; k < KEEP; ++k) {
-        held[k] = make_uint4(0, 0, 0, 0);
-        if (lo + k < hi) held[k] = recs[lo + k];
-        su += held[k].x; sd += held[k].y; sp += held[k].z;
-    }
-    for (long long i = lo + KEEP; i < hi; ++i) { const uint4 v = recs[i]; su += v.x; sd += v.y; sp += v.z; }
-    // inclusive scan over the 1024 threads: shuffles inside a warp, then the 32 warp totals
-    unsigned long long iu = su, id = sd, ip = sp;
+    __shared__ unsigned s_w[3][32];
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    asm volatile("griddepcontrol.wait;" ::: "memory");      // the counts are complete and visible
+    unsigned long long cu = 0, cd = 0, cp = 0;              // totals of the chunks before this one
+    constexpr int PER = 4;                                  // consecutive records per thread; a chunk is 4096 records
+    for (long long g0 = 0; g0 < n_rec; g0 += PER * 1024) {
+        const long long i0 = g0 + (long long)threadIdx.x * PER;
+        uint4 held[PER];
+        unsigned su = 0, sd = 0, sp = 0;                    // a chunk's counts fit 32 bits (at most 4096 blocks a record)
 #pragma unroll
-    for (int off = 1; off < 32; off <<= 1) {
-        const unsigned long long au = __shfl_up_sync(0xffffffffu, iu, off);
-        const unsigned long long ad = __shfl_up_sync(0xffffffffu, id, off);
-        const unsigned long long ap = __shfl_up_sync(0xffffffffu, ip, off);
-        if (lane >= off) { iu += au; id += ad; ip += ap; }
-    }
-    if (lane == 31) { s_u[wid] = iu; s_d[wid] = id; s_p[wid] = ip; }
-    __syncthreads();
-    if (wid == 0) {
-        unsigned long long wu = s_u[lane], wd = s_d[lane], wp = s_p[lane];
+        for (int k = 0; k < PER; ++k) {
+            held[k] = (i0 + k < n_rec) ? recs[i0 + k] : make_uint4(0, 0, 0, 0);
+            su += held[k].x; sd += held[k].y; sp += held[k].z;
+        }
+        // inclusive scan of the thread sums: inside a warp, then over the 32 warp totals
+        unsigned iu = su, id = sd, ip = sp;
 #pragma unroll
         for (int off = 1; off < 32; off <<= 1) {
-            const unsigned long long au = __shfl_up_sync(0xffffffffu, wu, off);
-            const unsigned long long ad = __shfl_up_sync(0xffffffffu, wd, off);
-            const unsigned long long ap = __shfl_up_sync(0xffffffffu, wp, off);
+            const unsigned au = __shfl_up_sync(0xffffffffu, iu, off);
+            const unsigned ad = __shfl_up_sync(0xffffffffu, id, off);
+            const unsigned ap = __shfl_up_sync(0xffffffffu, ip, off);
+            if (lane >= off) { iu += au; id += ad; ip += ap; }
+        }
+        __syncthreads();                                    // the previous chunk's warp totals have been read
+        if (lane == 31) { s_w[0][wid] = iu; s_w[1][wid] = id; s_w[2][wid] = ip; }
+        __syncthreads();
+        unsigned wu = s_w[0][lane], wd = s_w[1][lane], wp = s_w[2][lane];     // every warp scans the 32 totals
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const unsigned au = __shfl_up_sync(0xffffffffu, wu, off);
+            const unsigned ad = __shfl_up_sync(0xffffffffu, wd, off);
+            const unsigned ap = __shfl_up_sync(0xffffffffu, wp, off);
             if (lane >= off) { wu += au; wd += ad; wp += ap; }
         }
-        s_u[32 + lane] = wu; s_d[32 + lane] = wd; s_p[32 + lane] = wp;     // inclusive warp totals
-    }
-    __syncthreads();
-    if (wid > 0) { iu += s_u[32 + wid - 1]; id += s_d[32 + wid - 1]; ip += s_p[32 + wid - 1]; }
-    unsigned long long ru = iu - su, rd = id - sd, rp = ip - sp;
+        const unsigned tu = __shfl_sync(0xffffffffu, wu, 31), td = __shfl_sync(0xffffffffu, wd, 31),
+                       tp = __shfl_sync(0xffffffffu, wp, 31);
+        const unsigned bu = __shfl_sync(0xffffffffu, wu - s_w[0][lane], wid);  // totals of the warps before this one
+        const unsigned bd = __shfl_sync(0xffffffffu, wd - s_w[1][lane], wid);
+        const unsigned bp = __shfl_sync(0xffffffffu, wp - s_w[2][lane], wid);
+        unsigned long long ru = cu + bu + (iu - su), rd = cd + bd + (id - sd), rp = cp + bp + (ip - sp);
 #pragma unroll
-    for (int k = 0; k < KEEP; ++k) {
-        if (lo + k < hi) {
-            recs[lo + k] = make_uint4((unsigned)ru, (unsigned)rd, (unsigned)rp, held[k].w);
+        for (int k = 0; k < PER; ++k) {
+            if (i0 + k < n_rec) recs[i0 + k] = make_uint4((unsigned)ru, (unsigned)rd, (unsigned)rp, held[k].w);
             ru += held[k].x; rd += held[k].y; rp += held[k].z;
         }
-    }
-    for (long long i = lo + KEEP; i < hi; ++i) {
-        const uint4 v = recs[i];
-        recs[i] = make_uint4((unsigned)ru, (unsigned)rd, (unsigned)rp, v.w);
-        ru += v.x; rd += v.y; rp += v.z;
+        cu += tu; cd += td; cp += tp;
     }
     if (threadIdx.x == 1023) {
-        const unsigned long long tu = iu, td = id, tp = ip;
-        if (tu != (unsigned long long)p.L.n_unified || td != (unsigned long long)p.L.n_dense ||
-            tp != (unsigned long long)p.L.n_plist)
+        if (cu != (unsigned long long)p.L.n_unified || cd != (unsigned long long)p.L.n_dense ||
+            cp != (unsigned long long)p.L.n_plist)
             atomicOr(p.dev_status, (unsigned)MWU_DEV_BOUNDS);
-        recs[n_rec] = make_uint4((unsigned)tu, (unsigned)td, (unsigned)tp, 0u);
+        recs[n_rec] = make_uint4((unsigned)cu, (unsigned)cd, (unsigned)cp, 0u);
     }
     // the padding between the sections must read as zero (each gap is shorter than the alignment)
     for (int g = 0; g < 5; ++g)
@@ -198,144 +223,152 @@ __global__ void __launch_bounds__(1024) scan_kernel(Params p) {
     }
 }
 
+// row and block of a tile offset (the inverse of tile_offset)
+__device__ __forceinline__ void row_block_of(unsigned off, int b, unsigned *r, unsigned *i) {
+    const unsigned rr = (off >> 10) * 8u + ((off >> 7) & 7u);
+    const unsigned c = ((off >> 4) & 7u) ^ (rr & 7u);
+    *r = rr;
+    *i = (c * 16u + (off & 15u)) / (2u * (unsigned)b);
+}
+
 template <int B>
 __global__ void __launch_bounds__(128) fill_kernel(Params p) {
     constexpr int NBK = kStageK / B;
     constexpr unsigned MASK = (NBK >= 32) ? 0xffffffffu : ((1u << NBK) - 1u);
     constexpr int STORE = (B >= 8) ? 16 : 2 * B;            // bytes of one shared-memory store
     constexpr int G = 128 / STORE;                          // store slots of a 128-byte row
-    constexpr int NF = 3 * G;                               // (class, slot) counters, 8 bits each
-    constexpr int FW = NF / 4;                              // ... packed four to a word
+    constexpr int LPB = (B >= 4) ? B / 4 : 1;               // lanes that share a dense block's run of W
     const long long rec = blockIdx.x;
     const long long tile = rec / p.L.n_stages, stage = rec % p.L.n_stages;
     const int r = threadIdx.x, lane = r & 31, warp = r >> 5;
-    const PackedRec *recs = reinterpret_cast<const PackedRec *>(p.packed + p.L.off_rec);
+    const uint4 *recs = reinterpret_cast<const uint4 *>(p.packed + p.L.off_rec);
     uint2 *ulist = reinterpret_cast<uint2 *>(p.packed + p.L.off_ulist);
     unsigned short *dpos = reinterpret_cast<unsigned short *>(p.packed + p.L.off_dpos);
     unsigned char *dpay = p.packed + p.L.off_dpay;
     unsigned short *ppos = reinterpret_cast<unsigned short *>(p.packed + p.L.off_ppos);
-    const unsigned long long base_of[3] = {recs[rec].pbase, recs[rec].dbase, recs[rec].ubase};
 
-    __shared__ unsigned s_warp[4][FW];
-    __shared__ unsigned char s_len[NF];                     // blocks per (class, slot) in the record
+    __shared__ unsigned s_bal[4][3 * G];                    // per warp and (class, slot): the rows that have such a block
+    __shared__ unsigned short s_full[3][kTileRows + 1];     // per class and q: list entries of rounds 0 .. q-1
+    __shared__ unsigned s_more[3][kTileRows + 1];           // per class and q: slots that have a round q
+    __shared__ unsigned short s_off[3][kTileRows * NBK];    // tile offsets of each class list, in list order
     unsigned P, U;
     unsigned long long sgn;
     row_masks(p, tile, stage, r, &P, &U, &sgn);
     const unsigned D = ~P & ~U & MASK;
-    // class of block i: 0 pruned, 1 dense, 2 unified; its store slot
-    unsigned fld[FW];
-#pragma unroll
-    for (int w = 0; w < FW; ++w) fld[w] = 0;
+    // class of block i: 0 pruned, 1 dense, 2 unified.  occ[class]: the store slots this row fills with it
+    // (a row never has two blocks in one slot)
+    unsigned occ[3] = {0u, 0u, 0u};
 #pragma unroll
     for (int i = 0; i < NBK; ++i) {
-        const unsigned off = tile_offset((unsigned)r, (unsigned)i, B);
-        const unsigned slot = (off & 127u) / STORE;
-        const unsigned cls = ((U >> i) & 1u) ? 2u : (((D >> i) & 1u) ? 1u : 0u);
-        const unsigned fi = cls * G + slot;
-#pragma unroll
-        for (int w = 0; w < FW; ++w) fld[w] += ((fi >> 2) == (unsigned)w) ? (1u << (8 * (fi & 3u))) : 0u;
+        const unsigned slot = (tile_offset((unsigned)r, (unsigned)i, B) & 127u) / STORE;
+        const unsigned bit = 1u << slot;
+        occ[0] |= ((P >> i) & 1u) ? bit : 0u;
+        occ[1] |= ((D >> i) & 1u) ? bit : 0u;
+        occ[2] |= ((U >> i) & 1u) ? bit : 0u;
     }
-    // inclusive scan over the 128 rows (a field never exceeds 128, so fields do not carry)
-    unsigned inc[FW];
 #pragma unroll
-    for (int w = 0; w < FW; ++w) inc[w] = fld[w];
-    for (int off = 1; off < 32; off <<= 1) {
+    for (int c = 0; c < 3; ++c) {
 #pragma unroll
-        for (int w = 0; w < FW; ++w) {
-            const unsigned t = __shfl_up_sync(0xffffffffu, inc[w], off);
-            if (lane >= off) inc[w] += t;
+        for (int sl = 0; sl < G; ++sl) {
+            const unsigned bal = __ballot_sync(0xffffffffu, (occ[c] >> sl) & 1u);
+            if (lane == ((c * G + sl) & 31)) s_bal[warp][c * G + sl] = bal;
         }
     }
-    if (lane == 31) {
-#pragma unroll
-        for (int w = 0; w < FW; ++w) s_warp[warp][w] = inc[w];
-    }
     __syncthreads();
-    unsigned excl[FW];
+    // round-robin order of a class list: round q takes the q-th block of every slot that has one.
+    // Thread q (and thread 0 for q = 128) tabulates what comes before round q.
+    for (int q = r; q <= kTileRows; q += kTileRows) {
 #pragma unroll
-    for (int w = 0; w < FW; ++w) {
-        unsigned b0 = 0;
-        for (int ww = 0; ww < warp; ++ww) b0 += s_warp[ww][w];
-        excl[w] = b0 + inc[w] - fld[w];
-    }
-    if (r < NF) {
-        const unsigned tot = s_warp[0][r >> 2] + s_warp[1][r >> 2] + s_warp[2][r >> 2] + s_warp[3][r >> 2];
-        s_len[r] = (unsigned char)((tot >> (8 * (r & 3))) & 0xffu);
+        for (int c = 0; c < 3; ++c) {
+            unsigned full = 0, more = 0;
+#pragma unroll
+            for (int sl = 0; sl < G; ++sl) {
+                const unsigned len = __popc(s_bal[0][c * G + sl]) + __popc(s_bal[1][c * G + sl]) +
+                                     __popc(s_bal[2][c * G + sl]) + __popc(s_bal[3][c * G + sl]);
+                full += len < (unsigned)q ? len : (unsigned)q;
+                more |= (len > (unsigned)q) ? (1u << sl) : 0u;
+            }
+            s_full[c][q] = (unsigned short)full;
+            s_more[c][q] = more;
+        }
     }
     __syncthreads();
 
-    bool bad = false;
-    const long long n = tile * kTileRows + r;
-    constexpr unsigned BMASK = (B >= 32) ? 0xffffffffu : ((1u << B) - 1u);
+    // every block's place in its class list
+    const unsigned below = (1u << lane) - 1u;
 #pragma unroll 4
     for (int i = 0; i < NBK; ++i) {
         const unsigned off = tile_offset((unsigned)r, (unsigned)i, B);
         const unsigned slot = (off & 127u) / STORE;
         const unsigned cls = ((U >> i) & 1u) ? 2u : (((D >> i) & 1u) ? 1u : 0u);
-        const unsigned fi = cls * G + slot;
-        unsigned q = 0;                                     // earlier rows with the same class and slot
-#pragma unroll
-        for (int w = 0; w < FW; ++w) q += ((fi >> 2) == (unsigned)w) ? ((excl[w] >> (8 * (fi & 3u))) & 0xffu) : 0u;
-        // place in the round-robin order: q full rounds before it, then the lower slots of its round
-        unsigned idx = 0;
-#pragma unroll
-        for (int sl = 0; sl < G; ++sl) {
-            const unsigned len = s_len[cls * G + sl];
-            idx += (len < q ? len : q) + (((unsigned)sl < slot && len > q) ? 1u : 0u);
+        const unsigned f = cls * G + slot;
+        unsigned q = __popc(s_bal[warp][f] & below);        // earlier rows with the same class and slot
+        for (int ww = 0; ww < warp; ++ww) q += __popc(s_bal[ww][f]);
+        // q full rounds before it, then the lower slots of its own round
+        const unsigned idx = s_full[cls][q] + __popc(s_more[cls][q] & ((1u << slot) - 1u));
+        s_off[cls][idx] = (unsigned short)off;
+    }
+    asm volatile("griddepcontrol.wait;" ::: "memory");      // the record table holds the bases
+    const uint4 me = recs[rec], nx = recs[rec + 1];         // (ubase, dbase, pbase, live); the table ends with the totals
+    __syncthreads();
+
+    bool bad = false;
+    constexpr unsigned BMASK = (B >= 32) ? 0xffffffffu : ((1u << B) - 1u);
+    const unsigned len_u = nx.x - me.x, len_d = nx.y - me.y, len_p = nx.z - me.z;
+    if (len_u + len_d + len_p != (unsigned)(kTileRows * NBK)) bad = true;     // the table does not describe this record
+    else {
+        // pruned blocks: positions only
+        for (unsigned t = (unsigned)r; t < len_p; t += 128u) {
+            const unsigned long long e = (unsigned long long)me.z + t;
+            if (e < (unsigned long long)p.L.n_plist) ppos[e] = s_off[0][t];
+            else bad = true;
         }
-        const unsigned long long e = base_of[cls] + idx;
-        if (cls == 2u) {
-            const unsigned sb = (unsigned)(sgn >> (i * B)) & BMASK;
+        // unified blocks: sign bits, position, magnitude
+        for (unsigned t = (unsigned)r; t < len_u; t += 128u) {
+            const unsigned long long e = (unsigned long long)me.x + t;
+            const unsigned off = s_off[2][t];
+            unsigned rr, i;
+            row_block_of(off, B, &rr, &i);
+            const long long n = tile * kTileRows + rr;
+            const long long f = n * p.cols + stage * kStageK + (long long)i * B;
+            const unsigned sb = (__ldg(p.sign_bits + (f >> 5)) >> (f & 31)) & BMASK;
             const long long j = n * (p.cols / B) + stage * NBK + i;
             const unsigned ub = (unsigned)__bfloat16_as_ushort(__float2bfloat16_rn(__ldg(p.u + j)));
             if (e < (unsigned long long)p.L.n_unified) ulist[e] = make_uint2(spread_signs(sb, B), off | (ub << 16));
             else bad = true;
-        } else if (cls == 1u) {
-            if (e < (unsigned long long)p.L.n_dense) {
-                dpos[e] = (unsigned short)off;
-                const long long f = n * p.cols + stage * kStageK + i * B;
-                float v[B];
-                if (B >= 4) {
-#pragma unroll
-                    for (int l = 0; l < B; l += 4) {
-                        float4 a = __ldg(reinterpret_cast<const float4 *>(p.W + f + l));
-                        if (p.U) {
-                            const float4 d = __ldg(reinterpret_cast<const float4 *>(p.U + f + l));
-                            a.x = __fadd_rn(a.x, d.x); a.y = __fadd_rn(a.y, d.y); a.z = __fadd_rn(a.z, d.z); a.w = __fadd_rn(a.w, d.w);
-                        }
-                        v[l] = a.x; v[(l + 1) % B] = a.y; v[(l + 2) % B] = a.z; v[(l + 3) % B] = a.w;
-                    }
-                } else {
-                    float2 a = __ldg(reinterpret_cast<const float2 *>(p.W + f));
-                    if (p.U) {
-                        const float2 d = __ldg(reinterpret_cast<const float2 *>(p.U + f));
-                        a.x = __fadd_rn(a.x, d.x); a.y = __fadd_rn(a.y, d.y);
-                    }
-                    v[0] = a.x; v[1 % B] = a.y;
-                }
-                unsigned w[B / 2];
-#pragma unroll
-                for (int l = 0; l < B / 2; ++l) {
-                    const __nv_bfloat162 h = __floats2bfloat162_rn(v[2 * l], v[2 * l + 1]);
-                    w[l] = *reinterpret_cast<const unsigned *>(&h);
-                }
-                unsigned char *dst = dpay + e * (2 * B);
-                if (B == 16) {
-                    *reinterpret_cast<uint4 *>(dst) = make_uint4(w[0], w[1 % (B / 2)], w[2 % (B / 2)], w[3 % (B / 2)]);
-                    *reinterpret_cast<uint4 *>(dst + 16) = make_uint4(w[4 % (B / 2)], w[5 % (B / 2)], w[6 % (B / 2)], w[7 % (B / 2)]);
-                } else if (B == 8) {
-                    *reinterpret_cast<uint4 *>(dst) = make_uint4(w[0], w[1 % (B / 2)], w[2 % (B / 2)], w[3 % (B / 2)]);
-                } else if (B == 4) {
-                    *reinterpret_cast<uint2 *>(dst) = make_uint2(w[0], w[1 % (B / 2)]);
-                } else {
-                    *reinterpret_cast<unsigned *>(dst) = w[0];
-                }
-            } else {
-                bad = true;
-            }
-        } else {
-            if (e < (unsigned long long)p.L.n_plist) ppos[e] = (unsigned short)off;
+        }
+        // dense blocks: position, then the values, LPB lanes to a block
+        for (unsigned t = (unsigned)r; t < len_d; t += 128u) {
+            const unsigned long long e = (unsigned long long)me.y + t;
+            if (e < (unsigned long long)p.L.n_dense) dpos[e] = s_off[1][t];
             else bad = true;
+        }
+        for (unsigned q = (unsigned)r; q < len_d * (unsigned)LPB; q += 128u) {
+            const unsigned t = q / (unsigned)LPB, part = q % (unsigned)LPB;
+            const unsigned long long e = (unsigned long long)me.y + t;
+            if (e >= (unsigned long long)p.L.n_dense) continue;                  // flagged above
+            unsigned rr, i;
+            row_block_of(s_off[1][t], B, &rr, &i);
+            const long long f = (tile * kTileRows + rr) * p.cols + stage * kStageK + (long long)i * B + part * 4;
+            unsigned char *dst = dpay + e * (2 * B) + part * 8;
+            if (B >= 4) {
+                float4 a = __ldg(reinterpret_cast<const float4 *>(p.W + f));
+                if (p.U) {
+                    const float4 d = __ldg(reinterpret_cast<const float4 *>(p.U + f));
+                    a.x = __fadd_rn(a.x, d.x); a.y = __fadd_rn(a.y, d.y); a.z = __fadd_rn(a.z, d.z); a.w = __fadd_rn(a.w, d.w);
+                }
+                const __nv_bfloat162 h0 = __floats2bfloat162_rn(a.x, a.y), h1 = __floats2bfloat162_rn(a.z, a.w);
+                *reinterpret_cast<uint2 *>(dst) = make_uint2(*reinterpret_cast<const unsigned *>(&h0),
+                                                             *reinterpret_cast<const unsigned *>(&h1));
+            } else {
+                float2 a = __ldg(reinterpret_cast<const float2 *>(p.W + f));
+                if (p.U) {
+                    const float2 d = __ldg(reinterpret_cast<const float2 *>(p.U + f));
+                    a.x = __fadd_rn(a.x, d.x); a.y = __fadd_rn(a.y, d.y);
+                }
+                const __nv_bfloat162 h0 = __floats2bfloat162_rn(a.x, a.y);
+                *reinterpret_cast<unsigned *>(dst) = *reinterpret_cast<const unsigned *>(&h0);
+            }
         }
     }
     if (bad) atomicOr(p.dev_status, (unsigned)MWU_DEV_BOUNDS);
@@ -393,14 +426,30 @@ extern "C" int mwu_pack(const mwu_proj_desc *desc, const float *W, const float *
         {p.L.off_dpay + 2 * (size_t)desc->block * p.L.n_dense, p.L.off_ppos},
         {p.L.off_ppos + 2 * (size_t)p.L.n_plist, p.L.total}};
     for (int g = 0; g < 5; ++g) { p.gap[g][0] = gaps[g][0]; p.gap[g][1] = gaps[g][1] > gaps[g][0] ? gaps[g][1] : gaps[g][0]; }
-    pack::count_kernel<<<(unsigned)n_rec, 128, 0, st>>>(p);
-    pack::scan_kernel<<<1, 1024, 0, st>>>(p);
-    switch (desc->block) {
-        case 2: pack::fill_kernel<2><<<(unsigned)n_rec, 128, 0, st>>>(p); break;
-        case 4: pack::fill_kernel<4><<<(unsigned)n_rec, 128, 0, st>>>(p); break;
-        case 8: pack::fill_kernel<8><<<(unsigned)n_rec, 128, 0, st>>>(p); break;
-        default: pack::fill_kernel<16><<<(unsigned)n_rec, 128, 0, st>>>(p); break;
+    pack::count_kernel<<<(unsigned)(p.L.n_tiles * ((p.L.n_stages + 31) / 32)), 32 * pack::COUNT_WARPS, 0, st>>>(p);
+    // the next two start while their predecessor drains (programmatic stream serialization) and wait
+    // for its memory themselves
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.stream = st;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cfg.gridDim = dim3(1);
+    cfg.blockDim = dim3(1024);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, pack::scan_kernel, p);
+    cfg.gridDim = dim3((unsigned)n_rec);
+    cfg.blockDim = dim3(128);
+    if (e == cudaSuccess) {
+        switch (desc->block) {
+            case 2: e = cudaLaunchKernelEx(&cfg, pack::fill_kernel<2>, p); break;
+            case 4: e = cudaLaunchKernelEx(&cfg, pack::fill_kernel<4>, p); break;
+            case 8: e = cudaLaunchKernelEx(&cfg, pack::fill_kernel<8>, p); break;
+            default: e = cudaLaunchKernelEx(&cfg, pack::fill_kernel<16>, p); break;
+        }
     }
+    if (e != cudaSuccess) return MWU_ERR_CUDA;
     count_launch(3);
     return cudaGetLastError() == cudaSuccess ? MWU_OK : MWU_ERR_CUDA;
 }
