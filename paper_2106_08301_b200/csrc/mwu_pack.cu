@@ -28,21 +28,22 @@ struct Params {
     unsigned *dev_status;
     long long rows, cols;
     int b;
+    long long bpr;                  // blocks per row: cols / b
+    unsigned n_stages;              // L.n_stages, for 32-bit record arithmetic (records < 2^31)
     PackedLayout L;
     unsigned long long gap[5][2];   // byte ranges between the sections (alignment padding), zeroed by scan_kernel
 };
 
 // class masks of row r of a record; padding rows are all-pruned
-__device__ __forceinline__ void row_masks(const Params &p, long long tile, long long stage, int r,
+__device__ __forceinline__ void row_masks(const Params &p, int nb, long long tile, long long stage, int r,
                                           unsigned *P, unsigned *U, unsigned long long *sgn) {
-    const int nb = kStageK / p.b;
     const unsigned mask = (nb >= 32) ? 0xffffffffu : ((1u << nb) - 1u);
     const long long n = tile * kTileRows + r;
     *P = mask;
     *U = 0;
     *sgn = 0;
     if (n < p.rows) {
-        const long long j0 = n * (p.cols / p.b) + stage * nb;
+        const long long j0 = n * p.bpr + stage * nb;
         *P = (p.pruned_bitmap[j0 >> 5] >> (j0 & 31)) & mask;
         *U = (p.unified_bitmap[j0 >> 5] >> (j0 & 31)) & mask & ~*P;
         const long long f = n * p.cols + stage * kStageK;
@@ -93,12 +94,12 @@ constexpr int COUNT_WARPS = 16;                         // each takes 8 of the t
 __global__ void __launch_bounds__(32 * COUNT_WARPS) count_kernel(Params p) {
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const long long chunks = (p.L.n_stages + 31) / 32;      // 32 records of a tile at a time: lane = record (stage)
+    const unsigned chunks = (p.n_stages + 31u) / 32u;       // 32 records of a tile at a time: lane = record (stage)
     const long long tile = blockIdx.x / chunks;
-    const long long stage = (blockIdx.x % chunks) * 32 + lane;
+    const long long stage = (long long)(blockIdx.x % chunks) * 32 + lane;
     const int nb = kStageK / p.b;
     const unsigned mask = (nb >= 32) ? 0xffffffffu : ((1u << nb) - 1u);
-    const long long bpr = p.cols / p.b;                     // blocks per row
+    const long long bpr = p.bpr;                            // blocks per row
     constexpr int RPW = kTileRows / COUNT_WARPS;
     __shared__ unsigned s_cu[COUNT_WARPS][32], s_cp[COUNT_WARPS][32], s_live[COUNT_WARPS][32];
     unsigned cu = 0, cp = 0, live = 0;
@@ -238,8 +239,9 @@ __global__ void __launch_bounds__(128) fill_kernel(Params p) {
     constexpr int STORE = (B >= 8) ? 16 : 2 * B;            // bytes of one shared-memory store
     constexpr int G = 128 / STORE;                          // store slots of a 128-byte row
     constexpr int LPB = (B >= 4) ? B / 4 : 1;               // lanes that share a dense block's run of W
-    const long long rec = blockIdx.x;
-    const long long tile = rec / p.L.n_stages, stage = rec % p.L.n_stages;
+    const unsigned rec = blockIdx.x;
+    const unsigned tile_u = rec / p.n_stages;
+    const long long tile = tile_u, stage = rec - tile_u * p.n_stages;
     const int r = threadIdx.x, lane = r & 31, warp = r >> 5;
     const uint4 *recs = reinterpret_cast<const uint4 *>(p.packed + p.L.off_rec);
     uint2 *ulist = reinterpret_cast<uint2 *>(p.packed + p.L.off_ulist);
@@ -248,12 +250,13 @@ __global__ void __launch_bounds__(128) fill_kernel(Params p) {
     unsigned short *ppos = reinterpret_cast<unsigned short *>(p.packed + p.L.off_ppos);
 
     __shared__ unsigned s_bal[4][3 * G];                    // per warp and (class, slot): the rows that have such a block
+    __shared__ unsigned char s_before[4][3 * G], s_len[3 * G];   // ... how many in the warps before, and in all
     __shared__ unsigned short s_full[3][kTileRows + 1];     // per class and q: list entries of rounds 0 .. q-1
     __shared__ unsigned s_more[3][kTileRows + 1];           // per class and q: slots that have a round q
     __shared__ unsigned short s_off[3][kTileRows * NBK];    // tile offsets of each class list, in list order
     unsigned P, U;
     unsigned long long sgn;
-    row_masks(p, tile, stage, r, &P, &U, &sgn);
+    row_masks(p, NBK, tile, stage, r, &P, &U, &sgn);
     const unsigned D = ~P & ~U & MASK;
     // class of block i: 0 pruned, 1 dense, 2 unified.  occ[class]: the store slots this row fills with it
     // (a row never has two blocks in one slot)
@@ -275,6 +278,16 @@ __global__ void __launch_bounds__(128) fill_kernel(Params p) {
         }
     }
     __syncthreads();
+    // blocks per (class, slot) in the record, and in the warps before each warp (population counts
+    // are few to a clock, so each is taken once per CTA, not once per thread)
+    for (int t = r; t < 4 * 3 * G; t += kTileRows) {
+        const int ww = t / (3 * G), f = t % (3 * G);
+        unsigned before = 0;
+        for (int w2 = 0; w2 < ww; ++w2) before += __popc(s_bal[w2][f]);
+        s_before[ww][f] = (unsigned char)before;
+        if (ww == 3) s_len[f] = (unsigned char)(before + __popc(s_bal[3][f]));
+    }
+    __syncthreads();
     // round-robin order of a class list: round q takes the q-th block of every slot that has one.
     // Thread q (and thread 0 for q = 128) tabulates what comes before round q.
     for (int q = r; q <= kTileRows; q += kTileRows) {
@@ -283,8 +296,7 @@ __global__ void __launch_bounds__(128) fill_kernel(Params p) {
             unsigned full = 0, more = 0;
 #pragma unroll
             for (int sl = 0; sl < G; ++sl) {
-                const unsigned len = __popc(s_bal[0][c * G + sl]) + __popc(s_bal[1][c * G + sl]) +
-                                     __popc(s_bal[2][c * G + sl]) + __popc(s_bal[3][c * G + sl]);
+                const unsigned len = s_len[c * G + sl];
                 full += len < (unsigned)q ? len : (unsigned)q;
                 more |= (len > (unsigned)q) ? (1u << sl) : 0u;
             }
@@ -302,8 +314,8 @@ __global__ void __launch_bounds__(128) fill_kernel(Params p) {
         const unsigned slot = (off & 127u) / STORE;
         const unsigned cls = ((U >> i) & 1u) ? 2u : (((D >> i) & 1u) ? 1u : 0u);
         const unsigned f = cls * G + slot;
-        unsigned q = __popc(s_bal[warp][f] & below);        // earlier rows with the same class and slot
-        for (int ww = 0; ww < warp; ++ww) q += __popc(s_bal[ww][f]);
+        // earlier rows with the same class and slot
+        const unsigned q = s_before[warp][f] + __popc(s_bal[warp][f] & below);
         // q full rounds before it, then the lower slots of its own round
         const unsigned idx = s_full[cls][q] + __popc(s_more[cls][q] & ((1u << slot) - 1u));
         s_off[cls][idx] = (unsigned short)off;
@@ -415,6 +427,8 @@ extern "C" int mwu_pack(const mwu_proj_desc *desc, const float *W, const float *
     p.packed = (unsigned char *)packed;
     p.dev_status = dev_status;
     p.rows = desc->rows; p.cols = desc->cols; p.b = desc->block;
+    p.bpr = desc->cols / desc->block;
+    p.n_stages = (unsigned)p.L.n_stages;
     cudaStream_t st = (cudaStream_t)cuda_stream;
     // header and the gaps between sections must read as zero: scan_kernel writes all 32 header
     // words and clears the gaps
