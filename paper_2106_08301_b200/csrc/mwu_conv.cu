@@ -155,6 +155,7 @@ template <int BW>
 __global__ void __launch_bounds__(PREP_THREADS) conv_prep_kernel(const Params p, unsigned short *Wd, int taps, int C,
                                                                  unsigned n_rec, const unsigned short *x,
                                                                  unsigned short *xt, int HW, int tiles_hw, int tiles_c) {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the tensor-core kernel may set itself up meanwhile
     if (blockIdx.x < n_rec) {
         MWU_CHECK_HEADER(p);
         decode_taps_record<BW>(p, Wd, taps, C, blockIdx.x);
@@ -173,6 +174,7 @@ __global__ void __launch_bounds__(PREP_THREADS) nchw_to_nhwc_kernel(const unsign
 // (rows beyond `rows` are written as zeros)
 __global__ void __launch_bounds__(256) permute_taps_kernel(const unsigned short *Wd, long long ldw, long long rows,
                                                            long long n_pad, int taps, int C, unsigned short *out) {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const long long K = (long long)taps * C, total = n_pad * K;
     for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
         const long long row = i / K, kk = i - row * K;
@@ -218,6 +220,9 @@ mwu_conv_taps_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_co
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
+    // launched with programmatic stream serialization: the set-up above ran while the kernel that
+    // prepares the operands was still finishing; its memory is complete from here on
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const unsigned tmem_base = *reinterpret_cast<volatile unsigned *>(&sm->tmem_base);
 
     if (warp == 0) {
@@ -461,8 +466,18 @@ static int run_taps(ConvParams &p, const void *X_nchw, int n, int c, int h, int 
         return MWU_ERR_CUDA;
     const long long tiles = (long long)n * p.tiles_per_img * p.n_ntiles;
     const int grid = (int)(tiles < sm_count ? tiles : sm_count);
-    mwu_conv_taps_kernel<<<grid, C_THREADS, smem, st>>>(tmap_x, tmap_w, p);
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(C_THREADS);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
     count_launch();
+    if (cudaLaunchKernelEx(&cfg, mwu_conv_taps_kernel, tmap_x, tmap_w, p) != cudaSuccess) return MWU_ERR_CUDA;
     return cudaGetLastError() == cudaSuccess ? MWU_OK : MWU_ERR_CUDA;
 }
 

@@ -39,6 +39,7 @@ constexpr int DEC_THREADS = 128;
 template <int BW>
 __global__ void __launch_bounds__(DEC_THREADS)
 mwu_decode_kernel(const Params p, __nv_bfloat16 *Wd, long long ldw) {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the GEMM behind may set itself up meanwhile
     MWU_CHECK_HEADER(p);
     __shared__ __align__(1024) unsigned char tile[REC_BYTES];
     constexpr int ENT = DecodeCfg<BW, DEC_THREADS>::ENT;
@@ -198,6 +199,9 @@ mwu_dense_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
     cluster_sync_all();                                 // both CTAs' barriers exist before any remote arrive
     tc_fence_after();
     const unsigned tmem_base = *reinterpret_cast<volatile unsigned *>(&sm->tmem_base);
+    // launched with programmatic stream serialization: everything above ran while the kernel before
+    // (the one that expands the weights) was still finishing; its memory is complete from here on
+    asm volatile("griddepcontrol.wait;" ::: "memory");
 
     // the masks of tile nt: a view into the table, or a fresh copy in the role's own buffer
     auto load_live = [&](unsigned char *table, long long nt) -> const unsigned char * {
@@ -459,13 +463,15 @@ cudaError_t launch_dense(const CUtensorMap &tmap_x, const CUtensorMap &tmap_w, c
     cfg.blockDim = dim3(D_THREADS);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = 2;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = 2;
     count_launch();
     return cudaLaunchKernelEx(&cfg, kern, tmap_x, tmap_w, tmap_y, p);
 }
