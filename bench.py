@@ -39,6 +39,27 @@ L2_BYTES = 126 * 1024 * 1024
 FLUSH_BYTES = 256 * 1024 * 1024
 
 
+def recorded_traffic(workload: str):
+    """DRAM bytes per call of the product kernels, from the ncu captures summarised in
+    profiles/dram_traffic.txt; None when the table has no row for the workload or the kernel sources
+    have changed since the capture (the row carries a digest of them)."""
+    import glob
+    import hashlib
+    path = os.path.join(ROOT, "profiles", "dram_traffic.txt")
+    if not os.path.exists(path):
+        return None
+    h = hashlib.sha256()
+    for f in sorted(glob.glob(os.path.join(ROOT, "paper_2106_08301_b200", "csrc", "*"))):
+        h.update(os.path.basename(f).encode())
+        h.update(open(f, "rb").read())
+    digest = h.hexdigest()[:16]
+    for ln in open(path):
+        cells = [c.strip() for c in ln.strip().strip("|").split("|")]
+        if len(cells) == 4 and cells[0] == workload and cells[3] == digest and cells[2].isdigit():
+            return int(cells[2])
+    return None
+
+
 def measured_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -533,7 +554,8 @@ def run_gpu(args):
             roof["kernel"] = ("mwu_conv_implicit" if is_conv else "mwu_gemm") + (
                 " (decode kernel + two-operand tensor-core kernel, timed together)" if ws_bytes else " (fused kernel)")
             roof["roofline_ms"] = max(t_flops, t_bytes) * 1e3
-            roof["traffic"] = None       # DRAM bytes come from ncu captures, not from this run
+            # DRAM bytes come from an ncu capture of this call, not from this run; null once the kernels changed
+            roof["traffic"] = recorded_traffic(wl.name) if (ws_bytes and not args.m and not group) else None
             roof["projection"] = roof_proj
             line["roofline"] = roof
             if not is_conv and W.numel() >= (1 << 22):
