@@ -41,22 +41,24 @@ FLUSH_BYTES = 256 * 1024 * 1024
 
 def recorded_traffic(workload: str):
     """DRAM bytes per call of the product kernels, from the ncu captures summarised in
-    profiles/dram_traffic.txt; None when the table has no row for the workload or the kernel sources
-    have changed since the capture (the row carries a digest of them)."""
-    import glob
+    profiles/dram_traffic.txt; None when the table has no row for the workload or the sources of
+    those kernels have changed since the capture (the row names them and carries their digest)."""
     import hashlib
     path = os.path.join(ROOT, "profiles", "dram_traffic.txt")
     if not os.path.exists(path):
         return None
-    h = hashlib.sha256()
-    for f in sorted(glob.glob(os.path.join(ROOT, "paper_2106_08301_b200", "csrc", "*"))):
-        h.update(os.path.basename(f).encode())
-        h.update(open(f, "rb").read())
-    digest = h.hexdigest()[:16]
     for ln in open(path):
         cells = [c.strip() for c in ln.strip().strip("|").split("|")]
-        if len(cells) == 4 and cells[0] == workload and cells[3] == digest and cells[2].isdigit():
-            return int(cells[2])
+        if len(cells) != 5 or cells[0] != workload or not cells[2].isdigit():
+            continue
+        h = hashlib.sha256()
+        try:
+            for name in cells[4].split():
+                h.update(name.encode())
+                h.update(open(os.path.join(ROOT, "paper_2106_08301_b200", "csrc", name), "rb").read())
+        except OSError:
+            return None
+        return int(cells[2]) if h.hexdigest()[:16] == cells[3] else None
     return None
 
 

@@ -2114,30 +2114,36 @@ __global__ void __launch_bounds__(FIN_THREADS) multipass_kernel(Params p, float 
 // over the group's columns with shuffles (the pairing of the block keys continued across blocks);
 // the rows of a group are then summed as a pairwise tree in shared memory.  Everything is fp64 with
 // one rounding per operation, in a fixed order: the keys do not depend on the launch shape.
+template <int GC>                                      // columns of a group: 16, 32 or 64
 __global__ void __launch_bounds__(256) group_stats_kernel(Params p, double *gkey, long long rows, long long cols) {
     __shared__ double s_row[256][4];
-    const unsigned gc = p.group_cols, gr = p.group_rows;
-    const unsigned nsl = 64u / gc;                      // group slices per CTA tile: 4, 2 or 1
-    const unsigned lanes_per_slice = gc / 4u;
+    constexpr unsigned gc = GC;
+    const unsigned gr = p.group_rows;
+    constexpr unsigned nsl = 64u / gc;                  // group slices per CTA tile: 4, 2 or 1
+    constexpr unsigned lanes_per_slice = gc / 4u;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const long long row0 = (long long)blockIdx.y * 256, col0 = (long long)blockIdx.x * 64;
     const long long col = col0 + (lane & 15) * 4;
+    const long long first = (row0 + warp * 32 + (lane >> 4)) * cols + col;      // this thread's rows: every second one from here
+    const bool l1 = p.use_l1 != 0;
 #pragma unroll 4
     for (int it = 0; it < 16; ++it) {
         const int r = warp * 32 + it * 2 + (lane >> 4);
         const long long row = row0 + r;
+        const long long at = first + (long long)it * 2 * cols;
         float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
         if (row < rows && col < cols) {
-            v = __ldg(reinterpret_cast<const float4 *>(p.W + row * cols + col));
+            v = __ldg(reinterpret_cast<const float4 *>(p.W + at));
             if (p.U) {
-                const float4 d = __ldg(reinterpret_cast<const float4 *>(p.U + row * cols + col));
+                const float4 d = __ldg(reinterpret_cast<const float4 *>(p.U + at));
                 v.x = __fadd_rn(v.x, d.x); v.y = __fadd_rn(v.y, d.y); v.z = __fadd_rn(v.z, d.z); v.w = __fadd_rn(v.w, d.w);
             }
         }
         const double a0 = (double)fabsf(v.x), a1 = (double)fabsf(v.y), a2 = (double)fabsf(v.z), a3 = (double)fabsf(v.w);
         double t;
-        if (p.use_l1) t = __dadd_rn(__dadd_rn(a0, a1), __dadd_rn(a2, a3));
+        if (l1) t = __dadd_rn(__dadd_rn(a0, a1), __dadd_rn(a2, a3));
         else t = __dadd_rn(__fma_rn(a0, a0, __dmul_rn(a1, a1)), __fma_rn(a2, a2, __dmul_rn(a3, a3)));   // squares are exact
+#pragma unroll
         for (unsigned m = 1; m < lanes_per_slice; m <<= 1) t = __dadd_rn(t, __shfl_xor_sync(0xffffffffu, t, m));
         if (((unsigned)lane & (lanes_per_slice - 1u)) == 0u) s_row[r][((unsigned)lane & 15u) / lanes_per_slice] = t;
     }
@@ -2188,11 +2194,27 @@ __global__ void __launch_bounds__(FIN_THREADS) group_select_kernel(const double 
             if ((k & mask) == prefix) atomicAdd(&s_hist[(unsigned)(k >> shift) & 255u], 1u);
         }
         __syncthreads();
-        if (threadIdx.x == 0) {
-            unsigned r = s_r, d = 0;
-            while (d < 255u && s_hist[d] < r) { r -= s_hist[d]; ++d; }
-            s_r = r;
-            s_prefix = prefix | ((u64)d << shift);
+        if (threadIdx.x < 32) {
+            // the digit holding the r-th key: eight bins a lane, a shuffle scan over the lanes
+            const unsigned lane = threadIdx.x;
+            unsigned mine[8], sum = 0;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) { mine[j] = s_hist[lane * 8 + j]; sum += mine[j]; }
+            unsigned incl = sum;
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const unsigned t = __shfl_up_sync(0xffffffffu, incl, off);
+                if (lane >= (unsigned)off) incl += t;
+            }
+            const unsigned r = s_r;
+            const unsigned hit = __ballot_sync(0xffffffffu, incl >= r);      // never empty: the keys left are >= r
+            const unsigned owner = hit ? (unsigned)__ffs(hit) - 1u : 31u;
+            if (lane == owner) {
+                unsigned left = r - (incl - sum), d = 0;
+                while (d < 7u && mine[d] < left) { left -= mine[d]; ++d; }
+                s_r = left;
+                s_prefix = prefix | ((u64)(lane * 8u + d) << shift);
+            }
         }
         mask |= (u64)255 << shift;
         __syncthreads();
@@ -2288,7 +2310,11 @@ static cudaError_t launch_project(const mwu::proj::Params &p, const mwu_proj_des
     if (p.gprune) {
         // grouped pruning: the groups' keys, then the groups to zero (a bit per group)
         const dim3 grid((unsigned)((desc->cols + 63) / 64), (unsigned)((desc->rows + 255) / 256));
-        group_stats_kernel<<<grid, 256, 0, st>>>(p, gkey, desc->rows, desc->cols);
+        switch (desc->prune_group_cols) {
+            case 16: group_stats_kernel<16><<<grid, 256, 0, st>>>(p, gkey, desc->rows, desc->cols); break;
+            case 32: group_stats_kernel<32><<<grid, 256, 0, st>>>(p, gkey, desc->rows, desc->cols); break;
+            default: group_stats_kernel<64><<<grid, 256, 0, st>>>(p, gkey, desc->rows, desc->cols); break;
+        }
         const unsigned n_groups = (unsigned)mwu::n_groups_of(desc);
         const unsigned per_group = (unsigned)(desc->prune_group_rows * desc->prune_group_cols / desc->block);
         group_select_kernel<<<1, FIN_THREADS, 0, st>>>(gkey, n_groups, (unsigned)(desc->k_prune / per_group), gprune);
