@@ -258,7 +258,6 @@ mwu_dense_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
             const long long nt = nt_;
             const unsigned buf = mine, use_phase = (unsigned)((k >> 1) & 1);
             const unsigned char *lv = load_live(mine ? sm->live_mma_b : sm->live_mma, nt);
-            bool ready = false;
             if (!mbar_wait(smem_u32(&sm->tempty[buf]), use_phase ^ 1u, abort)) ok = false;
             if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
             // the hand-over: tiles 0 .. k-1 have been issued
@@ -275,21 +274,16 @@ mwu_dense_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
             unsigned phase = ring / D_STAGES;
             tc_fence_after();
             bool first = true;
+            // The stage loop holds no vote and no warp barrier: every lane executes the same barrier
+            // probes as one warp instruction and so takes the same decisions; what the warp does
+            // between two stages has to fit into the time the MMAs of one stage take.
             for (int ks = 0; ks < n_stages; ++ks) {
                 const unsigned live = lv[ks];
                 if (!live) continue;
-                if (!ready) {
-                    if (!mbar_wait_spin(smem_u32(&sm->full[stage]), phase, abort)) ok = false;
-                    if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
-                }
+                if (!mbar_wait_spin(smem_u32(&sm->full[stage]), phase, abort)) { ok = false; break; }
                 tc_fence_after();
                 const unsigned long long adesc = make_desc(smem_u32(sA + stage * D_A_BYTES));
                 const unsigned long long bdesc = make_desc(smem_u32(sB + stage * D_B_BYTES));
-                {
-                    const int nstage = (stage + 1 == D_STAGES) ? 0 : stage + 1;
-                    const unsigned nphase = (stage + 1 == D_STAGES) ? (phase ^ 1u) : phase;
-                    ready = __all_sync(0xffffffffu, mbar_test(smem_u32(&sm->full[nstage]), nphase));
-                }
                 if (elect_one()) {
 #pragma unroll
                     for (int k4 = 0; k4 < 4; ++k4) {
@@ -303,10 +297,9 @@ mwu_dense_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
                 }
                 first = false;
                 issued_any = true;
-                __syncwarp();
                 if (++stage == D_STAGES) { stage = 0; phase ^= 1u; }
             }
-            if (!ok) break;
+            if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
             if (lane == 0) {
                 *ho_ring = (unsigned)stage + phase * D_STAGES;
                 __threadfence_block();
