@@ -59,7 +59,7 @@ typedef enum {
 
 /* How mwu_project organises its kernels.  Every choice gives the same bits. */
 typedef enum {
-    MWU_ALGO_AUTO = 0,       /* one pass from 32768 blocks on, multi pass below                */
+    MWU_ALGO_AUTO = 0,       /* one pass from 8192 blocks on, multi pass below                 */
     MWU_ALGO_ONE_PASS = 1,   /* outputs written in one sweep over W with thresholds estimated
                                 from a sample, then the few blocks near a threshold corrected */
     MWU_ALGO_MULTI_PASS = 2  /* statistics pass, exact thresholds, emit pass                  */

@@ -556,7 +556,7 @@ static void fill_common(Params &p, const mwu_proj_desc *desc, const void *packed
 
 // Activation rows from which expanding the weights once per call beats decoding them again for
 // every 512-row activation tile.
-static const int64_t kDecodeOnceMinRows = 1024;
+static const int64_t kDecodeOnceMinRows = 1;
 
 static bool encode_bf16_2d(mwu::gemm::EncodeTiledFn encode, CUtensorMap *tmap, const void *ptr, int64_t inner,
                            int64_t outer, int64_t ld, int box_rows) {

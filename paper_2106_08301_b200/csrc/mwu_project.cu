@@ -56,7 +56,7 @@ constexpr int SAMP_THREADS = 1024;
 constexpr int SAMP_PER = NSAMP / SAMP_THREADS;
 static_assert(SAMP_PER == 4, "sample_select ranks one level-A key with the four threads that hold 16 samples");
 constexpr int STAGE_ENTRIES = 64;  // per-warp staging of candidate-list entries in pass_kernel
-constexpr long long ONE_PASS_MIN_BLOCKS = 32768;   // below: launch latency decides, multi-pass has fewer launches
+constexpr long long ONE_PASS_MIN_BLOCKS = 8192;    // below: launch latency decides, multi-pass has fewer launches
 constexpr int PASS_LOADS = 4;      // 16-byte loads of bin codes a thread keeps in flight in the selection passes
 constexpr int FIN_THREADS = 1024;   // block size of the kernels whose last CTA finalises
 static_assert(NB_MAX / FIN_THREADS <= 64, "scan_hist searches one thread's bins with one warp, two per lane");

@@ -114,10 +114,11 @@ def test_gemm_ws_degenerate_classes_and_dead_stages():
     check_gemm_ws(W, 16, n_zero + 500, n_zero, 1500)
 
 
-def test_gemm_ws_falls_back_without_workspace_or_for_few_rows():
+def test_gemm_ws_falls_back_without_workspace_or_with_a_short_one():
     W = inputs.normal_weights(256, 128, 0.02, 88)
     desc, bufs, packed, p = project_and_pack(W, 8, 2000, 1000)
-    assert B.mwu_gemm_workspace_bytes(desc, 200) == 0
+    assert B.mwu_gemm_workspace_bytes(desc, 0) == 0
+    assert B.mwu_gemm_workspace_bytes(desc, 200) == 256 * 128 * 2       # the expanded weights, bf16
     for M in (200, 1024):
         X = inputs.normal_activations_bf16((M, 128), 3)
         ref = O.gemm(X.to(torch.float64).numpy(), O.decoded_weights(p, 8))
