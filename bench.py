@@ -558,6 +558,11 @@ def run_gpu(args):
             roof["roofline_ms"] = max(t_flops, t_bytes) * 1e3
             # DRAM bytes come from an ncu capture of this call, not from this run; null once the kernels changed
             roof["traffic"] = recorded_traffic(wl.name) if (ws_bytes and not args.m and not group) else None
+            roof["traffic_source"] = ("ncu capture of this call (dram__bytes_read.sum + dram__bytes_write.sum), recorded "
+                                      "with a digest of the kernels' sources; the digest still matches"
+                                      if roof["traffic"] is not None else
+                                      "none: no capture recorded for this workload and launch configuration, or the "
+                                      "kernels changed since it was taken")
             roof["projection"] = roof_proj
             line["roofline"] = roof
             if not is_conv and W.numel() >= (1 << 22):
