@@ -258,12 +258,15 @@ mwu_dense_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
             const long long nt = nt_;
             const unsigned buf = mine, use_phase = (unsigned)((k >> 1) & 1);
             const unsigned char *lv = load_live(mine ? sm->live_mma_b : sm->live_mma, nt);
-            if (!mbar_wait(smem_u32(&sm->tempty[buf]), use_phase ^ 1u, abort)) ok = false;
+            if (!mbar_wait_spin(smem_u32(&sm->tempty[buf]), use_phase ^ 1u, abort)) ok = false;
             if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
             // the hand-over: tiles 0 .. k-1 have been issued
             if (*ho_tiles != (unsigned)k) {
                 const long long t0 = clock64();
+                unsigned polls = 0;
                 while (*ho_tiles != (unsigned)k) {
+                    // with a long reduction this issuer idles for a whole tile: it sleeps between looks
+                    if (++polls > 64u) __nanosleep(256);
                     if (*abort) { ok = false; break; }
                     if (clock64() - t0 > WAIT_LIMIT_CYCLES) { *abort = 1; ok = false; break; }
                 }

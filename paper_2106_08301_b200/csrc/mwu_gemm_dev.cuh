@@ -112,24 +112,25 @@ __device__ __forceinline__ bool mbar_test(unsigned bar, unsigned parity) {
 }
 // bounded wait: false when aborted or out of time (then *abort is set)
 __device__ __forceinline__ bool mbar_wait(unsigned bar, unsigned parity, volatile int *abort) {
-    // Polling, not a suspended try_wait: a waiter that went to sleep on a barrier which the OTHER CTA
-    // of the pair completes (a multicast commit, a remote arrive) was seen to wake a microsecond or
-    // two late, which serialised the pair's epilogue with the next tile's MMAs.
+    // A short wait is polled (a waiter suspended in try_wait wakes a few hundred cycles late); a long
+    // one, an epilogue warp waiting out a tile of a long reduction, sleeps in try_wait and leaves the
+    // issue slots and the power to the warps that work.
 #pragma unroll 1
-    for (int i = 0; i < 4096; ++i)
+    for (int i = 0; i < 128; ++i)
         if (mbar_test(bar, parity)) return true;
     const long long t0 = clock64();
 #pragma unroll 1
     while (true) {
-#pragma unroll 1
-        for (int i = 0; i < 64; ++i)
-            if (mbar_test(bar, parity)) return true;
+        if (mbar_try_wait(bar, parity)) return true;
         if (*abort) return false;
         if (clock64() - t0 > WAIT_LIMIT_CYCLES) { *abort = 1; return false; }
     }
 }
-// kept as a name of its own where a single latency-critical thread waits
+// the same for a single latency-critical warp (producer, MMA issuer): polled for much longer first
 __device__ __forceinline__ bool mbar_wait_spin(unsigned bar, unsigned parity, volatile int *abort) {
+#pragma unroll 1
+    for (int i = 0; i < 4096; ++i)
+        if (mbar_test(bar, parity)) return true;
     return mbar_wait(bar, parity, abort);
 }
 template <int BYTES>
