@@ -250,7 +250,8 @@ __global__ void __launch_bounds__(128) fill_kernel(Params p) {
     unsigned short *ppos = reinterpret_cast<unsigned short *>(p.packed + p.L.off_ppos);
 
     __shared__ unsigned s_bal[4][3 * G];                    // per warp and (class, slot): the rows that have such a block
-    __shared__ unsigned char s_before[4][3 * G], s_len[3 * G];   // ... how many in the warps before, and in all
+    __shared__ unsigned char s_before[4][3 * G];            // ... how many in the warps before
+    __shared__ __align__(4) unsigned char s_len[3 * G];     // ... and in all (at most 128 each: a byte)
     __shared__ unsigned short s_full[3][kTileRows + 1];     // per class and q: list entries of rounds 0 .. q-1
     __shared__ unsigned s_more[3][kTileRows + 1];           // per class and q: slots that have a round q
     __shared__ unsigned short s_off[3][kTileRows * NBK];    // tile offsets of each class list, in list order
@@ -293,12 +294,16 @@ __global__ void __launch_bounds__(128) fill_kernel(Params p) {
     for (int q = r; q <= kTileRows; q += kTileRows) {
 #pragma unroll
         for (int c = 0; c < 3; ++c) {
+            // four slots at a time: bytewise minimum summed with a dot product, bytewise compare
+            // gathered into a bit per slot
             unsigned full = 0, more = 0;
+            const unsigned q4 = (unsigned)q * 0x01010101u;
+            const unsigned *len4 = reinterpret_cast<const unsigned *>(s_len + c * G);
 #pragma unroll
-            for (int sl = 0; sl < G; ++sl) {
-                const unsigned len = s_len[c * G + sl];
-                full += len < (unsigned)q ? len : (unsigned)q;
-                more |= (len > (unsigned)q) ? (1u << sl) : 0u;
+            for (int w = 0; w < G / 4; ++w) {
+                const unsigned l4 = len4[w];
+                full = __dp4a(__vminu4(l4, q4), 0x01010101u, full);
+                more |= (((__vcmpgtu4(l4, q4) & 0x80808080u) * 0x00204081u) >> 28) << (4 * w);
             }
             s_full[c][q] = (unsigned short)full;
             s_more[c][q] = more;
@@ -327,42 +332,40 @@ __global__ void __launch_bounds__(128) fill_kernel(Params p) {
     bool bad = false;
     constexpr unsigned BMASK = (B >= 32) ? 0xffffffffu : ((1u << B) - 1u);
     const unsigned len_u = nx.x - me.x, len_d = nx.y - me.y, len_p = nx.z - me.z;
-    if (len_u + len_d + len_p != (unsigned)(kTileRows * NBK)) bad = true;     // the table does not describe this record
+    // the record's three list ranges must lie inside the sections (checked once, not per entry)
+    if (len_u + len_d + len_p != (unsigned)(kTileRows * NBK) ||
+        (unsigned long long)me.x + len_u > (unsigned long long)p.L.n_unified ||
+        (unsigned long long)me.y + len_d > (unsigned long long)p.L.n_dense ||
+        (unsigned long long)me.z + len_p > (unsigned long long)p.L.n_plist)
+        bad = true;                                          // the table does not describe this record
     else {
+        const long long row_base = tile * kTileRows;
+        const long long f_base = row_base * p.cols + stage * kStageK;          // first weight of the record
         // pruned blocks: positions only
-        for (unsigned t = (unsigned)r; t < len_p; t += 128u) {
-            const unsigned long long e = (unsigned long long)me.z + t;
-            if (e < (unsigned long long)p.L.n_plist) ppos[e] = s_off[0][t];
-            else bad = true;
-        }
+        unsigned short *pp = ppos + me.z;
+        for (unsigned t = (unsigned)r; t < len_p; t += 128u) pp[t] = s_off[0][t];
         // unified blocks: sign bits, position, magnitude
+        uint2 *ul = ulist + me.x;
+        const long long j_base = row_base * p.bpr + stage * NBK;
         for (unsigned t = (unsigned)r; t < len_u; t += 128u) {
-            const unsigned long long e = (unsigned long long)me.x + t;
             const unsigned off = s_off[2][t];
             unsigned rr, i;
             row_block_of(off, B, &rr, &i);
-            const long long n = tile * kTileRows + rr;
-            const long long f = n * p.cols + stage * kStageK + (long long)i * B;
+            const long long f = f_base + (long long)rr * p.cols + i * B;
             const unsigned sb = (__ldg(p.sign_bits + (f >> 5)) >> (f & 31)) & BMASK;
-            const long long j = n * (p.cols / B) + stage * NBK + i;
-            const unsigned ub = (unsigned)__bfloat16_as_ushort(__float2bfloat16_rn(__ldg(p.u + j)));
-            if (e < (unsigned long long)p.L.n_unified) ulist[e] = make_uint2(spread_signs(sb, B), off | (ub << 16));
-            else bad = true;
+            const unsigned ub = (unsigned)__bfloat16_as_ushort(__float2bfloat16_rn(__ldg(p.u + j_base + (long long)rr * p.bpr + i)));
+            ul[t] = make_uint2(spread_signs(sb, B), off | (ub << 16));
         }
         // dense blocks: position, then the values, LPB lanes to a block
-        for (unsigned t = (unsigned)r; t < len_d; t += 128u) {
-            const unsigned long long e = (unsigned long long)me.y + t;
-            if (e < (unsigned long long)p.L.n_dense) dpos[e] = s_off[1][t];
-            else bad = true;
-        }
+        unsigned short *dp = dpos + me.y;
+        for (unsigned t = (unsigned)r; t < len_d; t += 128u) dp[t] = s_off[1][t];
+        unsigned char *pay = dpay + (unsigned long long)me.y * (2 * B);
         for (unsigned q = (unsigned)r; q < len_d * (unsigned)LPB; q += 128u) {
             const unsigned t = q / (unsigned)LPB, part = q % (unsigned)LPB;
-            const unsigned long long e = (unsigned long long)me.y + t;
-            if (e >= (unsigned long long)p.L.n_dense) continue;                  // flagged above
             unsigned rr, i;
             row_block_of(s_off[1][t], B, &rr, &i);
-            const long long f = (tile * kTileRows + rr) * p.cols + stage * kStageK + (long long)i * B + part * 4;
-            unsigned char *dst = dpay + e * (2 * B) + part * 8;
+            const long long f = f_base + (long long)rr * p.cols + i * B + part * 4;
+            unsigned char *dst = pay + q * 8u;               // = t * 2B + part * 8 when a block takes LPB lanes
             if (B >= 4) {
                 float4 a = __ldg(reinterpret_cast<const float4 *>(p.W + f));
                 if (p.U) {
@@ -379,7 +382,7 @@ __global__ void __launch_bounds__(128) fill_kernel(Params p) {
                     a.x = __fadd_rn(a.x, d.x); a.y = __fadd_rn(a.y, d.y);
                 }
                 const __nv_bfloat162 h0 = __floats2bfloat162_rn(a.x, a.y);
-                *reinterpret_cast<unsigned *>(dst) = *reinterpret_cast<const unsigned *>(&h0);
+                *reinterpret_cast<unsigned *>(pay + q * 4u) = *reinterpret_cast<const unsigned *>(&h0);
             }
         }
     }
